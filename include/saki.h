@@ -1,0 +1,192 @@
+/*
+ * saki.h - C ABI of the B200-native SAKI per-position routing library.
+ *
+ * For every generated position the library takes the full-vocabulary row of
+ * student logits s and teacher logits t and computes, on the GPU:
+ *   1. p = softmax(s/temperature), T = softmax(t/temperature)  (Section 3.1)
+ *   2. the geometric bridge q = p^(1-lambda) T^lambda / Z with the largest
+ *      lambda in [0,1] such that KL(q || p) <= eps              (Eqs. "bridge",
+ *      "trust_region"; endpoints: Appendix J)
+ *   3. the maximal coupling of the student's proposal x with q: accept with
+ *      probability min(1, q(x)/p(x)), otherwise draw the committed token from
+ *      [q-p]_+ / TV(p,q); TV(p,q) is the correction probability (Eqs.
+ *      "accept", "residual", Proposition 1)
+ *   4. the routed loss: -A log pi(x), A = -(log p(x) - log T(x)), at accepted
+ *      positions (Eqs. "k1_loss_token", "k1_advantage_token"); -log pi(v*),
+ *      v* = argmax T, at corrected positions (Eq. "teacher_mode_loss")
+ *   5. the gradient of that loss with respect to the student logits
+ *      (Eq. "general_objective"; lambda, q, the coupling outcome and A are
+ *      constants of differentiation)
+ *   6. for drafted blocks, the left-to-right first-rejection resolve of
+ *      Section 3.5 / Appendix I.
+ *
+ * Conventions
+ *   - Every pointer in the structs below is a DEVICE pointer owned by the
+ *     caller unless a comment says HOST.  The library never frees or keeps
+ *     them.  Input and output buffers must not overlap.
+ *   - Calls are asynchronous on the given CUDA stream (a cudaStream_t passed
+ *     as void*; NULL = the legacy default stream) and return after host-side
+ *     validation and launch.  Outputs are valid once the stream has run.
+ *   - No exception, abort or device trap crosses this boundary.  Bad
+ *     arguments return an error code with nothing launched; bad DATA (a
+ *     non-finite logit, a proposal id outside [0,V)) flags the row in
+ *     `row_status`, zeroes its float outputs and gradient row and sets its
+ *     ids to -1.
+ *   - Random numbers: Philox4x32-10, key = (seed lo, seed hi), counter =
+ *     (row lo, row hi, stage, block); stage 0 proposal Gumbel noise (word
+ *     v%4 of block v/4), 1 acceptance uniform, 2 residual draw, 3 bonus draw
+ *     (word 0 of block 0).  A word w gives the uniform ((w>>9)+0.5) 2^-23.
+ *     `row` is the GLOBAL row id row_offset + i, so results do not depend on
+ *     how a batch is chunked or sharded.
+ *   - Results are deterministic: same inputs, same GPU model, same outputs.
+ */
+#ifndef SAKI_H_
+#define SAKI_H_
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define SAKI_API __attribute__((visibility("default")))
+#else
+#define SAKI_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SAKI_OK = 0,
+  SAKI_ERR_INVALID_ARG = 1, /* NULL required pointer, N < 0, V < 2, ld < V, eps NaN or < 0,
+                               temperature <= 0 or NaN, K outside [1,16], bad dtype */
+  SAKI_ERR_UNSUPPORTED = 2, /* no CUDA device of compute capability 10.x, or a layout the
+                               kernels do not serve */
+  SAKI_ERR_CUDA = 3,        /* a CUDA runtime call failed; text via saki_last_error() */
+  SAKI_ERR_ROW_STATUS = 4   /* returned only by saki_check(): some row was flagged */
+} saki_status;
+
+typedef enum { SAKI_F32 = 0, SAKI_BF16 = 1 } saki_dtype;
+
+/* row_status bits */
+#define SAKI_ROW_SATURATED    1u  /* lambda = 1: KL(T||p) <= eps (Appendix J, teacher endpoint) */
+#define SAKI_ROW_EPS_ZERO     2u  /* eps <= 0: lambda = 0, q = p, never corrected (Appendix J) */
+#define SAKI_ROW_MASKED       4u  /* mask[i] = 0: loss 0, gradient row 0 (M_t of Eq. "general_objective") */
+#define SAKI_ROW_NONFINITE    8u  /* a logit of the row is NaN or +-Inf */
+#define SAKI_ROW_BAD_ID      16u  /* proposal id outside [0,V) */
+#define SAKI_ROW_TIMEOUT     32u  /* a bounded on-device wait expired; the row's outputs are void */
+#define SAKI_ROW_NOT_COMPUTED 64u /* block verification: position after the first rejection */
+
+/* Inputs of one routing call over N positions. */
+typedef struct {
+  const void* student_logits; /* [N,V] stored logits s, unit stride along V, row stride ld_s ELEMENTS */
+  const void* teacher_logits; /* [N,V] stored logits t, row stride ld_t elements */
+  int64_t ld_s, ld_t;         /* >= V */
+  int64_t N;                  /* >= 0; 0 is a no-op */
+  int32_t V;                  /* >= 2 */
+  int32_t dtype;              /* saki_dtype of both logit arrays (and of dlogits) */
+  const int32_t* proposal;    /* [N] the student's sampled token z_t ~ p_t (Section 3.3). Required */
+  const uint8_t* mask;        /* [N] valid-response mask M_t, or NULL = all valid */
+  float eps;                  /* trust-region radius of Eq. "trust_region", >= 0 */
+  float temperature;          /* > 0; divides both logit rows */
+  uint64_t seed;              /* Philox key */
+  uint64_t row_offset;        /* global id of row 0 */
+} saki_in;
+
+/* Per-position outputs (the token-aligned metadata of Appendix K).  Any pointer
+ * may be NULL (= not wanted) except `corrected` and `token`. Arrays of length N. */
+typedef struct {
+  uint8_t* corrected;    /* C_t: 1 = proposal rejected, token drawn from the residual */
+  int32_t* token;        /* committed token y_t (= proposal when accepted) */
+  int32_t* teacher_top1; /* v*_t = argmax_v t[v], lowest index among exact ties */
+  float* lambda;         /* solved coefficient */
+  float* kl;             /* KL(q||p) at lambda, nats */
+  float* tv;             /* TV(p,q) = residual mass = correction probability */
+  float* accept_prob;    /* min(1, q(x)/p(x)) */
+  float* logp_x;         /* log p(x), log q(x), log T(x) at the proposal */
+  float* logq_x;
+  float* logT_x;
+  float* logp_y;         /* log p(y), log q(y) at the committed token */
+  float* logq_y;
+  float* loss;           /* routed loss of the position, NOT scaled by grad_scale; 0 where masked */
+  uint32_t* row_status;  /* SAKI_ROW_* bits */
+} saki_out;
+
+/* Steps 1-4 above for N positions (no gradient).  `in`/`out` are HOST structs
+ * read during the call.  Returns SAKI_OK after the kernels are enqueued. */
+SAKI_API int saki_route_fwd(const saki_in* in, const saki_out* out, void* cuda_stream);
+
+/* Steps 1-5: as saki_route_fwd, plus dlogits[i,:] = grad_scale * d loss_i / d s[i,:]
+ * in the logits' dtype (round to nearest even), row stride ld_g >= V elements.
+ * grad_scale is the caller's 1/N_valid (Appendix L, "Normalization"). */
+SAKI_API int saki_route_fwd_bwd(const saki_in* in, const saki_out* out, void* dlogits,
+                       int64_t ld_g, float grad_scale, void* cuda_stream);
+
+/* The same computation with every array in HOST memory (pageable or pinned):
+ * the library stages rows through device buffers it allocates and caches,
+ * overlapping the copies with the kernels on its own streams, and returns
+ * when all outputs are in host memory.  `dlogits` may be NULL (forward only). */
+SAKI_API int saki_route_host(const saki_in* in_host, const saki_out* out_host,
+                    void* dlogits_host, int64_t ld_g, float grad_scale);
+
+/* Block verification (Section 3.5, Appendix I) of B drafted blocks of K tokens. */
+typedef struct {
+  const void* student_logits; /* [B,K+1,V]: position j of sequence b at element offset
+                                 b*ss_seq + j*ss_pos; unit stride along V */
+  const void* teacher_logits; /* [B,K+1,V], strides ts_seq, ts_pos (elements) */
+  int64_t ss_seq, ss_pos, ts_seq, ts_pos;
+  int64_t B;                  /* >= 0 */
+  int32_t K;                  /* 1..16 drafted tokens per block */
+  int32_t V;
+  int32_t dtype;
+  const int32_t* draft;       /* [B,K] drafted ids, row stride draft_ld */
+  int64_t draft_ld;
+  float eps, temperature;
+  uint64_t seed;
+  uint64_t seq_offset;        /* global id of sequence 0; position j of sequence b uses the
+                                 random stream of row (seq_offset+b)*(K+1)+j */
+} saki_spec_in;
+
+typedef struct {
+  int32_t* n_accept;           /* [B] length of the accepted prefix, 0..K */
+  int32_t* next_token;         /* [B] residual draw at the first rejection, else a draw from q
+                                  at the bonus position K; -1 if that row was flagged */
+  uint8_t* next_is_correction; /* [B] 1 if next_token is a correction */
+  saki_out per_pos;            /* arrays of length B*(K+1), row b*(K+1)+j; `corrected` and
+                                  `token` required; rows after the first rejection are zeroed
+                                  and carry SAKI_ROW_NOT_COMPUTED; `loss` is not written */
+} saki_spec_out;
+
+SAKI_API int saki_spec_verify(const saki_spec_in* in, const saki_spec_out* out, void* cuda_stream);
+
+/* Harness utility (the proposal is an input of the method: z_t ~ p_t, Section
+ * 3.3): out[i] = argmax_v (logits[i,v]/temperature + G_v) with Gumbel noise
+ * G_v = -log(-log((w_v+0.5) 2^-32)) from stage 0 of row row_offset+i; lowest
+ * index on ties.  Keys are formed in float64. */
+SAKI_API int saki_sample_proposal(const void* logits, int64_t ld, int64_t N, int32_t V,
+                         int32_t dtype, float temperature, uint64_t seed,
+                         uint64_t row_offset, int32_t* out, void* cuda_stream);
+
+/* Synchronises the stream, then reports and clears the number of rows flagged
+ * NONFINITE, BAD_ID or TIMEOUT by calls on this device since the last check.
+ * Returns SAKI_ERR_ROW_STATUS if that number is non-zero.  n_flagged may be NULL. */
+SAKI_API int saki_check(void* cuda_stream, uint64_t* n_flagged);
+
+/* Selects the row kernel: 0 = automatic, 1 = the general kernel (one block per
+ * row, any V and layout), 2 = the register-resident cluster kernel (bf16 rows,
+ * 16-byte aligned, V within its capacity; other inputs fall back to 1).
+ * Process-wide; meant for tests and benchmarks.  Returns the previous value. */
+SAKI_API int saki_set_kernel(int which);
+
+/* Number of kernels this library has launched in this process (all threads). */
+SAKI_API uint64_t saki_launch_count(void);
+
+/* Text of the last error on the calling thread ("" if none). Never NULL. */
+SAKI_API const char* saki_last_error(void);
+
+/* Library version, major*10000 + minor*100 + patch. */
+SAKI_API int saki_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SAKI_H_ */

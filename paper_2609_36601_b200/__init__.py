@@ -1,1 +1,7 @@
-"""B200-native SAKI per-position routing."""
+"""B200-native SAKI per-position routing: thin Python binding over the C-ABI
+library built from csrc/.  Importing the package does not load the CUDA
+library; the first call does, and raises if it is missing (no CPU fallback)."""
+from .binding import (  # noqa: F401
+    load_library, route_fwd, route_fwd_bwd, route_host, spec_verify, sample_proposal,
+    check, set_kernel, launch_count, last_error, version, SakiError,
+)

@@ -1,0 +1,244 @@
+"""Thin ctypes binding of the C-ABI library: argument marshalling only.
+
+Every function takes torch tensors (device memory and streams are torch's),
+passes raw pointers, sizes and strides to the library, and returns torch
+tensors.  There is no CPU fallback: if the library is missing or cannot be
+loaded the first call raises."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsaki.so")
+_lib = None
+
+SAKI_F32, SAKI_BF16 = 0, 1
+ROW_SATURATED, ROW_EPS_ZERO, ROW_MASKED, ROW_NONFINITE, ROW_BAD_ID, ROW_TIMEOUT, ROW_NOT_COMPUTED = 1, 2, 4, 8, 16, 32, 64
+
+_FLOAT_FIELDS = ("lambda", "kl", "tv", "accept_prob", "logp_x", "logq_x", "logT_x", "logp_y", "logq_y", "loss")
+EXPORTS = ("saki_route_fwd", "saki_route_fwd_bwd", "saki_route_host", "saki_spec_verify",
+           "saki_sample_proposal", "saki_check", "saki_set_kernel", "saki_launch_count",
+           "saki_last_error", "saki_version")
+
+
+class SakiError(RuntimeError):
+    def __init__(self, code, text):
+        super().__init__(f"saki error {code}: {text}")
+        self.code = code
+
+
+class SakiIn(C.Structure):
+    _fields_ = [("student_logits", C.c_void_p), ("teacher_logits", C.c_void_p),
+                ("ld_s", C.c_int64), ("ld_t", C.c_int64), ("N", C.c_int64),
+                ("V", C.c_int32), ("dtype", C.c_int32),
+                ("proposal", C.c_void_p), ("mask", C.c_void_p),
+                ("eps", C.c_float), ("temperature", C.c_float),
+                ("seed", C.c_uint64), ("row_offset", C.c_uint64)]
+
+
+class SakiOut(C.Structure):
+    _fields_ = [("corrected", C.c_void_p), ("token", C.c_void_p), ("teacher_top1", C.c_void_p)] + \
+               [(f, C.c_void_p) for f in _FLOAT_FIELDS] + [("row_status", C.c_void_p)]
+
+
+class SakiSpecIn(C.Structure):
+    _fields_ = [("student_logits", C.c_void_p), ("teacher_logits", C.c_void_p),
+                ("ss_seq", C.c_int64), ("ss_pos", C.c_int64), ("ts_seq", C.c_int64), ("ts_pos", C.c_int64),
+                ("B", C.c_int64), ("K", C.c_int32), ("V", C.c_int32), ("dtype", C.c_int32),
+                ("draft", C.c_void_p), ("draft_ld", C.c_int64),
+                ("eps", C.c_float), ("temperature", C.c_float),
+                ("seed", C.c_uint64), ("seq_offset", C.c_uint64)]
+
+
+class SakiSpecOut(C.Structure):
+    _fields_ = [("n_accept", C.c_void_p), ("next_token", C.c_void_p), ("next_is_correction", C.c_void_p),
+                ("per_pos", SakiOut)]
+
+
+def load_library(path: str | None = None):
+    """Loads libsaki.so (built in-tree by `python -m paper_2609_36601_b200.build`)."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or LIB_PATH
+    if not os.path.exists(p):
+        raise SakiError(-1, f"{p} not found: build it with `python -m paper_2609_36601_b200.build`; "
+                            "there is no CPU fallback")
+    lib = C.CDLL(p)
+    lib.saki_route_fwd.argtypes = [C.POINTER(SakiIn), C.POINTER(SakiOut), C.c_void_p]
+    lib.saki_route_fwd_bwd.argtypes = [C.POINTER(SakiIn), C.POINTER(SakiOut), C.c_void_p, C.c_int64, C.c_float, C.c_void_p]
+    lib.saki_route_host.argtypes = [C.POINTER(SakiIn), C.POINTER(SakiOut), C.c_void_p, C.c_int64, C.c_float]
+    lib.saki_spec_verify.argtypes = [C.POINTER(SakiSpecIn), C.POINTER(SakiSpecOut), C.c_void_p]
+    lib.saki_sample_proposal.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_float,
+                                         C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p]
+    lib.saki_check.argtypes = [C.c_void_p, C.POINTER(C.c_uint64)]
+    lib.saki_set_kernel.argtypes = [C.c_int]
+    lib.saki_launch_count.restype = C.c_uint64
+    lib.saki_last_error.restype = C.c_char_p
+    for f in ("saki_route_fwd", "saki_route_fwd_bwd", "saki_route_host", "saki_spec_verify",
+              "saki_sample_proposal", "saki_check", "saki_set_kernel", "saki_version"):
+        getattr(lib, f).restype = C.c_int
+    _lib = lib
+    return lib
+
+
+def _raise(lib, rc):
+    if rc != 0:
+        raise SakiError(rc, lib.saki_last_error().decode())
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return SAKI_F32
+    if t.dtype == torch.bfloat16:
+        return SAKI_BF16
+    raise SakiError(1, f"unsupported logits dtype {t.dtype}")
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _alloc_out(n: int, device, pinned=False):
+    kw = dict(device=device)
+    if pinned:
+        kw = dict(device="cpu", pin_memory=True)
+    out = {"corrected": torch.empty(n, dtype=torch.uint8, **kw),
+           "token": torch.empty(n, dtype=torch.int32, **kw),
+           "teacher_top1": torch.empty(n, dtype=torch.int32, **kw),
+           "row_status": torch.empty(n, dtype=torch.int32, **kw)}
+    for f in _FLOAT_FIELDS:
+        out[f] = torch.empty(n, dtype=torch.float32, **kw)
+    return out
+
+
+def _out_struct(out: dict) -> SakiOut:
+    so = SakiOut()
+    for name, _ in SakiOut._fields_:
+        t = out.get(name)
+        setattr(so, name, t.data_ptr() if t is not None else None)
+    return so
+
+
+def _check_rows(s, t):
+    if s.dim() != 2 or t.shape != s.shape or t.dtype != s.dtype or s.stride(1) != 1 or t.stride(1) != 1:
+        raise SakiError(1, "student/teacher logits must be [N,V] of the same dtype with unit stride along V")
+
+
+def _in_struct(s, t, proposal, mask, eps, temperature, seed, row_offset) -> SakiIn:
+    si = SakiIn()
+    si.student_logits, si.teacher_logits = s.data_ptr(), t.data_ptr()
+    si.ld_s, si.ld_t = (s.stride(0) if s.shape[0] > 1 else s.shape[1]), (t.stride(0) if t.shape[0] > 1 else t.shape[1])
+    si.N, si.V, si.dtype = s.shape[0], s.shape[1], _dtype_code(s)
+    si.proposal = proposal.data_ptr()
+    si.mask = mask.data_ptr() if mask is not None else None
+    si.eps, si.temperature, si.seed, si.row_offset = eps, temperature, seed, row_offset
+    return si
+
+
+def route_fwd(s, t, proposal, eps, temperature=1.0, seed=0, row_offset=0, mask=None, out=None, stream=None):
+    """saki_route_fwd on device tensors; returns the dict of per-position output tensors."""
+    lib = load_library()
+    _check_rows(s, t)
+    out = out if out is not None else _alloc_out(s.shape[0], s.device)
+    si, so = _in_struct(s, t, proposal, mask, eps, temperature, seed, row_offset), _out_struct(out)
+    _raise(lib, lib.saki_route_fwd(C.byref(si), C.byref(so), _stream_ptr(stream)))
+    return out
+
+
+def route_fwd_bwd(s, t, proposal, eps, temperature=1.0, seed=0, row_offset=0, mask=None, grad_scale=1.0,
+                  out=None, dlogits=None, stream=None):
+    """saki_route_fwd_bwd on device tensors; returns (outputs dict, dlogits)."""
+    lib = load_library()
+    _check_rows(s, t)
+    out = out if out is not None else _alloc_out(s.shape[0], s.device)
+    if dlogits is None:
+        dlogits = torch.empty_like(s)
+    ld_g = dlogits.stride(0) if dlogits.shape[0] > 1 else dlogits.shape[1]
+    si, so = _in_struct(s, t, proposal, mask, eps, temperature, seed, row_offset), _out_struct(out)
+    _raise(lib, lib.saki_route_fwd_bwd(C.byref(si), C.byref(so), dlogits.data_ptr(), ld_g, grad_scale,
+                                       _stream_ptr(stream)))
+    return out, dlogits
+
+
+def route_host(s, t, proposal, eps, temperature=1.0, seed=0, row_offset=0, mask=None, grad_scale=1.0,
+               backward=True, out=None, dlogits=None):
+    """saki_route_host: every tensor lives in HOST memory (pinned for full copy speed); the library
+    stages the rows through the GPU and returns when the host outputs are complete."""
+    lib = load_library()
+    _check_rows(s, t)
+    if s.is_cuda:
+        raise SakiError(1, "route_host takes host tensors")
+    out = out if out is not None else _alloc_out(s.shape[0], "cpu", pinned=True)
+    if backward and dlogits is None:
+        dlogits = torch.empty(s.shape, dtype=s.dtype, pin_memory=True)
+    ld_g = (dlogits.stride(0) if dlogits.shape[0] > 1 else dlogits.shape[1]) if backward else 0
+    si, so = _in_struct(s, t, proposal, mask, eps, temperature, seed, row_offset), _out_struct(out)
+    _raise(lib, lib.saki_route_host(C.byref(si), C.byref(so), dlogits.data_ptr() if backward else None, ld_g,
+                                    grad_scale))
+    return out, dlogits
+
+
+def spec_verify(s, t, draft, eps, temperature=1.0, seed=0, seq_offset=0, stream=None):
+    """saki_spec_verify on device tensors s, t: [B,K+1,V], draft: [B,K] int32."""
+    lib = load_library()
+    if s.dim() != 3 or t.shape != s.shape or t.dtype != s.dtype or s.stride(2) != 1 or t.stride(2) != 1:
+        raise SakiError(1, "logits must be [B,K+1,V] with unit stride along V")
+    B, K1, V = s.shape
+    per = _alloc_out(B * K1, s.device)
+    res = {"n_accept": torch.empty(B, dtype=torch.int32, device=s.device),
+           "next_token": torch.empty(B, dtype=torch.int32, device=s.device),
+           "next_is_correction": torch.empty(B, dtype=torch.uint8, device=s.device), "per_pos": per}
+    si = SakiSpecIn()
+    si.student_logits, si.teacher_logits = s.data_ptr(), t.data_ptr()
+    si.ss_seq, si.ss_pos, si.ts_seq, si.ts_pos = s.stride(0), s.stride(1), t.stride(0), t.stride(1)
+    si.B, si.K, si.V, si.dtype = B, K1 - 1, V, _dtype_code(s)
+    si.draft, si.draft_ld = draft.data_ptr(), (draft.stride(0) if B > 1 else draft.shape[1])
+    si.eps, si.temperature, si.seed, si.seq_offset = eps, temperature, seed, seq_offset
+    so = SakiSpecOut()
+    so.n_accept, so.next_token, so.next_is_correction = (res["n_accept"].data_ptr(), res["next_token"].data_ptr(),
+                                                        res["next_is_correction"].data_ptr())
+    so.per_pos = _out_struct(per)
+    _raise(lib, lib.saki_spec_verify(C.byref(si), C.byref(so), _stream_ptr(stream)))
+    return res
+
+
+def sample_proposal(s, temperature=1.0, seed=0, row_offset=0, stream=None):
+    """saki_sample_proposal: x_i ~ softmax(s_i / temperature) by Philox-keyed Gumbel-max."""
+    lib = load_library()
+    out = torch.empty(s.shape[0], dtype=torch.int32, device=s.device)
+    ld = s.stride(0) if s.shape[0] > 1 else s.shape[1]
+    _raise(lib, lib.saki_sample_proposal(s.data_ptr(), ld, s.shape[0], s.shape[1], _dtype_code(s), temperature,
+                                         seed, row_offset, out.data_ptr(), _stream_ptr(stream)))
+    return out
+
+
+def check(stream=None) -> int:
+    """saki_check: synchronises the stream and returns the number of rows flagged since the last check."""
+    lib = load_library()
+    n = C.c_uint64(0)
+    rc = lib.saki_check(_stream_ptr(stream), C.byref(n))
+    if rc not in (0, 4):
+        _raise(lib, rc)
+    return int(n.value)
+
+
+def set_kernel(which: int) -> int:
+    return load_library().saki_set_kernel(which)
+
+
+def launch_count() -> int:
+    return int(load_library().saki_launch_count())
+
+
+def last_error() -> str:
+    return load_library().saki_last_error().decode()
+
+
+def version() -> int:
+    return load_library().saki_version()

@@ -1,0 +1,394 @@
+// C ABI of the SAKI routing library: host-side validation, kernel selection,
+// the proposal-sampling utility, the block-verification resolve and the
+// host-buffer convenience entry.  See include/saki.h for the contract.
+#include "saki_common.cuh"
+#include <atomic>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <vector>
+#include <algorithm>
+
+namespace saki {
+
+static thread_local char g_err[512] = "";
+static std::atomic<uint64_t> g_launches{0};
+static std::atomic<int> g_kernel{0};
+
+static int fail(int code, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+  return code;
+}
+static int cuda_fail(cudaError_t e, const char* what) {
+  return fail(SAKI_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+// device-resident count of flagged rows (one per device that loads the library)
+__device__ unsigned long long g_flagged_rows = 0ull;
+
+static int device_ready(unsigned long long** flagged) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return fail(SAKI_ERR_UNSUPPORTED, "no CUDA device: %s", cudaGetErrorString(e));
+  int major = 0;
+  e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+  if (major != 10) return fail(SAKI_ERR_UNSUPPORTED, "device compute capability %d.x: this library is built for sm_100a only", major);
+  e = cudaGetSymbolAddress((void**)flagged, g_flagged_rows);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress");
+  return SAKI_OK;
+}
+
+static int check_common(const void* s, const void* t, int64_t n, int32_t V, int32_t dtype, float eps, float tau) {
+  if (n < 0) return fail(SAKI_ERR_INVALID_ARG, "negative row count");
+  if (V < 2) return fail(SAKI_ERR_INVALID_ARG, "V must be >= 2 (got %d)", V);
+  if (dtype != SAKI_F32 && dtype != SAKI_BF16) return fail(SAKI_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+  if (!(eps >= 0.f)) return fail(SAKI_ERR_INVALID_ARG, "eps must be >= 0 and not NaN");
+  if (!(tau > 0.f) || std::isinf(tau)) return fail(SAKI_ERR_INVALID_ARG, "temperature must be finite and > 0");
+  if (n > 0 && (!s || !t)) return fail(SAKI_ERR_INVALID_ARG, "NULL logits pointer");
+  return SAKI_OK;
+}
+
+static int dispatch_rows(const RowParams& p, int dtype, cudaStream_t st) {
+  int launches = 0;
+  cudaError_t e;
+  bool served = false;
+  const int which = g_kernel.load();
+  if (which != 1 && cluster_can_serve(p, dtype)) {
+    e = launch_cluster(p, st, &launches, &served);
+    if (e != cudaSuccess) return cuda_fail(e, "cluster kernel launch");
+  }
+  if (!served) {
+    e = launch_general(p, dtype, st, &launches);
+    if (e != cudaSuccess) return cuda_fail(e, "general kernel launch");
+  }
+  g_launches += (uint64_t)launches;
+  return SAKI_OK;
+}
+
+static int route_impl(const saki_in* in, const saki_out* out, void* dlogits, int64_t ld_g, float grad_scale,
+                      bool bwd, void* stream) {
+  g_err[0] = 0;
+  if (!in || !out) return fail(SAKI_ERR_INVALID_ARG, "NULL argument struct");
+  int rc = check_common(in->student_logits, in->teacher_logits, in->N, in->V, in->dtype, in->eps, in->temperature);
+  if (rc) return rc;
+  if (in->ld_s < in->V || in->ld_t < in->V) return fail(SAKI_ERR_INVALID_ARG, "row stride smaller than V");
+  if (in->N > 0 && !in->proposal) return fail(SAKI_ERR_INVALID_ARG, "NULL proposal pointer");
+  if (in->N > 0 && (!out->corrected || !out->token)) return fail(SAKI_ERR_INVALID_ARG, "out.corrected and out.token are required");
+  if (bwd) {
+    if (in->N > 0 && !dlogits) return fail(SAKI_ERR_INVALID_ARG, "NULL dlogits pointer");
+    if (ld_g < in->V) return fail(SAKI_ERR_INVALID_ARG, "gradient row stride smaller than V");
+    if (!std::isfinite(grad_scale)) return fail(SAKI_ERR_INVALID_ARG, "grad_scale must be finite");
+  }
+  if (in->N == 0) return SAKI_OK;
+  unsigned long long* flagged = nullptr;
+  rc = device_ready(&flagged);
+  if (rc) return rc;
+  RowParams p;
+  memset(&p, 0, sizeof(p));
+  p.s = in->student_logits; p.t = in->teacher_logits;
+  p.s_seq = in->ld_s; p.s_pos = 0; p.t_seq = in->ld_t; p.t_pos = 0;
+  p.n_rows = in->N; p.V = in->V; p.K1 = 1; p.spec = 0;
+  p.proposal = in->proposal; p.prop_ld = 0; p.mask = in->mask;
+  p.eps = in->eps; p.temperature = in->temperature; p.seed = in->seed; p.row_offset = in->row_offset;
+  p.out = *out;
+  p.dlogits = bwd ? dlogits : nullptr; p.ld_g = ld_g; p.grad_scale = grad_scale;
+  p.flagged = flagged;
+  return dispatch_rows(p, in->dtype, (cudaStream_t)stream);
+}
+
+// ---- block verification: per-sequence first-rejection resolve (Section 3.5) ----
+__global__ void spec_resolve_kernel(int64_t B, int K, saki_out o, int32_t* n_accept, int32_t* next_token,
+                                    uint8_t* next_is_corr) {
+  const int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  const int K1 = K + 1;
+  int n = K, stopped = 0, next = -1, isc = 0;
+  for (int j = 0; j < K; ++j) {
+    const int64_t r = b * K1 + j;
+    if (o.token[r] < 0) { n = j; stopped = 1; break; }            // flagged row: cannot verify further
+    if (o.corrected[r]) { n = j; stopped = 1; next = o.token[r]; isc = 1; break; }
+  }
+  if (!stopped) next = o.token[b * K1 + K];                        // bonus draw (or -1 if flagged)
+  n_accept[b] = n; next_token[b] = next; next_is_corr[b] = (uint8_t)isc;
+  if (stopped) {                                                   // later positions sit on an invalid prefix
+    const RowResult z = zero_row(SAKI_ROW_NOT_COMPUTED);
+    for (int j = n + 1; j < K1; ++j) write_row(o, b * K1 + j, z, false);
+  }
+}
+
+// ---- proposal utility: Gumbel-max with per-element Philox noise ----
+template <typename T>
+__global__ void __launch_bounds__(256) proposal_kernel(const T* logits, int64_t ld, int64_t N, int V, double tau,
+                                                        uint64_t seed, uint64_t row_offset, int32_t* out) {
+  __shared__ double skey[8];
+  __shared__ int sidx[8];
+  for (int64_t row = blockIdx.x; row < N; row += gridDim.x) {
+    const T* s = logits + row * ld;
+    const uint64_t rid = row_offset + (uint64_t)row;
+    double best = -INFINITY;
+    int bi = 0x7fffffff;
+    for (int blk = threadIdx.x; blk * 4 < V; blk += blockDim.x) {
+      uint32_t w[4];
+      philox4x32_10((uint32_t)rid, (uint32_t)(rid >> 32), STAGE_PROPOSE, (uint32_t)blk, (uint32_t)seed,
+                    (uint32_t)(seed >> 32), w);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int v = blk * 4 + k;
+        if (v < V) {
+          const double u = ((double)w[k] + 0.5) * (1.0 / 4294967296.0);
+          const double key = (double)ld_as_float(s, v) / tau - log(-log(u));
+          if (key > best) { best = key; bi = v; }
+        }
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const double ob = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (ob > best || (ob == best && oi < bi)) { best = ob; bi = oi; }
+    }
+    if ((threadIdx.x & 31) == 0) { skey[threadIdx.x >> 5] = best; sidx[threadIdx.x >> 5] = bi; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      for (int w = 1; w < 8; ++w)
+        if (skey[w] > best || (skey[w] == best && sidx[w] < bi)) { best = skey[w]; bi = sidx[w]; }
+      out[row] = bi;
+    }
+    __syncthreads();
+  }
+}
+
+// ---- host-buffer entry: staged, double-buffered ----
+struct HostStage {
+  std::mutex mu;
+  int dev = -1;
+  cudaStream_t st[2] = {nullptr, nullptr};
+  void* buf[2] = {nullptr, nullptr};
+  size_t cap[2] = {0, 0};
+};
+static HostStage g_stage;
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace saki
+
+using namespace saki;
+
+extern "C" {
+
+SAKI_API int saki_route_fwd(const saki_in* in, const saki_out* out, void* cuda_stream) {
+  return route_impl(in, out, nullptr, 0, 0.f, false, cuda_stream);
+}
+
+SAKI_API int saki_route_fwd_bwd(const saki_in* in, const saki_out* out, void* dlogits, int64_t ld_g, float grad_scale,
+                       void* cuda_stream) {
+  return route_impl(in, out, dlogits, ld_g, grad_scale, true, cuda_stream);
+}
+
+SAKI_API int saki_spec_verify(const saki_spec_in* in, const saki_spec_out* out, void* cuda_stream) {
+  g_err[0] = 0;
+  if (!in || !out) return fail(SAKI_ERR_INVALID_ARG, "NULL argument struct");
+  int rc = check_common(in->student_logits, in->teacher_logits, in->B, in->V, in->dtype, in->eps, in->temperature);
+  if (rc) return rc;
+  if (in->K < 1 || in->K > 16) return fail(SAKI_ERR_INVALID_ARG, "K must be in [1,16] (got %d)", in->K);
+  if (in->ss_pos < in->V || in->ts_pos < in->V) return fail(SAKI_ERR_INVALID_ARG, "position stride smaller than V");
+  if (in->ss_seq < in->ss_pos || in->ts_seq < in->ts_pos) return fail(SAKI_ERR_INVALID_ARG, "sequence stride smaller than position stride");
+  if (in->B > 0 && (!in->draft || in->draft_ld < in->K)) return fail(SAKI_ERR_INVALID_ARG, "bad draft pointer or stride");
+  if (in->B > 0 && (!out->n_accept || !out->next_token || !out->next_is_correction || !out->per_pos.corrected ||
+                    !out->per_pos.token))
+    return fail(SAKI_ERR_INVALID_ARG, "n_accept, next_token, next_is_correction, per_pos.corrected and per_pos.token are required");
+  if (in->B == 0) return SAKI_OK;
+  unsigned long long* flagged = nullptr;
+  rc = device_ready(&flagged);
+  if (rc) return rc;
+  RowParams p;
+  memset(&p, 0, sizeof(p));
+  p.s = in->student_logits; p.t = in->teacher_logits;
+  p.s_seq = in->ss_seq; p.s_pos = in->ss_pos; p.t_seq = in->ts_seq; p.t_pos = in->ts_pos;
+  p.K1 = in->K + 1; p.n_rows = in->B * p.K1; p.V = in->V; p.spec = 1;
+  p.proposal = in->draft; p.prop_ld = in->draft_ld; p.mask = nullptr;
+  p.eps = in->eps; p.temperature = in->temperature; p.seed = in->seed;
+  p.row_offset = in->seq_offset * (uint64_t)p.K1;
+  p.out = out->per_pos;
+  p.out.loss = nullptr;
+  p.dlogits = nullptr; p.ld_g = 0; p.grad_scale = 0.f; p.flagged = flagged;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  rc = dispatch_rows(p, in->dtype, st);
+  if (rc) return rc;
+  const int th = 128;
+  spec_resolve_kernel<<<(unsigned)((in->B + th - 1) / th), th, 0, st>>>(in->B, in->K, p.out, out->n_accept,
+                                                                        out->next_token, out->next_is_correction);
+  g_launches += 1;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, "resolve kernel launch");
+  return SAKI_OK;
+}
+
+SAKI_API int saki_sample_proposal(const void* logits, int64_t ld, int64_t N, int32_t V, int32_t dtype, float temperature,
+                         uint64_t seed, uint64_t row_offset, int32_t* out, void* cuda_stream) {
+  g_err[0] = 0;
+  int rc = check_common(logits, logits, N, V, dtype, 0.f, temperature);
+  if (rc) return rc;
+  if (ld < V) return fail(SAKI_ERR_INVALID_ARG, "row stride smaller than V");
+  if (N > 0 && !out) return fail(SAKI_ERR_INVALID_ARG, "NULL output pointer");
+  if (N == 0) return SAKI_OK;
+  unsigned long long* flagged = nullptr;
+  rc = device_ready(&flagged);
+  if (rc) return rc;
+  const int grid = (int)std::min<int64_t>(N, 148 * 8);
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (dtype == SAKI_BF16)
+    proposal_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)logits, ld, N, V, (double)temperature,
+                                                         seed, row_offset, out);
+  else
+    proposal_kernel<float><<<grid, 256, 0, st>>>((const float*)logits, ld, N, V, (double)temperature, seed,
+                                                 row_offset, out);
+  g_launches += 1;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, "proposal kernel launch");
+  return SAKI_OK;
+}
+
+SAKI_API int saki_check(void* cuda_stream, uint64_t* n_flagged) {
+  g_err[0] = 0;
+  unsigned long long* flagged = nullptr;
+  int rc = device_ready(&flagged);
+  if (rc) return rc;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  cudaError_t e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+  unsigned long long h = 0, zero = 0;
+  e = cudaMemcpy(&h, flagged, sizeof(h), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy");
+  e = cudaMemcpy(flagged, &zero, sizeof(zero), cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy");
+  if (n_flagged) *n_flagged = h;
+  if (h) return fail(SAKI_ERR_ROW_STATUS, "%llu row(s) flagged (non-finite logits, bad proposal id or timeout)", h);
+  return SAKI_OK;
+}
+
+SAKI_API int saki_route_host(const saki_in* in, const saki_out* out, void* dlogits, int64_t ld_g, float grad_scale) {
+  g_err[0] = 0;
+  if (!in || !out) return fail(SAKI_ERR_INVALID_ARG, "NULL argument struct");
+  int rc = check_common(in->student_logits, in->teacher_logits, in->N, in->V, in->dtype, in->eps, in->temperature);
+  if (rc) return rc;
+  if (in->ld_s < in->V || in->ld_t < in->V) return fail(SAKI_ERR_INVALID_ARG, "row stride smaller than V");
+  if (dlogits && ld_g < in->V) return fail(SAKI_ERR_INVALID_ARG, "gradient row stride smaller than V");
+  if (in->N > 0 && (!in->proposal || !out->corrected || !out->token))
+    return fail(SAKI_ERR_INVALID_ARG, "proposal, out.corrected and out.token are required");
+  if (in->N == 0) return SAKI_OK;
+  unsigned long long* flagged = nullptr;
+  rc = device_ready(&flagged);
+  if (rc) return rc;
+
+  std::lock_guard<std::mutex> lock(g_stage.mu);
+  int dev = 0;
+  cudaGetDevice(&dev);
+  cudaError_t e;
+  if (g_stage.dev != dev) {   // (re)create the staging streams on this device
+    for (int k = 0; k < 2; ++k) {
+      if (g_stage.buf[k]) { cudaFree(g_stage.buf[k]); g_stage.buf[k] = nullptr; g_stage.cap[k] = 0; }
+      if (g_stage.st[k]) { cudaStreamDestroy(g_stage.st[k]); g_stage.st[k] = nullptr; }
+      e = cudaStreamCreateWithFlags(&g_stage.st[k], cudaStreamNonBlocking);
+      if (e != cudaSuccess) return cuda_fail(e, "cudaStreamCreate");
+    }
+    g_stage.dev = dev;
+  }
+  const size_t es = in->dtype == SAKI_BF16 ? 2 : 4;
+  const size_t Vp = align_up((size_t)in->V, 16);   // padded device row stride: rows stay 16-byte aligned
+  // rows per chunk: about 192 MB of logits per buffer
+  int64_t chunk = (int64_t)std::max<size_t>(1, (size_t)192 << 20) / (int64_t)(2 * Vp * es);
+  chunk = std::max<int64_t>(1, std::min<int64_t>(chunk, in->N));
+  const size_t row_bytes = Vp * es;
+  // device layout of one chunk
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  const size_t o_s = take(chunk * row_bytes), o_t = take(chunk * row_bytes);
+  const size_t o_g = dlogits ? take(chunk * row_bytes) : 0;
+  const size_t o_prop = take(chunk * 4), o_mask = take(chunk);
+  const size_t o_corr = take(chunk), o_tok = take(chunk * 4), o_top = take(chunk * 4), o_stat = take(chunk * 4);
+  size_t o_f[10];
+  for (int k = 0; k < 10; ++k) o_f[k] = take(chunk * 4);
+  const size_t total = off;
+  for (int k = 0; k < 2; ++k) {
+    if (g_stage.cap[k] < total) {
+      if (g_stage.buf[k]) cudaFree(g_stage.buf[k]);
+      g_stage.buf[k] = nullptr; g_stage.cap[k] = 0;
+      e = cudaMalloc(&g_stage.buf[k], total);
+      if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc (staging)");
+      g_stage.cap[k] = total;
+    }
+  }
+  float* const host_f[10] = {out->lambda, out->kl, out->tv, out->accept_prob, out->logp_x,
+                             out->logq_x, out->logT_x, out->logp_y, out->logq_y, out->loss};
+  int result = SAKI_OK;
+  int k = 0;
+  for (int64_t r0 = 0; r0 < in->N && result == SAKI_OK; r0 += chunk, k ^= 1) {
+    const int64_t n = std::min<int64_t>(chunk, in->N - r0);
+    char* base = (char*)g_stage.buf[k];
+    cudaStream_t st = g_stage.st[k];
+    const char* hs = (const char*)in->student_logits + (size_t)r0 * in->ld_s * es;
+    const char* ht = (const char*)in->teacher_logits + (size_t)r0 * in->ld_t * es;
+    e = cudaMemcpy2DAsync(base + o_s, row_bytes, hs, in->ld_s * es, in->V * es, n, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess)
+      e = cudaMemcpy2DAsync(base + o_t, row_bytes, ht, in->ld_t * es, in->V * es, n, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess)
+      e = cudaMemcpyAsync(base + o_prop, in->proposal + r0, n * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && in->mask) e = cudaMemcpyAsync(base + o_mask, in->mask + r0, n, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) { result = cuda_fail(e, "host-to-device copy"); break; }
+    saki_in din = *in;
+    din.student_logits = base + o_s; din.teacher_logits = base + o_t; din.ld_s = din.ld_t = (int64_t)Vp;
+    din.N = n; din.proposal = (const int32_t*)(base + o_prop);
+    din.mask = in->mask ? (const uint8_t*)(base + o_mask) : nullptr;
+    din.row_offset = in->row_offset + (uint64_t)r0;
+    saki_out dout;
+    dout.corrected = (uint8_t*)(base + o_corr); dout.token = (int32_t*)(base + o_tok);
+    dout.teacher_top1 = (int32_t*)(base + o_top); dout.row_status = (uint32_t*)(base + o_stat);
+    float** df[10] = {&dout.lambda, &dout.kl, &dout.tv, &dout.accept_prob, &dout.logp_x,
+                      &dout.logq_x, &dout.logT_x, &dout.logp_y, &dout.logq_y, &dout.loss};
+    for (int q = 0; q < 10; ++q) *df[q] = (float*)(base + o_f[q]);
+    result = route_impl(&din, &dout, dlogits ? base + o_g : nullptr, (int64_t)Vp, grad_scale, dlogits != nullptr, st);
+    if (result != SAKI_OK) break;
+    e = cudaMemcpyAsync(out->corrected + r0, dout.corrected, n, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(out->token + r0, dout.token, n * 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess && out->teacher_top1)
+      e = cudaMemcpyAsync(out->teacher_top1 + r0, dout.teacher_top1, n * 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess && out->row_status)
+      e = cudaMemcpyAsync(out->row_status + r0, dout.row_status, n * 4, cudaMemcpyDeviceToHost, st);
+    for (int q = 0; q < 10 && e == cudaSuccess; ++q)
+      if (host_f[q]) e = cudaMemcpyAsync(host_f[q] + r0, *df[q], n * 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess && dlogits)
+      e = cudaMemcpy2DAsync((char*)dlogits + (size_t)r0 * ld_g * es, ld_g * es, base + o_g, row_bytes, in->V * es, n,
+                            cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) { result = cuda_fail(e, "device-to-host copy"); break; }
+    // the other buffer is reused two chunks later: its stream must have drained by then
+    if (r0 + chunk < in->N) {
+      e = cudaStreamSynchronize(g_stage.st[k ^ 1]);
+      if (e != cudaSuccess) { result = cuda_fail(e, "cudaStreamSynchronize"); break; }
+    }
+  }
+  for (int q = 0; q < 2; ++q) {
+    e = cudaStreamSynchronize(g_stage.st[q]);
+    if (e != cudaSuccess && result == SAKI_OK) result = cuda_fail(e, "cudaStreamSynchronize");
+  }
+  return result;
+}
+
+SAKI_API int saki_set_kernel(int which) {
+  if (which < 0 || which > 2) which = 0;
+  return g_kernel.exchange(which);
+}
+
+SAKI_API uint64_t saki_launch_count(void) { return g_launches.load(); }
+
+SAKI_API const char* saki_last_error(void) { return g_err; }
+
+SAKI_API int saki_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,110 @@
+// Shared declarations of the SAKI routing library (device + host side).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "../../include/saki.h"
+
+namespace saki {
+
+enum { STAGE_PROPOSE = 0, STAGE_ACCEPT = 1, STAGE_RESIDUAL = 2, STAGE_BONUS = 3 };
+
+// Everything a row kernel needs; passed by value as the kernel parameter.
+// Plain routing and block verification share it: row i is position
+// j = i % K1 of sequence b = i / K1 (K1 = 1 for plain routing).
+struct RowParams {
+  const void* s;
+  const void* t;
+  int64_t s_seq, s_pos, t_seq, t_pos;  // element strides (plain: s_seq = ld_s, s_pos = 0)
+  int64_t n_rows;
+  int32_t V;
+  int32_t K1;                          // positions per sequence; the last one is the bonus row if spec
+  int32_t spec;                        // 1: block verification (proposal from draft, bonus row)
+  const int32_t* proposal;             // plain: [N]; spec: draft [B,K] with row stride prop_ld
+  int64_t prop_ld;
+  const uint8_t* mask;
+  float eps;
+  float temperature;
+  uint64_t seed;
+  uint64_t row_offset;
+  saki_out out;
+  void* dlogits;                       // NULL: forward only
+  int64_t ld_g;
+  float grad_scale;
+  unsigned long long* flagged;         // device counter of flagged rows
+};
+
+// ---- Philox4x32-10 (Salmon et al., SC'11), written from the published round function ----
+__host__ __device__ inline void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                              uint32_t k0, uint32_t k1, uint32_t out[4]) {
+  const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    uint64_t p0 = (uint64_t)M0 * c0;
+    uint64_t p1 = (uint64_t)M1 * c2;
+    uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+    uint32_t n1 = (uint32_t)p1;
+    uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+    uint32_t n3 = (uint32_t)p0;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    k0 += W0; k1 += W1;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// the one uniform a (row, stage) pair owns: an odd multiple of 2^-24 in (0,1)
+__host__ __device__ inline double scalar_uniform(uint64_t seed, uint64_t row, uint32_t stage) {
+  uint32_t w[4];
+  philox4x32_10((uint32_t)row, (uint32_t)(row >> 32), stage, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), w);
+  return ((double)(w[0] >> 9) + 0.5) * (1.0 / 8388608.0);
+}
+
+template <typename T> __device__ __forceinline__ float ld_as_float(const T* p, int64_t i);
+template <> __device__ __forceinline__ float ld_as_float<float>(const float* p, int64_t i) { return p[i]; }
+template <> __device__ __forceinline__ float ld_as_float<__nv_bfloat16>(const __nv_bfloat16* p, int64_t i) {
+  return __bfloat162float(p[i]);
+}
+template <typename T> __device__ __forceinline__ void st_from_float(T* p, int64_t i, float v);
+template <> __device__ __forceinline__ void st_from_float<float>(float* p, int64_t i, float v) { p[i] = v; }
+template <> __device__ __forceinline__ void st_from_float<__nv_bfloat16>(__nv_bfloat16* p, int64_t i, float v) {
+  p[i] = __float2bfloat16_rn(v);
+}
+
+// Per-row scalar results, written by one thread.
+struct RowResult {
+  int corrected, token, vstar;
+  float lambda, kl, tv, accept, logp_x, logq_x, logT_x, logp_y, logq_y, loss;
+  uint32_t status;
+};
+
+__device__ inline void write_row(const saki_out& o, int64_t i, const RowResult& r, bool write_loss) {
+  o.corrected[i] = (uint8_t)r.corrected;
+  o.token[i] = r.token;
+  if (o.teacher_top1) o.teacher_top1[i] = r.vstar;
+  if (o.lambda) o.lambda[i] = r.lambda;
+  if (o.kl) o.kl[i] = r.kl;
+  if (o.tv) o.tv[i] = r.tv;
+  if (o.accept_prob) o.accept_prob[i] = r.accept;
+  if (o.logp_x) o.logp_x[i] = r.logp_x;
+  if (o.logq_x) o.logq_x[i] = r.logq_x;
+  if (o.logT_x) o.logT_x[i] = r.logT_x;
+  if (o.logp_y) o.logp_y[i] = r.logp_y;
+  if (o.logq_y) o.logq_y[i] = r.logq_y;
+  if (o.loss && write_loss) o.loss[i] = r.loss;
+  if (o.row_status) o.row_status[i] = r.status;
+}
+
+__device__ inline RowResult zero_row(uint32_t status) {
+  RowResult r;
+  r.corrected = 0; r.token = -1; r.vstar = -1;
+  r.lambda = r.kl = r.tv = r.accept = r.logp_x = r.logq_x = r.logT_x = r.logp_y = r.logq_y = r.loss = 0.f;
+  r.status = status;
+  return r;
+}
+
+// host-side launchers (defined in the kernel translation units)
+cudaError_t launch_general(const RowParams& p, int dtype, cudaStream_t st, int* n_launches);
+cudaError_t launch_cluster(const RowParams& p, cudaStream_t st, int* n_launches, bool* served);
+bool cluster_can_serve(const RowParams& p, int dtype);
+
+}  // namespace saki

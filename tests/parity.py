@@ -1,0 +1,98 @@
+"""Element-by-element comparison of the CUDA path with the float64 oracle.
+
+Tolerances (written here so that the tests state them):
+  flags and ids       bit-exact, except rows whose oracle decision margin is
+                      below 1e-6 (|u - accept_prob| for the acceptance test;
+                      distance of the inverse-CDF target from the nearer cell
+                      edge as a fraction of the total for the draws), which are
+                      counted and returned
+  lambda, TV          |delta| <= 1e-5
+  other fp32 scalars  |delta| <= 1e-5 (kl, accept_prob) or 1e-5 (1+|ref|) (log-probs)
+  loss                |delta| <= 1e-4 |ref| + 2e-6
+  gradient, fp32      |delta| <= 1e-5 max(1, max|g_row|) ... see grad_check
+  gradient, bf16      |delta| <= 2e-3 where |g_ref| < 1; elsewhere within one
+                      bf16 ulp of the oracle's rounded value; and relative
+                      error <= 2^-7 on entries with |g_ref| >= 1e-30 (small
+                      entries must not be flushed to zero)
+"""
+import math
+
+import numpy as np
+import torch
+
+import oracle as O
+
+MARGIN = 1e-6
+
+
+def to_np64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to("cpu").to(torch.float64).numpy()
+
+
+def bf16_ulp(x):
+    x = np.abs(np.asarray(x, dtype=np.float64))
+    _, e = np.frexp(np.maximum(x, 2.0 ** -126))
+    return np.ldexp(1.0, (e - 1) - 7)
+
+
+def grad_check(g_gpu: np.ndarray, g_ref: np.ndarray, dtype: str):
+    """g_ref is the oracle gradient already rounded to the output dtype."""
+    d = np.abs(g_gpu - g_ref)
+    if dtype == "f32":
+        tol = 1e-6 + 2e-6 * np.abs(g_ref)
+        assert np.all(d <= tol), f"fp32 gradient error {d.max():.3e}"
+        return dict(max_abs=float(d.max()), n_ulp=0)
+    small = np.abs(g_ref) < 1.0
+    assert np.all(d[small] <= 2e-3), f"bf16 gradient max-abs error {d[small].max():.3e}"
+    big_ok = d[~small] <= bf16_ulp(g_ref[~small]) * 1.0000001
+    assert np.all(big_ok), "bf16 gradient entry with |g|>=1 off by more than one ulp"
+    nz = np.abs(g_ref) >= 1e-30
+    rel = d[nz] / np.abs(g_ref[nz])
+    assert np.all(rel <= 2.0 ** -7 * 1.0000001), f"bf16 gradient relative error {rel.max():.3e}"
+    return dict(max_abs=float(d[small].max()) if small.any() else 0.0,
+                n_ulp=int(np.count_nonzero(g_gpu != g_ref)))
+
+
+def compare_rows(gpu: dict, ref: dict, rows=None, check_loss=True):
+    """gpu: dict of torch tensors (all rows); ref: oracle dict over `rows`.
+    Returns the number of margin-exempt rows."""
+    n_total = len(gpu["token"])
+    rows = np.arange(n_total) if rows is None else np.asarray(list(rows))
+    g = {k: v.detach().cpu().numpy()[rows] for k, v in gpu.items() if isinstance(v, torch.Tensor)}
+    exempt = (np.minimum(ref["margin_accept"], ref["margin_draw"]) < MARGIN)
+    ok = ~exempt
+    assert np.array_equal(g["teacher_top1"], ref["teacher_top1"]), "teacher argmax differs"
+    assert np.array_equal(g["row_status"].astype(np.uint32), ref["status"]), \
+        f"row status differs: {g['row_status'][:8]} vs {ref['status'][:8]}"
+    assert np.array_equal(g["corrected"][ok], ref["corrected"][ok]), "accept/correct flags differ"
+    assert np.array_equal(g["token"][ok], ref["token"][ok]), \
+        f"committed tokens differ at rows {rows[ok][g['token'][ok] != ref['token'][ok]][:5]}"
+    for name, key, tol in (("lambda", "lam", 1e-5), ("tv", "tv", 1e-5), ("kl", "kl", 1e-5),
+                           ("accept_prob", "accept_prob", 1e-5)):
+        d = np.abs(g[name].astype(np.float64) - ref[key])
+        assert np.all(d <= tol), f"{name}: max error {d.max():.3e}"
+    same = ok & (g["corrected"] == ref["corrected"]) & (g["token"] == ref["token"])
+    for name in ("logp_x", "logq_x", "logT_x", "logp_y", "logq_y"):
+        d = np.abs(g[name].astype(np.float64) - ref[name])[same]
+        assert np.all(d <= 1e-5 * (1 + np.abs(ref[name][same]))), f"{name}: max error {d.max():.3e}"
+    if check_loss:
+        d = np.abs(g["loss"].astype(np.float64) - ref["loss"])[same]
+        assert np.all(d <= 1e-4 * np.abs(ref["loss"][same]) + 2e-6), f"loss: max error {d.max():.3e}"
+    return int(exempt.sum())
+
+
+def max_errors(gpu: dict, ref: dict, rows=None):
+    n_total = len(gpu["token"])
+    rows = np.arange(n_total) if rows is None else np.asarray(list(rows))
+    g = {k: v.detach().cpu().numpy()[rows] for k, v in gpu.items() if isinstance(v, torch.Tensor)}
+    return {name: float(np.abs(g[name].astype(np.float64) - ref[key]).max())
+            for name, key in (("lambda", "lam"), ("tv", "tv"), ("kl", "kl"), ("accept_prob", "accept_prob"))}
+
+
+def oracle_inputs(d: dict, rows=None):
+    """The identical bytes the GPU sees, widened exactly to float64 on the host."""
+    s, t = d["s"], d["t"]
+    if rows is not None:
+        idx = torch.as_tensor(list(rows), device=s.device)
+        s, t = s[idx], t[idx]
+    return to_np64(s), to_np64(t)

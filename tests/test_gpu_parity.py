@@ -1,0 +1,183 @@
+"""Parity of the CUDA path (through the C ABI) with the float64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+import paper_2609_36601_b200 as P
+from paper_2609_36601_b200 import synth
+from parity import compare_rows, grad_check, oracle_inputs, to_np64
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+KERNELS = {"general": 1, "auto": 0}
+
+
+@pytest.fixture(params=list(KERNELS))
+def kernel(request):
+    prev = P.set_kernel(KERNELS[request.param])
+    yield request.param
+    P.set_kernel(prev)
+
+
+def _route_oracle(d, w, rows=None, mask=None, want_grad=True, row_offset=0, grad_scale=1.0, eps=None):
+    s64, t64 = oracle_inputs(d)
+    x = d["proposal"].cpu().numpy()
+    return O.route(s64, t64, x, w.eps if eps is None else eps, w.temperature, w.seed, row_offset, mask=mask,
+                   grad_scale=grad_scale, want_grad=want_grad, grad_dtype=w.dtype, rows=rows)
+
+
+def _check_fwd_bwd(d, w, rows=None, mask=None, row_offset=0, grad_scale=1.0, eps=None):
+    e = w.eps if eps is None else eps
+    m = None if mask is None else torch.as_tensor(mask, dtype=torch.uint8, device=DEV)
+    out_f = P.route_fwd(d["s"], d["t"], d["proposal"], e, w.temperature, w.seed, row_offset, mask=m)
+    out, g = P.route_fwd_bwd(d["s"], d["t"], d["proposal"], e, w.temperature, w.seed, row_offset, mask=m,
+                             grad_scale=grad_scale)
+    torch.cuda.synchronize()
+    for k in out:   # forward-only and forward+backward agree bit for bit
+        assert torch.equal(out[k], out_f[k]), k
+    ref = _route_oracle(d, w, rows, mask, True, row_offset, grad_scale, eps)
+    n_exempt = compare_rows(out, ref, rows)
+    rr = np.arange(len(d["proposal"])) if rows is None else np.asarray(list(rows))
+    gg = to_np64(g)[rr]
+    same = (out["corrected"].cpu().numpy()[rr] == ref["corrected"])
+    stats = grad_check(gg[same], ref["grad"][same], w.dtype)
+    return out, ref, n_exempt, stats
+
+
+def test_cfg1_tiny_fp32_all_rows(kernel):
+    w = synth.WORKLOADS["cfg1"]
+    d = synth.generate(w, DEV)
+    # the proposal utility agrees with the oracle's Gumbel-max (outside the margin)
+    x_gpu = P.sample_proposal(d["s"], w.temperature, w.seed).cpu().numpy()
+    x_ref, gaps = O.sample_proposal(to_np64(d["s"]), w.temperature, w.seed)
+    assert np.array_equal(x_gpu[gaps >= 1e-6], x_ref[gaps >= 1e-6])
+    d["proposal"] = torch.as_tensor(x_ref, device=DEV)
+    out, ref, n_exempt, stats = _check_fwd_bwd(d, w)
+    assert n_exempt <= 2
+    assert 0.15 < np.median(ref["tv"]) < 0.2237      # Pinsker cap sqrt(eps/2)
+
+
+@pytest.mark.parametrize("V,N,dtype", [(1000, 9, "bf16"), (4099, 5, "bf16"), (33, 7, "f32"), (2, 4, "f32"),
+                                        (20000, 3, "bf16")])
+def test_ragged_shapes(kernel, V, N, dtype):
+    w = synth.Workload("t", N, V, dtype, 0.1, 1.5, V > 100, 77, 9, temperature=0.9)
+    d = synth.generate(w, DEV)
+    _check_fwd_bwd(d, w, row_offset=(1 << 33) + 5, grad_scale=0.125)
+
+
+def test_strided_rows_and_mask(kernel):
+    w = synth.Workload("t", 12, 3000, "bf16", 0.05, 1.0, True, 78, 10)
+    d = synth.generate(w, DEV)
+    pad = torch.zeros((12, 3000 + 72), dtype=torch.bfloat16, device=DEV)
+    for k in ("s", "t"):
+        buf = pad.clone()
+        buf[:, :3000] = d[k]
+        d[k] = buf[:, :3000]            # row stride 3072
+    mask = np.array([1, 0] * 6, dtype=np.uint8)
+    out, ref, _, _ = _check_fwd_bwd(d, w, mask=mask)
+    assert np.all(out["loss"].cpu().numpy()[mask == 0] == 0)
+
+
+def test_eps_zero_and_saturation(kernel):
+    w = synth.Workload("t", 16, 2048, "bf16", 0.0, 0.5, True, 79, 11)
+    d = synth.generate(w, DEV)
+    out, ref, _, _ = _check_fwd_bwd(d, w, eps=0.0)
+    assert torch.all(out["corrected"] == 0) and torch.all(out["lambda"] == 0)
+    assert torch.all((out["row_status"] & 2) != 0)
+    out, ref, _, _ = _check_fwd_bwd(d, w, eps=5.0)
+    assert torch.all(out["lambda"] == 1) and torch.all((out["row_status"] & 1) != 0)
+    out, ref, _, _ = _check_fwd_bwd(d, w, eps=0.3)
+    sat = (ref["status"] & 1) != 0
+    assert 0 < sat.sum() < 16, "want a mix of saturated and interior rows"
+
+
+def test_flagged_rows(kernel):
+    w = synth.Workload("t", 6, 1500, "bf16", 0.1, 1.5, True, 80, 12)
+    d = synth.generate(w, DEV)
+    d["s"][1, 700] = float("nan")
+    d["t"][2, 3] = float("inf")
+    d["t"][3, 1499] = float("-inf")
+    d["proposal"][4] = 1500
+    d["proposal"][5] = -1
+    P.check()
+    out, ref, _, _ = _check_fwd_bwd(d, w)
+    st = out["row_status"].cpu().numpy()
+    assert list(st[1:]) == [8, 8, 8, 16, 16] and st[0] == 0
+    assert torch.all(out["token"][1:] == -1)
+    assert P.check() == 10          # 5 rows x (fwd + fwd_bwd)
+    assert P.check() == 0
+
+
+def test_empty_and_bad_arguments():
+    z = torch.zeros((0, 128), dtype=torch.bfloat16, device=DEV)
+    out, g = P.route_fwd_bwd(z, z, torch.zeros(0, dtype=torch.int32, device=DEV), 0.1)
+    assert g.shape == (0, 128)
+    s = torch.zeros((2, 128), dtype=torch.bfloat16, device=DEV)
+    x = torch.zeros(2, dtype=torch.int32, device=DEV)
+    for kw in (dict(eps=-1.0), dict(eps=float("nan")), dict(eps=0.1, temperature=0.0)):
+        with pytest.raises(P.SakiError) as ei:
+            P.route_fwd(s, s, x, **kw)
+        assert ei.value.code == 1
+    with pytest.raises(P.SakiError):
+        P.route_fwd(s[:, :1], s[:, :1], x, 0.1)     # V < 2
+
+
+def test_determinism_and_chunk_invariance(kernel):
+    w = synth.Workload("t", 40, 5000, "bf16", 0.1, 1.5, True, 81, 13)
+    d = synth.generate(w, DEV)
+    a, ga = P.route_fwd_bwd(d["s"], d["t"], d["proposal"], w.eps, seed=w.seed)
+    b, gb = P.route_fwd_bwd(d["s"], d["t"], d["proposal"], w.eps, seed=w.seed)
+    c, gc = P.route_fwd_bwd(d["s"][17:], d["t"][17:], d["proposal"][17:], w.eps, seed=w.seed, row_offset=17)
+    torch.cuda.synchronize()
+    for k in a:
+        assert torch.equal(a[k], b[k]) and torch.equal(a[k][17:], c[k]), k
+    assert torch.equal(ga, gb) and torch.equal(ga[17:], gc)
+
+
+def test_spec_verify_small(kernel):
+    B, K, V = 48, 4, 3000
+    w = synth.Workload("t", B * (K + 1), V, "bf16", 0.2, 1.5, True, 82, 14, K=K)
+    d = synth.generate(w, DEV)
+    s3, t3 = d["s"].view(B, K + 1, V), d["t"].view(B, K + 1, V)
+    draft = d["proposal"].view(B, K + 1)[:, :K].contiguous()
+    draft[5, 1] = V + 3                    # a bad id stops verification of that sequence
+    res = P.spec_verify(s3, t3, draft, w.eps, seed=w.seed, seq_offset=3)
+    torch.cuda.synchronize()
+    ref = O.spec_verify(to_np64(s3), to_np64(t3), draft.cpu().numpy(), w.eps, seed=w.seed, seq_offset=3)
+    ok = ref["margin"] >= 1e-6
+    assert np.array_equal(res["n_accept"].cpu().numpy()[ok], ref["n_accept"][ok])
+    assert np.array_equal(res["next_token"].cpu().numpy()[ok], ref["next_token"][ok])
+    assert np.array_equal(res["next_is_correction"].cpu().numpy()[ok], ref["next_is_correction"][ok])
+    assert len(set(ref["n_accept"])) >= 3
+    per = {k: v.cpu().numpy().reshape(B, K + 1) for k, v in res["per_pos"].items()}
+    for b in np.nonzero(ok)[0]:
+        for j in range(K + 1):
+            r = ref["per_pos"][b][j]
+            assert per["row_status"][b, j] == r["status"], (b, j)
+            assert per["token"][b, j] == r["token"] and per["corrected"][b, j] == r["corrected"]
+            for name, key in (("lambda", "lam"), ("tv", "tv"), ("kl", "kl"), ("accept_prob", "accept_prob")):
+                assert abs(per[name][b, j] - r[key]) <= 1e-5, (name, b, j)
+            for name in ("logp_y", "logq_y", "logp_x", "logq_x"):
+                assert abs(per[name][b, j] - r[name]) <= 1e-5 * (1 + abs(r[name])), (name, b, j)
+    assert ref["n_accept"][5] <= 1 and res["next_token"][5].item() == ref["next_token"][5]
+
+
+def test_proposal_utility_bf16():
+    w = synth.Workload("t", 64, 7001, "bf16", 0.1, 1.5, True, 83, 15, temperature=0.8)
+    d = synth.generate(w, DEV)
+    x_gpu = P.sample_proposal(d["s"], w.temperature, w.seed, row_offset=11).cpu().numpy()
+    x_ref, gaps = O.sample_proposal(to_np64(d["s"]), w.temperature, w.seed, row_offset=11)
+    assert np.array_equal(x_gpu[gaps >= 1e-6], x_ref[gaps >= 1e-6])
+
+
+def test_host_entry_matches_device_entry(kernel):
+    w = synth.Workload("t", 700, 2500, "bf16", 0.1, 1.5, True, 84, 16)
+    d = synth.generate(w, DEV)
+    out, g = P.route_fwd_bwd(d["s"], d["t"], d["proposal"], w.eps, seed=w.seed, grad_scale=0.5)
+    hs, ht = d["s"].cpu().pin_memory(), d["t"].cpu().pin_memory()
+    hout, hg = P.route_host(hs, ht, d["proposal"].cpu(), w.eps, seed=w.seed, grad_scale=0.5)
+    torch.cuda.synchronize()
+    for k in out:
+        assert torch.equal(out[k].cpu(), hout[k]), k
+    assert torch.equal(g.cpu(), hg)
