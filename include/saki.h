@@ -177,6 +177,10 @@ SAKI_API int saki_check(void* cuda_stream, uint64_t* n_flagged);
  * Process-wide; meant for tests and benchmarks.  Returns the previous value. */
 SAKI_API int saki_set_kernel(int which);
 
+/* Which row kernel the calling thread's last routing call used: 1 general, 2 cluster,
+ * 0 if none yet. */
+SAKI_API int saki_last_kernel(void);
+
 /* Number of kernels this library has launched in this process (all threads). */
 SAKI_API uint64_t saki_launch_count(void);
 

@@ -20,7 +20,7 @@ ROW_SATURATED, ROW_EPS_ZERO, ROW_MASKED, ROW_NONFINITE, ROW_BAD_ID, ROW_TIMEOUT,
 
 _FLOAT_FIELDS = ("lambda", "kl", "tv", "accept_prob", "logp_x", "logq_x", "logT_x", "logp_y", "logq_y", "loss")
 EXPORTS = ("saki_route_fwd", "saki_route_fwd_bwd", "saki_route_host", "saki_spec_verify",
-           "saki_sample_proposal", "saki_check", "saki_set_kernel", "saki_launch_count",
+           "saki_sample_proposal", "saki_check", "saki_set_kernel", "saki_last_kernel", "saki_launch_count",
            "saki_last_error", "saki_version")
 
 
@@ -79,7 +79,7 @@ def load_library(path: str | None = None):
     lib.saki_launch_count.restype = C.c_uint64
     lib.saki_last_error.restype = C.c_char_p
     for f in ("saki_route_fwd", "saki_route_fwd_bwd", "saki_route_host", "saki_spec_verify",
-              "saki_sample_proposal", "saki_check", "saki_set_kernel", "saki_version"):
+              "saki_sample_proposal", "saki_check", "saki_set_kernel", "saki_last_kernel", "saki_version"):
         getattr(lib, f).restype = C.c_int
     _lib = lib
     return lib
@@ -230,6 +230,11 @@ def check(stream=None) -> int:
 
 def set_kernel(which: int) -> int:
     return load_library().saki_set_kernel(which)
+
+
+def last_kernel() -> int:
+    """1 = general kernel, 2 = cluster kernel (the calling thread's last routing call)."""
+    return load_library().saki_last_kernel()
 
 
 def launch_count() -> int:

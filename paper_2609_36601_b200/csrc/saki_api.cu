@@ -16,6 +16,7 @@ namespace saki {
 static thread_local char g_err[512] = "";
 static std::atomic<uint64_t> g_launches{0};
 static std::atomic<int> g_kernel{0};
+static thread_local int g_last_kernel = 0;
 
 static int fail(int code, const char* fmt, ...) {
   va_list ap;
@@ -68,6 +69,7 @@ static int dispatch_rows(const RowParams& p, int dtype, cudaStream_t st) {
     if (e != cudaSuccess) return cuda_fail(e, "general kernel launch");
   }
   g_launches += (uint64_t)launches;
+  g_last_kernel = served ? 2 : 1;
   return SAKI_OK;
 }
 
@@ -384,6 +386,8 @@ SAKI_API int saki_set_kernel(int which) {
   if (which < 0 || which > 2) which = 0;
   return g_kernel.exchange(which);
 }
+
+SAKI_API int saki_last_kernel(void) { return g_last_kernel; }
 
 SAKI_API uint64_t saki_launch_count(void) { return g_launches.load(); }
 

@@ -66,6 +66,20 @@ def test_ragged_shapes(kernel, V, N, dtype):
     _check_fwd_bwd(d, w, row_offset=(1 << 33) + 5, grad_scale=0.125)
 
 
+@pytest.mark.parametrize("V,N,eps,sigma", [(2048, 5, 0.1, 1.5), (32000, 24, 0.05, 1.0), (50048, 10, 0.1, 1.5),
+                                           (151936, 12, 0.1, 1.5), (163840, 3, 0.01, 2.0), (151936, 6, 1.0, 0.5)])
+def test_cluster_kernel_shapes(V, N, eps, sigma):
+    """The register-resident cluster kernel at every cluster size (1, 2, 4, 8 CTAs per row)."""
+    prev = P.set_kernel(2)
+    try:
+        w = synth.Workload("t", N, V, "bf16", eps, sigma, True, 90 + N, 21)
+        d = synth.generate(w, DEV)
+        _check_fwd_bwd(d, w, row_offset=7)
+        assert P.last_kernel() == 2
+    finally:
+        P.set_kernel(prev)
+
+
 def test_strided_rows_and_mask(kernel):
     w = synth.Workload("t", 12, 3000, "bf16", 0.05, 1.0, True, 78, 10)
     d = synth.generate(w, DEV)
