@@ -1,0 +1,309 @@
+#!/usr/bin/env python
+"""Benchmark of the SAKI routing hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload cfg3] [--rows R] [--no-e2e] [--no-cpu]
+
+One "step" is one pass of the whole hot path (log-softmax x2, lambda solve,
+coupling + TV, routed loss, fused gradient) over one batch of synthetic
+positions: one saki_route_fwd_bwd call.  Prints ONE JSON line.
+
+  value     routed positions/s with the logits resident in HBM (whole job)
+  e2e       the same through saki_route_host: inputs in pinned host memory,
+            host<->device copies inside the timed region
+  roofline  algorithmic HBM bytes (read both logit rows once, write the
+            gradient row once) / measured kernel time, against the measured
+            copy bandwidth of this machine's B200s
+  cpu_baseline  the float64 test oracle, as it stands, on a bounded sample
+
+With N > 1 (under torchrun) every rank routes its own batch of the same
+shape (rows are independent: no collective on the data path); the time is
+the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "routed positions/sec (fwd+bwd, V=151936 bf16)"
+UNIT = "positions/s"
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one cluster-kernel launch divided by the
+# positions it routed (ncu capture summarised in profiles/); None until measured
+TRAFFIC_BYTES_PER_POSITION = None
+
+
+def _peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        time.sleep(0.15)
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.f.read().splitlines():
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1])); mx.append(float(c[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, c[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        if sm:
+            busy = [x for x in sm if x > 0.5 * max(sm)] or sm
+            out.update(sm_mhz=statistics.median(busy), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def _oracle_sample(w, d, rows, grad=True):
+    """Times the float64 oracle on `rows` rows of the workload (host cores)."""
+    import numpy as np
+    import torch
+    import oracle as O
+    idx = torch.arange(rows)
+    s = d["s"][idx.to(d["s"].device)].to("cpu").to(torch.float64).numpy()
+    t = d["t"][idx.to(d["t"].device)].to("cpu").to(torch.float64).numpy()
+    x = d["proposal"][:rows].to("cpu").numpy()
+    t0 = time.perf_counter()
+    ref = O.route(s, t, x, w.eps, w.temperature, w.seed, 0, want_grad=grad, grad_dtype=w.dtype)
+    dt = time.perf_counter() - t0
+    return rows / dt, dt, ref
+
+
+def run_reference(args):
+    """The reference arm: the float64 oracle on a bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import torch
+    from paper_2609_36601_b200 import synth
+    w = synth.WORKLOADS[args.workload]
+    rows = args.ref_rows
+    d = synth.generate(w, "cpu", rows=rows)
+    for _ in range(min(args.warmup, 1)):
+        _oracle_sample(w, d, min(rows, 2))
+    tot_rows, tot_t = 0, 0.0
+    for _ in range(args.steps):
+        r, dt, _ = _oracle_sample(w, d, rows)
+        tot_rows += rows
+        tot_t += dt
+    v = tot_rows / tot_t
+    line = {"metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * tot_t / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "impl": "reference",
+            "config": {"workload": _describe(w), "sample": f"{rows} rows per step"},
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
+                             "sample": f"first {rows} rows of {w.name}, forward + gradient, {args.steps} steps"},
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def _describe(w):
+    return (f"{w.name}: N={w.N} positions, V={w.V}, {w.dtype} logits, eps={w.eps}, temperature={w.temperature}, "
+            f"teacher noise sigma={w.sigma}, fused fwd+bwd with {w.dtype} dlogits")
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2609_36601_b200 as P
+    from paper_2609_36601_b200 import synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    P.load_library()
+
+    w = synth.WORKLOADS[args.workload]
+    if args.rows:
+        w = synth.shrink(w, args.rows)
+    d = synth.generate(w, dev)
+    s, t, x = d["s"], d["t"], d["proposal"]
+    row_offset = rank * w.N                      # ranks route disjoint global rows
+    g = torch.empty_like(s)
+    out = None
+    stream = torch.cuda.current_stream()
+
+    def step():
+        nonlocal out
+        out, _ = P.route_fwd_bwd(s, t, x, w.eps, w.temperature, w.seed, row_offset, grad_scale=1.0 / w.N,
+                                 out=out, dlogits=g, stream=stream)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local) if rank == 0 else None
+    l0 = P.launch_count()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    ev[0].record(stream)
+    for k in range(args.steps):
+        step()
+        ev[k + 1].record(stream)
+    torch.cuda.synchronize()
+    launches = P.launch_count() - l0
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if sampler else None
+    per_step = [ev[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]
+    total_ms = ev[0].elapsed_time(ev[-1])
+    if world > 1:
+        tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    ms_per_step = total_ms / args.steps
+    value = world * w.N / (ms_per_step * 1e-3)
+    n_flagged = P.check()
+    kernel_used = P.last_kernel()
+
+    # ---- end to end: host buffers through saki_route_host
+    e2e = None
+    if not args.no_e2e:
+        hs, ht = s.to("cpu").pin_memory(), t.to("cpu").pin_memory()
+        hx = x.to("cpu").pin_memory()
+        hg = torch.empty(s.shape, dtype=s.dtype, pin_memory=True)
+        hout = None
+        esz = s.element_size()
+        h2d = 2 * s.numel() * esz + hx.numel() * 4
+        d2h = s.numel() * esz + w.N * (1 + 4 * 13)
+        n_e2e = max(1, min(args.steps, args.e2e_steps))
+        hout, _ = P.route_host(hs, ht, hx, w.eps, w.temperature, w.seed, row_offset, grad_scale=1.0 / w.N,
+                               out=hout, dlogits=hg)      # warm-up: staging buffers get allocated
+        if world > 1:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            hout, _ = P.route_host(hs, ht, hx, w.eps, w.temperature, w.seed, row_offset, grad_scale=1.0 / w.N,
+                                   out=hout, dlogits=hg)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        if world > 1:
+            tt = torch.tensor([dt], device=dev, dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            dt = float(tt.item())
+        e2e = {"value": world * w.N * n_e2e / dt, "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": n_e2e, "host_memory": "pinned"}
+        same = all(torch.equal(hout[k], out[k].cpu()) for k in ("corrected", "token", "lambda"))
+        e2e["matches_device_path"] = bool(same)
+        del hs, ht, hg
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = _peaks()
+    bpp = synth.bytes_per_position(w, backward=True)
+    kern_ms = statistics.mean(per_step)          # one kernel launch per step
+    achieved = bpp * w.N / (kern_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "peak_kind": f"of {peak_kind} (device-to-device copy, MEASURED_PEAKS.json)"
+                if peak_kind == "measured" else "of fallback",
+                "traffic": (TRAFFIC_BYTES_PER_POSITION * w.N) if TRAFFIC_BYTES_PER_POSITION else None,
+                "algorithmic_bytes_per_launch": bpp * w.N, "kernel": "saki::cluster_kernel<8>" if kernel_used == 2
+                else "saki::general_kernel", "kernel_ms": kern_ms,
+                "frac_of_nominal_8TBs": achieved / 8000.0}
+
+    stats = {"correction_rate": float(out["corrected"].float().mean().item()),
+             "median_tv": float(out["tv"].median().item()), "mean_lambda": float(out["lambda"].mean().item()),
+             "frac_saturated": float(((out["row_status"] & 1) != 0).float().mean().item()),
+             "rows_flagged": n_flagged}
+
+    cpu = None
+    if not args.no_cpu:
+        v, dt, ref = _oracle_sample(w, d, args.cpu_rows)
+        import numpy as np
+        agree = int(np.sum(out["corrected"][:args.cpu_rows].cpu().numpy() == ref["corrected"]))
+        cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": f"first {args.cpu_rows} rows of {w.name}, forward + gradient, {dt:.1f} s on one host core "
+                         f"(of {os.cpu_count()}); accept/correct flags agree with the GPU on {agree}/{args.cpu_rows}"}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": _describe(w), "l2": "inputs (2 x %.1f GB) exceed L2; no flush needed" %
+                       (s.numel() * s.element_size() / 1e9), "parallelism": f"rows sharded over {world} GPU(s), no collective"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
+            "stats": stats, "achieved_gbs": achieved}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg3")
+    ap.add_argument("--rows", type=int, default=0, help="cut the workload to its first R rows (profiling)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-rows", type=int, default=128)
+    ap.add_argument("--ref-rows", type=int, default=32)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -8,10 +8,12 @@
 // only the landing zone of the NEXT row's slice, fetched by one 1-D bulk
 // async copy per row (cp.async.bulk + mbarrier) while the current row is
 // being computed.  Passes over the registers:
-//   max      packed bf16 maxima of both rows
-//   lse      2 exponentials/element: both log-sum-exps, moments of the
-//            teacher-student logit difference under p (initial guess of
-//            lambda), KL(T||p) (saturation test), teacher argmax index
+//   lse      2 exponentials/element: both log-sum-exps (computed under the
+//            CTA's own maxima rounded up to whole powers of two, then moved
+//            exactly onto the row's maxima, which the CTAs exchange while the
+//            pass runs), moments of the teacher-student logit difference under
+//            p (initial guess of lambda), KL(T||p) (saturation test), teacher
+//            argmax index
 //   solve    1 exponential/element per evaluation of KL(q_beta||p) and its
 //            slope; Newton on sqrt(KL) inside a bisection bracket, typically
 //            two evaluations (Eqs. "bridge", "trust_region")
@@ -20,10 +22,12 @@
 //            "residual"), and the gradient row written straight from
 //            registers (Eq. "general_objective")
 // Per-element work is float32 (packed f32x2 FMAs, ex2.approx); every
-// cross-thread combination and every per-row scalar is float64.  Partial sums
-// travel warp -> all CTAs of the cluster through distributed shared memory,
-// one cluster barrier per pass; each CTA then forms the same scalars
-// redundantly, so control flow is uniform across the cluster.
+// cross-thread combination and every per-row scalar is float64.  Per-warp
+// partial sums travel to all CTAs of the cluster as asynchronous
+// distributed-shared-memory stores that complete on the receiver's mbarrier
+// (no cluster barrier, no fence on the row loop); each CTA then forms the
+// same scalars redundantly from the same numbers in the same order, so
+// control flow is uniform across the cluster.
 #include "saki_common.cuh"
 #include <cooperative_groups.h>
 #include <math_constants.h>
@@ -40,26 +44,35 @@ constexpr int EPT = CHUNKS * 8;         // elements per thread
 constexpr int NPAIR = EPT / 2;          // packed registers per thread per row
 constexpr int SLICE_CAP = CT * EPT;     // elements of one row a CTA can hold
 constexpr int MAX_CS = 8;
-constexpr int NV = 8;                   // doubles per partial-sum vector
+constexpr int NSLOT = MAX_CS * CW;      // per-warp partial slots of a cluster
+constexpr int NV = 8;                   // doubles per partial vector
 constexpr uint32_t SENTINEL = 0xFF7FFF7Fu;   // two bf16 "most negative finite": exp -> 0, difference 0
 
+constexpr int BC_DOUBLES = 40;
 constexpr int OFF_S = 0;
 constexpr int OFF_T = SLICE_CAP * 2;
-constexpr int OFF_RED = OFF_T + SLICE_CAP * 2;                  // [2][MAX_CS*CW][NV] doubles
-constexpr int OFF_BC = OFF_RED + 2 * MAX_CS * CW * NV * 8;      // broadcast scalars
-constexpr int BC_DOUBLES = 32;
-constexpr int OFF_MBAR = OFF_BC + BC_DOUBLES * 8;
-constexpr int SMEM_BYTES = OFF_MBAR + 16;
+constexpr int OFF_RED = OFF_T + SLICE_CAP * 2;                  // [2][NV][NSLOT] doubles: per-warp partials
+constexpr int OFF_MX = OFF_RED + 2 * NV * NSLOT * 8;            // [2][MAX_CS][2] doubles: per-CTA maxima
+constexpr int OFF_GAT = OFF_MX + 2 * MAX_CS * 2 * 8;            // [NV] doubles: cluster totals
+constexpr int OFF_BC = OFF_GAT + NV * 8;                        // [2][BC_DOUBLES] broadcast scalars
+constexpr int OFF_WMAX = OFF_BC + 2 * BC_DOUBLES * 8;           // [2][2][CW] floats: per-warp maxima
+constexpr int OFF_SCR = OFF_WMAX + 2 * 2 * CW * 4;              // [2][EPT] bf16: one thread's elements in index order
+constexpr int OFF_MBAR = OFF_SCR + 2 * EPT * 2;                 // copy barrier, 2 exchange barriers, 2 maxima barriers
+constexpr int SMEM_BYTES = OFF_MBAR + 5 * 8 + 8;
+static_assert(OFF_MBAR % 8 == 0 && OFF_SCR % 16 == 0, "alignment");
 
 constexpr double LN2 = 0.693147180559945309417232121458;
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // ~2 s: give up on a bulk copy
+constexpr double INV_LN2 = 1.44269504088896340735992468100;
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // ~2 s: give up on a wait
 
 enum { MODE_SOLVE = 0, MODE_FINAL = 1, MODE_FLAGGED = 2 };
-// broadcast slots
-enum { BC_MODE = 0, BC_BETA, BC_CB, BC_KB, BC_LO, BC_HI, BC_ITER,       // solver
-       BC_IQ, BC_IP, BC_KG, BC_TOK, BC_STATUS, BC_CORR, BC_LAMBDA,        // final pass
-       BC_GLAM, BC_G0, BC_G1, BC_ACC, BC_LPX, BC_LTX, BC_LOSS, BC_VSTAR,
-       BC_OWNER_WARP, BC_BEFORE, BC_TARGET, BC_TAKE_LAST, BC_MS, BC_MT, BC_BAD, BC_KL, BC_TV };
+// broadcast slots (one set per row buffer)
+enum { BC_MODE = 0, BC_BETA, BC_CB, BC_KB, BC_LO, BC_HI, BC_ITER,                    // solver
+       BC_CL, BC_KQ, BC_IQ, BC_IP, BC_KG, BC_TOK, BC_STATUS, BC_CORR, BC_LAMBDA,    // final pass
+       BC_GLAM, BC_G0, BC_G1, BC_ACC, BC_LPX, BC_LTX, BC_LOSS, BC_VSTAR, BC_KL, BC_TV,
+       BC_OWNER_WARP, BC_BEFORE, BC_TARGET, BC_TAKE_LAST, BC_RSS,
+       BC_UACC, BC_UDRAW, BC_SX, BC_TX, BC_COUNT };
+static_assert(BC_COUNT <= BC_DOUBLES, "broadcast area too small");
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -90,10 +103,56 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {   // round
 __device__ __forceinline__ float2 ex2f2(float2 a) { return make_float2(ex2f(a.x), ex2f(a.y)); }
 __device__ __forceinline__ float2 splat(float a) { return make_float2(a, a); }
 
-// ---- bulk async copy global -> this CTA's shared memory, completion on an mbarrier ----
+// ---- short float64 routines for the scalar phases (one thread, latency-bound) ----
+// log2(1 + (i+0.5)/16) and 2^(i/16), i = 0..15
+__constant__ double LOG2_CENTER[16] = {
+    0.044394119358453436, 0.12928301694496647, 0.20945336562894978, 0.28540221886224837,
+    0.3575520046180837,   0.42626475470209796, 0.4918530963296747,  0.5545888516776374,
+    0.6147098441152082,   0.6724253419714956,  0.7279204545631992,  0.7813597135246596,
+    0.8328900141647416,   0.8826430493618412,  0.9307373375628862,  0.9772799234999164};
+__constant__ double EXP2_SIXTEENTH[16] = {
+    1.0,                1.0442737824274138, 1.0905077326652577, 1.1387886347566916,
+    1.189207115002721,  1.241857812073484,  1.2968395546510096, 1.3542555469368927,
+    1.4142135623730951, 1.4768261459394993, 1.5422108254079407, 1.6104903319492543,
+    1.681792830507429,  1.7562521603732995, 1.8340080864093424, 1.9152065613971474};
+
+__device__ __forceinline__ double rcp_fast(double x) {   // |x| within float range; rel. error ~1e-14
+  double r = (double)__frcp_rn((float)x);
+  r = r * (2.0 - x * r);
+  return r * (2.0 - x * r);
+}
+// x > 0, normal.  Mantissa m in [1,2) is compared with the centre c of its sixteenth:
+// log2 m = log2 c + (2/ln 2) atanh((m-c)/(m+c)), |(m-c)/(m+c)| <= 1/64: three series terms.
+__device__ __forceinline__ double log2_fast(double x) {
+  const long long bits = __double_as_longlong(x);
+  const int e = (int)((bits >> 52) & 0x7ff) - 1023;
+  const int i = (int)((bits >> 48) & 0xf);
+  const double m = __longlong_as_double((bits & 0x000fffffffffffffLL) | 0x3ff0000000000000LL);
+  const double c = 1.0 + ((double)i + 0.5) * 0.0625;
+  const double s = (m - c) * rcp_fast(m + c);
+  const double z = s * s;
+  const double p = 1.0 + z * (1.0 / 3.0 + z * (1.0 / 5.0 + z * (1.0 / 7.0)));
+  return ((double)e + LOG2_CENTER[i]) + (2.0 * INV_LN2) * s * p;
+}
+// any finite x; underflows to 0.  x = n + i/16 + f, |f| <= 1/32.
+__device__ __forceinline__ double exp2_fast(double x) {
+  if (x < -1020.0) return 0.0;
+  if (x > 1020.0) x = 1020.0;
+  const double t = rint(x * 16.0);
+  const int ti = (int)t;
+  const double y = (x - t * 0.0625) * LN2;                 // |y| <= 0.0217
+  const double p = 1.0 + y * (1.0 + y * (0.5 + y * (1.0 / 6.0 + y * (1.0 / 24.0 + y * (1.0 / 120.0 + y * (1.0 / 720.0))))));
+  const double r = p * EXP2_SIXTEENTH[ti & 15];
+  return __longlong_as_double(__double_as_longlong(r) + ((long long)(ti >> 4) << 52));
+}
+
+__device__ __forceinline__ double pow2_exact(int n) {     // 2^n for n <= 0; 0 far below the float range
+  return n < -120 ? 0.0 : (double)__uint_as_float((uint32_t)(127 + n) << 23);
+}
+
+// ---- mbarriers, bulk async copies, asynchronous distributed-shared-memory stores ----
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count));
-  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
@@ -108,7 +167,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
                : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
-// bounded wait: false if the copy did not land within the limit
+// bounded wait: false if the phase did not complete within the limit
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
@@ -117,78 +176,31 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
   }
   return true;
 }
-
-// ---- cluster-wide combination of per-thread partial vectors ----
-// ops: components [0,NSUM) are summed, [NSUM,NSUM+NMAX) maximised, then NMIN minimised.
-template <int NSUM, int NMAX, int NMIN>
-__device__ __forceinline__ double comb(int k, double a, double b) {
-  if (k < NSUM) return a + b;
-  if (k < NSUM + NMAX) return fmax(a, b);
-  return fmin(a, b);
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t local_smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_smem_addr), "r"(rank));
+  return r;
 }
-template <int NSUM, int NMAX, int NMIN>
-__device__ __forceinline__ double ident(int k) {
-  if (k < NSUM) return 0.0;
-  if (k < NSUM + NMAX) return -CUDART_INF;
-  return CUDART_INF;
+// store 8 bytes into a peer CTA's shared memory; the peer's mbarrier counts the bytes
+__device__ __forceinline__ void st_async_f64(uint32_t remote_addr, double v, uint32_t remote_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b64 [%0], %1, [%2];"
+               ::"r"(remote_addr), "l"(__double_as_longlong(v)), "r"(remote_bar) : "memory");
 }
 
-// After the call, warp 0 of every CTA holds the cluster-wide result in v[] (all
-// lanes); the per-warp partials of every CTA sit in red[parity][rank*CW+warp][k].
-template <int CS, int NSUM, int NMAX, int NMIN>
-__device__ __forceinline__ void cluster_combine(double (&v)[NSUM + NMAX + NMIN], double* red, int parity,
-                                                unsigned rank, int warp, int lane) {
-  constexpr int N = NSUM + NMAX + NMIN;
-  static_assert(N <= NV, "vector too long");
+__device__ __forceinline__ double warp_sum(double a) {
 #pragma unroll
-  for (int k = 0; k < N; ++k) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v[k] = comb<NSUM, NMAX, NMIN>(k, v[k], __shfl_xor_sync(0xffffffffu, v[k], o));
-  }
-  double* mine = red + ((size_t)parity * MAX_CS * CW + rank * CW + warp) * NV;
-  if (CS == 1) {
-    if (lane == 0) {
-#pragma unroll
-      for (int k = 0; k < N; ++k) mine[k] = v[k];
-    }
-    __syncthreads();
-  } else {
-    cg::cluster_group cl = cg::this_cluster();
-    if (lane < CS) {
-      double* dst = cl.map_shared_rank(mine, lane);
-#pragma unroll
-      for (int k = 0; k < N; ++k) dst[k] = v[k];
-    }
-    cl.sync();
-  }
-  if (warp == 0) {
-    double acc[N];
-#pragma unroll
-    for (int k = 0; k < N; ++k) acc[k] = ident<NSUM, NMAX, NMIN>(k);
-    for (int slot = lane; slot < CS * CW; slot += 32) {
-      const double* src = red + ((size_t)parity * MAX_CS * CW + slot) * NV;
-#pragma unroll
-      for (int k = 0; k < N; ++k) acc[k] = comb<NSUM, NMAX, NMIN>(k, acc[k], src[k]);
-    }
-#pragma unroll
-    for (int k = 0; k < N; ++k) {
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) acc[k] = comb<NSUM, NMAX, NMIN>(k, acc[k], __shfl_xor_sync(0xffffffffu, acc[k], o));
-      v[k] = acc[k];
-    }
-  }
+  for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+  return a;
 }
-
-struct RowCtx {   // per-row values every thread needs (all cluster-uniform)
-  int64_t row;
-  uint64_t rid;
-  int x;
-  bool bonus, masked;
-};
+__device__ __forceinline__ double warp_min(double a) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) a = fmin(a, __shfl_xor_sync(0xffffffffu, a, o));
+  return a;
+}
 
 struct Consts {   // per-launch constants of the scalar phases
-  double tau, eps, c64, grad_scale;
-  uint64_t seed;
+  double tau, rtau, eps, c64, rc64, grad_scale;
+  float sqrt_eps;
   int V;
 };
 
@@ -196,208 +208,192 @@ struct Consts {   // per-launch constants of the scalar phases
 // threads hold the row in registers; they are kept out of line so that their
 // register needs do not add to the row loop's.
 
-// after pass "lse": log-sum-exps, saturation test, initial guess of lambda
-__device__ __noinline__ void scalar_after_lse(volatile double* bc, const double* v, Consts K, float k0, float k1,
-                                              int x, bool bonus, bool row_timeout) {
-  const double SsT = v[0], StT = v[1], tau = K.tau, eps = K.eps;
-  uint32_t status = 0;
-  if (row_timeout) status = SAKI_ROW_TIMEOUT;
-  else if (!isfinite(v[0] + v[1] + v[2] + v[3] + v[4] + v[5]) || !(SsT > 0.0) || !(StT > 0.0)) status = SAKI_ROW_NONFINITE;
-  else if (!bonus && (x < 0 || x >= K.V)) status = SAKI_ROW_BAD_ID;
-  bc[BC_STATUS] = (double)status;
-  bc[BC_VSTAR] = (v[6] >= 0.0 && v[6] < (double)K.V) ? v[6] : 0.0;
-  if (status) { bc[BC_MODE] = MODE_FLAGGED; return; }
-  const double G0 = LN2 * (log2(SsT) - (double)k0), G1 = LN2 * (log2(StT) - (double)k1);
-  bc[BC_G0] = G0; bc[BC_G1] = G1;
-  double lam = -1.0;
-  if (!(eps > 0.0)) { lam = 0.0; status |= SAKI_ROW_EPS_ZERO; }
-  else {
-    const double m1 = v[2] / SsT, m2 = v[3] / SsT, m3 = v[4] / SsT;
-    const double kl1 = (v[5] / StT) / tau - (G1 - G0);       // KL(T || p)
-    if (kl1 <= eps) { lam = 1.0; status |= SAKI_ROW_SATURATED; }
-    else {
-      // KL(beta) ~ beta^2/2 Var_p(d) + beta^3/3 kappa3_p(d)
-      const double vd = fmax((m2 - m1 * m1) / (tau * tau), 1e-300);
-      const double k3 = (m3 - 3.0 * m1 * m2 + 2.0 * m1 * m1 * m1) / (tau * tau * tau);
-      double b = sqrt(2.0 * eps / vd);
-      for (int it = 0; it < 3; ++it) {
-        const double den = vd + (2.0 / 3.0) * fmin(b, 1.0) * k3;
-        if (den > 0.25 * vd) b = sqrt(2.0 * eps / den);
-      }
-      if (!(b > 1e-7)) b = 1e-7;
-      if (b > 0.98) b = 0.98;
-      const float cb = (float)(K.c64 * b);
-      const double be = (double)cb / K.c64;   // the coefficient the pass really evaluates
-      bc[BC_MODE] = MODE_SOLVE; bc[BC_BETA] = be; bc[BC_CB] = (double)cb;
-      bc[BC_KB] = (double)(float)((1.0 - be) * (double)k0 + be * (double)k1);
-      bc[BC_LO] = 0.0; bc[BC_HI] = 1.0; bc[BC_ITER] = 0.0;
+// The coupling decision, the routed loss and the constants of pass "final".
+__device__ __forceinline__ void decide(double* bc, const Consts& K, double lam, double Glam, double G0, double G1,
+                                       double k0, double k1, double rSs, uint32_t status, int vstar, bool bonus,
+                                       bool masked, int x) {
+  const double Lam = Glam - (1.0 - lam) * G0 - lam * G1;     // log Z(lambda)
+  double lp_x = 0.0, lT_x = 0.0, acc = 1.0;
+  int corrected = 0;
+  if (!bonus) {
+    lp_x = LN2 * (K.c64 * bc[BC_SX]) - G0;
+    lT_x = LN2 * (K.c64 * bc[BC_TX]) - G1;
+    if (lam > 0.0) {
+      acc = exp2_fast(fmin(0.0, lam * (lT_x - lp_x) - Lam) * INV_LN2);
+      corrected = (bc[BC_UACC] < acc) ? 0 : 1;
     }
   }
-  bc[BC_STATUS] = (double)status;
-  if (lam >= 0.0) {   // endpoint: no solve
-    bc[BC_MODE] = MODE_FINAL; bc[BC_LAMBDA] = lam;
-    bc[BC_GLAM] = lam == 0.0 ? G0 : G1;
+  double loss = 0.0, coef = 0.0;   // a corrected row's loss, -log p(v*), is filled in when the row is written
+  int tok = -1;
+  if (masked) status |= SAKI_ROW_MASKED;
+  else if (!bonus) {
+    if (!corrected) { loss = (lp_x - lT_x) * lp_x; coef = -(lp_x - lT_x); tok = x; }
+    else { coef = 1.0; tok = vstar; }
   }
+  // final pass: q_i = e_q * iq, p_i = e_p * ip with exponent shifts kq, k0
+  const float cl = (float)(K.c64 * lam);
+  const float kq = (float)((1.0 - lam) * k0 + lam * k1);
+  bc[BC_LAMBDA] = lam; bc[BC_GLAM] = Glam;
+  bc[BC_CL] = (double)cl; bc[BC_KQ] = (double)kq;
+  bc[BC_IQ] = (double)(float)exp2_fast(-(Glam * INV_LN2 + (double)kq));   // 1 / predicted sum of e_q
+  bc[BC_IP] = (double)(float)rSs;                                           // 1 / sum of e_p
+  bc[BC_KG] = K.grad_scale * coef * K.rtau;                  // gradient = KG * (p - onehot(tok))
+  bc[BC_TOK] = (double)tok; bc[BC_STATUS] = (double)status; bc[BC_CORR] = (double)corrected;
+  bc[BC_ACC] = acc; bc[BC_LPX] = lp_x; bc[BC_LTX] = lT_x; bc[BC_LOSS] = loss;
+  bc[BC_MODE] = MODE_FINAL;
 }
 
-// after one evaluation of pass "solve": safeguarded Newton step on sqrt(KL)
-__device__ __noinline__ void scalar_after_solve(volatile double* bc, const double* v, Consts K, float k0, float k1) {
-  const double tau = K.tau, eps = K.eps;
-  const double beta = bc[BC_BETA], G0 = bc[BC_G0];
+// after pass "lse": v = {Ss, St, M1, M2, M3, N1, argmax index} on the row's shifts k0, k1
+__device__ __noinline__ void scalar_after_lse(double* bc, const double* v, Consts K, float k0f, float k1f, int x,
+                                              bool bonus, bool masked, bool row_timeout) {
+  const double SsT = v[0], StT = v[1], eps = K.eps, k0 = (double)k0f, k1 = (double)k1f;
+  uint32_t status = 0;
+  const double chk = ((v[0] + v[1]) + (v[2] + v[3])) + (v[4] + v[5]);
+  if (row_timeout) status = SAKI_ROW_TIMEOUT;
+  else if (!(fabs(chk) < CUDART_INF) || !(SsT > 0.0) || !(StT > 0.0)) status = SAKI_ROW_NONFINITE;
+  else if (!bonus && (x < 0 || x >= K.V)) status = SAKI_ROW_BAD_ID;
+  const int vstar = (v[6] >= 0.0 && v[6] < (double)K.V) ? (int)v[6] : 0;
+  bc[BC_VSTAR] = (double)vstar;
+  if (status) { bc[BC_STATUS] = (double)status; bc[BC_MODE] = MODE_FLAGGED; return; }
+  const double rSs = rcp_fast(SsT), rSt = rcp_fast(StT);
+  const double G0 = LN2 * (log2_fast(SsT) - k0), G1 = LN2 * (log2_fast(StT) - k1);
+  bc[BC_G0] = G0; bc[BC_G1] = G1; bc[BC_RSS] = rSs;
+  if (!(eps > 0.0)) {          // student-only endpoint
+    bc[BC_KL] = 0.0;
+    decide(bc, K, 0.0, G0, G0, G1, k0, k1, rSs, status | SAKI_ROW_EPS_ZERO, vstar, bonus, masked, x);
+    return;
+  }
+  const double rtau = K.rtau;
+  const double m1 = v[2] * rSs, m2 = v[3] * rSs, m3 = v[4] * rSs;
+  const double kl1 = (v[5] * rSt) * rtau - (G1 - G0);       // KL(T || p)
+  if (kl1 <= eps) {            // teacher endpoint
+    bc[BC_KL] = kl1;
+    decide(bc, K, 1.0, G1, G0, G1, k0, k1, rSs, status | SAKI_ROW_SATURATED, vstar, bonus, masked, x);
+    return;
+  }
+  // initial guess from KL(beta) ~ beta^2/2 Var_p(d) + beta^3/3 kappa3_p(d); float32 is plenty
+  const float rt = (float)rtau;
+  const float vd = fmaxf((float)(m2 - m1 * m1) * rt * rt, 1e-30f);
+  const float k3 = (float)(m3 - 3.0 * m1 * m2 + 2.0 * m1 * m1 * m1) * rt * rt * rt;
+  const float e2 = 2.f * (float)eps;
+  float b = sqrtf(__fdividef(e2, vd));
+#pragma unroll
+  for (int it = 0; it < 3; ++it) {
+    const float den = vd + (2.f / 3.f) * fminf(b, 1.f) * k3;
+    if (den > 0.25f * vd) b = sqrtf(__fdividef(e2, den));
+  }
+  if (!(b > 1e-7f)) b = 1e-7f;
+  if (b > 0.98f) b = 0.98f;
+  const float cb = (float)(K.c64 * (double)b);
+  const double be = (double)cb * K.rc64;   // the coefficient the pass really evaluates
+  bc[BC_STATUS] = (double)status;
+  bc[BC_BETA] = be; bc[BC_CB] = (double)cb;
+  bc[BC_KB] = (double)(float)((1.0 - be) * k0 + be * k1);
+  bc[BC_LO] = 0.0; bc[BC_HI] = 1.0; bc[BC_ITER] = 0.0;
+  bc[BC_MODE] = MODE_SOLVE;
+}
+
+// after one evaluation of pass "solve": safeguarded Newton step on sqrt(KL); v = {S0, S1, S2}
+__device__ __noinline__ void scalar_after_solve(double* bc, const double* v, Consts K, float k0f, float k1f, int x,
+                                                bool bonus, bool masked) {
+  const double eps = K.eps, rtau = K.rtau;
+  const double beta = bc[BC_BETA], G0 = bc[BC_G0], kb = bc[BC_KB];
   double lo = bc[BC_LO], hi = bc[BC_HI];
   const int iter = (int)bc[BC_ITER] + 1;
-  const double G = LN2 * (log2(v[0]) - (double)(float)bc[BC_KB]);
-  const double mu = v[1] / v[0], var = fmax(v[2] / v[0] - mu * mu, 0.0);
-  const double kl = beta * mu / tau - G + G0;         // KL(q_beta || p)
-  const double slope = beta * var / (tau * tau);      // d KL / d beta
+  const double r0 = rcp_fast(v[0]);
+  const double G = LN2 * (log2_fast(v[0]) - kb);
+  const double mu = v[1] * r0, var = fmax(v[2] * r0 - mu * mu, 0.0);
+  const double kl = beta * mu * rtau - G + G0;          // KL(q_beta || p)
+  const double slope = beta * var * rtau * rtau;        // d KL / d beta
   if (kl <= eps) lo = fmax(lo, beta); else hi = fmin(hi, beta);
-  // KL is nearly quadratic in beta, so its square root is nearly linear
+  // KL is nearly quadratic in beta, so its square root is nearly linear: Newton on sqrt(KL).
+  // The step is a correction, so float32 suffices for it once eps - KL is formed in float64.
   double step;
-  const double klp = fmax(kl, 1e-300);
-  if (slope > 0.0 && isfinite(kl)) step = (sqrt(eps) - sqrt(klp)) * 2.0 * sqrt(klp) / slope;
-  else step = 0.5 * (lo + hi) - beta;
+  if (slope > 1e-30 && kl > 1e-30 && kl < 1e30) {
+    const float rk = sqrtf((float)kl);
+    step = (double)__fdividef((float)(eps - kl) * (2.f * rk), (K.sqrt_eps + rk) * (float)slope);
+  } else step = 0.5 * (lo + hi) - beta;
   double nb = beta + step;
   bool bisected = false;
   if (!(nb > lo && nb < hi)) { nb = 0.5 * (lo + hi); bisected = true; }
   const bool done = (!bisected && fabs(nb - beta) <= 2e-4 * beta) || iter >= 40 || (hi - lo) < 1e-9;
   if (done) {
     const float cl = (float)(K.c64 * nb);
-    const double lam = (double)cl / K.c64;
+    const double lam = (double)cl * K.rc64;
     const double dle = lam - beta;
-    bc[BC_MODE] = MODE_FINAL; bc[BC_LAMBDA] = lam;
-    // second-order prediction of G at lambda from this evaluation
-    bc[BC_GLAM] = G + dle * mu / tau + 0.5 * dle * dle * var / (tau * tau);
+    // second-order predictions at lambda from this evaluation
+    bc[BC_KL] = kl + dle * slope;
+    decide(bc, K, lam, G + dle * mu * rtau + 0.5 * dle * dle * var * rtau * rtau, G0, bc[BC_G1], (double)k0f,
+           (double)k1f, bc[BC_RSS], (uint32_t)bc[BC_STATUS], (int)bc[BC_VSTAR], bonus, masked, x);
   } else {
     const float cbn = (float)(K.c64 * nb);
-    const double be = (double)cbn / K.c64;
+    const double be = (double)cbn * K.rc64;
     bc[BC_BETA] = be; bc[BC_CB] = (double)cbn;
-    bc[BC_KB] = (double)(float)((1.0 - be) * (double)k0 + be * (double)k1);
+    bc[BC_KB] = (double)(float)((1.0 - be) * (double)k0f + be * (double)k1f);
     bc[BC_LO] = lo; bc[BC_HI] = hi; bc[BC_ITER] = (double)iter;
   }
 }
 
-// before pass "final": the coupling decision, the routed loss, the pass constants
-__device__ __noinline__ void scalar_decide(volatile double* bc, Consts K, float k0, float k1, const __nv_bfloat16* g_s,
-                                           const __nv_bfloat16* g_t, int x, uint64_t rid, bool bonus, bool masked) {
-  const double lam = bc[BC_LAMBDA], G0 = bc[BC_G0], G1 = bc[BC_G1], Glam = bc[BC_GLAM];
-  const double Lam = Glam - (1.0 - lam) * G0 - lam * G1;     // log Z(lambda)
-  const int vstar = (int)bc[BC_VSTAR];
-  double lp_x = 0.0, lT_x = 0.0, acc = 1.0;
-  int corrected = 0;
-  if (!bonus) {
-    lp_x = LN2 * (K.c64 * (double)__bfloat162float(g_s[x])) - G0;
-    lT_x = LN2 * (K.c64 * (double)__bfloat162float(g_t[x])) - G1;
-    if (lam > 0.0) {
-      acc = exp(fmin(0.0, lam * (lT_x - lp_x) - Lam));
-      corrected = (scalar_uniform(K.seed, rid, STAGE_ACCEPT) < acc) ? 0 : 1;
-    }
-  }
-  double loss = 0.0, coef = 0.0;
-  int tok = -1;
-  uint32_t status = (uint32_t)bc[BC_STATUS];
-  if (masked) status |= SAKI_ROW_MASKED;
-  else if (!bonus) {
-    if (!corrected) { loss = (lp_x - lT_x) * lp_x; coef = -(lp_x - lT_x); tok = x; }
-    else {
-      const double lp_v = LN2 * (K.c64 * (double)__bfloat162float(g_s[vstar])) - G0;
-      loss = -lp_v; coef = 1.0; tok = vstar;
-    }
-  }
-  // final pass: q_i = e_q * iq, p_i = e_p * ip with exponent shifts kq, k0
-  const float cl = (float)(K.c64 * lam);
-  const float kq = (float)((1.0 - lam) * (double)k0 + lam * (double)k1);
-  const double log2S0 = Glam / LN2 + (double)kq;             // predicted log2 of the sum of e_q
-  const double log2Ss = G0 / LN2 + (double)k0;
-  bc[BC_CB] = (double)cl; bc[BC_KB] = (double)kq;
-  bc[BC_IQ] = (double)(float)exp2(-log2S0);
-  bc[BC_IP] = (double)(float)exp2(-log2Ss);
-  bc[BC_KG] = K.grad_scale * coef / K.tau;                   // gradient = KG * (p - onehot(tok))
-  bc[BC_TOK] = (double)tok; bc[BC_STATUS] = (double)status; bc[BC_CORR] = (double)corrected;
-  bc[BC_ACC] = acc; bc[BC_LPX] = lp_x; bc[BC_LTX] = lT_x; bc[BC_LOSS] = loss;
-}
-
-// after pass "final": KL and TV at lambda; for a draw, the warp that owns the target
-__device__ __noinline__ void scalar_after_final(volatile double* bc, const double* v, const double* warp_part, int n_warps,
-                                                Consts K, uint64_t rid, bool bonus) {
-  const double lam = bc[BC_LAMBDA], G0 = bc[BC_G0], G1 = bc[BC_G1];
-  const double Glam = (lam == 0.0) ? G0 : (lam == 1.0 ? G1 : LN2 * (log2(v[0]) - (double)(float)bc[BC_KB]));
-  const double mu = v[1] / v[0];
-  bc[BC_GLAM] = Glam;
-  bc[BC_KL] = (lam > 0.0) ? (lam * mu / K.tau - Glam + G0) : 0.0;
-  bc[BC_TV] = (lam > 0.0) ? v[2] : 0.0;
-  bc[BC_OWNER_WARP] = -1.0;
-  if (!(bonus || bc[BC_CORR] != 0.0)) return;
-  // ordered scan of the per-warp weights (index order = CTA rank, then warp)
+// for a draw: the warp that owns the inverse-CDF target (ordered scan of per-warp weights)
+__device__ __noinline__ void scalar_find_owner(double* bc, const double* warp_part, int n_warps) {
   double total = 0.0;
-  for (int w = 0; w < n_warps; ++w) total += warp_part[w * NV + 3];
-  const double u = scalar_uniform(K.seed, rid, bonus ? STAGE_BONUS : STAGE_RESIDUAL);
-  const double target = u * total;
+  for (int w = 0; w < n_warps; ++w) total += warp_part[w];
+  const double target = bc[BC_UDRAW] * total;
   int owner = -1;
   double before = 0.0;
   for (int w = 0; w < n_warps; ++w) {
-    if (before + warp_part[w * NV + 3] > target) { owner = w; break; }
-    before += warp_part[w * NV + 3];
+    if (before + warp_part[w] > target) { owner = w; break; }
+    before += warp_part[w];
   }
   double take_last = 0.0;
   if (owner < 0) {   // rounding left no crossing: last position with positive weight
     take_last = 1.0; before = 0.0;
-    for (int w = n_warps - 1; w >= 0; --w) if (warp_part[w * NV + 3] > 0.0) { owner = w; break; }
+    for (int w = n_warps - 1; w >= 0; --w) if (warp_part[w] > 0.0) { owner = w; break; }
     if (owner < 0) owner = 0;
   }
   bc[BC_OWNER_WARP] = (double)owner; bc[BC_BEFORE] = before; bc[BC_TARGET] = target; bc[BC_TAKE_LAST] = take_last;
 }
 
-__device__ __noinline__ void write_result(volatile double* bc, const RowParams& P, int64_t row, int corrected, int y,
-                                          bool bonus, double c64, const __nv_bfloat16* g_s, const __nv_bfloat16* g_t) {
+__device__ __noinline__ void write_result(const double* bc, saki_out out, bool write_loss, int64_t row, int corrected,
+                                          int y, bool bonus, double c64, const __nv_bfloat16* g_s,
+                                          const __nv_bfloat16* g_t) {
   RowResult r;
   const double lam = bc[BC_LAMBDA], G0 = bc[BC_G0], G1 = bc[BC_G1], Glam = bc[BC_GLAM];
   const double Lam = Glam - (1.0 - lam) * G0 - lam * G1;
   const double lp_x = bc[BC_LPX], lT_x = bc[BC_LTX];
-  const double lp_y = LN2 * (c64 * (double)__bfloat162float(g_s[y])) - G0;
-  const double lT_y = LN2 * (c64 * (double)__bfloat162float(g_t[y])) - G1;
+  const uint32_t status = (uint32_t)bc[BC_STATUS];
   r.corrected = corrected; r.token = y; r.vstar = (int)bc[BC_VSTAR];
   r.lambda = (float)lam; r.kl = (float)bc[BC_KL]; r.tv = (float)bc[BC_TV];
   r.accept = bonus ? 0.f : (float)bc[BC_ACC];
   r.logp_x = (float)lp_x; r.logT_x = (float)lT_x;
   r.logq_x = bonus ? 0.f : (float)(lp_x + lam * (lT_x - lp_x) - Lam);
-  r.logp_y = (float)lp_y; r.logq_y = (float)(lp_y + lam * (lT_y - lp_y) - Lam);
-  r.loss = (float)bc[BC_LOSS]; r.status = (uint32_t)bc[BC_STATUS];
-  write_row(P.out, row, r, !P.spec);
-}
-
-// the thread that owns the inverse-CDF target walks its elements in index order (from global memory: L2)
-__device__ __noinline__ int rewalk(volatile double* bc, const __nv_bfloat16* g_s, const __nv_bfloat16* g_t, int first,
-                                   int n_el, double running, bool last_mode, bool bonus, float c32, float k0, int V) {
-  const float cl = (float)bc[BC_CB], kq = (float)bc[BC_KB], iq = (float)bc[BC_IQ], ip = (float)bc[BC_IP];
-  const double target = bc[BC_TARGET];
-  int y = -1, last_pos = -1;
-  for (int e = 0; e < n_el; ++e) {
-    const float sf = __bfloat162float(g_s[first + e]), tf = __bfloat162float(g_t[first + e]);
-    const float d = tf - sf;
-    const float ep = ex2f(fmaf(sf, c32, k0));
-    const float eq = ex2f(fmaf(d, cl, fmaf(sf, c32, kq)));
-    const float w = bonus ? eq * iq : fmaxf(fmaf(eq, iq, -(ep * ip)), 0.f);
-    if (w > 0.f) last_pos = first + e;
-    running += (double)w;
-    if (!last_mode && running > target) { y = first + e; break; }
-  }
-  if (y < 0) y = (last_pos >= 0) ? last_pos : min(V - 1, first + max(n_el - 1, 0));
-  return y;
+  r.loss = (float)bc[BC_LOSS];
+  if (corrected || bonus) {
+    const double lp_y = LN2 * (c64 * (double)__bfloat162float(g_s[y])) - G0;
+    const double lT_y = LN2 * (c64 * (double)__bfloat162float(g_t[y])) - G1;
+    r.logp_y = (float)lp_y; r.logq_y = (float)(lp_y + lam * (lT_y - lp_y) - Lam);
+    if (corrected && !(status & SAKI_ROW_MASKED))   // teacher-mode loss: -log p(v*)
+      r.loss = (float)-(LN2 * (c64 * (double)__bfloat162float(g_s[r.vstar])) - G0);
+  } else { r.logp_y = r.logp_x; r.logq_y = r.logq_x; }
+  r.status = status;
+  write_row(out, row, r, write_loss);
 }
 
 template <int CS>
 __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const int n_clusters) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  unsigned rank = 0;
-  if (CS > 1) rank = cg::this_cluster().block_rank();
+  const unsigned rank = cg::this_cluster().block_rank();
   const int cluster_id = blockIdx.x / CS;
 
   const __nv_bfloat16* slot_s = (const __nv_bfloat16*)(smem + OFF_S);
   const __nv_bfloat16* slot_t = (const __nv_bfloat16*)(smem + OFF_T);
   double* red = (double*)(smem + OFF_RED);
-  volatile double* bc = (volatile double*)(smem + OFF_BC);
-  uint64_t* mbar = (uint64_t*)(smem + OFF_MBAR);
+  double* mx = (double*)(smem + OFF_MX);
+  double* gat = (double*)(smem + OFF_GAT);
+  float* wmax = (float*)(smem + OFF_WMAX);
+  uint64_t* mbar = (uint64_t*)(smem + OFF_MBAR);   // [0] row copy, [1..2] partial exchange, [3..4] maxima exchange
+  const uint32_t red_s = smem_addr(red), mx_s = smem_addr(mx), bar_s = smem_addr(mbar);
 
   const int V = P.V;
   const int slice_len = ((V + CS - 1) / CS + 7) & ~7;
@@ -409,8 +405,8 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
 
   const float c32 = (float)(1.4426950408889634 / (double)P.temperature);     // log2(e)/temperature
   Consts K;
-  K.tau = (double)P.temperature; K.eps = (double)P.eps; K.c64 = (double)c32; K.grad_scale = (double)P.grad_scale;
-  K.seed = P.seed; K.V = V;
+  K.tau = (double)P.temperature; K.rtau = 1.0 / K.tau; K.eps = (double)P.eps; K.c64 = (double)c32;
+  K.rc64 = 1.0 / K.c64; K.grad_scale = (double)P.grad_scale; K.sqrt_eps = sqrtf(P.eps); K.V = V;
 
   auto row_ptrs = [&](int64_t row, const __nv_bfloat16*& s, const __nv_bfloat16*& t) {
     const int64_t b = row / P.K1;
@@ -421,29 +417,49 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
   auto issue = [&](int64_t row) {   // one thread: fetch this CTA's slice of both rows
     const __nv_bfloat16 *s, *t;
     row_ptrs(row, s, t);
-    mbar_expect_tx(mbar, 2u * slice_bytes);
+    mbar_expect_tx(&mbar[0], 2u * slice_bytes);
     if (slice_bytes) {
-      bulk_load(smem + OFF_S, s + slice_start, slice_bytes, mbar);
-      bulk_load(smem + OFF_T, t + slice_start, slice_bytes, mbar);
+      bulk_load(smem + OFF_S, s + slice_start, slice_bytes, &mbar[0]);
+      bulk_load(smem + OFF_T, t + slice_start, slice_bytes, &mbar[0]);
     }
   };
+  // one exchange: every warp sends its N-vector to slot rank*CW+warp of red[p] in every CTA
+  auto push = [&](const double* v, int n, int p) {
+    if (lane < CS) {
+      const uint32_t dst = map_to_rank(red_s + (uint32_t)(((p * NV) * NSLOT + rank * CW + warp) * 8), lane);
+      const uint32_t bar = map_to_rank(bar_s + (uint32_t)((1 + p) * 8), lane);
+#pragma unroll
+      for (int k = 0; k < NV; ++k)
+        if (k < n) st_async_f64(dst + (uint32_t)(k * NSLOT * 8), v[k], bar);
+    }
+  };
+  // cluster total of component k (fixed order, the same in every CTA); is_min: minimum instead of sum
+  auto gather = [&](int p, int k, bool is_min) {
+    const double* base = red + (size_t)(p * NV + k) * NSLOT;
+    double a = is_min ? CUDART_INF : 0.0;
+    for (int slot = lane; slot < CS * CW; slot += 32) a = is_min ? fmin(a, base[slot]) : a + base[slot];
+    return is_min ? warp_min(a) : warp_sum(a);
+  };
 
-  if (tid == 0) mbar_init(mbar, 1);
-  __syncthreads();
+  if (tid == 0) {
+#pragma unroll
+    for (int i = 0; i < 5; ++i) mbar_init(&mbar[i], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  cg::this_cluster().sync();   // every CTA's barriers exist before any peer signals them
   if (tid == 0 && cluster_id < P.n_rows) issue(cluster_id);
-  uint32_t phase = 0;
-  int parity = 0;
-  bool dead = false;   // a bulk copy timed out: this CTA stops fetching and flags its rows
+  uint32_t phase = 0, xph0 = 0, xph1 = 0, mph0 = 0, mph1 = 0;
+  int parity = 0, rb = 0;
+  bool dead = false;   // a wait timed out: this CTA stops fetching and the cluster flags its rows
 
-  for (int64_t row = cluster_id; row < P.n_rows; row += n_clusters) {
-    RowCtx rc;
-    rc.row = row;
-    rc.rid = P.row_offset + (uint64_t)row;
+  for (int64_t row = cluster_id; row < P.n_rows; row += n_clusters, rb ^= 1) {
+    double* bc = (double*)(smem + OFF_BC) + rb * BC_DOUBLES;
+    const uint64_t rid = P.row_offset + (uint64_t)row;
     const int64_t seq = row / P.K1;
     const int pos = (int)(row - seq * P.K1);
-    rc.bonus = P.spec && (pos == P.K1 - 1);
-    rc.x = rc.bonus ? 0 : (P.spec ? P.proposal[seq * P.prop_ld + pos] : P.proposal[row]);
-    rc.masked = (P.mask != nullptr) && (P.mask[row] == 0);
+    const bool bonus = P.spec && (pos == P.K1 - 1);
+    const int x = bonus ? 0 : (P.spec ? P.proposal[seq * P.prop_ld + pos] : P.proposal[row]);
+    const bool masked = (P.mask != nullptr) && (P.mask[row] == 0);
     const __nv_bfloat16 *g_s, *g_t;
     row_ptrs(row, g_s, g_t);
     __nv_bfloat16* g_out = P.dlogits ? (__nv_bfloat16*)P.dlogits + row * P.ld_g : nullptr;
@@ -451,7 +467,7 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
     // ------------------------------------------------ stage: shared slot -> registers
     bool timed_out = dead;
     if (!dead) {
-      if (!mbar_wait_bounded(mbar, phase)) timed_out = true;
+      if (!mbar_wait_bounded(&mbar[0], phase)) timed_out = true;
       else phase ^= 1u;
     }
     uint32_t sr[NPAIR], tr[NPAIR];
@@ -468,18 +484,8 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
       sr[4 * j + 0] = a.x; sr[4 * j + 1] = a.y; sr[4 * j + 2] = a.z; sr[4 * j + 3] = a.w;
       tr[4 * j + 0] = b.x; tr[4 * j + 1] = b.y; tr[4 * j + 2] = b.z; tr[4 * j + 3] = b.w;
     }
-    const int any_timeout = __syncthreads_or(timed_out ? 1 : 0);   // also: every thread has drained the slot
-    if (any_timeout) dead = true;
-    if (tid == 0 && !dead) {
-      const int64_t next = row + n_clusters;
-      if (next < P.n_rows) {
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        issue(next);
-      }
-    }
-
-    // ------------------------------------------------ pass "max"
-    float ms, mt;
+    // maxima of this CTA's slice (packed bf16), via shuffles and one CTA barrier
+    float my_mt;
     {
       uint32_t a = sr[0], b = tr[0];
 #pragma unroll
@@ -487,27 +493,58 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
         a = max_bf16x2(a, sr[i]);
         b = max_bf16x2(b, tr[i]);
       }
-      const float2 fa = unpack_bf16x2(a), fb = unpack_bf16x2(b);
-      ms = fmaxf(fa.x, fa.y);
-      mt = fmaxf(fb.x, fb.y);
+      const float2 fb0 = unpack_bf16x2(b);
+      my_mt = fmaxf(fb0.x, fb0.y);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        a = max_bf16x2(a, __shfl_xor_sync(0xffffffffu, a, o));
+        b = max_bf16x2(b, __shfl_xor_sync(0xffffffffu, b, o));
+      }
+      if (lane == 0) {
+        const float2 fa = unpack_bf16x2(a), fb = unpack_bf16x2(b);
+        wmax[(rb * 2 + 0) * CW + warp] = fmaxf(fa.x, fa.y);
+        wmax[(rb * 2 + 1) * CW + warp] = fmaxf(fb.x, fb.y);
+      }
     }
-    const float my_mt = mt;
-    {
-      double v[3] = {dead ? 1.0 : 0.0, (double)ms, (double)mt};
-      // component 0 is a flag: its maximum says whether any CTA of the cluster timed out
-      cluster_combine<CS, 0, 3, 0>(v, red, parity, rank, warp, lane);
-      parity ^= 1;
-      if (tid == 0) { bc[BC_BAD] = v[0]; bc[BC_MS] = v[1]; bc[BC_MT] = v[2]; }
-      __syncthreads();
-      ms = (float)bc[BC_MS];
-      mt = (float)bc[BC_MT];
+    const int any_timeout = __syncthreads_or(timed_out ? 1 : 0);   // also: every thread has drained the slot
+    if (any_timeout) dead = true;
+    if (tid == 0) {
+      const int64_t next = row + n_clusters;
+      if (!dead && next < P.n_rows) {
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        issue(next);
+      }
+      mbar_expect_tx(&mbar[3 + rb], (uint32_t)(CS * 16));          // maxima of all CTAs
+      mbar_expect_tx(&mbar[1 + parity], (uint32_t)(CS * CW * 7 * 8));   // partials of pass "lse"
     }
-    const bool row_timeout = bc[BC_BAD] != 0.0;
-    const float k0 = -(c32 * ms), k1 = -(c32 * mt);   // shifts: every exponent argument <= 0
+    float ms_r = wmax[(rb * 2 + 0) * CW], mt_r = wmax[(rb * 2 + 1) * CW];
+#pragma unroll
+    for (int w = 1; w < CW; ++w) {
+      ms_r = fmaxf(ms_r, wmax[(rb * 2 + 0) * CW + w]);
+      mt_r = fmaxf(mt_r, wmax[(rb * 2 + 1) * CW + w]);
+    }
+    if (tid < CS) {   // this CTA's maxima to every CTA (a CTA that timed out sends NaN: the row is flagged)
+      const uint32_t dst = map_to_rank(mx_s + (uint32_t)(((rb * MAX_CS) + rank) * 16), tid);
+      const uint32_t bar = map_to_rank(bar_s + (uint32_t)((3 + rb) * 8), tid);
+      st_async_f64(dst, dead ? CUDART_NAN : (double)ms_r, bar);
+      st_async_f64(dst + 8, (double)mt_r, bar);
+    }
+    // whole-number shifts: every exponent argument is <= 0, and sums taken under different
+    // shifts differ by exact powers of two
+    const float k0r = -ceilf(c32 * fmaxf(ms_r, -1e30f)), k1r = -ceilf(c32 * fmaxf(mt_r, -1e30f));
 
-    // teacher argmax: lowest index holding the row maximum (exact compare on stored values)
+    // row scalars that do not depend on the passes, fetched off the critical path
+    if (tid == 32) bc[BC_UACC] = scalar_uniform(P.seed, rid, STAGE_ACCEPT);
+    if (tid == 64) bc[BC_UDRAW] = scalar_uniform(P.seed, rid, bonus ? STAGE_BONUS : STAGE_RESIDUAL);
+    if (tid == 96) {
+      const bool ok = (x >= 0 && x < V);
+      bc[BC_SX] = ok ? (double)__bfloat162float(g_s[x]) : 0.0;
+      bc[BC_TX] = ok ? (double)__bfloat162float(g_t[x]) : 0.0;
+    }
+
+    // teacher argmax candidate of this thread (exact compare on stored values, lowest index)
     double cand = CUDART_INF;
-    if (my_mt == mt) {
+    if (my_mt == mt_r) {
 #pragma unroll
       for (int j = 0; j < CHUNKS; ++j) {
         int cj = j + rot;
@@ -516,16 +553,18 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           const float2 f = unpack_bf16x2(tr[4 * j + k]);
-          if (f.x == mt) cand = fmin(cand, (double)(e0 + 2 * k));
-          if (f.y == mt) cand = fmin(cand, (double)(e0 + 2 * k + 1));
+          if (f.x == mt_r) cand = fmin(cand, (double)(e0 + 2 * k));
+          if (f.y == mt_r) cand = fmin(cand, (double)(e0 + 2 * k + 1));
         }
       }
     }
 
     // ------------------------------------------------ pass "lse"
+    float k0, k1;        // the row's shifts
+    bool row_timeout;
     {
       float2 Ss = splat(0.f), St = splat(0.f), M1 = splat(0.f), M2 = splat(0.f), M3 = splat(0.f), N1 = splat(0.f);
-      const float2 cc = splat(c32), kk0 = splat(k0), kk1 = splat(k1), neg1 = splat(-1.f);
+      const float2 cc = splat(c32), kk0 = splat(k0r), kk1 = splat(k1r), neg1 = splat(-1.f);
 #pragma unroll
       for (int i = 0; i < NPAIR; ++i) {
         const float2 sf = unpack_fresh(sr[i]), tf = unpack_fresh(tr[i]);
@@ -541,11 +580,42 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
         M3 = __ffma2_rn(t2, d, M3);
         N1 = __ffma2_rn(et, d, N1);
       }
+      // the row's maxima have arrived meanwhile: move the partial sums onto the row's shifts
+      bool mx_timeout = false;
+      if (!mbar_wait_bounded(&mbar[3 + rb], rb ? mph1 : mph0)) mx_timeout = true;
+      if (rb) mph1 ^= 1u; else mph0 ^= 1u;
+      float gms = -CUDART_INF_F, gmt = -CUDART_INF_F;
+      bool poisoned = mx_timeout;
+#pragma unroll
+      for (int r = 0; r < CS; ++r) {
+        const double a = mx[(rb * MAX_CS + r) * 2 + 0], b = mx[(rb * MAX_CS + r) * 2 + 1];
+        if (a != a) poisoned = true;
+        gms = fmaxf(gms, (float)a); gmt = fmaxf(gmt, (float)b);
+      }
+      row_timeout = poisoned;
+      if (mx_timeout) dead = true;
+      k0 = -ceilf(c32 * fmaxf(gms, -1e30f)); k1 = -ceilf(c32 * fmaxf(gmt, -1e30f));
+      const double fs = pow2_exact((int)(k0 - k0r)), ft = pow2_exact((int)(k1 - k1r));
       auto tot = [](const float2 a) { return (double)a.x + (double)a.y; };
-      double v[7] = {tot(Ss), tot(St), tot(M1), tot(M2), tot(M3), tot(N1), cand};
-      cluster_combine<CS, 6, 0, 1>(v, red, parity, rank, warp, lane);
+      double v[7] = {fs * tot(Ss), ft * tot(St), fs * tot(M1), fs * tot(M2), fs * tot(M3), ft * tot(N1),
+                     (mt_r == gmt) ? cand : CUDART_INF};
+#pragma unroll
+      for (int k = 0; k < 6; ++k) v[k] = warp_sum(v[k]);
+      v[6] = warp_min(v[6]);
+      push(v, 7, parity);
+      if (warp < 7) {
+        if (!mbar_wait_bounded(&mbar[1 + parity], parity ? xph1 : xph0)) dead = true;
+        const double g = gather(parity, warp, warp == 6);
+        if (lane == 0) gat[warp] = g;
+      }
+      if (parity) xph1 ^= 1u; else xph0 ^= 1u;
       parity ^= 1;
-      if (tid == 0) scalar_after_lse(bc, v, K, k0, k1, rc.x, rc.bonus, row_timeout);
+      __syncthreads();
+      if (tid == 0) {
+        scalar_after_lse(bc, gat, K, k0, k1, x, bonus, masked, row_timeout);
+        if ((int)bc[BC_MODE] == MODE_SOLVE) mbar_expect_tx(&mbar[1 + parity], (uint32_t)(CS * CW * 3 * 8));
+        else if ((int)bc[BC_MODE] == MODE_FINAL) mbar_expect_tx(&mbar[1 + parity], (uint32_t)(CS * CW * 3 * 8));
+      }
       __syncthreads();
     }
 
@@ -566,10 +636,20 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
         S2[h] = __ffma2_rn(t1, d, S2[h]);
       }
       auto tot = [](const float2 (&a)[2]) { return ((double)a[0].x + (double)a[0].y) + ((double)a[1].x + (double)a[1].y); };
-      double v[3] = {tot(S0), tot(S1), tot(S2)};
-      cluster_combine<CS, 3, 0, 0>(v, red, parity, rank, warp, lane);
+      double v[3] = {warp_sum(tot(S0)), warp_sum(tot(S1)), warp_sum(tot(S2))};
+      push(v, 3, parity);
+      if (warp < 3) {
+        if (!mbar_wait_bounded(&mbar[1 + parity], parity ? xph1 : xph0)) dead = true;
+        const double g = gather(parity, warp, false);
+        if (lane == 0) gat[warp] = g;
+      }
+      if (parity) xph1 ^= 1u; else xph0 ^= 1u;
       parity ^= 1;
-      if (tid == 0) scalar_after_solve(bc, v, K, k0, k1);
+      __syncthreads();
+      if (tid == 0) {
+        scalar_after_solve(bc, gat, K, k0, k1, x, bonus, masked);
+        mbar_expect_tx(&mbar[1 + parity], (uint32_t)(CS * CW * 3 * 8));   // next evaluation, or pass "final"
+      }
       __syncthreads();
     }
 
@@ -588,23 +668,19 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
           if (e0 < my_len) *reinterpret_cast<uint4*>(g_out + slice_start + e0) = make_uint4(0, 0, 0, 0);
         }
       }
-      __syncthreads();
       continue;
     }
 
-    // ------------------------------------------------ the coupling decision
-    if (tid == 0) scalar_decide(bc, K, k0, k1, g_s, g_t, rc.x, rc.rid, rc.bonus, rc.masked);
-    __syncthreads();
-
     // ------------------------------------------------ pass "final"
+    const bool need_draw = bonus || bc[BC_CORR] != 0.0;
     float my_part;       // this thread's ordered weight for the inverse-CDF draw
+    const float cl = (float)bc[BC_CL], kq = (float)bc[BC_KQ];
+    const float iq = (float)bc[BC_IQ], ip = (float)bc[BC_IP];
     {
-      const float cl = (float)bc[BC_CB], kq = (float)bc[BC_KB];
-      const float iq = (float)bc[BC_IQ], ip = (float)bc[BC_IP];
       const float KGf = (float)bc[BC_KG];
       const float kg = (float)(bc[BC_KG] * (double)ip);     // gradient entry = e_p * kg
       const bool want_g = (g_out != nullptr);
-      float2 Sq[2] = {splat(0.f), splat(0.f)}, S1[2] = {splat(0.f), splat(0.f)}, R[2] = {splat(0.f), splat(0.f)};
+      float2 Sq[2] = {splat(0.f), splat(0.f)}, R[2] = {splat(0.f), splat(0.f)};
       const float2 cc = splat(c32), cll = splat(cl), kqq = splat(kq), kk0 = splat(k0), neg1 = splat(-1.f);
       const float2 iqq = splat(iq), nip = splat(-ip), kgg = splat(kg);
 #pragma unroll
@@ -618,7 +694,6 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
           const float2 ep = ex2f2(__ffma2_rn(sf, cc, kk0));
           const float2 eq = ex2f2(__ffma2_rn(d, cll, __ffma2_rn(sf, cc, kqq)));
           Sq[h] = __fadd2_rn(Sq[h], eq);
-          S1[h] = __ffma2_rn(eq, d, S1[h]);
           float2 r = __ffma2_rn(eq, iqq, __fmul2_rn(ep, nip));     // q_i - p_i
           r.x = fmaxf(r.x, 0.f); r.y = fmaxf(r.y, 0.f);
           R[h] = __fadd2_rn(R[h], r);
@@ -634,9 +709,7 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
       }
       const float sq_f = (Sq[0].x + Sq[0].y) + (Sq[1].x + Sq[1].y);
       const float r_f = (R[0].x + R[0].y) + (R[1].x + R[1].y);
-      my_part = rc.bonus ? sq_f * iq : r_f;
-      auto tot = [](const float2 (&a)[2]) { return ((double)a[0].x + (double)a[0].y) + ((double)a[1].x + (double)a[1].y); };
-      double v[4] = {tot(Sq), tot(S1), (double)r_f, (double)my_part};
+      my_part = bonus ? sq_f * iq : r_f;
       // the thread that owns the supervised token subtracts the one-hot part of the gradient
       if (want_g) {
         const int tok = (int)bc[BC_TOK];
@@ -646,46 +719,90 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
           g_out[tok] = __float2bfloat16_rn(fmaf(ep, kg, -KGf));
         }
       }
-      cluster_combine<CS, 4, 0, 0>(v, red, parity, rank, warp, lane);
-      if (tid == 0)
-        scalar_after_final(bc, v, red + (size_t)parity * MAX_CS * CW * NV, CS * CW, K, rc.rid, rc.bonus);
+      double v[3] = {warp_sum((double)sq_f), warp_sum((double)r_f), warp_sum((double)my_part)};
+      push(v, 3, parity);
+      if (warp == 0) {
+        if (!mbar_wait_bounded(&mbar[1 + parity], parity ? xph1 : xph0)) dead = true;
+        const double tv = gather(parity, 1, false);
+        if (lane == 0) {
+          bc[BC_TV] = (bc[BC_LAMBDA] > 0.0) ? tv : 0.0;
+          if (need_draw) scalar_find_owner(bc, red + (size_t)(parity * NV + 2) * NSLOT, CS * CW);
+          else if (rank == 0) write_result(bc, P.out, !P.spec, row, 0, x, false, K.c64, g_s, g_t);
+        }
+      }
+      if (parity) xph1 ^= 1u; else xph0 ^= 1u;
       parity ^= 1;
-      __syncthreads();
     }
 
-    // ------------------------------------------------ commit: write the row's outputs
-    const bool need_draw = rc.bonus || bc[BC_CORR] != 0.0;
-    if (!need_draw) {
-      if (rank == 0 && tid == 0) write_result(bc, P, row, 0, rc.x, false, K.c64, g_s, g_t);
-    } else if ((int)rank * CW + warp == (int)bc[BC_OWNER_WARP]) {
-      // inverse CDF inside the owning warp: lanes are in index order
-      const double target = bc[BC_TARGET], before = bc[BC_BEFORE];
-      const bool take_last = bc[BC_TAKE_LAST] != 0.0;
-      double inc = (double)my_part;
+    // ------------------------------------------------ the draw (corrected and bonus rows only)
+    if (need_draw) {
+      __syncthreads();
+      if ((int)rank * CW + warp == (int)bc[BC_OWNER_WARP]) {
+        // inverse CDF inside the owning warp: lanes are in index order
+        const double target = bc[BC_TARGET], before = bc[BC_BEFORE];
+        const bool take_last = bc[BC_TAKE_LAST] != 0.0;
+        double inc = (double)my_part;
 #pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const double up = __shfl_up_sync(0xffffffffu, inc, o);
-        if (lane >= o) inc += up;
-      }
-      const unsigned pos = __ballot_sync(0xffffffffu, my_part > 0.f);
-      const unsigned hit = take_last ? 0u : __ballot_sync(0xffffffffu, before + inc > target);
-      int owner_lane;
-      bool last_mode = take_last;
-      if (hit) owner_lane = __ffs(hit) - 1;
-      else { owner_lane = pos ? 31 - __clz(pos) : 0; last_mode = true; }
-      if (lane == owner_lane) {
-        const int first = slice_start + thr_first;
+        for (int o = 1; o < 32; o <<= 1) {
+          const double up = __shfl_up_sync(0xffffffffu, inc, o);
+          if (lane >= o) inc += up;
+        }
+        const unsigned posm = __ballot_sync(0xffffffffu, my_part > 0.f);
+        const unsigned hit = take_last ? 0u : __ballot_sync(0xffffffffu, before + inc > target);
+        int owner_lane;
+        bool last_mode = take_last;
+        if (hit) owner_lane = __ffs(hit) - 1;
+        else { owner_lane = posm ? 31 - __clz(posm) : 0; last_mode = true; }
+        // the owning thread lays its 80 elements out in index order; the warp walks them together
+        uint32_t* scr_s = (uint32_t*)(smem + OFF_SCR);
+        uint32_t* scr_t = scr_s + NPAIR;
+        if (lane == owner_lane) {
+#pragma unroll
+          for (int j = 0; j < CHUNKS; ++j) {
+            int cj = j + rot;
+            if (cj == CHUNKS) cj = 0;
+            *reinterpret_cast<uint4*>(scr_s + cj * 4) = make_uint4(sr[4 * j], sr[4 * j + 1], sr[4 * j + 2], sr[4 * j + 3]);
+            *reinterpret_cast<uint4*>(scr_t + cj * 4) = make_uint4(tr[4 * j], tr[4 * j + 1], tr[4 * j + 2], tr[4 * j + 3]);
+          }
+        }
+        __syncwarp();
+        double running = __shfl_sync(0xffffffffu, before + inc - (double)my_part, owner_lane);
+        const int first = slice_start + (warp * 32 + owner_lane) * EPT;
         const int n_el = max(0, min(EPT, slice_start + my_len - first));
-        const int y = rewalk(bc, g_s, g_t, first, n_el, before + inc - (double)my_part, last_mode, rc.bonus, c32, k0, V);
-        write_result(bc, P, row, rc.bonus ? 0 : 1, y, rc.bonus, K.c64, g_s, g_t);
+        int y = -1, last_pos = -1;
+        const __nv_bfloat16* es = (const __nv_bfloat16*)scr_s;
+        const __nv_bfloat16* et = (const __nv_bfloat16*)scr_t;
+        for (int base = 0; base < n_el && y < 0; base += 32) {
+          const int e = base + lane;
+          float w = 0.f;
+          if (e < n_el) {
+            const float sf = __bfloat162float(es[e]), tf = __bfloat162float(et[e]);
+            const float d = tf - sf;
+            const float ep = ex2f(fmaf(sf, c32, k0));
+            const float eq = ex2f(fmaf(d, cl, fmaf(sf, c32, kq)));
+            w = bonus ? eq * iq : fmaxf(fmaf(eq, iq, -(ep * ip)), 0.f);
+          }
+          double wi = (double)w;
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const double up = __shfl_up_sync(0xffffffffu, wi, o);
+            if (lane >= o) wi += up;
+          }
+          const unsigned pm = __ballot_sync(0xffffffffu, w > 0.f);
+          const unsigned hm = last_mode ? 0u : __ballot_sync(0xffffffffu, running + wi > target);
+          if (pm) last_pos = first + base + 31 - __clz(pm);
+          if (hm) y = first + base + __ffs(hm) - 1;
+          running += __shfl_sync(0xffffffffu, wi, 31);
+        }
+        if (y < 0) y = (last_pos >= 0) ? last_pos : min(V - 1, first + max(n_el - 1, 0));
+        if (lane == 0) write_result(bc, P.out, !P.spec, row, bonus ? 0 : 1, y, bonus, K.c64, g_s, g_t);
       }
     }
-    __syncthreads();   // the broadcast slots are rewritten by the next row
   }
 
   // a CTA that gave up on a copy still waits (bounded) for what it has in flight before leaving
-  if (dead && tid == 0) (void)mbar_wait_bounded(mbar, phase);
-  if (CS > 1) cg::this_cluster().sync();   // no CTA leaves while a peer may still write its shared memory
+  if (dead && tid == 0) (void)mbar_wait_bounded(&mbar[0], phase);
+  cg::this_cluster().sync();   // no CTA leaves while a peer may still write its shared memory
 }
 
 // ---------------------------------------------------------------- host side
