@@ -172,13 +172,16 @@ SAKI_API int saki_sample_proposal(const void* logits, int64_t ld, int64_t N, int
 SAKI_API int saki_check(void* cuda_stream, uint64_t* n_flagged);
 
 /* Selects the row kernel: 0 = automatic, 1 = the general kernel (one block per
- * row, any V and layout), 2 = the register-resident cluster kernel (bf16 rows,
- * 16-byte aligned, V within its capacity; other inputs fall back to 1).
- * Process-wide; meant for tests and benchmarks.  Returns the previous value. */
+ * row, float64, any V, dtype and layout), 2 = the register-resident cluster
+ * kernel (one row per cluster of up to 8 blocks), 3 = the row-per-SM kernel
+ * (one row per block; shared memory plus L2).  2 and 3 serve bf16 rows with
+ * 16-byte aligned rows and V a multiple of 8, V >= 2048 (2: V <= 163840);
+ * other inputs fall back to 1.  Automatic prefers 3.  Process-wide; meant for
+ * tests and benchmarks.  Returns the previous value. */
 SAKI_API int saki_set_kernel(int which);
 
 /* Which row kernel the calling thread's last routing call used: 1 general, 2 cluster,
- * 0 if none yet. */
+ * 3 row-per-SM, 0 if none yet. */
 SAKI_API int saki_last_kernel(void);
 
 /* Number of kernels this library has launched in this process (all threads). */

@@ -60,16 +60,23 @@ static int dispatch_rows(const RowParams& p, int dtype, cudaStream_t st) {
   cudaError_t e;
   bool served = false;
   const int which = g_kernel.load();
-  if (which != 1 && cluster_can_serve(p, dtype)) {
+  int used = 1;
+  if ((which == 0 || which == 3) && rowsm_can_serve(p, dtype)) {
+    e = launch_rowsm(p, st, &launches, &served);
+    if (e != cudaSuccess) return cuda_fail(e, "row-per-SM kernel launch");
+    if (served) used = 3;
+  }
+  if (!served && which == 2 && cluster_can_serve(p, dtype)) {
     e = launch_cluster(p, st, &launches, &served);
     if (e != cudaSuccess) return cuda_fail(e, "cluster kernel launch");
+    if (served) used = 2;
   }
   if (!served) {
     e = launch_general(p, dtype, st, &launches);
     if (e != cudaSuccess) return cuda_fail(e, "general kernel launch");
   }
   g_launches += (uint64_t)launches;
-  g_last_kernel = served ? 2 : 1;
+  g_last_kernel = used;
   return SAKI_OK;
 }
 
@@ -383,7 +390,7 @@ SAKI_API int saki_route_host(const saki_in* in, const saki_out* out, void* dlogi
 }
 
 SAKI_API int saki_set_kernel(int which) {
-  if (which < 0 || which > 2) which = 0;
+  if (which < 0 || which > 3) which = 0;
   return g_kernel.exchange(which);
 }
 

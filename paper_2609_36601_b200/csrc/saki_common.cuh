@@ -106,5 +106,7 @@ __device__ inline RowResult zero_row(uint32_t status) {
 cudaError_t launch_general(const RowParams& p, int dtype, cudaStream_t st, int* n_launches);
 cudaError_t launch_cluster(const RowParams& p, cudaStream_t st, int* n_launches, bool* served);
 bool cluster_can_serve(const RowParams& p, int dtype);
+cudaError_t launch_rowsm(const RowParams& p, cudaStream_t st, int* n_launches, bool* served);
+bool rowsm_can_serve(const RowParams& p, int dtype);
 
 }  // namespace saki

@@ -1,0 +1,330 @@
+// Device-side pieces shared by the two bf16 row kernels: packed-bf16 helpers,
+// mbarrier / bulk-copy wrappers, the short float64 routines and the per-row
+// scalar phases (lambda guess and solve step, coupling decision, result write).
+#pragma once
+#include "saki_common.cuh"
+#include <math_constants.h>
+
+namespace saki {
+
+constexpr int BC_DOUBLES = 40;             // doubles of one broadcast area
+constexpr double LN2 = 0.693147180559945309417232121458;
+constexpr double INV_LN2 = 1.44269504088896340735992468100;
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // ~2 s: give up on a wait
+
+enum { MODE_SOLVE = 0, MODE_FINAL = 1, MODE_FLAGGED = 2 };
+// broadcast slots (one set per row buffer)
+enum { BC_MODE = 0, BC_BETA, BC_CB, BC_KB, BC_LO, BC_HI, BC_ITER,                    // solver
+       BC_CL, BC_KQ, BC_IQ, BC_IP, BC_KG, BC_TOK, BC_STATUS, BC_CORR, BC_LAMBDA,    // final pass
+       BC_GLAM, BC_G0, BC_G1, BC_ACC, BC_LPX, BC_LTX, BC_LOSS, BC_VSTAR, BC_KL, BC_TV,
+       BC_OWNER_WARP, BC_BEFORE, BC_TARGET, BC_TAKE_LAST, BC_RSS,
+       BC_UACC, BC_UDRAW, BC_SX, BC_TX, BC_COUNT };
+static_assert(BC_COUNT <= BC_DOUBLES, "broadcast area too small");
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ float ex2f(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float2 unpack_bf16x2(uint32_t r) {
+  return make_float2(__uint_as_float(r << 16), __uint_as_float(r & 0xffff0000u));
+}
+// Same, but opaque to the optimiser: each pass re-derives the floats from the
+// packed registers instead of keeping 160 unpacked values alive across passes.
+__device__ __forceinline__ float2 unpack_fresh(uint32_t r) {
+  asm volatile("" : "+r"(r));
+  return unpack_bf16x2(r);
+}
+__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {   // round to nearest even
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+__device__ __forceinline__ float2 ex2f2(float2 a) { return make_float2(ex2f(a.x), ex2f(a.y)); }
+__device__ __forceinline__ float2 splat(float a) { return make_float2(a, a); }
+
+// ---- short float64 routines for the scalar phases (one thread, latency-bound) ----
+// log2(1 + (i+0.5)/16) and 2^(i/16), i = 0..15
+static __constant__ double LOG2_CENTER[16] = {
+    0.044394119358453436, 0.12928301694496647, 0.20945336562894978, 0.28540221886224837,
+    0.3575520046180837,   0.42626475470209796, 0.4918530963296747,  0.5545888516776374,
+    0.6147098441152082,   0.6724253419714956,  0.7279204545631992,  0.7813597135246596,
+    0.8328900141647416,   0.8826430493618412,  0.9307373375628862,  0.9772799234999164};
+static __constant__ double EXP2_SIXTEENTH[16] = {
+    1.0,                1.0442737824274138, 1.0905077326652577, 1.1387886347566916,
+    1.189207115002721,  1.241857812073484,  1.2968395546510096, 1.3542555469368927,
+    1.4142135623730951, 1.4768261459394993, 1.5422108254079407, 1.6104903319492543,
+    1.681792830507429,  1.7562521603732995, 1.8340080864093424, 1.9152065613971474};
+
+__device__ __forceinline__ double rcp_fast(double x) {   // |x| within float range; rel. error ~1e-14
+  double r = (double)__frcp_rn((float)x);
+  r = r * (2.0 - x * r);
+  return r * (2.0 - x * r);
+}
+// x > 0, normal.  Mantissa m in [1,2) is compared with the centre c of its sixteenth:
+// log2 m = log2 c + (2/ln 2) atanh((m-c)/(m+c)), |(m-c)/(m+c)| <= 1/64: three series terms.
+__device__ __forceinline__ double log2_fast(double x) {
+  const long long bits = __double_as_longlong(x);
+  const int e = (int)((bits >> 52) & 0x7ff) - 1023;
+  const int i = (int)((bits >> 48) & 0xf);
+  const double m = __longlong_as_double((bits & 0x000fffffffffffffLL) | 0x3ff0000000000000LL);
+  const double c = 1.0 + ((double)i + 0.5) * 0.0625;
+  const double s = (m - c) * rcp_fast(m + c);
+  const double z = s * s;
+  const double p = 1.0 + z * (1.0 / 3.0 + z * (1.0 / 5.0 + z * (1.0 / 7.0)));
+  return ((double)e + LOG2_CENTER[i]) + (2.0 * INV_LN2) * s * p;
+}
+// any finite x; underflows to 0.  x = n + i/16 + f, |f| <= 1/32.
+__device__ __forceinline__ double exp2_fast(double x) {
+  if (x < -1020.0) return 0.0;
+  if (x > 1020.0) x = 1020.0;
+  const double t = rint(x * 16.0);
+  const int ti = (int)t;
+  const double y = (x - t * 0.0625) * LN2;                 // |y| <= 0.0217
+  const double p = 1.0 + y * (1.0 + y * (0.5 + y * (1.0 / 6.0 + y * (1.0 / 24.0 + y * (1.0 / 120.0 + y * (1.0 / 720.0))))));
+  const double r = p * EXP2_SIXTEENTH[ti & 15];
+  return __longlong_as_double(__double_as_longlong(r) + ((long long)(ti >> 4) << 52));
+}
+
+__device__ __forceinline__ double pow2_exact(int n) {     // 2^n for n <= 0; 0 far below the float range
+  return n < -120 ? 0.0 : (double)__uint_as_float((uint32_t)(127 + n) << 23);
+}
+
+// ---- mbarriers, bulk async copies, asynchronous distributed-shared-memory stores ----
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_load(void* dst_smem, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_addr(dst_smem)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// bounded wait: false if the phase did not complete within the limit
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (clock64() - t0 > WAIT_LIMIT_CYCLES) return false;
+  }
+  return true;
+}
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t local_smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_smem_addr), "r"(rank));
+  return r;
+}
+// store 8 bytes into a peer CTA's shared memory; the peer's mbarrier counts the bytes
+__device__ __forceinline__ void st_async_f64(uint32_t remote_addr, double v, uint32_t remote_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b64 [%0], %1, [%2];"
+               ::"r"(remote_addr), "l"(__double_as_longlong(v)), "r"(remote_bar) : "memory");
+}
+
+__device__ __forceinline__ double warp_sum(double a) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+  return a;
+}
+__device__ __forceinline__ double warp_min(double a) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) a = fmin(a, __shfl_xor_sync(0xffffffffu, a, o));
+  return a;
+}
+
+struct Consts {   // per-launch constants of the scalar phases
+  double tau, rtau, eps, c64, rc64, grad_scale;
+  float sqrt_eps;
+  int V;
+};
+
+// The scalar phases run on one thread per CTA, in float64, while all other
+// threads hold the row in registers; they are kept out of line so that their
+// register needs do not add to the row loop's.
+
+// The coupling decision, the routed loss and the constants of pass "final".
+__device__ __forceinline__ void decide(double* bc, const Consts& K, double lam, double Glam, double G0, double G1,
+                                       double k0, double k1, double rSs, uint32_t status, int vstar, bool bonus,
+                                       bool masked, int x) {
+  const double Lam = Glam - (1.0 - lam) * G0 - lam * G1;     // log Z(lambda)
+  double lp_x = 0.0, lT_x = 0.0, acc = 1.0;
+  int corrected = 0;
+  if (!bonus) {
+    lp_x = LN2 * (K.c64 * bc[BC_SX]) - G0;
+    lT_x = LN2 * (K.c64 * bc[BC_TX]) - G1;
+    if (lam > 0.0) {
+      acc = exp2_fast(fmin(0.0, lam * (lT_x - lp_x) - Lam) * INV_LN2);
+      corrected = (bc[BC_UACC] < acc) ? 0 : 1;
+    }
+  }
+  double loss = 0.0, coef = 0.0;   // a corrected row's loss, -log p(v*), is filled in when the row is written
+  int tok = -1;
+  if (masked) status |= SAKI_ROW_MASKED;
+  else if (!bonus) {
+    if (!corrected) { loss = (lp_x - lT_x) * lp_x; coef = -(lp_x - lT_x); tok = x; }
+    else { coef = 1.0; tok = vstar; }
+  }
+  // final pass: q_i = e_q * iq, p_i = e_p * ip with exponent shifts kq, k0
+  const float cl = (float)(K.c64 * lam);
+  const float kq = (float)((1.0 - lam) * k0 + lam * k1);
+  bc[BC_LAMBDA] = lam; bc[BC_GLAM] = Glam;
+  bc[BC_CL] = (double)cl; bc[BC_KQ] = (double)kq;
+  bc[BC_IQ] = (double)(float)exp2_fast(-(Glam * INV_LN2 + (double)kq));   // 1 / predicted sum of e_q
+  bc[BC_IP] = (double)(float)rSs;                                           // 1 / sum of e_p
+  bc[BC_KG] = K.grad_scale * coef * K.rtau;                  // gradient = KG * (p - onehot(tok))
+  bc[BC_TOK] = (double)tok; bc[BC_STATUS] = (double)status; bc[BC_CORR] = (double)corrected;
+  bc[BC_ACC] = acc; bc[BC_LPX] = lp_x; bc[BC_LTX] = lT_x; bc[BC_LOSS] = loss;
+  bc[BC_MODE] = MODE_FINAL;
+}
+
+// after pass "lse": v = {Ss, St, M1, M2, M3, N1, argmax index} on the row's shifts k0, k1
+static __device__ __noinline__ void scalar_after_lse(double* bc, const double* v, Consts K, float k0f, float k1f, int x,
+                                              bool bonus, bool masked, bool row_timeout) {
+  const double SsT = v[0], StT = v[1], eps = K.eps, k0 = (double)k0f, k1 = (double)k1f;
+  uint32_t status = 0;
+  const double chk = ((v[0] + v[1]) + (v[2] + v[3])) + (v[4] + v[5]);
+  if (row_timeout) status = SAKI_ROW_TIMEOUT;
+  else if (!(fabs(chk) < CUDART_INF) || !(SsT > 0.0) || !(StT > 0.0)) status = SAKI_ROW_NONFINITE;
+  else if (!bonus && (x < 0 || x >= K.V)) status = SAKI_ROW_BAD_ID;
+  const int vstar = (v[6] >= 0.0 && v[6] < (double)K.V) ? (int)v[6] : 0;
+  bc[BC_VSTAR] = (double)vstar;
+  if (status) { bc[BC_STATUS] = (double)status; bc[BC_MODE] = MODE_FLAGGED; return; }
+  const double rSs = rcp_fast(SsT), rSt = rcp_fast(StT);
+  const double G0 = LN2 * (log2_fast(SsT) - k0), G1 = LN2 * (log2_fast(StT) - k1);
+  bc[BC_G0] = G0; bc[BC_G1] = G1; bc[BC_RSS] = rSs;
+  if (!(eps > 0.0)) {          // student-only endpoint
+    bc[BC_KL] = 0.0;
+    decide(bc, K, 0.0, G0, G0, G1, k0, k1, rSs, status | SAKI_ROW_EPS_ZERO, vstar, bonus, masked, x);
+    return;
+  }
+  const double rtau = K.rtau;
+  const double m1 = v[2] * rSs, m2 = v[3] * rSs, m3 = v[4] * rSs;
+  const double kl1 = (v[5] * rSt) * rtau - (G1 - G0);       // KL(T || p)
+  if (kl1 <= eps) {            // teacher endpoint
+    bc[BC_KL] = kl1;
+    decide(bc, K, 1.0, G1, G0, G1, k0, k1, rSs, status | SAKI_ROW_SATURATED, vstar, bonus, masked, x);
+    return;
+  }
+  // initial guess from KL(beta) ~ beta^2/2 Var_p(d) + beta^3/3 kappa3_p(d); float32 is plenty
+  const float rt = (float)rtau;
+  const float vd = fmaxf((float)(m2 - m1 * m1) * rt * rt, 1e-30f);
+  const float k3 = (float)(m3 - 3.0 * m1 * m2 + 2.0 * m1 * m1 * m1) * rt * rt * rt;
+  const float e2 = 2.f * (float)eps;
+  float b = sqrtf(__fdividef(e2, vd));
+#pragma unroll
+  for (int it = 0; it < 3; ++it) {
+    const float den = vd + (2.f / 3.f) * fminf(b, 1.f) * k3;
+    if (den > 0.25f * vd) b = sqrtf(__fdividef(e2, den));
+  }
+  if (!(b > 1e-7f)) b = 1e-7f;
+  if (b > 0.98f) b = 0.98f;
+  const float cb = (float)(K.c64 * (double)b);
+  const double be = (double)cb * K.rc64;   // the coefficient the pass really evaluates
+  bc[BC_STATUS] = (double)status;
+  bc[BC_BETA] = be; bc[BC_CB] = (double)cb;
+  bc[BC_KB] = (double)(float)((1.0 - be) * k0 + be * k1);
+  bc[BC_LO] = 0.0; bc[BC_HI] = 1.0; bc[BC_ITER] = 0.0;
+  bc[BC_MODE] = MODE_SOLVE;
+}
+
+// after one evaluation of pass "solve": safeguarded Newton step on sqrt(KL); v = {S0, S1, S2}
+static __device__ __noinline__ void scalar_after_solve(double* bc, const double* v, Consts K, float k0f, float k1f, int x,
+                                                bool bonus, bool masked) {
+  const double eps = K.eps, rtau = K.rtau;
+  const double beta = bc[BC_BETA], G0 = bc[BC_G0], kb = bc[BC_KB];
+  double lo = bc[BC_LO], hi = bc[BC_HI];
+  const int iter = (int)bc[BC_ITER] + 1;
+  const double r0 = rcp_fast(v[0]);
+  const double G = LN2 * (log2_fast(v[0]) - kb);
+  const double mu = v[1] * r0, var = fmax(v[2] * r0 - mu * mu, 0.0);
+  const double kl = beta * mu * rtau - G + G0;          // KL(q_beta || p)
+  const double slope = beta * var * rtau * rtau;        // d KL / d beta
+  if (kl <= eps) lo = fmax(lo, beta); else hi = fmin(hi, beta);
+  // KL is nearly quadratic in beta, so its square root is nearly linear: Newton on sqrt(KL).
+  // The step is a correction, so float32 suffices for it once eps - KL is formed in float64.
+  double step;
+  if (slope > 1e-30 && kl > 1e-30 && kl < 1e30) {
+    const float rk = sqrtf((float)kl);
+    step = (double)__fdividef((float)(eps - kl) * (2.f * rk), (K.sqrt_eps + rk) * (float)slope);
+  } else step = 0.5 * (lo + hi) - beta;
+  double nb = beta + step;
+  bool bisected = false;
+  if (!(nb > lo && nb < hi)) { nb = 0.5 * (lo + hi); bisected = true; }
+  const bool done = (!bisected && fabs(nb - beta) <= 2e-4 * beta) || iter >= 40 || (hi - lo) < 1e-9;
+  if (done) {
+    const float cl = (float)(K.c64 * nb);
+    const double lam = (double)cl * K.rc64;
+    const double dle = lam - beta;
+    // second-order predictions at lambda from this evaluation
+    bc[BC_KL] = kl + dle * slope;
+    decide(bc, K, lam, G + dle * mu * rtau + 0.5 * dle * dle * var * rtau * rtau, G0, bc[BC_G1], (double)k0f,
+           (double)k1f, bc[BC_RSS], (uint32_t)bc[BC_STATUS], (int)bc[BC_VSTAR], bonus, masked, x);
+  } else {
+    const float cbn = (float)(K.c64 * nb);
+    const double be = (double)cbn * K.rc64;
+    bc[BC_BETA] = be; bc[BC_CB] = (double)cbn;
+    bc[BC_KB] = (double)(float)((1.0 - be) * (double)k0f + be * (double)k1f);
+    bc[BC_LO] = lo; bc[BC_HI] = hi; bc[BC_ITER] = (double)iter;
+  }
+}
+
+// for a draw: the warp that owns the inverse-CDF target (ordered scan of per-warp weights)
+static __device__ __noinline__ void scalar_find_owner(double* bc, const double* warp_part, int n_warps) {
+  double total = 0.0;
+  for (int w = 0; w < n_warps; ++w) total += warp_part[w];
+  const double target = bc[BC_UDRAW] * total;
+  int owner = -1;
+  double before = 0.0;
+  for (int w = 0; w < n_warps; ++w) {
+    if (before + warp_part[w] > target) { owner = w; break; }
+    before += warp_part[w];
+  }
+  double take_last = 0.0;
+  if (owner < 0) {   // rounding left no crossing: last position with positive weight
+    take_last = 1.0; before = 0.0;
+    for (int w = n_warps - 1; w >= 0; --w) if (warp_part[w] > 0.0) { owner = w; break; }
+    if (owner < 0) owner = 0;
+  }
+  bc[BC_OWNER_WARP] = (double)owner; bc[BC_BEFORE] = before; bc[BC_TARGET] = target; bc[BC_TAKE_LAST] = take_last;
+}
+
+static __device__ __noinline__ void write_result(const double* bc, saki_out out, bool write_loss, int64_t row, int corrected,
+                                          int y, bool bonus, double c64, const __nv_bfloat16* g_s,
+                                          const __nv_bfloat16* g_t) {
+  RowResult r;
+  const double lam = bc[BC_LAMBDA], G0 = bc[BC_G0], G1 = bc[BC_G1], Glam = bc[BC_GLAM];
+  const double Lam = Glam - (1.0 - lam) * G0 - lam * G1;
+  const double lp_x = bc[BC_LPX], lT_x = bc[BC_LTX];
+  const uint32_t status = (uint32_t)bc[BC_STATUS];
+  r.corrected = corrected; r.token = y; r.vstar = (int)bc[BC_VSTAR];
+  r.lambda = (float)lam; r.kl = (float)bc[BC_KL]; r.tv = (float)bc[BC_TV];
+  r.accept = bonus ? 0.f : (float)bc[BC_ACC];
+  r.logp_x = (float)lp_x; r.logT_x = (float)lT_x;
+  r.logq_x = bonus ? 0.f : (float)(lp_x + lam * (lT_x - lp_x) - Lam);
+  r.loss = (float)bc[BC_LOSS];
+  if (corrected || bonus) {
+    const double lp_y = LN2 * (c64 * (double)__bfloat162float(g_s[y])) - G0;
+    const double lT_y = LN2 * (c64 * (double)__bfloat162float(g_t[y])) - G1;
+    r.logp_y = (float)lp_y; r.logq_y = (float)(lp_y + lam * (lT_y - lp_y) - Lam);
+    if (corrected && !(status & SAKI_ROW_MASKED))   // teacher-mode loss: -log p(v*)
+      r.loss = (float)-(LN2 * (c64 * (double)__bfloat162float(g_s[r.vstar])) - G0);
+  } else { r.logp_y = r.logp_x; r.logq_y = r.logq_x; }
+  r.status = status;
+  write_row(out, row, r, write_loss);
+}
+
+
+}  // namespace saki

@@ -10,7 +10,7 @@ from parity import compare_rows, grad_check, oracle_inputs, to_np64
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
-KERNELS = {"general": 1, "auto": 0}
+KERNELS = {"general": 1, "cluster": 2, "auto": 0}
 
 
 @pytest.fixture(params=list(KERNELS))
@@ -68,14 +68,20 @@ def test_ragged_shapes(kernel, V, N, dtype):
 
 @pytest.mark.parametrize("V,N,eps,sigma", [(2048, 5, 0.1, 1.5), (32000, 24, 0.05, 1.0), (50048, 10, 0.1, 1.5),
                                            (151936, 12, 0.1, 1.5), (163840, 3, 0.01, 2.0), (151936, 6, 1.0, 0.5)])
-def test_cluster_kernel_shapes(V, N, eps, sigma):
-    """The register-resident cluster kernel at every cluster size (1, 2, 4, 8 CTAs per row)."""
-    prev = P.set_kernel(2)
+@pytest.mark.parametrize("which", [2, 3])
+def test_fast_kernel_shapes(V, N, eps, sigma, which):
+    """The two bf16 hot-path kernels: the cluster kernel at every cluster size (1, 2, 4, 8 blocks
+    per row) and the row-per-SM kernel with and without a part of the row left in L2."""
+    prev = P.set_kernel(which)
     try:
         w = synth.Workload("t", N, V, "bf16", eps, sigma, True, 90 + N, 21)
         d = synth.generate(w, DEV)
         _check_fwd_bwd(d, w, row_offset=7)
-        assert P.last_kernel() == 2
+        assert P.last_kernel() == which
+        if V <= 50048:      # more rows than blocks: every block routes several rows back to back
+            w = synth.Workload("t", 400, V, "bf16", eps, sigma, True, 91 + N, 22)
+            d = synth.generate(w, DEV)
+            _check_fwd_bwd(d, w, rows=range(0, 400, 7))
     finally:
         P.set_kernel(prev)
 
