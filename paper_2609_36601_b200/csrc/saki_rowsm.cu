@@ -26,12 +26,18 @@
 // combinations and per-row scalars are float64.
 #include "saki_device.cuh"
 #include <mutex>
+#ifdef SAKI_PHASE_TIMING
+#include <cstdio>
+#endif
 
 namespace saki {
 
-constexpr int RT = 1024;                // threads per CTA
+#ifndef SAKI_ROWSM_THREADS
+#define SAKI_ROWSM_THREADS 1024
+#endif
+constexpr int RT = SAKI_ROWSM_THREADS;  // threads per CTA
 constexpr int RW = RT / 32;             // warps per CTA
-constexpr int KS_MAX = 6;               // resident steps per warp (a step = 32 chunks of 8 elements)
+constexpr int KS_MAX = 6 * (1024 / RT);   // resident steps per warp (a step = 32 chunks of 8 elements)
 constexpr int RES_CHUNKS = KS_MAX * 32; // resident chunks per warp and row
 constexpr int RNV = 8;                  // doubles per partial vector
 
@@ -43,10 +49,36 @@ constexpr int ROFF_WMAX = ROFF_BC + BC_DOUBLES * 8;              // [2][RW] floa
 constexpr int ROFF_MBAR = ROFF_WMAX + 2 * RW * 4;
 constexpr int RSMEM_BYTES = ROFF_MBAR + 16;
 
-__device__ __forceinline__ void prefetch_l2(const void* src, uint32_t bytes) {
-  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+// L2 residency hints: the part of a row that is re-read from L2 in every pass is marked
+// evict-last; everything that passes through L2 once (the shared-memory resident part, the
+// gradient row) is marked evict-first so that it does not push the re-read part out.
+__device__ __forceinline__ uint64_t policy_evict_last() {
+  uint64_t p;
+  asm("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
 }
-__device__ __forceinline__ uint4 ld_l2(const __nv_bfloat16* p) { return __ldcg(reinterpret_cast<const uint4*>(p)); }
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t p;
+  asm("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void prefetch_l2(const void* src, uint32_t bytes, uint64_t pol) {
+  asm volatile("cp.async.bulk.prefetch.L2.global.L2::cache_hint [%0], %1, %2;" ::"l"(src), "r"(bytes), "l"(pol) : "memory");
+}
+__device__ __forceinline__ void bulk_load_hint(void* dst_smem, const void* src, uint32_t bytes, uint64_t* bar, uint64_t pol) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+               ::"r"(smem_addr(dst_smem)), "l"(src), "r"(bytes), "r"(smem_addr(bar)), "l"(pol) : "memory");
+}
+__device__ __forceinline__ uint4 ld_l2(const __nv_bfloat16* p, uint64_t pol) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4], %5;"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(pol));
+  return v;
+}
+__device__ __forceinline__ void st_stream(__nv_bfloat16* p, uint4 v, uint64_t pol) {
+  asm volatile("st.global.L2::cache_hint.v4.b32 [%0], {%1, %2, %3, %4}, %5;"
+               ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "l"(pol) : "memory");
+}
 
 __device__ __forceinline__ double warp_sum_d(double a) {
 #pragma unroll
@@ -69,12 +101,26 @@ struct Seg {   // this warp's share of a row, in chunks of 8 elements
   int steps, res;      // steps of 32 chunks; the first `res` of them are shared-memory resident
 };
 
-// Visits this thread's chunks in step order: body(a, b, chunk, valid) with the packed student /
-// teacher words of the chunk.  Global (L2) chunks are fetched one step ahead.
+__device__ __forceinline__ float pow2f_exact(float n) {   // 2^n for whole n, clamped to the normal float range
+  const int i = (int)fminf(fmaxf(n, -126.f), 127.f);
+  return __uint_as_float((uint32_t)(127 + i) << 23);
+}
+
+// Visits this thread's chunks in step order: body(a, b, chunk, valid) -> bool (false = stop) with the
+// packed student / teacher words of the chunk.  Global (L2) chunks are fetched two steps ahead.
 template <typename Body>
 __device__ __forceinline__ void for_each_chunk(const Seg& sg, int lane, const uint4* res_s, const uint4* res_t,
-                                               const __nv_bfloat16* g_s, const __nv_bfloat16* g_t, Body&& body) {
+                                               const __nv_bfloat16* g_s, const __nv_bfloat16* g_t, uint64_t pol,
+                                               Body&& body) {
   const uint4 sent = make_uint4(0xFF7FFF7Fu, 0xFF7FFF7Fu, 0xFF7FFF7Fu, 0xFF7FFF7Fu);   // exp -> 0, difference 0
+  const int t0 = sg.c0 + sg.res * 32 + lane;       // this lane's first global chunk
+  uint4 a1 = sent, b1 = sent, a2 = sent, b2 = sent;
+  if (sg.steps > sg.res) {                           // start the first global fetches before the resident part
+    if (t0 < sg.c1) { a1 = ld_l2(g_s + (size_t)t0 * 8, pol); b1 = ld_l2(g_t + (size_t)t0 * 8, pol); }
+    if (sg.steps > sg.res + 1 && t0 + 32 < sg.c1) {
+      a2 = ld_l2(g_s + (size_t)(t0 + 32) * 8, pol); b2 = ld_l2(g_t + (size_t)(t0 + 32) * 8, pol);
+    }
+  }
 #pragma unroll
   for (int k = 0; k < KS_MAX; ++k) {
     if (k < sg.res) {
@@ -82,32 +128,38 @@ __device__ __forceinline__ void for_each_chunk(const Seg& sg, int lane, const ui
       const bool valid = c < sg.c1;
       uint4 a = sent, b = sent;
       if (valid) { a = res_s[k * 32 + lane]; b = res_t[k * 32 + lane]; }
-      body(a, b, c, valid);
+      if (!body(a, b, c, valid)) return;
     }
   }
-  if (sg.steps > sg.res) {
-    int c = sg.c0 + sg.res * 32 + lane;
-    uint4 na = sent, nb = sent;
-    if (c < sg.c1) { na = ld_l2(g_s + (size_t)c * 8); nb = ld_l2(g_t + (size_t)c * 8); }
-    for (int k = sg.res; k < sg.steps; ++k) {
-      const uint4 a = na, b = nb;
-      const int cc = c;
-      c += 32;
-      na = sent; nb = sent;
-      if (k + 1 < sg.steps && c < sg.c1) { na = ld_l2(g_s + (size_t)c * 8); nb = ld_l2(g_t + (size_t)c * 8); }
-      body(a, b, cc, cc < sg.c1);
-    }
+  int c = t0;
+  for (int k = sg.res; k < sg.steps; ++k) {
+    const uint4 a = a1, b = b1;
+    a1 = a2; b1 = b2; a2 = sent; b2 = sent;
+    const int cn = c + 64;
+    if (k + 2 < sg.steps && cn < sg.c1) { a2 = ld_l2(g_s + (size_t)cn * 8, pol); b2 = ld_l2(g_t + (size_t)cn * 8, pol); }
+    if (!body(a, b, c, c < sg.c1)) return;
+    c += 32;
   }
 }
 
+#ifdef SAKI_PHASE_TIMING
+#define RTS(i) do { const long long _n = clock64(); tacc[i] += _n - tlast; tlast = _n; } while (0)
+#else
+#define RTS(i) do { } while (0)
+#endif
+
 __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
   extern __shared__ __align__(128) unsigned char smem[];
+#ifdef SAKI_PHASE_TIMING
+  long long tacc[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+  long long tlast = clock64();
+  int t_rows = 0;
+#endif
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint4* res_s = reinterpret_cast<const uint4*>(smem + ROFF_S) + warp * RES_CHUNKS;
   const uint4* res_t = reinterpret_cast<const uint4*>(smem + ROFF_T) + warp * RES_CHUNKS;
   double* red = (double*)(smem + ROFF_RED);
   double* bc = (double*)(smem + ROFF_BC);
-  float* wmax = (float*)(smem + ROFF_WMAX);
   uint64_t* mbar = (uint64_t*)(smem + ROFF_MBAR);
 
   const int V = P.V;
@@ -127,6 +179,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
   Consts K;
   K.tau = (double)P.temperature; K.rtau = 1.0 / K.tau; K.eps = (double)P.eps; K.c64 = (double)c32;
   K.rc64 = 1.0 / K.c64; K.grad_scale = (double)P.grad_scale; K.sqrt_eps = sqrtf(P.eps); K.V = V;
+  const uint64_t pol_last = policy_evict_last(), pol_first = policy_evict_first();
 
   auto row_ptrs = [&](int64_t row, const __nv_bfloat16*& s, const __nv_bfloat16*& t) {
     const int64_t b = row / P.K1;
@@ -134,22 +187,18 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
     s = (const __nv_bfloat16*)P.s + b * P.s_seq + (int64_t)j * P.s_pos;
     t = (const __nv_bfloat16*)P.t + b * P.t_seq + (int64_t)j * P.t_pos;
   };
-  // lane 0 of each warp: fetch the warp's resident part of `row`, and pull the rest towards L2
+  // lane 0 of each warp: fetch the warp's resident part of `row` into shared memory
   auto issue = [&](int64_t row) {
     const __nv_bfloat16 *s, *t;
     row_ptrs(row, s, t);
     mbar_expect_tx(mbar, 2u * res_bytes);
     if (res_bytes) {
-      bulk_load((void*)res_s, s + (size_t)sg.c0 * 8, res_bytes, mbar);
-      bulk_load((void*)res_t, t + (size_t)sg.c0 * 8, res_bytes, mbar);
-    }
-    if (l2_bytes) {
-      prefetch_l2(s + (size_t)l2_first * 8, l2_bytes);
-      prefetch_l2(t + (size_t)l2_first * 8, l2_bytes);
+      bulk_load_hint((void*)res_s, s + (size_t)sg.c0 * 8, res_bytes, mbar, pol_first);
+      bulk_load_hint((void*)res_t, t + (size_t)sg.c0 * 8, res_bytes, mbar, pol_first);
     }
   };
-  // sum (or minimum, from component n_sum on) of n per-warp vectors: warp 0 ends up with the totals in v[]
-  auto combine = [&](double* v, int n, int n_sum) {
+  // n per-warp vectors -> red; after the barrier warp 0 holds in v[k] the sum over warps of component k
+  auto combine = [&](double* v, int n) {
     if (lane == 0) {
 #pragma unroll
       for (int k = 0; k < RNV; ++k) if (k < n) red[k * RW + warp] = v[k];
@@ -157,7 +206,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
     __syncthreads();
     if (warp == 0) {
 #pragma unroll
-      for (int k = 0; k < RNV; ++k) if (k < n) v[k] = (k < n_sum) ? warp_sum_d(red[k * RW + lane]) : warp_min_d(red[k * RW + lane]);
+      for (int k = 0; k < RNV; ++k) if (k < n) v[k] = warp_sum_d(lane < RW ? red[k * RW + lane] : 0.0);
     }
   };
 
@@ -181,32 +230,14 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
     row_ptrs(row, g_s, g_t);
     __nv_bfloat16* g_out = P.dlogits ? (__nv_bfloat16*)P.dlogits + row * P.ld_g : nullptr;
     const int64_t next_row = row + gridDim.x;
-    bool next_issued = false;
 
-    bool timed_out = dead;
-    if (!dead) {
-      if (!mbar_wait_bounded(mbar, phase)) timed_out = true;
-      else phase ^= 1u;
+    RTS(0);
+    // the part of the row that is not shared-memory resident: pull it towards L2 now; the passes
+    // start with the resident part, which gives these lines time to arrive
+    if (lane == 0 && l2_bytes) {
+      prefetch_l2(g_s + (size_t)l2_first * 8, l2_bytes, pol_last);
+      prefetch_l2(g_t + (size_t)l2_first * 8, l2_bytes, pol_last);
     }
-
-    // ------------------------------------------------ pass "max"
-    float my_mt;
-    {
-      uint32_t a = 0xFF7FFF7Fu, b = 0xFF7FFF7Fu;
-      for_each_chunk(sg, lane, res_s, res_t, g_s, g_t, [&](const uint4& s4, const uint4& t4, int, bool) {
-        a = max_bf16x2(max_bf16x2(a, max_bf16x2(s4.x, s4.y)), max_bf16x2(s4.z, s4.w));
-        b = max_bf16x2(max_bf16x2(b, max_bf16x2(t4.x, t4.y)), max_bf16x2(t4.z, t4.w));
-      });
-      const float2 fa = unpack_bf16x2(a), fb = unpack_bf16x2(b);
-      my_mt = fmaxf(fb.x, fb.y);
-      const float wa = warp_max_f(fmaxf(fa.x, fa.y)), wb = warp_max_f(my_mt);
-      if (lane == 0) { wmax[warp] = wa; wmax[RW + warp] = wb; }
-    }
-    const int any_timeout = __syncthreads_or(timed_out ? 1 : 0);
-    if (any_timeout) dead = true;
-    const float ms = warp_max_f(wmax[lane]), mt = warp_max_f(wmax[RW + lane]);
-    const float k0 = -ceilf(c32 * fmaxf(ms, -1e30f)), k1 = -ceilf(c32 * fmaxf(mt, -1e30f));   // shifts: arguments <= 0
-
     // row scalars that do not depend on the passes
     if (tid == 32) bc[BC_UACC] = scalar_uniform(P.seed, rid, STAGE_ACCEPT);
     if (tid == 64) bc[BC_UDRAW] = scalar_uniform(P.seed, rid, bonus ? STAGE_BONUS : STAGE_RESIDUAL);
@@ -215,29 +246,45 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       bc[BC_SX] = ok ? (double)__bfloat162float(g_s[x]) : 0.0;
       bc[BC_TX] = ok ? (double)__bfloat162float(g_t[x]) : 0.0;
     }
-
-    // teacher argmax: threads that saw the row maximum look for its lowest index
-    double cand = CUDART_INF;
-    if (my_mt == mt) {
-      for_each_chunk(sg, lane, res_s, res_t, g_s, g_t, [&](const uint4&, const uint4& t4, int c, bool valid) {
-        if (valid) {
-          const uint32_t w[4] = {t4.x, t4.y, t4.z, t4.w};
-#pragma unroll
-          for (int k = 3; k >= 0; --k) {
-            const float2 f = unpack_bf16x2(w[k]);
-            if (f.y == mt) cand = fmin(cand, (double)(c * 8 + 2 * k + 1));
-            if (f.x == mt) cand = fmin(cand, (double)(c * 8 + 2 * k));
-          }
-        }
-      });
+    if (!dead) {
+      if (!mbar_wait_bounded(mbar, phase)) dead = true;
+      else phase ^= 1u;
     }
+    RTS(1);
 
-    // ------------------------------------------------ pass "lse"
+    // ------------------------------------------------ pass "lse" (no separate maximum pass)
+    // Each thread sums under its own running shifts -ceil(c * running max): whole numbers, so that
+    // changing a shift, and later bringing all threads onto the row's shifts, multiplies the sums
+    // by exact powers of two.
     {
       float2 Ss = splat(0.f), St = splat(0.f), M1 = splat(0.f), M2 = splat(0.f), M3 = splat(0.f), N1 = splat(0.f);
-      const float2 cc = splat(c32), kk0 = splat(k0), kk1 = splat(k1), neg1 = splat(-1.f);
-      for_each_chunk(sg, lane, res_s, res_t, g_s, g_t, [&](const uint4& s4, const uint4& t4, int, bool) {
+      float ms_run = -CUDART_INF_F, mt_run = -CUDART_INF_F, ks = 1e30f, kt = 1e30f;
+      int my_arg = 0x7fffffff;                   // lowest index of this thread's teacher maximum
+      const float2 cc = splat(c32), neg1 = splat(-1.f);
+      for_each_chunk(sg, lane, res_s, res_t, g_s, g_t, pol_last, [&](const uint4& s4, const uint4& t4, int c, bool valid) {
         const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
+        const float2 cms = unpack_bf16x2(max_bf16x2(max_bf16x2(sw[0], sw[1]), max_bf16x2(sw[2], sw[3])));
+        const float2 cmt = unpack_bf16x2(max_bf16x2(max_bf16x2(tw[0], tw[1]), max_bf16x2(tw[2], tw[3])));
+        const float cm_s = fmaxf(cms.x, cms.y), cm_t = fmaxf(cmt.x, cmt.y);
+        if (valid && cm_s > ms_run) {
+          const float nk = -ceilf(c32 * fmaxf(cm_s, -1e30f));
+          const float2 f = splat(pow2f_exact(nk - ks));
+          Ss = __fmul2_rn(Ss, f); M1 = __fmul2_rn(M1, f); M2 = __fmul2_rn(M2, f); M3 = __fmul2_rn(M3, f);
+          ks = nk; ms_run = cm_s;
+        }
+        if (valid && cm_t > mt_run) {
+          const float nk = -ceilf(c32 * fmaxf(cm_t, -1e30f));
+          const float2 f = splat(pow2f_exact(nk - kt));
+          St = __fmul2_rn(St, f); N1 = __fmul2_rn(N1, f);
+          kt = nk; mt_run = cm_t;
+#pragma unroll
+          for (int i = 3; i >= 0; --i) {
+            const float2 f2 = unpack_bf16x2(tw[i]);
+            if (f2.y == cm_t) my_arg = c * 8 + 2 * i + 1;
+            if (f2.x == cm_t) my_arg = c * 8 + 2 * i;
+          }
+        }
+        const float2 kk0 = splat(ks), kk1 = splat(kt);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const float2 sf = unpack_bf16x2(sw[i]), tf = unpack_bf16x2(tw[i]);
@@ -253,21 +300,77 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           M3 = __ffma2_rn(t2, d, M3);
           N1 = __ffma2_rn(et, d, N1);
         }
+        return true;
       });
+      RTS(2);
+      // warp: common shifts (the smallest), teacher argmax, sums
+      float kws = ks, kwt = kt, wmt = mt_run;
+      int warg = my_arg;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        kws = fminf(kws, __shfl_xor_sync(0xffffffffu, kws, o));
+        kwt = fminf(kwt, __shfl_xor_sync(0xffffffffu, kwt, o));
+        const float om = __shfl_xor_sync(0xffffffffu, wmt, o);
+        const int oa = __shfl_xor_sync(0xffffffffu, warg, o);
+        if (om > wmt || (om == wmt && oa < warg)) { wmt = om; warg = oa; }
+      }
+      const double fs = (double)pow2f_exact(kws - ks), ft = (double)pow2f_exact(kwt - kt);
+      const bool has_s = ks < 1e29f, has_t = kt < 1e29f;
       auto tot = [](const float2 a) { return (double)a.x + (double)a.y; };
-      double v[7] = {warp_sum_d(tot(Ss)), warp_sum_d(tot(St)), warp_sum_d(tot(M1)), warp_sum_d(tot(M2)),
-                     warp_sum_d(tot(M3)), warp_sum_d(tot(N1)), warp_min_d(cand)};
-      combine(v, 7, 6);
-      if (tid == 0) scalar_after_lse(bc, v, K, k0, k1, x, bonus, masked, dead);
+      double v[6] = {has_s ? fs * tot(Ss) : 0.0, has_t ? ft * tot(St) : 0.0, has_s ? fs * tot(M1) : 0.0,
+                     has_s ? fs * tot(M2) : 0.0, has_s ? fs * tot(M3) : 0.0, has_t ? ft * tot(N1) : 0.0};
+#pragma unroll
+      for (int k = 0; k < 6; ++k) v[k] = warp_sum_d(v[k]);
+      if (lane == 0) {
+#pragma unroll
+        for (int k = 0; k < 6; ++k) red[k * RW + warp] = v[k];
+        red[6 * RW + warp] = (double)kws; red[7 * RW + warp] = (double)kwt;
+        float* wm = (float*)(smem + ROFF_WMAX);
+        wm[warp] = wmt; ((int*)wm)[RW + warp] = warg;
+      }
+      const int any_dead = __syncthreads_or(dead ? 1 : 0);
+      RTS(3);
+      if (warp == 0) {   // block: the row's shifts, argmax, sums
+        const int wl = lane < RW ? lane : 0;       // lanes beyond the warp count repeat warp 0 with zero weight
+        const double ksw = lane < RW ? red[6 * RW + wl] : 1e30, ktw = lane < RW ? red[7 * RW + wl] : 1e30;
+        double k0d = ksw, k1d = ktw;
+        const float* wm = (const float*)(smem + ROFF_WMAX);
+        float gmt = lane < RW ? wm[wl] : -CUDART_INF_F;
+        int garg = ((const int*)wm)[RW + wl];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          k0d = fmin(k0d, __shfl_xor_sync(0xffffffffu, k0d, o));
+          k1d = fmin(k1d, __shfl_xor_sync(0xffffffffu, k1d, o));
+          const float om = __shfl_xor_sync(0xffffffffu, gmt, o);
+          const int oa = __shfl_xor_sync(0xffffffffu, garg, o);
+          if (om > gmt || (om == gmt && oa < garg)) { gmt = om; garg = oa; }
+        }
+        const double fsw = ksw < 1e29 ? (double)pow2f_exact((float)(k0d - ksw)) : 0.0;
+        const double ftw = ktw < 1e29 ? (double)pow2f_exact((float)(k1d - ktw)) : 0.0;
+        double a[7];
+        a[0] = warp_sum_d(fsw * red[0 * RW + wl]); a[1] = warp_sum_d(ftw * red[1 * RW + wl]);
+        a[2] = warp_sum_d(fsw * red[2 * RW + wl]); a[3] = warp_sum_d(fsw * red[3 * RW + wl]);
+        a[4] = warp_sum_d(fsw * red[4 * RW + wl]); a[5] = warp_sum_d(ftw * red[5 * RW + wl]);
+        a[6] = (double)garg;
+        RTS(4);
+        if (lane == 0) {
+          bc[BC_K0] = k0d; bc[BC_K1] = k1d;
+          scalar_after_lse(bc, a, K, (float)k0d, (float)k1d, x, bonus, masked, any_dead != 0);
+        }
+      }
+      if (any_dead) dead = true;
+      RTS(5);
       __syncthreads();
     }
+    const float k0 = (float)bc[BC_K0], k1 = (float)bc[BC_K1];   // the row's shifts: exponent arguments <= 0
 
     // ------------------------------------------------ pass "solve" (repeated)
     while ((int)bc[BC_MODE] == MODE_SOLVE) {
+      RTS(6);
       const float cb = (float)bc[BC_CB], kb = (float)bc[BC_KB];
       float2 S0 = splat(0.f), S1 = splat(0.f), S2 = splat(0.f);
       const float2 cc = splat(c32), cbb = splat(cb), kbb = splat(kb), neg1 = splat(-1.f);
-      for_each_chunk(sg, lane, res_s, res_t, g_s, g_t, [&](const uint4& s4, const uint4& t4, int, bool) {
+      for_each_chunk(sg, lane, res_s, res_t, g_s, g_t, pol_last, [&](const uint4& s4, const uint4& t4, int, bool) {
         const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -279,11 +382,15 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           S1 = __fadd2_rn(S1, t1);
           S2 = __ffma2_rn(t1, d, S2);
         }
+        return true;
       });
+      RTS(7);
       auto tot = [](const float2 a) { return (double)a.x + (double)a.y; };
       double v[3] = {warp_sum_d(tot(S0)), warp_sum_d(tot(S1)), warp_sum_d(tot(S2))};
-      combine(v, 3, 3);
+      combine(v, 3);
+      RTS(8);
       if (tid == 0) scalar_after_solve(bc, v, K, k0, k1, x, bonus, masked);
+      RTS(9);
       __syncthreads();
     }
 
@@ -296,7 +403,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       if (g_out) {
         for (int k = 0; k < sg.steps; ++k) {
           const int c = sg.c0 + k * 32 + lane;
-          if (c < sg.c1) __stcs(reinterpret_cast<uint4*>(g_out + (size_t)c * 8), make_uint4(0, 0, 0, 0));
+          if (c < sg.c1) st_stream(g_out + (size_t)c * 8, make_uint4(0, 0, 0, 0), pol_first);
         }
       }
       __syncwarp();
@@ -309,20 +416,21 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
     }
 
     // ------------------------------------------------ pass "final"
+    RTS(10);
     const bool need_draw = bonus || bc[BC_CORR] != 0.0;
     const float cl = (float)bc[BC_CL], kq = (float)bc[BC_KQ];
     const float iq = (float)bc[BC_IQ], ip = (float)bc[BC_IP];
     const int tok = (int)bc[BC_TOK];
     const float KGf = (float)bc[BC_KG];
     const float kg = (float)(bc[BC_KG] * (double)ip);     // gradient entry = e_p * kg
-    float warp_part;   // this warp's ordered weight for the inverse-CDF draw
     {
       const bool want_g = (g_out != nullptr);
       float2 Sq = splat(0.f), R = splat(0.f);
       const float2 cc = splat(c32), cll = splat(cl), kqq = splat(kq), kk0 = splat(k0), neg1 = splat(-1.f);
       const float2 iqq = splat(iq), nip = splat(-ip), kgg = splat(kg);
       int n_res_done = 0;
-      for_each_chunk(sg, lane, res_s, res_t, g_s, g_t, [&](const uint4& s4, const uint4& t4, int c, bool valid) {
+      bool next_issued = false;
+      for_each_chunk(sg, lane, res_s, res_t, g_s, g_t, pol_last, [&](const uint4& s4, const uint4& t4, int c, bool valid) {
         const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
         uint32_t gp[4];
 #pragma unroll
@@ -348,7 +456,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           const uint32_t neu = (e & 1) ? ((old & 0x0000ffffu) | (g16 << 16)) : ((old & 0xffff0000u) | g16);
           if (wi == 0) gp[0] = neu; else if (wi == 1) gp[1] = neu; else if (wi == 2) gp[2] = neu; else gp[3] = neu;
         }
-        if (want_g && valid) __stcs(reinterpret_cast<uint4*>(g_out + (size_t)c * 8), make_uint4(gp[0], gp[1], gp[2], gp[3]));
+        if (want_g && valid) st_stream(g_out + (size_t)c * 8, make_uint4(gp[0], gp[1], gp[2], gp[3]), pol_first);
         // once the warp has read its resident part for the last time, the next row's may land there
         // (a row that still needs its draw re-reads the resident part: its copy is issued after the draw)
         if (++n_res_done == sg.res && !need_draw) {
@@ -359,20 +467,21 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           }
           next_issued = true;
         }
+        return true;
       });
       if (!next_issued && !need_draw && lane == 0 && !dead && next_row < P.n_rows) issue(next_row);   // no elements
+      RTS(11);
       const float sq_f = Sq.x + Sq.y, r_f = R.x + R.y;
       const double part = warp_sum_d((double)(bonus ? sq_f * iq : r_f));
-      warp_part = (float)part;
       double v[3] = {warp_sum_d((double)sq_f), warp_sum_d((double)r_f), part};
-      combine(v, 2, 2);
+      combine(v, 2);
+      RTS(12);
       if (lane == 0) red[2 * RW + warp] = part;     // ordered per-warp weights (read after the next barrier)
       if (tid == 0) {
         bc[BC_TV] = (bc[BC_LAMBDA] > 0.0) ? v[1] : 0.0;
         if (!need_draw) write_result(bc, P.out, !P.spec, row, 0, x, false, K.c64, g_s, g_t);
       }
     }
-    (void)warp_part;
 
     // ------------------------------------------------ the draw (corrected and bonus rows only)
     if (need_draw) {
@@ -385,8 +494,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
         double running = bc[BC_BEFORE];
         int y = -1, last_pos = -1;
         const float2 cc = splat(c32), cll = splat(cl), kqq = splat(kq), kk0 = splat(k0), neg1 = splat(-1.f);
-        for_each_chunk(sg, lane, res_s, res_t, g_s, g_t, [&](const uint4& s4, const uint4& t4, int c, bool valid) {
-          if (y >= 0) return;
+        for_each_chunk(sg, lane, res_s, res_t, g_s, g_t, pol_last, [&](const uint4& s4, const uint4& t4, int c, bool valid) {
           const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
           float w[8];
 #pragma unroll
@@ -429,6 +537,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           if (hit) y = __shfl_sync(0xffffffffu, found, __ffs(hit) - 1);
           if (posm) last_pos = __shfl_sync(0xffffffffu, lastp, 31 - __clz(posm));
           running += __shfl_sync(0xffffffffu, inc, 31);
+          return y < 0;                                   // stop at the crossing
         });
         if (y < 0) y = (last_pos >= 0) ? last_pos : min(V - 1, sg.c1 * 8 - 1);
         if (lane == 0) write_result(bc, P.out, !P.spec, row, bonus ? 0 : 1, y, bonus, K.c64, g_s, g_t);
@@ -439,9 +548,19 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
         issue(next_row);
       }
     }
+    RTS(13);
     __syncthreads();   // the broadcast area and the partial-sum area are rewritten by the next row
   }
 
+#ifdef SAKI_PHASE_TIMING
+  for (int64_t row = blockIdx.x; row < P.n_rows; row += gridDim.x) ++t_rows;
+  if ((tid == 0 || tid == 1023) && (blockIdx.x == 0 || blockIdx.x == 77) && t_rows > 0)
+    printf("blk %d tid %d rows %d | endbar %lld copy-wait %lld | lse %lld warp+bar %lld gather %lld scalar %lld | "
+           "bar %lld solve %lld combine %lld scalar %lld | bar %lld final %lld combine %lld tail %lld (cycles per row)\n",
+           (int)blockIdx.x, tid, t_rows, tacc[0] / t_rows, tacc[1] / t_rows, tacc[2] / t_rows, tacc[3] / t_rows,
+           tacc[4] / t_rows, tacc[5] / t_rows, tacc[6] / t_rows, tacc[7] / t_rows, tacc[8] / t_rows, tacc[9] / t_rows,
+           tacc[10] / t_rows, tacc[11] / t_rows, tacc[12] / t_rows, tacc[13] / t_rows);
+#endif
   // a CTA that gave up on a copy still waits (bounded) for what it has in flight before leaving
   if (dead && tid == 0) (void)mbar_wait_bounded(mbar, phase);
 }
