@@ -268,17 +268,17 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
 #pragma unroll
       for (int i = 0; i < NPAIR; ++i) {
         const float2 sf = unpack_fresh(sr[i]), tf = unpack_fresh(tr[i]);
-        const float2 d = __ffma2_rn(sf, neg1, tf);
-        const float2 es = ex2f2(__ffma2_rn(sf, cc, kk0));
-        const float2 et = ex2f2(__ffma2_rn(tf, cc, kk1));
-        Ss = __fadd2_rn(Ss, es);
-        St = __fadd2_rn(St, et);
-        const float2 t1 = __fmul2_rn(es, d);
-        M1 = __fadd2_rn(M1, t1);
-        const float2 t2 = __fmul2_rn(t1, d);
-        M2 = __fadd2_rn(M2, t2);
-        M3 = __ffma2_rn(t2, d, M3);
-        N1 = __ffma2_rn(et, d, N1);
+        const float2 d = ffma2(sf, neg1, tf);
+        const float2 es = ex2f2(ffma2(sf, cc, kk0));
+        const float2 et = ex2f2(ffma2(tf, cc, kk1));
+        Ss = fadd2(Ss, es);
+        St = fadd2(St, et);
+        const float2 t1 = fmul2(es, d);
+        M1 = fadd2(M1, t1);
+        const float2 t2 = fmul2(t1, d);
+        M2 = fadd2(M2, t2);
+        M3 = ffma2(t2, d, M3);
+        N1 = ffma2(et, d, N1);
       }
       // the row's maxima have arrived meanwhile: move the partial sums onto the row's shifts
       TS(4);
@@ -333,12 +333,12 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
       for (int i = 0; i < NPAIR; ++i) {
         const int h = i & 1;
         const float2 sf = unpack_fresh(sr[i]), tf = unpack_fresh(tr[i]);
-        const float2 d = __ffma2_rn(sf, neg1, tf);
-        const float2 e = ex2f2(__ffma2_rn(d, cbb, __ffma2_rn(sf, cc, kbb)));
-        S0[h] = __fadd2_rn(S0[h], e);
-        const float2 t1 = __fmul2_rn(e, d);
-        S1[h] = __fadd2_rn(S1[h], t1);
-        S2[h] = __ffma2_rn(t1, d, S2[h]);
+        const float2 d = ffma2(sf, neg1, tf);
+        const float2 e = ex2f2(ffma2(d, cbb, ffma2(sf, cc, kbb)));
+        S0[h] = fadd2(S0[h], e);
+        const float2 t1 = fmul2(e, d);
+        S1[h] = fadd2(S1[h], t1);
+        S2[h] = ffma2(t1, d, S2[h]);
       }
       auto tot = [](const float2 (&a)[2]) { return ((double)a[0].x + (double)a[0].y) + ((double)a[1].x + (double)a[1].y); };
       TS(9);
@@ -403,14 +403,14 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
         for (int k = 0; k < 4; ++k) {
           const int i = 4 * j + k, h = k & 1;
           const float2 sf = unpack_fresh(sr[i]), tf = unpack_fresh(tr[i]);
-          const float2 d = __ffma2_rn(sf, neg1, tf);
-          const float2 ep = ex2f2(__ffma2_rn(sf, cc, kk0));
-          const float2 eq = ex2f2(__ffma2_rn(d, cll, __ffma2_rn(sf, cc, kqq)));
-          Sq[h] = __fadd2_rn(Sq[h], eq);
-          float2 r = __ffma2_rn(eq, iqq, __fmul2_rn(ep, nip));     // q_i - p_i
+          const float2 d = ffma2(sf, neg1, tf);
+          const float2 ep = ex2f2(ffma2(sf, cc, kk0));
+          const float2 eq = ex2f2(ffma2(d, cll, ffma2(sf, cc, kqq)));
+          Sq[h] = fadd2(Sq[h], eq);
+          float2 r = ffma2(eq, iqq, fmul2(ep, nip));     // q_i - p_i
           r.x = fmaxf(r.x, 0.f); r.y = fmaxf(r.y, 0.f);
-          R[h] = __fadd2_rn(R[h], r);
-          const float2 gv = __fmul2_rn(ep, kgg);
+          R[h] = fadd2(R[h], r);
+          const float2 gv = fmul2(ep, kgg);
           gp[k] = pack_bf16x2(gv.x, gv.y);
         }
         if (want_g) {

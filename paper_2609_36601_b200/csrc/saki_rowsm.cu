@@ -33,7 +33,7 @@
 namespace saki {
 
 #ifndef SAKI_ROWSM_THREADS
-#define SAKI_ROWSM_THREADS 1024
+#define SAKI_ROWSM_THREADS 512
 #endif
 constexpr int RT = SAKI_ROWSM_THREADS;  // threads per CTA
 constexpr int RW = RT / 32;             // warps per CTA
@@ -44,8 +44,9 @@ constexpr int RNV = 8;                  // doubles per partial vector
 constexpr int ROFF_S = 0;                                        // [RW][RES_CHUNKS] uint4
 constexpr int ROFF_T = RW * RES_CHUNKS * 16;
 constexpr int ROFF_RED = 2 * RW * RES_CHUNKS * 16;               // [RNV][RW] doubles
-constexpr int ROFF_BC = ROFF_RED + RNV * RW * 8;                 // [BC_DOUBLES] doubles
-constexpr int ROFF_WMAX = ROFF_BC + BC_DOUBLES * 8;              // [2][RW] floats
+constexpr int ROFF_GAT = ROFF_RED + RNV * RW * 8;                // [16] doubles: block totals
+constexpr int ROFF_BC = ROFF_GAT + 16 * 8;                       // [2][BC_DOUBLES] doubles, alternating by row
+constexpr int ROFF_WMAX = ROFF_BC + 2 * BC_DOUBLES * 8;          // [2][RW] floats
 constexpr int ROFF_MBAR = ROFF_WMAX + 2 * RW * 4;
 constexpr int RSMEM_BYTES = ROFF_MBAR + 16;
 
@@ -106,25 +107,45 @@ __device__ __forceinline__ float pow2f_exact(float n) {   // 2^n for whole n, cl
   return __uint_as_float((uint32_t)(127 + i) << 23);
 }
 
+constexpr int LOOKAHEAD = 2;            // global (L2) chunks in flight per thread
+constexpr int PF_STEPS = 8;             // first touch of a row: lines are requested this many steps ahead
+
+__device__ __forceinline__ void prefetch_line_l2(const void* p) {
+  asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+}
+
 // Visits this thread's chunks in step order: body(a, b, chunk, valid) -> bool (false = stop) with the
-// packed student / teacher words of the chunk.  Global (L2) chunks are fetched two steps ahead.
-template <typename Body>
+// packed student / teacher words of the chunk.  Global (L2) chunks are fetched LOOKAHEAD steps ahead,
+// the first ones before the resident part is processed.  FIRST_TOUCH: the row has not been read yet,
+// so its global part is additionally requested into L2 PF_STEPS steps ahead (one lane per 128-byte line).
+template <bool FIRST_TOUCH, typename Body>
 __device__ __forceinline__ void for_each_chunk(const Seg& sg, int lane, const uint4* res_s, const uint4* res_t,
                                                const __nv_bfloat16* g_s, const __nv_bfloat16* g_t, uint64_t pol,
                                                Body&& body) {
   const uint4 sent = make_uint4(0xFF7FFF7Fu, 0xFF7FFF7Fu, 0xFF7FFF7Fu, 0xFF7FFF7Fu);   // exp -> 0, difference 0
   const int t0 = sg.c0 + sg.res * 32 + lane;       // this lane's first global chunk
-  uint4 a1 = sent, b1 = sent, a2 = sent, b2 = sent;
-  if (sg.steps > sg.res) {                           // start the first global fetches before the resident part
-    if (t0 < sg.c1) { a1 = ld_l2(g_s + (size_t)t0 * 8, pol); b1 = ld_l2(g_t + (size_t)t0 * 8, pol); }
-    if (sg.steps > sg.res + 1 && t0 + 32 < sg.c1) {
-      a2 = ld_l2(g_s + (size_t)(t0 + 32) * 8, pol); b2 = ld_l2(g_t + (size_t)(t0 + 32) * 8, pol);
+  if (FIRST_TOUCH && (lane & 7) == 0) {
+#pragma unroll
+    for (int j = LOOKAHEAD; j < PF_STEPS; ++j) {
+      const int c = t0 + 32 * j;
+      if (c < sg.c1) { prefetch_line_l2(g_s + (size_t)c * 8); prefetch_line_l2(g_t + (size_t)c * 8); }
     }
   }
+  uint4 qa[LOOKAHEAD], qb[LOOKAHEAD];
 #pragma unroll
-  for (int k = 0; k < KS_MAX; ++k) {
-    if (k < sg.res) {
-      const int c = sg.c0 + k * 32 + lane;
+  for (int j = 0; j < LOOKAHEAD; ++j) {
+    qa[j] = sent; qb[j] = sent;
+    const int c = t0 + 32 * j;
+    if (c < sg.c1) { qa[j] = ld_l2(g_s + (size_t)c * 8, pol); qb[j] = ld_l2(g_t + (size_t)c * 8, pol); }
+  }
+  // resident part; kept rolled: the pass bodies are large and must stay in the instruction cache
+  const int full = (sg.c1 - sg.c0) >> 5;           // steps in which every lane has a chunk
+#pragma unroll 1
+  for (int k = 0; k < sg.res; ++k) {
+    const int c = sg.c0 + k * 32 + lane;
+    if (k < full) {
+      if (!body(res_s[k * 32 + lane], res_t[k * 32 + lane], c, true)) return;
+    } else {
       const bool valid = c < sg.c1;
       uint4 a = sent, b = sent;
       if (valid) { a = res_s[k * 32 + lane]; b = res_t[k * 32 + lane]; }
@@ -132,13 +153,23 @@ __device__ __forceinline__ void for_each_chunk(const Seg& sg, int lane, const ui
     }
   }
   int c = t0;
-  for (int k = sg.res; k < sg.steps; ++k) {
-    const uint4 a = a1, b = b1;
-    a1 = a2; b1 = b2; a2 = sent; b2 = sent;
-    const int cn = c + 64;
-    if (k + 2 < sg.steps && cn < sg.c1) { a2 = ld_l2(g_s + (size_t)cn * 8, pol); b2 = ld_l2(g_t + (size_t)cn * 8, pol); }
-    if (!body(a, b, c, c < sg.c1)) return;
-    c += 32;
+#pragma unroll 1
+  for (int k = sg.res; k < sg.steps; k += LOOKAHEAD) {
+#pragma unroll
+    for (int j = 0; j < LOOKAHEAD; ++j) {
+      if (k + j < sg.steps) {
+        const uint4 a = qa[j], b = qb[j];
+        const int cn = c + 32 * LOOKAHEAD;
+        qa[j] = sent; qb[j] = sent;
+        if (cn < sg.c1) { qa[j] = ld_l2(g_s + (size_t)cn * 8, pol); qb[j] = ld_l2(g_t + (size_t)cn * 8, pol); }
+        if (FIRST_TOUCH && (lane & 7) == 0) {
+          const int cp = c + 32 * PF_STEPS;
+          if (cp < sg.c1) { prefetch_line_l2(g_s + (size_t)cp * 8); prefetch_line_l2(g_t + (size_t)cp * 8); }
+        }
+        if (!body(a, b, c, c < sg.c1)) return;
+        c += 32;
+      }
+    }
   }
 }
 
@@ -159,7 +190,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
   const uint4* res_s = reinterpret_cast<const uint4*>(smem + ROFF_S) + warp * RES_CHUNKS;
   const uint4* res_t = reinterpret_cast<const uint4*>(smem + ROFF_T) + warp * RES_CHUNKS;
   double* red = (double*)(smem + ROFF_RED);
-  double* bc = (double*)(smem + ROFF_BC);
+  double* gat = (double*)(smem + ROFF_GAT);
   uint64_t* mbar = (uint64_t*)(smem + ROFF_MBAR);
 
   const int V = P.V;
@@ -197,17 +228,19 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       bulk_load_hint((void*)res_t, t + (size_t)sg.c0 * 8, res_bytes, mbar, pol_first);
     }
   };
-  // n per-warp vectors -> red; after the barrier warp 0 holds in v[k] the sum over warps of component k
-  auto combine = [&](double* v, int n) {
+  // n per-warp vectors -> gat[k] = sum over warps of component k; warp k adds up component k, so the
+  // serial part after the barrier is one shuffle tree deep
+  auto combine = [&](const double* v, int n) {
     if (lane == 0) {
 #pragma unroll
       for (int k = 0; k < RNV; ++k) if (k < n) red[k * RW + warp] = v[k];
     }
     __syncthreads();
-    if (warp == 0) {
-#pragma unroll
-      for (int k = 0; k < RNV; ++k) if (k < n) v[k] = warp_sum_d(lane < RW ? red[k * RW + lane] : 0.0);
+    if (warp < n) {
+      const double a = warp_sum_d(lane < RW ? red[warp * RW + lane] : 0.0);
+      if (lane == 0) gat[warp] = a;
     }
+    __syncthreads();
   };
 
   if (tid == 0) {
@@ -218,8 +251,10 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
   if (lane == 0 && (int64_t)blockIdx.x < P.n_rows) issue(blockIdx.x);
   uint32_t phase = 0;
   bool dead = false;
+  int rb = 0;
 
-  for (int64_t row = blockIdx.x; row < P.n_rows; row += gridDim.x) {
+  for (int64_t row = blockIdx.x; row < P.n_rows; row += gridDim.x, rb ^= 1) {
+    double* bc = (double*)(smem + ROFF_BC) + rb * BC_DOUBLES;   // this row's broadcast scalars
     const uint64_t rid = P.row_offset + (uint64_t)row;
     const int64_t seq = row / P.K1;
     const int pos = (int)(row - seq * P.K1);
@@ -232,12 +267,6 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
     const int64_t next_row = row + gridDim.x;
 
     RTS(0);
-    // the part of the row that is not shared-memory resident: pull it towards L2 now; the passes
-    // start with the resident part, which gives these lines time to arrive
-    if (lane == 0 && l2_bytes) {
-      prefetch_l2(g_s + (size_t)l2_first * 8, l2_bytes, pol_last);
-      prefetch_l2(g_t + (size_t)l2_first * 8, l2_bytes, pol_last);
-    }
     // row scalars that do not depend on the passes
     if (tid == 32) bc[BC_UACC] = scalar_uniform(P.seed, rid, STAGE_ACCEPT);
     if (tid == 64) bc[BC_UDRAW] = scalar_uniform(P.seed, rid, bonus ? STAGE_BONUS : STAGE_RESIDUAL);
@@ -261,7 +290,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       float ms_run = -CUDART_INF_F, mt_run = -CUDART_INF_F, ks = 1e30f, kt = 1e30f;
       int my_arg = 0x7fffffff;                   // lowest index of this thread's teacher maximum
       const float2 cc = splat(c32), neg1 = splat(-1.f);
-      for_each_chunk(sg, lane, res_s, res_t, g_s, g_t, pol_last, [&](const uint4& s4, const uint4& t4, int c, bool valid) {
+      for_each_chunk<true>(sg, lane, res_s, res_t, g_s, g_t, pol_last, [&](const uint4& s4, const uint4& t4, int c, bool valid) {
         const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
         const float2 cms = unpack_bf16x2(max_bf16x2(max_bf16x2(sw[0], sw[1]), max_bf16x2(sw[2], sw[3])));
         const float2 cmt = unpack_bf16x2(max_bf16x2(max_bf16x2(tw[0], tw[1]), max_bf16x2(tw[2], tw[3])));
@@ -269,13 +298,13 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
         if (valid && cm_s > ms_run) {
           const float nk = -ceilf(c32 * fmaxf(cm_s, -1e30f));
           const float2 f = splat(pow2f_exact(nk - ks));
-          Ss = __fmul2_rn(Ss, f); M1 = __fmul2_rn(M1, f); M2 = __fmul2_rn(M2, f); M3 = __fmul2_rn(M3, f);
+          Ss = fmul2(Ss, f); M1 = fmul2(M1, f); M2 = fmul2(M2, f); M3 = fmul2(M3, f);
           ks = nk; ms_run = cm_s;
         }
         if (valid && cm_t > mt_run) {
           const float nk = -ceilf(c32 * fmaxf(cm_t, -1e30f));
           const float2 f = splat(pow2f_exact(nk - kt));
-          St = __fmul2_rn(St, f); N1 = __fmul2_rn(N1, f);
+          St = fmul2(St, f); N1 = fmul2(N1, f);
           kt = nk; mt_run = cm_t;
 #pragma unroll
           for (int i = 3; i >= 0; --i) {
@@ -288,17 +317,17 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const float2 sf = unpack_bf16x2(sw[i]), tf = unpack_bf16x2(tw[i]);
-          const float2 d = __ffma2_rn(sf, neg1, tf);
-          const float2 es = ex2f2(__ffma2_rn(sf, cc, kk0));
-          const float2 et = ex2f2(__ffma2_rn(tf, cc, kk1));
-          Ss = __fadd2_rn(Ss, es);
-          St = __fadd2_rn(St, et);
-          const float2 t1 = __fmul2_rn(es, d);
-          M1 = __fadd2_rn(M1, t1);
-          const float2 t2 = __fmul2_rn(t1, d);
-          M2 = __fadd2_rn(M2, t2);
-          M3 = __ffma2_rn(t2, d, M3);
-          N1 = __ffma2_rn(et, d, N1);
+          const float2 d = ffma2(sf, neg1, tf);
+          const float2 es = ex2f2(ffma2(sf, cc, kk0));
+          const float2 et = ex2f2(ffma2(tf, cc, kk1));
+          Ss = fadd2(Ss, es);
+          St = fadd2(St, et);
+          const float2 t1 = fmul2(es, d);
+          M1 = fadd2(M1, t1);
+          const float2 t2 = fmul2(t1, d);
+          M2 = fadd2(M2, t2);
+          M3 = ffma2(t2, d, M3);
+          N1 = ffma2(et, d, N1);
         }
         return true;
       });
@@ -330,35 +359,41 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       }
       const int any_dead = __syncthreads_or(dead ? 1 : 0);
       RTS(3);
-      if (warp == 0) {   // block: the row's shifts, argmax, sums
-        const int wl = lane < RW ? lane : 0;       // lanes beyond the warp count repeat warp 0 with zero weight
+      if (warp < 7) {   // block level: warps 0-5 add up one sum each on the row's shifts, warp 6 finds the argmax
+        const int wl = lane < RW ? lane : 0;       // lanes beyond the warp count carry zero weight
         const double ksw = lane < RW ? red[6 * RW + wl] : 1e30, ktw = lane < RW ? red[7 * RW + wl] : 1e30;
         double k0d = ksw, k1d = ktw;
-        const float* wm = (const float*)(smem + ROFF_WMAX);
-        float gmt = lane < RW ? wm[wl] : -CUDART_INF_F;
-        int garg = ((const int*)wm)[RW + wl];
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
           k0d = fmin(k0d, __shfl_xor_sync(0xffffffffu, k0d, o));
           k1d = fmin(k1d, __shfl_xor_sync(0xffffffffu, k1d, o));
-          const float om = __shfl_xor_sync(0xffffffffu, gmt, o);
-          const int oa = __shfl_xor_sync(0xffffffffu, garg, o);
-          if (om > gmt || (om == gmt && oa < garg)) { gmt = om; garg = oa; }
         }
-        const double fsw = ksw < 1e29 ? (double)pow2f_exact((float)(k0d - ksw)) : 0.0;
-        const double ftw = ktw < 1e29 ? (double)pow2f_exact((float)(k1d - ktw)) : 0.0;
-        double a[7];
-        a[0] = warp_sum_d(fsw * red[0 * RW + wl]); a[1] = warp_sum_d(ftw * red[1 * RW + wl]);
-        a[2] = warp_sum_d(fsw * red[2 * RW + wl]); a[3] = warp_sum_d(fsw * red[3 * RW + wl]);
-        a[4] = warp_sum_d(fsw * red[4 * RW + wl]); a[5] = warp_sum_d(ftw * red[5 * RW + wl]);
-        a[6] = (double)garg;
-        RTS(4);
-        if (lane == 0) {
-          bc[BC_K0] = k0d; bc[BC_K1] = k1d;
-          scalar_after_lse(bc, a, K, (float)k0d, (float)k1d, x, bonus, masked, any_dead != 0);
+        if (warp < 6) {
+          const bool teacher = (warp == 1 || warp == 5);
+          const double kw = teacher ? ktw : ksw, kr = teacher ? k1d : k0d;
+          const double f = kw < 1e29 ? (double)pow2f_exact((float)(kr - kw)) : 0.0;
+          const double a = warp_sum_d(f * red[warp * RW + wl]);
+          if (lane == 0) { gat[warp] = a; if (warp == 0) { gat[7] = k0d; gat[8] = k1d; } }
+        } else {
+          const float* wm = (const float*)(smem + ROFF_WMAX);
+          float gmt = lane < RW ? wm[wl] : -CUDART_INF_F;
+          int garg = ((const int*)wm)[RW + wl];
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            const float om = __shfl_xor_sync(0xffffffffu, gmt, o);
+            const int oa = __shfl_xor_sync(0xffffffffu, garg, o);
+            if (om > gmt || (om == gmt && oa < garg)) { gmt = om; garg = oa; }
+          }
+          if (lane == 0) gat[6] = (double)garg;
         }
       }
       if (any_dead) dead = true;
+      __syncthreads();
+      RTS(4);
+      if (tid == 0) {
+        bc[BC_K0] = gat[7]; bc[BC_K1] = gat[8];
+        scalar_after_lse(bc, gat, K, (float)gat[7], (float)gat[8], x, bonus, masked, any_dead != 0);
+      }
       RTS(5);
       __syncthreads();
     }
@@ -370,26 +405,26 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       const float cb = (float)bc[BC_CB], kb = (float)bc[BC_KB];
       float2 S0 = splat(0.f), S1 = splat(0.f), S2 = splat(0.f);
       const float2 cc = splat(c32), cbb = splat(cb), kbb = splat(kb), neg1 = splat(-1.f);
-      for_each_chunk(sg, lane, res_s, res_t, g_s, g_t, pol_last, [&](const uint4& s4, const uint4& t4, int, bool) {
+      for_each_chunk<false>(sg, lane, res_s, res_t, g_s, g_t, pol_last, [&](const uint4& s4, const uint4& t4, int, bool) {
         const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const float2 sf = unpack_bf16x2(sw[i]), tf = unpack_bf16x2(tw[i]);
-          const float2 d = __ffma2_rn(sf, neg1, tf);
-          const float2 e = ex2f2(__ffma2_rn(d, cbb, __ffma2_rn(sf, cc, kbb)));
-          S0 = __fadd2_rn(S0, e);
-          const float2 t1 = __fmul2_rn(e, d);
-          S1 = __fadd2_rn(S1, t1);
-          S2 = __ffma2_rn(t1, d, S2);
+          const float2 d = ffma2(sf, neg1, tf);
+          const float2 e = ex2f2(ffma2(d, cbb, ffma2(sf, cc, kbb)));
+          S0 = fadd2(S0, e);
+          const float2 t1 = fmul2(e, d);
+          S1 = fadd2(S1, t1);
+          S2 = ffma2(t1, d, S2);
         }
         return true;
       });
       RTS(7);
       auto tot = [](const float2 a) { return (double)a.x + (double)a.y; };
-      double v[3] = {warp_sum_d(tot(S0)), warp_sum_d(tot(S1)), warp_sum_d(tot(S2))};
+      const double v[3] = {warp_sum_d(tot(S0)), warp_sum_d(tot(S1)), warp_sum_d(tot(S2))};
       combine(v, 3);
       RTS(8);
-      if (tid == 0) scalar_after_solve(bc, v, K, k0, k1, x, bonus, masked);
+      if (tid == 0) scalar_after_solve(bc, gat, K, k0, k1, x, bonus, masked);
       RTS(9);
       __syncthreads();
     }
@@ -411,7 +446,6 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         issue(next_row);
       }
-      __syncthreads();   // the broadcast area is rewritten by the next row
       continue;
     }
 
@@ -430,20 +464,20 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       const float2 iqq = splat(iq), nip = splat(-ip), kgg = splat(kg);
       int n_res_done = 0;
       bool next_issued = false;
-      for_each_chunk(sg, lane, res_s, res_t, g_s, g_t, pol_last, [&](const uint4& s4, const uint4& t4, int c, bool valid) {
+      for_each_chunk<false>(sg, lane, res_s, res_t, g_s, g_t, pol_last, [&](const uint4& s4, const uint4& t4, int c, bool valid) {
         const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
         uint32_t gp[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const float2 sf = unpack_bf16x2(sw[i]), tf = unpack_bf16x2(tw[i]);
-          const float2 d = __ffma2_rn(sf, neg1, tf);
-          const float2 ep = ex2f2(__ffma2_rn(sf, cc, kk0));
-          const float2 eq = ex2f2(__ffma2_rn(d, cll, __ffma2_rn(sf, cc, kqq)));
-          Sq = __fadd2_rn(Sq, eq);
-          float2 r = __ffma2_rn(eq, iqq, __fmul2_rn(ep, nip));     // q_i - p_i
+          const float2 d = ffma2(sf, neg1, tf);
+          const float2 ep = ex2f2(ffma2(sf, cc, kk0));
+          const float2 eq = ex2f2(ffma2(d, cll, ffma2(sf, cc, kqq)));
+          Sq = fadd2(Sq, eq);
+          float2 r = ffma2(eq, iqq, fmul2(ep, nip));     // q_i - p_i
           r.x = fmaxf(r.x, 0.f); r.y = fmaxf(r.y, 0.f);
-          R = __fadd2_rn(R, r);
-          const float2 gv = __fmul2_rn(ep, kgg);
+          R = fadd2(R, r);
+          const float2 gv = fmul2(ep, kgg);
           gp[i] = pack_bf16x2(gv.x, gv.y);
         }
         if ((tok >> 3) == c && tok >= 0) {   // the supervised token is in this chunk: subtract the one-hot part
@@ -473,19 +507,18 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       RTS(11);
       const float sq_f = Sq.x + Sq.y, r_f = R.x + R.y;
       const double part = warp_sum_d((double)(bonus ? sq_f * iq : r_f));
-      double v[3] = {warp_sum_d((double)sq_f), warp_sum_d((double)r_f), part};
+      const double v[3] = {warp_sum_d((double)sq_f), warp_sum_d((double)r_f), part};
+      if (lane == 0) red[2 * RW + warp] = part;     // ordered per-warp weights of the draw
       combine(v, 2);
       RTS(12);
-      if (lane == 0) red[2 * RW + warp] = part;     // ordered per-warp weights (read after the next barrier)
       if (tid == 0) {
-        bc[BC_TV] = (bc[BC_LAMBDA] > 0.0) ? v[1] : 0.0;
+        bc[BC_TV] = (bc[BC_LAMBDA] > 0.0) ? gat[1] : 0.0;
         if (!need_draw) write_result(bc, P.out, !P.spec, row, 0, x, false, K.c64, g_s, g_t);
       }
     }
 
     // ------------------------------------------------ the draw (corrected and bonus rows only)
     if (need_draw) {
-      __syncthreads();
       if (tid == 0) scalar_find_owner(bc, red + 2 * RW, RW);
       __syncthreads();
       if (warp == (int)bc[BC_OWNER_WARP]) {
@@ -494,15 +527,15 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
         double running = bc[BC_BEFORE];
         int y = -1, last_pos = -1;
         const float2 cc = splat(c32), cll = splat(cl), kqq = splat(kq), kk0 = splat(k0), neg1 = splat(-1.f);
-        for_each_chunk(sg, lane, res_s, res_t, g_s, g_t, pol_last, [&](const uint4& s4, const uint4& t4, int c, bool valid) {
+        for_each_chunk<false>(sg, lane, res_s, res_t, g_s, g_t, pol_last, [&](const uint4& s4, const uint4& t4, int c, bool valid) {
           const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
           float w[8];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const float2 sf = unpack_bf16x2(sw[i]), tf = unpack_bf16x2(tw[i]);
-            const float2 d = __ffma2_rn(sf, neg1, tf);
-            const float2 ep = ex2f2(__ffma2_rn(sf, cc, kk0));
-            const float2 eq = ex2f2(__ffma2_rn(d, cll, __ffma2_rn(sf, cc, kqq)));
+            const float2 d = ffma2(sf, neg1, tf);
+            const float2 ep = ex2f2(ffma2(sf, cc, kk0));
+            const float2 eq = ex2f2(ffma2(d, cll, ffma2(sf, cc, kqq)));
             w[2 * i] = bonus ? eq.x * iq : fmaxf(fmaf(eq.x, iq, -(ep.x * ip)), 0.f);
             w[2 * i + 1] = bonus ? eq.y * iq : fmaxf(fmaf(eq.y, iq, -(ep.y * ip)), 0.f);
           }
@@ -549,7 +582,8 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       }
     }
     RTS(13);
-    __syncthreads();   // the broadcast area and the partial-sum area are rewritten by the next row
+    // no barrier here: the next row uses the other broadcast buffer, and every other shared area is
+    // rewritten only after the next row's first block barrier
   }
 
 #ifdef SAKI_PHASE_TIMING
