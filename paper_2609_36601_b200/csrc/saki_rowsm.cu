@@ -37,7 +37,8 @@ namespace saki {
 #endif
 constexpr int RT = SAKI_ROWSM_THREADS;  // threads per CTA
 constexpr int RW = RT / 32;             // warps per CTA
-constexpr int KS_MAX = 6 * (1024 / RT);   // resident steps per warp (a step = 32 chunks of 8 elements)
+constexpr int KS_MAX = RT == 512 ? 13 : 6;  // resident steps per warp (a step = 32 chunks of 8 elements)
+constexpr int MAX_STEPS = 64;            // steps per warp the draw bookkeeping can hold (V <= 64*32*8*RW)
 constexpr int RES_CHUNKS = KS_MAX * 32; // resident chunks per warp and row
 constexpr int RNV = 8;                  // doubles per partial vector
 
@@ -47,7 +48,8 @@ constexpr int ROFF_RED = 2 * RW * RES_CHUNKS * 16;               // [RNV][RW] do
 constexpr int ROFF_GAT = ROFF_RED + RNV * RW * 8;                // [16] doubles: block totals
 constexpr int ROFF_BC = ROFF_GAT + 16 * 8;                       // [2][BC_DOUBLES] doubles, alternating by row
 constexpr int ROFF_WMAX = ROFF_BC + 2 * BC_DOUBLES * 8;          // [2][RW] floats
-constexpr int ROFF_MBAR = ROFF_WMAX + 2 * RW * 4;
+constexpr int ROFF_STEP = ROFF_WMAX + 2 * RW * 4;                // [RW][MAX_STEPS] floats: draw weight of each step
+constexpr int ROFF_MBAR = ROFF_STEP + RW * MAX_STEPS * 4;
 constexpr int RSMEM_BYTES = ROFF_MBAR + 16;
 
 // L2 residency hints: the part of a row that is re-read from L2 in every pass is marked
@@ -115,15 +117,17 @@ __device__ __forceinline__ void prefetch_line_l2(const void* p) {
 }
 
 // Visits this thread's chunks in step order: body(a, b, chunk, valid) -> bool (false = stop) with the
-// packed student / teacher words of the chunk.  Global (L2) chunks are fetched LOOKAHEAD steps ahead,
-// the first ones before the resident part is processed.  FIRST_TOUCH: the row has not been read yet,
-// so its global part is additionally requested into L2 PF_STEPS steps ahead (one lane per 128-byte line).
+// packed student / teacher words of the chunk.  Steps in which every lane has a chunk run without
+// predicates; global (L2) chunks are fetched LOOKAHEAD steps ahead, the first ones before the
+// resident part is processed.  FIRST_TOUCH: the row has not been read yet, so its global part is
+// additionally requested into L2 PF_STEPS steps ahead (one lane per 128-byte line).
 template <bool FIRST_TOUCH, typename Body>
 __device__ __forceinline__ void for_each_chunk(const Seg& sg, int lane, const uint4* res_s, const uint4* res_t,
                                                const __nv_bfloat16* g_s, const __nv_bfloat16* g_t, uint64_t pol,
                                                Body&& body) {
-  const uint4 sent = make_uint4(0xFF7FFF7Fu, 0xFF7FFF7Fu, 0xFF7FFF7Fu, 0xFF7FFF7Fu);   // exp -> 0, difference 0
-  const int t0 = sg.c0 + sg.res * 32 + lane;       // this lane's first global chunk
+  const int full = (sg.c1 - sg.c0) >> 5;            // steps in which every lane has a chunk
+  const int res_full = min(sg.res, full);
+  const int t0 = sg.c0 + sg.res * 32 + lane;        // this lane's first global chunk
   if (FIRST_TOUCH && (lane & 7) == 0) {
 #pragma unroll
     for (int j = LOOKAHEAD; j < PF_STEPS; ++j) {
@@ -134,42 +138,42 @@ __device__ __forceinline__ void for_each_chunk(const Seg& sg, int lane, const ui
   uint4 qa[LOOKAHEAD], qb[LOOKAHEAD];
 #pragma unroll
   for (int j = 0; j < LOOKAHEAD; ++j) {
-    qa[j] = sent; qb[j] = sent;
     const int c = t0 + 32 * j;
-    if (c < sg.c1) { qa[j] = ld_l2(g_s + (size_t)c * 8, pol); qb[j] = ld_l2(g_t + (size_t)c * 8, pol); }
+    if (sg.res + j < full) { qa[j] = ld_l2(g_s + (size_t)c * 8, pol); qb[j] = ld_l2(g_t + (size_t)c * 8, pol); }
   }
   // resident part; kept rolled: the pass bodies are large and must stay in the instruction cache
-  const int full = (sg.c1 - sg.c0) >> 5;           // steps in which every lane has a chunk
 #pragma unroll 1
-  for (int k = 0; k < sg.res; ++k) {
-    const int c = sg.c0 + k * 32 + lane;
-    if (k < full) {
-      if (!body(res_s[k * 32 + lane], res_t[k * 32 + lane], c, true)) return;
-    } else {
-      const bool valid = c < sg.c1;
-      uint4 a = sent, b = sent;
-      if (valid) { a = res_s[k * 32 + lane]; b = res_t[k * 32 + lane]; }
-      if (!body(a, b, c, valid)) return;
-    }
-  }
+  for (int k = 0; k < res_full; ++k)
+    if (!body(res_s[k * 32 + lane], res_t[k * 32 + lane], sg.c0 + k * 32 + lane, true)) return;
   int c = t0;
 #pragma unroll 1
-  for (int k = sg.res; k < sg.steps; k += LOOKAHEAD) {
+  for (int k = sg.res; k < full; k += LOOKAHEAD) {
 #pragma unroll
     for (int j = 0; j < LOOKAHEAD; ++j) {
-      if (k + j < sg.steps) {
+      if (k + j < full) {
         const uint4 a = qa[j], b = qb[j];
-        const int cn = c + 32 * LOOKAHEAD;
-        qa[j] = sent; qb[j] = sent;
-        if (cn < sg.c1) { qa[j] = ld_l2(g_s + (size_t)cn * 8, pol); qb[j] = ld_l2(g_t + (size_t)cn * 8, pol); }
+        if (k + j + LOOKAHEAD < full) {
+          const int cn = c + 32 * LOOKAHEAD;
+          qa[j] = ld_l2(g_s + (size_t)cn * 8, pol); qb[j] = ld_l2(g_t + (size_t)cn * 8, pol);
+        }
         if (FIRST_TOUCH && (lane & 7) == 0) {
           const int cp = c + 32 * PF_STEPS;
           if (cp < sg.c1) { prefetch_line_l2(g_s + (size_t)cp * 8); prefetch_line_l2(g_t + (size_t)cp * 8); }
         }
-        if (!body(a, b, c, c < sg.c1)) return;
+        if (!body(a, b, c, true)) return;
         c += 32;
       }
     }
+  }
+  if (full < sg.steps) {   // the last, partly filled step
+    const int cl = sg.c0 + full * 32 + lane;
+    const bool valid = cl < sg.c1;
+    uint4 a = make_uint4(0xFF7FFF7Fu, 0xFF7FFF7Fu, 0xFF7FFF7Fu, 0xFF7FFF7Fu), b = a;   // exp -> 0, difference 0
+    if (valid) {
+      if (full < sg.res) { a = res_s[full * 32 + lane]; b = res_t[full * 32 + lane]; }
+      else { a = ld_l2(g_s + (size_t)cl * 8, pol); b = ld_l2(g_t + (size_t)cl * 8, pol); }
+    }
+    body(a, b, cl, valid);
   }
 }
 
@@ -462,23 +466,34 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       float2 Sq = splat(0.f), R = splat(0.f);
       const float2 cc = splat(c32), cll = splat(cl), kqq = splat(kq), kk0 = splat(k0), neg1 = splat(-1.f);
       const float2 iqq = splat(iq), nip = splat(-ip), kgg = splat(kg);
+      float* step_w = (float*)(smem + ROFF_STEP) + warp * MAX_STEPS;   // draw weight of each of this warp's steps
       int n_res_done = 0;
       bool next_issued = false;
       for_each_chunk<false>(sg, lane, res_s, res_t, g_s, g_t, pol_last, [&](const uint4& s4, const uint4& t4, int c, bool valid) {
         const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
         uint32_t gp[4];
+        float2 sqc = splat(0.f), rc = splat(0.f);       // this chunk's share of Sq and R
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const float2 sf = unpack_bf16x2(sw[i]), tf = unpack_bf16x2(tw[i]);
           const float2 d = ffma2(sf, neg1, tf);
           const float2 ep = ex2f2(ffma2(sf, cc, kk0));
           const float2 eq = ex2f2(ffma2(d, cll, ffma2(sf, cc, kqq)));
-          Sq = fadd2(Sq, eq);
+          sqc = fadd2(sqc, eq);
           float2 r = ffma2(eq, iqq, fmul2(ep, nip));     // q_i - p_i
           r.x = fmaxf(r.x, 0.f); r.y = fmaxf(r.y, 0.f);
-          R = fadd2(R, r);
+          rc = fadd2(rc, r);
           const float2 gv = fmul2(ep, kgg);
           gp[i] = pack_bf16x2(gv.x, gv.y);
+        }
+        Sq = fadd2(Sq, sqc);
+        R = fadd2(R, rc);
+        if (need_draw) {   // ordered bookkeeping for the inverse-CDF draw: the weight of this step of the warp
+          float wsum = bonus ? (sqc.x + sqc.y) * iq : (rc.x + rc.y);
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
+          const int k = (c - sg.c0) >> 5;
+          if (lane == 0 && k < MAX_STEPS) step_w[k] = wsum;
         }
         if ((tok >> 3) == c && tok >= 0) {   // the supervised token is in this chunk: subtract the one-hot part
           const int e = tok & 7, wi = e >> 1;
@@ -492,7 +507,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
         }
         if (want_g && valid) st_stream(g_out + (size_t)c * 8, make_uint4(gp[0], gp[1], gp[2], gp[3]), pol_first);
         // once the warp has read its resident part for the last time, the next row's may land there
-        // (a row that still needs its draw re-reads the resident part: its copy is issued after the draw)
+        // (a row that still needs its draw may re-read one resident step: its copy is issued after the draw)
         if (++n_res_done == sg.res && !need_draw) {
           __syncwarp();
           if (lane == 0 && !dead && next_row < P.n_rows) {
@@ -506,8 +521,13 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       if (!next_issued && !need_draw && lane == 0 && !dead && next_row < P.n_rows) issue(next_row);   // no elements
       RTS(11);
       const float sq_f = Sq.x + Sq.y, r_f = R.x + R.y;
-      const double part = warp_sum_d((double)(bonus ? sq_f * iq : r_f));
-      const double v[3] = {warp_sum_d((double)sq_f), warp_sum_d((double)r_f), part};
+      double part = 0.0;                               // this warp's draw weight: its step weights, in order
+      if (need_draw) {
+        __syncwarp();
+        const int ns = min(sg.steps, MAX_STEPS);
+        for (int k = 0; k < ns; ++k) part += (double)step_w[k];
+      }
+      const double v[2] = {warp_sum_d((double)sq_f), warp_sum_d((double)r_f)};
       if (lane == 0) red[2 * RW + warp] = part;     // ordered per-warp weights of the draw
       combine(v, 2);
       RTS(12);
@@ -523,56 +543,73 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       __syncthreads();
       if (warp == (int)bc[BC_OWNER_WARP]) {
         const double target = bc[BC_TARGET];
-        const bool last_mode = bc[BC_TAKE_LAST] != 0.0;
+        bool last_mode = bc[BC_TAKE_LAST] != 0.0;
         double running = bc[BC_BEFORE];
-        int y = -1, last_pos = -1;
-        const float2 cc = splat(c32), cll = splat(cl), kqq = splat(kq), kk0 = splat(k0), neg1 = splat(-1.f);
-        for_each_chunk<false>(sg, lane, res_s, res_t, g_s, g_t, pol_last, [&](const uint4& s4, const uint4& t4, int c, bool valid) {
-          const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
-          float w[8];
+        const float* step_w = (const float*)(smem + ROFF_STEP) + warp * MAX_STEPS;
+        const int ns = min(sg.steps, MAX_STEPS);
+        // the step that holds the target (every lane walks the same few numbers)
+        int ks = -1, kpos = -1;
+        for (int k = 0; k < ns; ++k) {
+          const double w = (double)step_w[k];
+          if (w > 0.0) kpos = k;
+          if (!last_mode && running + w > target) { ks = k; break; }
+          running += w;
+        }
+        if (ks < 0) { last_mode = true; ks = max(kpos, 0); }   // rounding: last step with positive weight
+        const int c = sg.c0 + ks * 32 + lane;
+        const bool valid = c < sg.c1;
+        uint4 s4 = make_uint4(0xFF7FFF7Fu, 0xFF7FFF7Fu, 0xFF7FFF7Fu, 0xFF7FFF7Fu), t4 = s4;
+        if (valid) {
+          if (ks < sg.res) { s4 = res_s[ks * 32 + lane]; t4 = res_t[ks * 32 + lane]; }
+          else { s4 = ld_l2(g_s + (size_t)c * 8, pol_last); t4 = ld_l2(g_t + (size_t)c * 8, pol_last); }
+        }
+        const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
+        float w[8];
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const float2 sf = unpack_bf16x2(sw[i]), tf = unpack_bf16x2(tw[i]);
-            const float2 d = ffma2(sf, neg1, tf);
-            const float2 ep = ex2f2(ffma2(sf, cc, kk0));
-            const float2 eq = ex2f2(ffma2(d, cll, ffma2(sf, cc, kqq)));
-            w[2 * i] = bonus ? eq.x * iq : fmaxf(fmaf(eq.x, iq, -(ep.x * ip)), 0.f);
-            w[2 * i + 1] = bonus ? eq.y * iq : fmaxf(fmaf(eq.y, iq, -(ep.y * ip)), 0.f);
-          }
-          double mine = 0.0;
+        for (int i = 0; i < 4; ++i) {
+          const float2 sf = unpack_bf16x2(sw[i]), tf = unpack_bf16x2(tw[i]);
+          const float2 d = ffma2(sf, splat(-1.f), tf);
+          const float2 ep = ex2f2(ffma2(sf, splat(c32), splat(k0)));
+          const float2 eq = ex2f2(ffma2(d, splat(cl), ffma2(sf, splat(c32), splat(kq))));
+          w[2 * i] = bonus ? eq.x * iq : fmaxf(fmaf(eq.x, iq, -(ep.x * ip)), 0.f);
+          w[2 * i + 1] = bonus ? eq.y * iq : fmaxf(fmaf(eq.y, iq, -(ep.y * ip)), 0.f);
+        }
+        double mine = 0.0;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) mine += valid ? (double)w[i] : 0.0;
-          double inc = mine;
+        for (int i = 0; i < 8; ++i) mine += (double)w[i];
+        double inc = mine;
 #pragma unroll
-          for (int o = 1; o < 32; o <<= 1) {
-            const double up = __shfl_up_sync(0xffffffffu, inc, o);
-            if (lane >= o) inc += up;
-          }
-          const unsigned posm = __ballot_sync(0xffffffffu, mine > 0.0);
-          const unsigned hit = last_mode ? 0u : __ballot_sync(0xffffffffu, running + inc > target);
-          int found = -1, lastp = -1;
-          if (hit && lane == __ffs(hit) - 1) {           // walk the 8 elements of the crossing chunk
+        for (int o = 1; o < 32; o <<= 1) {
+          const double up = __shfl_up_sync(0xffffffffu, inc, o);
+          if (lane >= o) inc += up;
+        }
+        const unsigned posm = __ballot_sync(0xffffffffu, mine > 0.0);
+        const unsigned hit = last_mode ? 0u : __ballot_sync(0xffffffffu, running + inc > target);
+        int y = -1;
+        if (hit) {
+          int found = -1;
+          if (lane == __ffs(hit) - 1) {                   // walk the 8 elements of the crossing chunk
             double run = running + inc - mine;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
               run += (double)w[i];
               if (found < 0 && run > target) found = c * 8 + i;
             }
-            if (found < 0) {                              // rounding: last positive element of the chunk
+            if (found < 0) {
 #pragma unroll
               for (int i = 0; i < 8; ++i) if (w[i] > 0.f) found = c * 8 + i;
             }
           }
-          if (posm && lane == 31 - __clz(posm)) {
+          y = __shfl_sync(0xffffffffu, found, __ffs(hit) - 1);
+        } else if (posm) {                                // rounding: last positive element of the step
+          int lastp = -1;
+          if (lane == 31 - __clz(posm)) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) if (w[i] > 0.f) lastp = c * 8 + i;
           }
-          if (hit) y = __shfl_sync(0xffffffffu, found, __ffs(hit) - 1);
-          if (posm) last_pos = __shfl_sync(0xffffffffu, lastp, 31 - __clz(posm));
-          running += __shfl_sync(0xffffffffu, inc, 31);
-          return y < 0;                                   // stop at the crossing
-        });
-        if (y < 0) y = (last_pos >= 0) ? last_pos : min(V - 1, sg.c1 * 8 - 1);
+          y = __shfl_sync(0xffffffffu, lastp, 31 - __clz(posm));
+        }
+        if (y < 0) y = min(V - 1, max(sg.c0 * 8, sg.c1 * 8 - 1));
         if (lane == 0) write_result(bc, P.out, !P.spec, row, bonus ? 0 : 1, y, bonus, K.c64, g_s, g_t);
       }
       __syncwarp();
@@ -602,7 +639,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
 // ---------------------------------------------------------------- host side
 bool rowsm_can_serve(const RowParams& p, int dtype) {
   if (dtype != SAKI_BF16) return false;
-  if (p.V < 2048 || p.V % 8 != 0) return false;
+  if (p.V < 2048 || p.V % 8 != 0 || p.V > MAX_STEPS * 32 * 8 * RW) return false;
   auto al16 = [](const void* q) { return ((uintptr_t)q & 15) == 0; };
   if (!al16(p.s) || !al16(p.t)) return false;
   if (p.s_seq % 8 || p.s_pos % 8 || p.t_seq % 8 || p.t_pos % 8) return false;
