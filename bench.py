@@ -38,9 +38,10 @@ if ROOT not in sys.path:
 METRIC = "routed positions/sec (fwd+bwd, V=151936 bf16)"
 UNIT = "positions/s"
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one cluster-kernel launch divided by the
-# positions it routed (ncu capture summarised in profiles/); None until measured
-TRAFFIC_BYTES_PER_POSITION = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one rowsm_kernel launch divided by the positions it
+# routed: ncu capture on 2220 rows of the same workload (profiles/rowsm_kernel_cfg3.md); traffic grows
+# in proportion to the rows, so a full launch is this figure times N
+TRAFFIC_BYTES_PER_POSITION = 932506
 
 
 def _peaks():
@@ -255,8 +256,8 @@ def run_ours(args):
                 "peak_kind": f"of {peak_kind} (device-to-device copy, MEASURED_PEAKS.json)"
                 if peak_kind == "measured" else "of fallback",
                 "traffic": (TRAFFIC_BYTES_PER_POSITION * w.N) if TRAFFIC_BYTES_PER_POSITION else None,
-                "algorithmic_bytes_per_launch": bpp * w.N, "kernel": "saki::cluster_kernel<8>" if kernel_used == 2
-                else "saki::general_kernel", "kernel_ms": kern_ms,
+                "algorithmic_bytes_per_launch": bpp * w.N, "kernel": {3: "saki::rowsm_kernel", 2: "saki::cluster_kernel<8>"}.get(kernel_used, "saki::general_kernel"),
+                "kernel_ms": kern_ms,
                 "frac_of_nominal_8TBs": achieved / 8000.0}
 
     stats = {"correction_rate": float(out["corrected"].float().mean().item()),
@@ -296,7 +297,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--cpu-rows", type=int, default=128)
+    ap.add_argument("--cpu-rows", type=int, default=384)
     ap.add_argument("--ref-rows", type=int, default=32)
     args = ap.parse_args()
     if args.impl == "reference":

@@ -37,7 +37,7 @@ namespace saki {
 #endif
 constexpr int RT = SAKI_ROWSM_THREADS;  // threads per CTA
 constexpr int RW = RT / 32;             // warps per CTA
-constexpr int KS_MAX = RT == 512 ? 13 : 6;  // resident steps per warp (a step = 32 chunks of 8 elements)
+constexpr int KS_MAX = RT == 512 ? 13 : RT == 768 ? 8 : 6;  // resident steps per warp (a step = 32 chunks of 8 elements)
 constexpr int MAX_STEPS = 64;            // steps per warp the draw bookkeeping can hold (V <= 64*32*8*RW)
 constexpr int RES_CHUNKS = KS_MAX * 32; // resident chunks per warp and row
 constexpr int RNV = 8;                  // doubles per partial vector
