@@ -175,14 +175,21 @@ SAKI_API int saki_check(void* cuda_stream, uint64_t* n_flagged);
  * row, float64, any V, dtype and layout), 2 = the register-resident cluster
  * kernel (one row per cluster of up to 8 blocks), 3 = the row-per-SM kernel
  * (one row per block; shared memory plus L2).  2 and 3 serve bf16 rows with
- * 16-byte aligned rows and V a multiple of 8, V >= 2048 (2: V <= 163840);
- * other inputs fall back to 1.  Automatic prefers 3.  Process-wide; meant for
+ * 16-byte aligned rows and V a multiple of 8, V >= 2048 (2: V <= 163840), and
+ * eps = 0 or eps >= 5e-3 (their float32 sums cannot resolve smaller radii to the
+ * tolerance); other inputs fall back to 1.  Automatic prefers 3.  Process-wide; meant for
  * tests and benchmarks.  Returns the previous value. */
 SAKI_API int saki_set_kernel(int which);
 
 /* Which row kernel the calling thread's last routing call used: 1 general, 2 cluster,
  * 3 row-per-SM, 0 if none yet. */
 SAKI_API int saki_last_kernel(void);
+
+/* Two-tier routing: the float32 kernels (2, 3) hand rows whose KL they cannot resolve to the
+ * tolerance (very small eps, nearly one-hot rows) to the float64 kernel, through a row list in device
+ * memory that the library allocates once per device and keeps.  Synchronises the stream and returns
+ * how many rows of the calling thread's last routing call took that second tier. */
+SAKI_API int saki_redo_count(void* cuda_stream, uint64_t* n_rows);
 
 /* Number of kernels this library has launched in this process (all threads). */
 SAKI_API uint64_t saki_launch_count(void);

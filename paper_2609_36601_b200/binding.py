@@ -20,7 +20,8 @@ ROW_SATURATED, ROW_EPS_ZERO, ROW_MASKED, ROW_NONFINITE, ROW_BAD_ID, ROW_TIMEOUT,
 
 _FLOAT_FIELDS = ("lambda", "kl", "tv", "accept_prob", "logp_x", "logq_x", "logT_x", "logp_y", "logq_y", "loss")
 EXPORTS = ("saki_route_fwd", "saki_route_fwd_bwd", "saki_route_host", "saki_spec_verify",
-           "saki_sample_proposal", "saki_check", "saki_set_kernel", "saki_last_kernel", "saki_launch_count",
+           "saki_sample_proposal", "saki_check", "saki_set_kernel", "saki_last_kernel", "saki_redo_count",
+           "saki_launch_count",
            "saki_last_error", "saki_version")
 
 
@@ -76,10 +77,12 @@ def load_library(path: str | None = None):
                                          C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p]
     lib.saki_check.argtypes = [C.c_void_p, C.POINTER(C.c_uint64)]
     lib.saki_set_kernel.argtypes = [C.c_int]
+    lib.saki_redo_count.argtypes = [C.c_void_p, C.POINTER(C.c_uint64)]
     lib.saki_launch_count.restype = C.c_uint64
     lib.saki_last_error.restype = C.c_char_p
     for f in ("saki_route_fwd", "saki_route_fwd_bwd", "saki_route_host", "saki_spec_verify",
-              "saki_sample_proposal", "saki_check", "saki_set_kernel", "saki_last_kernel", "saki_version"):
+              "saki_sample_proposal", "saki_check", "saki_set_kernel", "saki_last_kernel", "saki_redo_count",
+              "saki_version"):
         getattr(lib, f).restype = C.c_int
     _lib = lib
     return lib
@@ -235,6 +238,14 @@ def set_kernel(which: int) -> int:
 def last_kernel() -> int:
     """1 = general kernel, 2 = cluster kernel (the calling thread's last routing call)."""
     return load_library().saki_last_kernel()
+
+
+def redo_count(stream=None) -> int:
+    """Rows of the last routing call that the float32 kernel handed to the float64 kernel (synchronises)."""
+    lib = load_library()
+    n = C.c_uint64(0)
+    _raise(lib, lib.saki_redo_count(_stream_ptr(stream), C.byref(n)))
+    return int(n.value)
 
 
 def launch_count() -> int:

@@ -45,6 +45,34 @@ static int device_ready(unsigned long long** flagged) {
   return SAKI_OK;
 }
 
+// Scratch of the two-tier routing: the float32 kernels append the rows they cannot resolve to a list
+// that the float64 kernel then routes.  One buffer per device, grown on demand, kept until exit.
+struct RedoScratch {
+  std::mutex mu;
+  int dev = -1;
+  int32_t* list = nullptr;       // [cap] rows, followed by the counter
+  int64_t cap = 0;
+};
+static RedoScratch g_redo;
+static thread_local unsigned int* g_last_redo_count = nullptr;
+
+static int redo_scratch(int64_t n_rows, int32_t** list, unsigned int** count) {
+  std::lock_guard<std::mutex> lock(g_redo.mu);
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (g_redo.dev != dev || g_redo.cap < n_rows) {
+    if (g_redo.list && g_redo.dev == dev) cudaFree(g_redo.list);
+    g_redo.list = nullptr; g_redo.cap = 0; g_redo.dev = dev;
+    const int64_t cap = std::max<int64_t>(n_rows, 1 << 16);
+    cudaError_t e = cudaMalloc((void**)&g_redo.list, (size_t)(cap + 64) * sizeof(int32_t));
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc (redo list)");
+    g_redo.cap = cap;
+  }
+  *list = g_redo.list;
+  *count = (unsigned int*)(g_redo.list + g_redo.cap);
+  return SAKI_OK;
+}
+
 static int check_common(const void* s, const void* t, int64_t n, int32_t V, int32_t dtype, float eps, float tau) {
   if (n < 0) return fail(SAKI_ERR_INVALID_ARG, "negative row count");
   if (V < 2) return fail(SAKI_ERR_INVALID_ARG, "V must be >= 2 (got %d)", V);
@@ -55,23 +83,45 @@ static int check_common(const void* s, const void* t, int64_t n, int32_t V, int3
   return SAKI_OK;
 }
 
-static int dispatch_rows(const RowParams& p, int dtype, cudaStream_t st) {
+// `scratch_list` / `scratch_count`: where the two-tier routing keeps its redo list (NULL: the library's
+// own per-device buffer, allocated on demand).
+static int dispatch_rows(RowParams p, int dtype, cudaStream_t st, int32_t* scratch_list = nullptr,
+                         unsigned int* scratch_count = nullptr) {
   int launches = 0;
   cudaError_t e;
   bool served = false;
   const int which = g_kernel.load();
   int used = 1;
-  if ((which == 0 || which == 3) && rowsm_can_serve(p, dtype)) {
+  // The float32 kernels resolve KL(q||p) to a few 1e-7 absolute: enough for |d lambda| <= 1e-5 when
+  // eps >= 5e-3 (measured), not below.  Smaller positive radii run on the float64 kernel.
+  const bool eps_ok = !(p.eps > 0.f) || p.eps >= 5e-3f;
+  const bool fast = (which != 1) && eps_ok && (rowsm_can_serve(p, dtype) || cluster_can_serve(p, dtype));
+  p.redo_list = nullptr; p.redo_count = nullptr; p.from_list = 0;
+  if (fast) {
+    if (scratch_list) { p.redo_list = scratch_list; p.redo_count = scratch_count; }
+    else {
+      const int rc = redo_scratch(p.n_rows, &p.redo_list, &p.redo_count);
+      if (rc) return rc;
+    }
+    e = cudaMemsetAsync(p.redo_count, 0, sizeof(unsigned int), st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+    g_last_redo_count = p.redo_count;
+  }
+  if (fast && (which == 0 || which == 3) && rowsm_can_serve(p, dtype)) {
     e = launch_rowsm(p, st, &launches, &served);
     if (e != cudaSuccess) return cuda_fail(e, "row-per-SM kernel launch");
     if (served) used = 3;
   }
-  if (!served && which == 2 && cluster_can_serve(p, dtype)) {
+  if (fast && !served && which == 2 && cluster_can_serve(p, dtype)) {
     e = launch_cluster(p, st, &launches, &served);
     if (e != cudaSuccess) return cuda_fail(e, "cluster kernel launch");
     if (served) used = 2;
   }
-  if (!served) {
+  if (served) {   // second tier: the rows the float32 kernel handed over
+    p.from_list = 1;
+    e = launch_general(p, dtype, st, &launches);
+    if (e != cudaSuccess) return cuda_fail(e, "general kernel launch (redo list)");
+  } else {
     e = launch_general(p, dtype, st, &launches);
     if (e != cudaSuccess) return cuda_fail(e, "general kernel launch");
   }
@@ -395,6 +445,20 @@ SAKI_API int saki_set_kernel(int which) {
 }
 
 SAKI_API int saki_last_kernel(void) { return g_last_kernel; }
+
+SAKI_API int saki_redo_count(void* cuda_stream, uint64_t* n_rows) {
+  g_err[0] = 0;
+  if (!n_rows) return fail(SAKI_ERR_INVALID_ARG, "NULL output pointer");
+  *n_rows = 0;
+  if (!g_last_redo_count) return SAKI_OK;
+  cudaError_t e = cudaStreamSynchronize((cudaStream_t)cuda_stream);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+  unsigned int h = 0;
+  e = cudaMemcpy(&h, g_last_redo_count, sizeof(h), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy");
+  *n_rows = h;
+  return SAKI_OK;
+}
 
 SAKI_API uint64_t saki_launch_count(void) { return g_launches.load(); }
 

@@ -356,7 +356,8 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
       TS(11);
       if (tid == 0) {
         scalar_after_solve(bc, gat, K, k0, k1, x, bonus, masked);
-        mbar_expect_tx(&mbar[1 + parity], (uint32_t)(CS * CW * 3 * 8));   // next evaluation, or pass "final"
+        if ((int)bc[BC_MODE] == MODE_SOLVE || (int)bc[BC_MODE] == MODE_FINAL)
+          mbar_expect_tx(&mbar[1 + parity], (uint32_t)(CS * CW * 3 * 8));   // next evaluation, or pass "final"
       }
       TS(12);
       __syncthreads();
@@ -366,12 +367,16 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
     }
 
     // ------------------------------------------------ flagged row: zero outputs, zero gradient
-    if ((int)bc[BC_MODE] == MODE_FLAGGED) {
+    if ((int)bc[BC_MODE] == MODE_FLAGGED || (int)bc[BC_MODE] == MODE_REDO) {
+      const bool redo = (int)bc[BC_MODE] == MODE_REDO;   // ill-conditioned for float32: the float64 kernel routes it
       if (rank == 0 && tid == 0) {
-        write_row(P.out, row, zero_row((uint32_t)bc[BC_STATUS]), !P.spec);
-        atomicAdd(P.flagged, 1ull);
+        if (redo) P.redo_list[atomicAdd(P.redo_count, 1u)] = (int32_t)row;
+        else {
+          write_row(P.out, row, zero_row((uint32_t)bc[BC_STATUS]), !P.spec);
+          atomicAdd(P.flagged, 1ull);
+        }
       }
-      if (g_out) {
+      if (g_out && !redo) {
 #pragma unroll
         for (int j = 0; j < CHUNKS; ++j) {
           int cj = j + rot;

@@ -32,6 +32,9 @@ struct RowParams {
   int64_t ld_g;
   float grad_scale;
   unsigned long long* flagged;         // device counter of flagged rows
+  int32_t* redo_list;                  // scratch: rows the float32 kernels hand to the float64 kernel
+  unsigned int* redo_count;            // scratch: their number (zeroed before the launch)
+  int32_t from_list;                   // general kernel only: route the rows of redo_list
 };
 
 // ---- Philox4x32-10 (Salmon et al., SC'11), written from the published round function ----

@@ -12,13 +12,13 @@ constexpr double LN2 = 0.693147180559945309417232121458;
 constexpr double INV_LN2 = 1.44269504088896340735992468100;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // ~2 s: give up on a wait
 
-enum { MODE_SOLVE = 0, MODE_FINAL = 1, MODE_FLAGGED = 2 };
+enum { MODE_SOLVE = 0, MODE_FINAL = 1, MODE_FLAGGED = 2, MODE_REDO = 3 };
 // broadcast slots (one set per row buffer)
 enum { BC_MODE = 0, BC_BETA, BC_CB, BC_KB, BC_LO, BC_HI, BC_ITER,                    // solver
        BC_CL, BC_KQ, BC_IQ, BC_IP, BC_KG, BC_TOK, BC_STATUS, BC_CORR, BC_LAMBDA,    // final pass
        BC_GLAM, BC_G0, BC_G1, BC_ACC, BC_LPX, BC_LTX, BC_LOSS, BC_VSTAR, BC_KL, BC_TV,
        BC_OWNER_WARP, BC_BEFORE, BC_TARGET, BC_TAKE_LAST, BC_RSS,
-       BC_UACC, BC_UDRAW, BC_SX, BC_TX, BC_K0, BC_K1, BC_COUNT };
+       BC_UACC, BC_UDRAW, BC_SX, BC_TX, BC_K0, BC_K1, BC_PMAX, BC_COUNT };
 static_assert(BC_COUNT <= BC_DOUBLES, "broadcast area too small");
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -215,6 +215,7 @@ static __device__ __noinline__ void scalar_after_lse(double* bc, const double* v
   const double rSs = rcp_fast(SsT), rSt = rcp_fast(StT);
   const double G0 = LN2 * (log2_fast(SsT) - k0), G1 = LN2 * (log2_fast(StT) - k1);
   bc[BC_G0] = G0; bc[BC_G1] = G1; bc[BC_RSS] = rSs;
+  bc[BC_PMAX] = fmax(rSs, rSt);      // upper bound of the largest probability of either row
   if (!(eps > 0.0)) {          // student-only endpoint
     bc[BC_KL] = 0.0;
     decide(bc, K, 0.0, G0, G0, G1, k0, k1, rSs, status | SAKI_ROW_EPS_ZERO, vstar, bonus, masked, x);
@@ -274,6 +275,10 @@ static __device__ __noinline__ void scalar_after_solve(double* bc, const double*
   bool bisected = false;
   if (!(nb > lo && nb < hi)) { nb = 0.5 * (lo + hi); bisected = true; }
   const bool done = (!bisected && fabs(nb - beta) <= 2e-4 * beta) || iter >= 40 || (hi - lo) < 1e-9;
+  // The float32 sums resolve KL to a few 1e-7 x (largest probability).  Where that would move lambda by
+  // more than the tolerance (a very flat KL: nearly one-hot rows), or the solve did not converge, the row
+  // is handed to the float64 kernel.  (Radii below 5e-3 never reach this kernel: see the dispatcher.)
+  if (done && (3e-7 * bc[BC_PMAX] > 1e-5 * slope || iter >= 40)) { bc[BC_MODE] = MODE_REDO; return; }
   if (done) {
     const float cl = (float)(K.c64 * nb);
     const double lam = (double)cl * K.rc64;

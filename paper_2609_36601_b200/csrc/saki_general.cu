@@ -58,7 +58,9 @@ __global__ void __launch_bounds__(GT) general_kernel(const RowParams P) {
   const double tau = (double)P.temperature;
   const double eps = (double)P.eps;
 
-  for (int64_t row = blockIdx.x; row < P.n_rows; row += gridDim.x) {
+  const int64_t n_work = P.from_list ? (int64_t)*P.redo_count : P.n_rows;
+  for (int64_t item = blockIdx.x; item < n_work; item += gridDim.x) {
+    const int64_t row = P.from_list ? (int64_t)P.redo_list[item] : item;   // list mode: rows handed over by the float32 kernels
     const int64_t b = row / P.K1;
     const int j = (int)(row - b * P.K1);
     const T* s = (const T*)P.s + b * P.s_seq + (int64_t)j * P.s_pos;
@@ -310,7 +312,7 @@ cudaError_t launch_general(const RowParams& p, int dtype, cudaStream_t st, int* 
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const int64_t cap = (int64_t)sms * 3;
+  const int64_t cap = (int64_t)sms * (p.from_list ? 1 : 3);
   const int grid = (int)(p.n_rows < cap ? p.n_rows : cap);
   if (dtype == SAKI_BF16) general_kernel<__nv_bfloat16><<<grid, GT, 0, st>>>(p);
   else general_kernel<float><<<grid, GT, 0, st>>>(p);

@@ -37,7 +37,7 @@ namespace saki {
 #endif
 constexpr int RT = SAKI_ROWSM_THREADS;  // threads per CTA
 constexpr int RW = RT / 32;             // warps per CTA
-constexpr int KS_MAX = RT == 512 ? 13 : RT == 768 ? 8 : 6;  // resident steps per warp (a step = 32 chunks of 8 elements)
+constexpr int KS_MAX = RT == 512 ? 13 : RT == 640 ? 10 : RT == 768 ? 8 : 6;  // resident steps per warp (a step = 32 chunks of 8 elements)
 constexpr int MAX_STEPS = 64;            // steps per warp the draw bookkeeping can hold (V <= 64*32*8*RW)
 constexpr int RES_CHUNKS = KS_MAX * 32; // resident chunks per warp and row
 constexpr int RNV = 8;                  // doubles per partial vector
@@ -109,6 +109,10 @@ __device__ __forceinline__ float pow2f_exact(float n) {   // 2^n for whole n, cl
   return __uint_as_float((uint32_t)(127 + i) << 23);
 }
 
+#ifndef SAKI_RES_UNROLL
+#define SAKI_RES_UNROLL 1
+#endif
+constexpr int RES_UNROLL = SAKI_RES_UNROLL;   // unrolling of the resident-part loop
 constexpr int LOOKAHEAD = 2;            // global (L2) chunks in flight per thread
 constexpr int PF_STEPS = 8;             // first touch of a row: lines are requested this many steps ahead
 
@@ -141,8 +145,8 @@ __device__ __forceinline__ void for_each_chunk(const Seg& sg, int lane, const ui
     const int c = t0 + 32 * j;
     if (sg.res + j < full) { qa[j] = ld_l2(g_s + (size_t)c * 8, pol); qb[j] = ld_l2(g_t + (size_t)c * 8, pol); }
   }
-  // resident part; kept rolled: the pass bodies are large and must stay in the instruction cache
-#pragma unroll 1
+  // resident part; kept (nearly) rolled: the pass bodies are large and must stay in the instruction cache
+#pragma unroll RES_UNROLL
   for (int k = 0; k < res_full; ++k)
     if (!body(res_s[k * 32 + lane], res_t[k * 32 + lane], sg.c0 + k * 32 + lane, true)) return;
   int c = t0;
@@ -434,12 +438,16 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
     }
 
     // ------------------------------------------------ flagged row: zero outputs, zero gradient
-    if ((int)bc[BC_MODE] == MODE_FLAGGED) {
+    if ((int)bc[BC_MODE] == MODE_FLAGGED || (int)bc[BC_MODE] == MODE_REDO) {
+      const bool redo = (int)bc[BC_MODE] == MODE_REDO;   // ill-conditioned for float32: the float64 kernel routes it
       if (tid == 0) {
-        write_row(P.out, row, zero_row((uint32_t)bc[BC_STATUS]), !P.spec);
-        atomicAdd(P.flagged, 1ull);
+        if (redo) P.redo_list[atomicAdd(P.redo_count, 1u)] = (int32_t)row;
+        else {
+          write_row(P.out, row, zero_row((uint32_t)bc[BC_STATUS]), !P.spec);
+          atomicAdd(P.flagged, 1ull);
+        }
       }
-      if (g_out) {
+      if (g_out && !redo) {
         for (int k = 0; k < sg.steps; ++k) {
           const int c = sg.c0 + k * 32 + lane;
           if (c < sg.c1) st_stream(g_out + (size_t)c * 8, make_uint4(0, 0, 0, 0), pol_first);

@@ -8,7 +8,8 @@ Tolerances (written here so that the tests state them):
                       counted and returned
   lambda, TV          |delta| <= 1e-5
   other fp32 scalars  |delta| <= 1e-5 (kl, accept_prob) or 1e-5 (1+|ref|) (log-probs)
-  loss                |delta| <= 1e-4 |ref| + 2e-6
+  loss                |delta| <= 1e-4 |ref| + 1e-6 (1 + |k1| + |log p(x)|), k1 = log p(x) - log T(x): the loss is
+                      k1 log p(x), and a log-sum-exp taken from float32 sums resolves each factor to ~1e-7
   gradient, fp32      |delta| <= 1e-5 max(1, max|g_row|) ... see grad_check
   gradient, bf16      |delta| <= 2e-3 where |g_ref| < 1; elsewhere within one
                       bf16 ulp of the oracle's rounded value; and relative
@@ -35,8 +36,11 @@ def bf16_ulp(x):
     return np.ldexp(1.0, (e - 1) - 7)
 
 
-def grad_check(g_gpu: np.ndarray, g_ref: np.ndarray, dtype: str):
-    """g_ref is the oracle gradient already rounded to the output dtype."""
+def grad_check(g_gpu: np.ndarray, g_ref: np.ndarray, dtype: str, tok=None):
+    """g_ref is the oracle gradient already rounded to the output dtype.  `tok[i]` is the supervised
+    token of row i: that entry is coef (p - 1), a difference that cancels when p is close to 1, so it is
+    held to the absolute bound only (the relative bound exists to keep small-p entries from being
+    flushed to zero, which does not apply to it)."""
     d = np.abs(g_gpu - g_ref)
     if dtype == "f32":
         tol = 1e-6 + 2e-6 * np.abs(g_ref)
@@ -47,6 +51,8 @@ def grad_check(g_gpu: np.ndarray, g_ref: np.ndarray, dtype: str):
     big_ok = d[~small] <= bf16_ulp(g_ref[~small]) * 1.0000001
     assert np.all(big_ok), "bf16 gradient entry with |g|>=1 off by more than one ulp"
     nz = np.abs(g_ref) >= 1e-30
+    if tok is not None:
+        nz[np.arange(len(tok)), np.asarray(tok)] = False
     rel = d[nz] / np.abs(g_ref[nz])
     assert np.all(rel <= 2.0 ** -7 * 1.0000001), f"bf16 gradient relative error {rel.max():.3e}"
     return dict(max_abs=float(d[small].max()) if small.any() else 0.0,
@@ -77,7 +83,8 @@ def compare_rows(gpu: dict, ref: dict, rows=None, check_loss=True):
         assert np.all(d <= 1e-5 * (1 + np.abs(ref[name][same]))), f"{name}: max error {d.max():.3e}"
     if check_loss:
         d = np.abs(g["loss"].astype(np.float64) - ref["loss"])[same]
-        assert np.all(d <= 1e-4 * np.abs(ref["loss"][same]) + 2e-6), f"loss: max error {d.max():.3e}"
+        floor = 1e-6 * (1.0 + np.abs(ref["logp_x"] - ref["logT_x"]) + np.abs(ref["logp_x"]))[same]   # the ~1e-7 resolution of a
+        assert np.all(d <= 1e-4 * np.abs(ref["loss"][same]) + floor), f"loss: max error {d.max():.3e}"   # float32 lse
     return int(exempt.sum())
 
 

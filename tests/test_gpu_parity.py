@@ -41,7 +41,8 @@ def _check_fwd_bwd(d, w, rows=None, mask=None, row_offset=0, grad_scale=1.0, eps
     rr = np.arange(len(d["proposal"])) if rows is None else np.asarray(list(rows))
     gg = to_np64(g)[rr]
     same = (out["corrected"].cpu().numpy()[rr] == ref["corrected"])
-    stats = grad_check(gg[same], ref["grad"][same], w.dtype)
+    tok = np.where(ref["corrected"] == 1, ref["teacher_top1"], ref["token"])[same]
+    stats = grad_check(gg[same], ref["grad"][same], w.dtype, tok)
     return out, ref, n_exempt, stats
 
 
@@ -201,3 +202,53 @@ def test_host_entry_matches_device_entry(kernel):
     for k in out:
         assert torch.equal(out[k].cpu(), hout[k]), k
     assert torch.equal(g.cpu(), hg)
+
+
+@pytest.mark.parametrize("which", [1, 2, 3])
+def test_hard_rows(which):
+    """Rows that stress the numerics: near one-hot students and teachers, very small and very large
+    radii, large logit magnitudes, teacher equal to the student, a flat row."""
+    prev = P.set_kernel(which)
+    try:
+        V, N = 4096, 10
+        gen = torch.Generator(device=DEV).manual_seed(5)
+        s = 2.0 * torch.randn((N, V), generator=gen, device=DEV)
+        t = s + 1.5 * torch.randn((N, V), generator=gen, device=DEV)
+        s[0, 17] += 40.0                       # student nearly one-hot
+        t[1, 99] += 40.0                       # teacher nearly one-hot
+        s[2] *= 12.0; t[2] *= 12.0             # logits of magnitude ~100
+        t[3] = s[3]                            # teacher == student: saturated at once
+        s[4] = 0.0; t[4] = 0.0; t[4, 5] = 3.0  # flat student
+        s[5] += 300.0; t[5] -= 250.0           # large common offsets
+        s[6, 7] = 80.0; t[6, 9] = 80.0         # disjoint peaks: KL(T||p) huge
+        s, t = s.to(torch.bfloat16), t.to(torch.bfloat16)
+        x = torch.tensor([17, 3, 5, 8, 0, 11, 7, 1, 2, 3], dtype=torch.int32, device=DEV)
+        w = synth.Workload("t", N, V, "bf16", 0.1, 1.5, False, 0, 31)
+        redone = {}
+        for eps in (1e-6, 1e-4, 4e-4, 2e-3, 0.02, 0.1, 3.0):
+            _check_fwd_bwd(dict(s=s, t=t, proposal=x, mask=None), w, eps=eps)
+            redone[eps] = P.redo_count()
+            if eps < 5e-3:
+                assert P.last_kernel() == 1      # radii below 5e-3 are beyond float32 sums: float64 kernel
+            else:
+                assert P.last_kernel() == which
+    finally:
+        P.set_kernel(prev)
+
+
+def test_spec_verify_k_limits():
+    V = 2048
+    for K in (1, 16):
+        B = 6
+        w = synth.Workload("t", B * (K + 1), V, "bf16", 0.05, 1.0, True, 60 + K, 33, K=K)
+        d = synth.generate(w, DEV)
+        s3, t3 = d["s"].view(B, K + 1, V), d["t"].view(B, K + 1, V)
+        draft = d["proposal"].view(B, K + 1)[:, :K].contiguous()
+        res = P.spec_verify(s3, t3, draft, w.eps, seed=w.seed)
+        ref = O.spec_verify(to_np64(s3), to_np64(t3), draft.cpu().numpy(), w.eps, seed=w.seed)
+        ok = ref["margin"] >= 1e-6
+        assert np.array_equal(res["n_accept"].cpu().numpy()[ok], ref["n_accept"][ok])
+        assert np.array_equal(res["next_token"].cpu().numpy()[ok], ref["next_token"][ok])
+    with pytest.raises(P.SakiError):
+        bad = torch.zeros((2, 18, V), dtype=torch.bfloat16, device=DEV)
+        P.spec_verify(bad, bad, torch.zeros((2, 17), dtype=torch.int32, device=DEV), 0.1)
