@@ -121,6 +121,23 @@ SAKI_API int saki_route_fwd(const saki_in* in, const saki_out* out, void* cuda_s
 SAKI_API int saki_route_fwd_bwd(const saki_in* in, const saki_out* out, void* dlogits,
                        int64_t ld_g, float grad_scale, void* cuda_stream);
 
+/* saki_route_fwd_bwd for callers that must not allocate device memory: code that runs while an
+ * allocator is locked or memory is fully committed (inside another framework's allocator callback, a
+ * real-time serving loop with a frozen memory plan, a process whose device memory is entirely handed to
+ * a pool it may not touch).  The paper has no counterpart; this is a property of the library only.
+ * Same arguments, outputs and results as saki_route_fwd_bwd.  The one piece of scratch the routing needs
+ * (the list of rows that the float32 kernel passes on to the float64 kernel) lives in a fixed device
+ * array inside the library (4 MB per device, held from library load to process exit) instead of a buffer
+ * allocated on first use, so the call makes no cudaMalloc / cudaFree and calls no allocating routine.
+ *   - N may not exceed 1,048,576 rows: larger batches return SAKI_ERR_INVALID_ARG; split them.
+ *   - The first call on a device looks up the array's device address (once, with that device current);
+ *     make that first call before any stream capture.
+ *   - All calls on a device share the array.  The library clears what must start at zero at the start of
+ *     every call, but two calls whose kernels overlap on the GPU (different streams, no ordering between
+ *     them) race on it: order them, or use saki_route_fwd_bwd for one of them. */
+SAKI_API int saki_route_fwd_bwd_noalloc(const saki_in* in, const saki_out* out, void* dlogits,
+                                        int64_t ld_g, float grad_scale, void* cuda_stream);
+
 /* The same computation with every array in HOST memory (pageable or pinned):
  * the library stages rows through device buffers it allocates and caches,
  * overlapping the copies with the kernels on its own streams, and returns

@@ -19,7 +19,7 @@ SAKI_F32, SAKI_BF16 = 0, 1
 ROW_SATURATED, ROW_EPS_ZERO, ROW_MASKED, ROW_NONFINITE, ROW_BAD_ID, ROW_TIMEOUT, ROW_NOT_COMPUTED = 1, 2, 4, 8, 16, 32, 64
 
 _FLOAT_FIELDS = ("lambda", "kl", "tv", "accept_prob", "logp_x", "logq_x", "logT_x", "logp_y", "logq_y", "loss")
-EXPORTS = ("saki_route_fwd", "saki_route_fwd_bwd", "saki_route_host", "saki_spec_verify",
+EXPORTS = ("saki_route_fwd", "saki_route_fwd_bwd", "saki_route_fwd_bwd_noalloc", "saki_route_host", "saki_spec_verify",
            "saki_sample_proposal", "saki_check", "saki_set_kernel", "saki_last_kernel", "saki_redo_count",
            "saki_launch_count",
            "saki_last_error", "saki_version")
@@ -71,6 +71,8 @@ def load_library(path: str | None = None):
     lib = C.CDLL(p)
     lib.saki_route_fwd.argtypes = [C.POINTER(SakiIn), C.POINTER(SakiOut), C.c_void_p]
     lib.saki_route_fwd_bwd.argtypes = [C.POINTER(SakiIn), C.POINTER(SakiOut), C.c_void_p, C.c_int64, C.c_float, C.c_void_p]
+    lib.saki_route_fwd_bwd_noalloc.argtypes = lib.saki_route_fwd_bwd.argtypes
+    lib.saki_route_fwd_bwd_noalloc.restype = C.c_int
     lib.saki_route_host.argtypes = [C.POINTER(SakiIn), C.POINTER(SakiOut), C.c_void_p, C.c_int64, C.c_float]
     lib.saki_spec_verify.argtypes = [C.POINTER(SakiSpecIn), C.POINTER(SakiSpecOut), C.c_void_p]
     lib.saki_sample_proposal.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_float,
@@ -105,6 +107,11 @@ def _stream_ptr(stream) -> int:
     if stream is None:
         stream = torch.cuda.current_stream()
     return int(stream.cuda_stream)
+
+
+def alloc_outputs(n: int, device):
+    """Preallocated per-position output tensors for the calls that take `out=`."""
+    return _alloc_out(n, device)
 
 
 def _alloc_out(n: int, device, pinned=False):
@@ -166,6 +173,20 @@ def route_fwd_bwd(s, t, proposal, eps, temperature=1.0, seed=0, row_offset=0, ma
     si, so = _in_struct(s, t, proposal, mask, eps, temperature, seed, row_offset), _out_struct(out)
     _raise(lib, lib.saki_route_fwd_bwd(C.byref(si), C.byref(so), dlogits.data_ptr(), ld_g, grad_scale,
                                        _stream_ptr(stream)))
+    return out, dlogits
+
+
+def route_fwd_bwd_noalloc(s, t, proposal, eps, out, dlogits, temperature=1.0, seed=0, row_offset=0, mask=None,
+                          grad_scale=1.0, stream=None):
+    """saki_route_fwd_bwd_noalloc: the variant for callers that cannot allocate device memory.  The caller
+    passes every buffer (`out`: dict of preallocated output tensors, `dlogits`); the library's own scratch
+    is a fixed device array, so nothing is allocated on the way (at most 1,048,576 rows per call)."""
+    lib = load_library()
+    _check_rows(s, t)
+    ld_g = dlogits.stride(0) if dlogits.shape[0] > 1 else dlogits.shape[1]
+    si, so = _in_struct(s, t, proposal, mask, eps, temperature, seed, row_offset), _out_struct(out)
+    _raise(lib, lib.saki_route_fwd_bwd_noalloc(C.byref(si), C.byref(so), dlogits.data_ptr(), ld_g, grad_scale,
+                                               _stream_ptr(stream)))
     return out, dlogits
 
 

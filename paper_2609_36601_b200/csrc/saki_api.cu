@@ -73,6 +73,33 @@ static int redo_scratch(int64_t n_rows, int32_t** list, unsigned int** count) {
   return SAKI_OK;
 }
 
+// Fixed scratch of saki_route_fwd_bwd_noalloc: the redo list of the two-tier routing for callers that must
+// not allocate.  SAKI_NOALLOC_MAX_ROWS row ids plus the counter; every device that loads the library holds
+// these 4 MB until the process exits.
+#define SAKI_NOALLOC_MAX_ROWS (1 << 20)
+static __device__ __align__(256) int32_t g_noalloc_scratch[SAKI_NOALLOC_MAX_ROWS + 64];
+static std::mutex g_noalloc_mu;
+static int32_t* g_noalloc_ptr[64] = {nullptr};   // device address of the array, per device ordinal
+
+// In host code the array's name is only a handle; the kernels need its device address, looked up once per
+// device with that device current.
+static int noalloc_scratch(int32_t** list, unsigned int** count) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+  if (dev < 0 || dev >= 64) return fail(SAKI_ERR_UNSUPPORTED, "device ordinal %d outside the table", dev);
+  std::lock_guard<std::mutex> lock(g_noalloc_mu);
+  if (!g_noalloc_ptr[dev]) {
+    int32_t* ptr = nullptr;
+    e = cudaGetSymbolAddress((void**)&ptr, g_noalloc_scratch);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress (fixed scratch)");
+    g_noalloc_ptr[dev] = ptr;
+  }
+  *list = g_noalloc_ptr[dev];
+  *count = (unsigned int*)(g_noalloc_ptr[dev] + SAKI_NOALLOC_MAX_ROWS);
+  return SAKI_OK;
+}
+
 static int check_common(const void* s, const void* t, int64_t n, int32_t V, int32_t dtype, float eps, float tau) {
   if (n < 0) return fail(SAKI_ERR_INVALID_ARG, "negative row count");
   if (V < 2) return fail(SAKI_ERR_INVALID_ARG, "V must be >= 2 (got %d)", V);
@@ -131,9 +158,12 @@ static int dispatch_rows(RowParams p, int dtype, cudaStream_t st, int32_t* scrat
 }
 
 static int route_impl(const saki_in* in, const saki_out* out, void* dlogits, int64_t ld_g, float grad_scale,
-                      bool bwd, void* stream) {
+                      bool bwd, void* stream, bool fixed_scratch = false) {
   g_err[0] = 0;
   if (!in || !out) return fail(SAKI_ERR_INVALID_ARG, "NULL argument struct");
+  if (fixed_scratch && in->N > SAKI_NOALLOC_MAX_ROWS)
+    return fail(SAKI_ERR_INVALID_ARG, "N = %lld exceeds the fixed scratch of this entry point (%d rows): split the batch",
+                (long long)in->N, SAKI_NOALLOC_MAX_ROWS);
   int rc = check_common(in->student_logits, in->teacher_logits, in->N, in->V, in->dtype, in->eps, in->temperature);
   if (rc) return rc;
   if (in->ld_s < in->V || in->ld_t < in->V) return fail(SAKI_ERR_INVALID_ARG, "row stride smaller than V");
@@ -158,6 +188,13 @@ static int route_impl(const saki_in* in, const saki_out* out, void* dlogits, int
   p.out = *out;
   p.dlogits = bwd ? dlogits : nullptr; p.ld_g = ld_g; p.grad_scale = grad_scale;
   p.flagged = flagged;
+  if (fixed_scratch) {
+    int32_t* list = nullptr;
+    unsigned int* count = nullptr;
+    rc = noalloc_scratch(&list, &count);
+    if (rc) return rc;
+    return dispatch_rows(p, in->dtype, (cudaStream_t)stream, list, count);
+  }
   return dispatch_rows(p, in->dtype, (cudaStream_t)stream);
 }
 
@@ -248,6 +285,11 @@ SAKI_API int saki_route_fwd(const saki_in* in, const saki_out* out, void* cuda_s
 SAKI_API int saki_route_fwd_bwd(const saki_in* in, const saki_out* out, void* dlogits, int64_t ld_g, float grad_scale,
                        void* cuda_stream) {
   return route_impl(in, out, dlogits, ld_g, grad_scale, true, cuda_stream);
+}
+
+SAKI_API int saki_route_fwd_bwd_noalloc(const saki_in* in, const saki_out* out, void* dlogits, int64_t ld_g,
+                                        float grad_scale, void* cuda_stream) {
+  return route_impl(in, out, dlogits, ld_g, grad_scale, true, cuda_stream, true);
 }
 
 SAKI_API int saki_spec_verify(const saki_spec_in* in, const saki_spec_out* out, void* cuda_stream) {
