@@ -113,72 +113,98 @@ __device__ __forceinline__ float pow2f_exact(float n) {   // 2^n for whole n, cl
 #define SAKI_RES_UNROLL 1
 #endif
 constexpr int RES_UNROLL = SAKI_RES_UNROLL;   // unrolling of the resident-part loop
-constexpr int LOOKAHEAD = 2;            // global (L2) chunks in flight per thread
-constexpr int PF_STEPS = 8;             // first touch of a row: lines are requested this many steps ahead
+#ifndef SAKI_RING
+#define SAKI_RING 4
+#endif
+constexpr int NST = SAKI_RING;          // ring stages: steps of the streamed part in flight per warp
+constexpr int KS_RES = KS_MAX - NST;    // resident steps of a warp whose segment does not fit entirely
 
-__device__ __forceinline__ void prefetch_line_l2(const void* p) {
-  asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+// 16-byte asynchronous copy global -> shared (through L2 only), grouped per thread
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint64_t pol) {
+  asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "l"(pol) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+  return v;
 }
 
-// Visits this thread's chunks in step order: body(a, b, chunk, valid) -> bool (false = stop) with the
-// packed student / teacher words of the chunk.  Steps in which every lane has a chunk run without
-// predicates; global (L2) chunks are fetched LOOKAHEAD steps ahead, the first ones before the
-// resident part is processed.  FIRST_TOUCH: the row has not been read yet, so its global part is
-// additionally requested into L2 PF_STEPS steps ahead (one lane per 128-byte line).
-template <bool FIRST_TOUCH, typename Body>
+// The streamed part of a warp's segment passes through a ring of NST steps in shared memory.  Every
+// lane owns one 16-byte slot per stage and array and fills it itself (cp.async), so no lane ever
+// reads what another lane copied: a thread's own wait_group is all the synchronisation there is.
+// Invariant between passes: the first NST streamed steps of the coming pass are in flight or landed,
+// one committed group per step (empty where there is nothing to copy).
+struct Ring {
+  uint32_t s_slot, t_slot;   // shared-memory address of this lane's slot of stage 0 (a stage is 512 bytes on)
+  int stage;                 // stage of the next step to consume
+};
+
+// issue the first NST streamed steps of a row (after everything in flight has landed)
+__device__ __forceinline__ void ring_prime(Ring& rg, const Seg& sg, int lane, const __nv_bfloat16* g_s,
+                                           const __nv_bfloat16* g_t, uint64_t pol) {
+  cp_async_wait<0>();
+  int st = rg.stage;
+#pragma unroll
+  for (int j = 0; j < NST; ++j) {
+    const int c = sg.c0 + (sg.res + j) * 32 + lane;
+    if (g_s != nullptr && sg.res < sg.steps && c < sg.c1) {
+      cp_async16(rg.s_slot + st * 512, g_s + (size_t)c * 8, pol);
+      cp_async16(rg.t_slot + st * 512, g_t + (size_t)c * 8, pol);
+    }
+    cp_async_commit();
+    st = (st + 1 == NST) ? 0 : st + 1;
+  }
+}
+
+// Visits this thread's chunks in step order: body(a, b, chunk, valid) with the packed student /
+// teacher words of the chunk.  Resident steps are read from shared memory; streamed steps come out of
+// the ring, and each one consumed requests the step NST further on: of this pass, or, past its end,
+// of the next pass, whose rows are wrap_s / wrap_t (the same row again, the next row after the
+// last pass, nullptr if nothing follows).
+template <typename Body>
 __device__ __forceinline__ void for_each_chunk(const Seg& sg, int lane, const uint4* res_s, const uint4* res_t,
-                                               const __nv_bfloat16* g_s, const __nv_bfloat16* g_t, uint64_t pol,
-                                               Body&& body) {
+                                               const __nv_bfloat16* g_s, const __nv_bfloat16* g_t,
+                                               const __nv_bfloat16* wrap_s, const __nv_bfloat16* wrap_t,
+                                               uint64_t pol, Ring& rg, Body&& body) {
   const int full = (sg.c1 - sg.c0) >> 5;            // steps in which every lane has a chunk
   const int res_full = min(sg.res, full);
-  const int t0 = sg.c0 + sg.res * 32 + lane;        // this lane's first global chunk
-  if (FIRST_TOUCH && (lane & 7) == 0) {
-#pragma unroll
-    for (int j = LOOKAHEAD; j < PF_STEPS; ++j) {
-      const int c = t0 + 32 * j;
-      if (c < sg.c1) { prefetch_line_l2(g_s + (size_t)c * 8); prefetch_line_l2(g_t + (size_t)c * 8); }
-    }
-  }
-  uint4 qa[LOOKAHEAD], qb[LOOKAHEAD];
-#pragma unroll
-  for (int j = 0; j < LOOKAHEAD; ++j) {
-    const int c = t0 + 32 * j;
-    if (sg.res + j < full) { qa[j] = ld_l2(g_s + (size_t)c * 8, pol); qb[j] = ld_l2(g_t + (size_t)c * 8, pol); }
-  }
   // resident part; kept (nearly) rolled: the pass bodies are large and must stay in the instruction cache
 #pragma unroll RES_UNROLL
-  for (int k = 0; k < res_full; ++k)
-    if (!body(res_s[k * 32 + lane], res_t[k * 32 + lane], sg.c0 + k * 32 + lane, true)) return;
-  int c = t0;
-#pragma unroll 1
-  for (int k = sg.res; k < full; k += LOOKAHEAD) {
-#pragma unroll
-    for (int j = 0; j < LOOKAHEAD; ++j) {
-      if (k + j < full) {
-        const uint4 a = qa[j], b = qb[j];
-        if (k + j + LOOKAHEAD < full) {
-          const int cn = c + 32 * LOOKAHEAD;
-          qa[j] = ld_l2(g_s + (size_t)cn * 8, pol); qb[j] = ld_l2(g_t + (size_t)cn * 8, pol);
-        }
-        if (FIRST_TOUCH && (lane & 7) == 0) {
-          const int cp = c + 32 * PF_STEPS;
-          if (cp < sg.c1) { prefetch_line_l2(g_s + (size_t)cp * 8); prefetch_line_l2(g_t + (size_t)cp * 8); }
-        }
-        if (!body(a, b, c, true)) return;
-        c += 32;
-      }
-    }
-  }
-  if (full < sg.steps) {   // the last, partly filled step
-    const int cl = sg.c0 + full * 32 + lane;
+  for (int k = 0; k < res_full; ++k) body(res_s[k * 32 + lane], res_t[k * 32 + lane], sg.c0 + k * 32 + lane, true);
+  const uint4 filler = make_uint4(0xFF7FFF7Fu, 0xFF7FFF7Fu, 0xFF7FFF7Fu, 0xFF7FFF7Fu);   // exp -> 0, difference 0
+  if (res_full < sg.res) {   // a partly filled resident step (the segment then has no streamed part)
+    const int cl = sg.c0 + res_full * 32 + lane;
     const bool valid = cl < sg.c1;
-    uint4 a = make_uint4(0xFF7FFF7Fu, 0xFF7FFF7Fu, 0xFF7FFF7Fu, 0xFF7FFF7Fu), b = a;   // exp -> 0, difference 0
-    if (valid) {
-      if (full < sg.res) { a = res_s[full * 32 + lane]; b = res_t[full * 32 + lane]; }
-      else { a = ld_l2(g_s + (size_t)cl * 8, pol); b = ld_l2(g_t + (size_t)cl * 8, pol); }
-    }
+    uint4 a = filler, b = filler;
+    if (valid) { a = res_s[res_full * 32 + lane]; b = res_t[res_full * 32 + lane]; }
     body(a, b, cl, valid);
   }
+  const int T = sg.steps - sg.res;                  // streamed steps: 0 or more than NST
+  int c = sg.c0 + sg.res * 32 + lane;
+  int stage = rg.stage;
+#pragma unroll 1
+  for (int i = 0; i < T; ++i) {
+    cp_async_wait<NST - 1>();
+    const bool valid = c < sg.c1;
+    uint4 a = filler, b = filler;
+    if (valid) { a = lds128(rg.s_slot + stage * 512); b = lds128(rg.t_slot + stage * 512); }
+    {   // the step NST further on takes this slot
+      int cn = c + 32 * NST;
+      const __nv_bfloat16 *ns = g_s, *nt = g_t;
+      if (i + NST >= T) { cn -= 32 * T; ns = wrap_s; nt = wrap_t; }
+      if (ns != nullptr && cn < sg.c1) {
+        cp_async16(rg.s_slot + stage * 512, ns + (size_t)cn * 8, pol);
+        cp_async16(rg.t_slot + stage * 512, nt + (size_t)cn * 8, pol);
+      }
+      cp_async_commit();
+    }
+    stage = (stage + 1 == NST) ? 0 : stage + 1;
+    body(a, b, c, valid);
+    c += 32;
+  }
+  rg.stage = stage;
 }
 
 #ifdef SAKI_PHASE_TIMING
@@ -193,6 +219,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
   long long tacc[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
   long long tlast = clock64();
   int t_rows = 0;
+  long long w_solve = 0, w_lse = 0, w_final = 0;
 #endif
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint4* res_s = reinterpret_cast<const uint4*>(smem + ROFF_S) + warp * RES_CHUNKS;
@@ -208,11 +235,13 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
   sg.c0 = min(n_chunks, warp * cpw);
   sg.c1 = min(n_chunks, sg.c0 + cpw);
   sg.steps = (sg.c1 - sg.c0 + 31) / 32;
-  sg.res = min(sg.steps, KS_MAX);
+  sg.res = sg.steps <= KS_MAX ? sg.steps : KS_RES;   // a segment that does not fit leaves NST steps to the ring
   const int res_chunks = min(sg.c1 - sg.c0, sg.res * 32);          // resident chunks of this warp
   const uint32_t res_bytes = (uint32_t)res_chunks * 16u;
-  const int l2_first = sg.c0 + res_chunks;                          // first chunk read from global memory
-  const uint32_t l2_bytes = (uint32_t)max(0, sg.c1 - l2_first) * 16u;
+  Ring rg;
+  rg.s_slot = smem_addr(res_s + KS_RES * 32 + lane);
+  rg.t_slot = smem_addr(res_t + KS_RES * 32 + lane);
+  rg.stage = 0;
 
   const float c32 = (float)(1.4426950408889634 / (double)P.temperature);     // log2(e)/temperature
   Consts K;
@@ -256,7 +285,12 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
-  if (lane == 0 && (int64_t)blockIdx.x < P.n_rows) issue(blockIdx.x);
+  if ((int64_t)blockIdx.x < P.n_rows) {
+    if (lane == 0) issue(blockIdx.x);
+    const __nv_bfloat16 *s0, *t0;
+    row_ptrs(blockIdx.x, s0, t0);
+    ring_prime(rg, sg, lane, s0, t0, pol_last);
+  }
   uint32_t phase = 0;
   bool dead = false;
   int rb = 0;
@@ -273,6 +307,8 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
     row_ptrs(row, g_s, g_t);
     __nv_bfloat16* g_out = P.dlogits ? (__nv_bfloat16*)P.dlogits + row * P.ld_g : nullptr;
     const int64_t next_row = row + gridDim.x;
+    const __nv_bfloat16 *n_s = nullptr, *n_t = nullptr;   // the next row of this CTA, if any
+    if (next_row < P.n_rows) row_ptrs(next_row, n_s, n_t);
 
     RTS(0);
     // row scalars that do not depend on the passes
@@ -298,7 +334,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       float ms_run = -CUDART_INF_F, mt_run = -CUDART_INF_F, ks = 1e30f, kt = 1e30f;
       int my_arg = 0x7fffffff;                   // lowest index of this thread's teacher maximum
       const float2 cc = splat(c32), neg1 = splat(-1.f);
-      for_each_chunk<true>(sg, lane, res_s, res_t, g_s, g_t, pol_last, [&](const uint4& s4, const uint4& t4, int c, bool valid) {
+      for_each_chunk(sg, lane, res_s, res_t, g_s, g_t, g_s, g_t, pol_last, rg, [&](const uint4& s4, const uint4& t4, int c, bool valid) {
         const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
         const float2 cms = unpack_bf16x2(max_bf16x2(max_bf16x2(sw[0], sw[1]), max_bf16x2(sw[2], sw[3])));
         const float2 cmt = unpack_bf16x2(max_bf16x2(max_bf16x2(tw[0], tw[1]), max_bf16x2(tw[2], tw[3])));
@@ -337,7 +373,6 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           M3 = ffma2(t2, d, M3);
           N1 = ffma2(et, d, N1);
         }
-        return true;
       });
       RTS(2);
       // warp: common shifts (the smallest), teacher argmax, sums
@@ -413,7 +448,10 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       const float cb = (float)bc[BC_CB], kb = (float)bc[BC_KB];
       float2 S0 = splat(0.f), S1 = splat(0.f), S2 = splat(0.f);
       const float2 cc = splat(c32), cbb = splat(cb), kbb = splat(kb), neg1 = splat(-1.f);
-      for_each_chunk<false>(sg, lane, res_s, res_t, g_s, g_t, pol_last, [&](const uint4& s4, const uint4& t4, int, bool) {
+#ifdef SAKI_PHASE_TIMING
+      const long long w_t0 = clock64();
+#endif
+      for_each_chunk(sg, lane, res_s, res_t, g_s, g_t, g_s, g_t, pol_last, rg, [&](const uint4& s4, const uint4& t4, int, bool) {
         const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -425,8 +463,10 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           S1 = fadd2(S1, t1);
           S2 = ffma2(t1, d, S2);
         }
-        return true;
       });
+#ifdef SAKI_PHASE_TIMING
+      w_solve += clock64() - w_t0; ++w_lse;
+#endif
       RTS(7);
       auto tot = [](const float2 a) { return (double)a.x + (double)a.y; };
       const double v[3] = {warp_sum_d(tot(S0)), warp_sum_d(tot(S1)), warp_sum_d(tot(S2))};
@@ -458,6 +498,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         issue(next_row);
       }
+      ring_prime(rg, sg, lane, n_s, n_t, pol_last);   // the ring holds steps of this row: refill it for the next
       continue;
     }
 
@@ -477,7 +518,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       float* step_w = (float*)(smem + ROFF_STEP) + warp * MAX_STEPS;   // draw weight of each of this warp's steps
       int n_res_done = 0;
       bool next_issued = false;
-      for_each_chunk<false>(sg, lane, res_s, res_t, g_s, g_t, pol_last, [&](const uint4& s4, const uint4& t4, int c, bool valid) {
+      for_each_chunk(sg, lane, res_s, res_t, g_s, g_t, n_s, n_t, pol_last, rg, [&](const uint4& s4, const uint4& t4, int c, bool valid) {
         const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
         uint32_t gp[4];
         float2 sqc = splat(0.f), rc = splat(0.f);       // this chunk's share of Sq and R
@@ -524,7 +565,6 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           }
           next_issued = true;
         }
-        return true;
       });
       if (!next_issued && !need_draw && lane == 0 && !dead && next_row < P.n_rows) issue(next_row);   // no elements
       RTS(11);
@@ -633,6 +673,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
 
 #ifdef SAKI_PHASE_TIMING
   for (int64_t row = blockIdx.x; row < P.n_rows; row += gridDim.x) ++t_rows;
+  if (lane == 0 && blockIdx.x == 5 && t_rows > 0) printf("warp %d solve loop %lld cycles per row, %lld evaluations in %d rows, %d steps\n", warp, w_solve / t_rows, w_lse, t_rows, sg.steps);
   if ((tid == 0 || tid == 1023) && (blockIdx.x == 0 || blockIdx.x == 77) && t_rows > 0)
     printf("blk %d tid %d rows %d | endbar %lld copy-wait %lld | lse %lld warp+bar %lld gather %lld scalar %lld | "
            "bar %lld solve %lld combine %lld scalar %lld | bar %lld final %lld combine %lld tail %lld (cycles per row)\n",
@@ -640,6 +681,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
            tacc[4] / t_rows, tacc[5] / t_rows, tacc[6] / t_rows, tacc[7] / t_rows, tacc[8] / t_rows, tacc[9] / t_rows,
            tacc[10] / t_rows, tacc[11] / t_rows, tacc[12] / t_rows, tacc[13] / t_rows);
 #endif
+  cp_async_wait<0>();
   // a CTA that gave up on a copy still waits (bounded) for what it has in flight before leaving
   if (dead && tid == 0) (void)mbar_wait_bounded(mbar, phase);
 }
