@@ -316,16 +316,17 @@ static __device__ __noinline__ void scalar_find_owner(double* bc, const double* 
   bc[BC_OWNER_WARP] = (double)owner; bc[BC_BEFORE] = before; bc[BC_TARGET] = target; bc[BC_TAKE_LAST] = take_last;
 }
 
-static __device__ __noinline__ void write_result(const double* bc, saki_out out, bool write_loss, int64_t row, int corrected,
-                                          int y, bool bonus, double c64, const __nv_bfloat16* g_s,
-                                          const __nv_bfloat16* g_t) {
+// tv: the row's total variation (the caller may hold it before bc[BC_TV] is written)
+static __device__ __noinline__ void write_result_tv(const double* bc, saki_out out, bool write_loss, int64_t row, int corrected,
+                                             int y, bool bonus, double c64, const __nv_bfloat16* g_s,
+                                             const __nv_bfloat16* g_t, double tv) {
   RowResult r;
   const double lam = bc[BC_LAMBDA], G0 = bc[BC_G0], G1 = bc[BC_G1], Glam = bc[BC_GLAM];
   const double Lam = Glam - (1.0 - lam) * G0 - lam * G1;
   const double lp_x = bc[BC_LPX], lT_x = bc[BC_LTX];
   const uint32_t status = (uint32_t)bc[BC_STATUS];
   r.corrected = corrected; r.token = y; r.vstar = (int)bc[BC_VSTAR];
-  r.lambda = (float)lam; r.kl = (float)bc[BC_KL]; r.tv = (float)bc[BC_TV];
+  r.lambda = (float)lam; r.kl = (float)bc[BC_KL]; r.tv = (float)tv;
   r.accept = bonus ? 0.f : (float)bc[BC_ACC];
   r.logp_x = (float)lp_x; r.logT_x = (float)lT_x;
   r.logq_x = bonus ? 0.f : (float)(lp_x + lam * (lT_x - lp_x) - Lam);
@@ -339,6 +340,11 @@ static __device__ __noinline__ void write_result(const double* bc, saki_out out,
   } else { r.logp_y = r.logp_x; r.logq_y = r.logq_x; }
   r.status = status;
   write_row(out, row, r, write_loss);
+}
+__device__ __forceinline__ void write_result(const double* bc, saki_out out, bool write_loss, int64_t row, int corrected,
+                                             int y, bool bonus, double c64, const __nv_bfloat16* g_s,
+                                             const __nv_bfloat16* g_t) {
+  write_result_tv(bc, out, write_loss, row, corrected, y, bonus, c64, g_s, g_t, bc[BC_TV]);
 }
 
 

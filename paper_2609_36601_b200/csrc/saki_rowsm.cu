@@ -41,6 +41,7 @@ constexpr int KS_MAX = RT == 512 ? 13 : RT == 640 ? 10 : RT == 768 ? 8 : 6;  // 
 constexpr int MAX_STEPS = 64;            // steps per warp the draw bookkeeping can hold (V <= 64*32*8*RW)
 constexpr int RES_CHUNKS = KS_MAX * 32; // resident chunks per warp and row
 constexpr int RNV = 8;                  // doubles per partial vector
+static_assert(RW >= 12, "warps 8-11 do side work while warps 0-6 gather");
 
 constexpr int ROFF_S = 0;                                        // [RW][RES_CHUNKS] uint4
 constexpr int ROFF_T = RW * RES_CHUNKS * 16;
@@ -131,80 +132,92 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   return v;
 }
 
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t w) {
+  asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(w) : "memory");
+}
+constexpr uint32_t FILLER = 0xFF7FFF7Fu;          // two bf16 of the most negative finite value: exp -> 0, difference 0
+constexpr uint32_t T_OFF = RW * RES_CHUNKS * 16;  // a teacher slot lies this far behind its student slot
+
 // The streamed part of a warp's segment passes through a ring of NST steps in shared memory.  Every
-// lane owns one 16-byte slot per stage and array and fills it itself (cp.async), so no lane ever
-// reads what another lane copied: a thread's own wait_group is all the synchronisation there is.
-// Invariant between passes: the first NST streamed steps of the coming pass are in flight or landed,
-// one committed group per step (empty where there is nothing to copy).
+// lane owns one 16-byte slot per stage and array and fills it itself (cp.async, or the filler where
+// the row has no chunk for it), so no lane ever reads what another lane wrote: a thread's own
+// wait_group is all the synchronisation there is.  Invariant between passes: the first NST streamed
+// steps of the coming pass are in flight or landed, one committed group per step.
 struct Ring {
-  uint32_t s_slot, t_slot;   // shared-memory address of this lane's slot of stage 0 (a stage is 512 bytes on)
-  int stage;                 // stage of the next step to consume
+  uint32_t base;   // shared-memory address of this lane's student slot of stage 0 (a stage is 512 bytes on)
+  uint32_t slot;   // slot of the next step to consume
 };
 
-// issue the first NST streamed steps of a row (after everything in flight has landed)
+// request the first NST streamed steps of a row (g_s == nullptr: no row) once everything in flight has landed
 __device__ __forceinline__ void ring_prime(Ring& rg, const Seg& sg, int lane, const __nv_bfloat16* g_s,
                                            const __nv_bfloat16* g_t, uint64_t pol) {
   cp_async_wait<0>();
-  int st = rg.stage;
+  if (sg.res == sg.steps) return;          // nothing is streamed
+  uint32_t slot = rg.slot;
 #pragma unroll
   for (int j = 0; j < NST; ++j) {
     const int c = sg.c0 + (sg.res + j) * 32 + lane;
-    if (g_s != nullptr && sg.res < sg.steps && c < sg.c1) {
-      cp_async16(rg.s_slot + st * 512, g_s + (size_t)c * 8, pol);
-      cp_async16(rg.t_slot + st * 512, g_t + (size_t)c * 8, pol);
+    if (g_s != nullptr && c < sg.c1) {
+      cp_async16(slot, g_s + (size_t)c * 8, pol);
+      cp_async16(slot + T_OFF, g_t + (size_t)c * 8, pol);
+    } else {
+      sts128(slot, FILLER);
+      sts128(slot + T_OFF, FILLER);
     }
     cp_async_commit();
-    st = (st + 1 == NST) ? 0 : st + 1;
+    slot += 512;
+    if (slot == rg.base + NST * 512) slot = rg.base;
   }
 }
 
 // Visits this thread's chunks in step order: body(a, b, chunk, valid) with the packed student /
-// teacher words of the chunk.  Resident steps are read from shared memory; streamed steps come out of
-// the ring, and each one consumed requests the step NST further on: of this pass, or, past its end,
-// of the next pass, whose rows are wrap_s / wrap_t (the same row again, the next row after the
-// last pass, nullptr if nothing follows).
+// teacher words of the chunk (the filler where valid is false).  Resident steps are read from shared
+// memory; streamed steps come out of the ring, and each one consumed requests the step NST further
+// on: of this pass, or, past its end, of the next pass, whose rows are wrap_s / wrap_t (the same row
+// again, the next row after the last pass, nullptr if nothing follows).
 template <typename Body>
 __device__ __forceinline__ void for_each_chunk(const Seg& sg, int lane, const uint4* res_s, const uint4* res_t,
                                                const __nv_bfloat16* g_s, const __nv_bfloat16* g_t,
                                                const __nv_bfloat16* wrap_s, const __nv_bfloat16* wrap_t,
                                                uint64_t pol, Ring& rg, Body&& body) {
-  const int full = (sg.c1 - sg.c0) >> 5;            // steps in which every lane has a chunk
-  const int res_full = min(sg.res, full);
-  // resident part; kept (nearly) rolled: the pass bodies are large and must stay in the instruction cache
+  // resident part (slots past the end of the segment hold the filler); kept rolled: the pass bodies
+  // are large and must stay in the instruction cache
+  int c = sg.c0 + lane;
 #pragma unroll RES_UNROLL
-  for (int k = 0; k < res_full; ++k) body(res_s[k * 32 + lane], res_t[k * 32 + lane], sg.c0 + k * 32 + lane, true);
-  const uint4 filler = make_uint4(0xFF7FFF7Fu, 0xFF7FFF7Fu, 0xFF7FFF7Fu, 0xFF7FFF7Fu);   // exp -> 0, difference 0
-  if (res_full < sg.res) {   // a partly filled resident step (the segment then has no streamed part)
-    const int cl = sg.c0 + res_full * 32 + lane;
-    const bool valid = cl < sg.c1;
-    uint4 a = filler, b = filler;
-    if (valid) { a = res_s[res_full * 32 + lane]; b = res_t[res_full * 32 + lane]; }
-    body(a, b, cl, valid);
-  }
+  for (int k = 0; k < sg.res; ++k, c += 32) body(res_s[k * 32 + lane], res_t[k * 32 + lane], c, c < sg.c1);
   const int T = sg.steps - sg.res;                  // streamed steps: 0 or more than NST
-  int c = sg.c0 + sg.res * 32 + lane;
-  int stage = rg.stage;
+  if (T <= 0) return;
+  const int c_first = c;
+  int cn = c + 32 * NST;                            // the chunk requested next, and where it comes from
+  int lim = sg.c1;
+  const __nv_bfloat16* ns = g_s + (size_t)cn * 8;
+  const __nv_bfloat16* nt = g_t + (size_t)cn * 8;
+  uint32_t slot = rg.slot;
+  const uint32_t slot_end = rg.base + NST * 512;
 #pragma unroll 1
-  for (int i = 0; i < T; ++i) {
-    cp_async_wait<NST - 1>();
-    const bool valid = c < sg.c1;
-    uint4 a = filler, b = filler;
-    if (valid) { a = lds128(rg.s_slot + stage * 512); b = lds128(rg.t_slot + stage * 512); }
-    {   // the step NST further on takes this slot
-      int cn = c + 32 * NST;
-      const __nv_bfloat16 *ns = g_s, *nt = g_t;
-      if (i + NST >= T) { cn -= 32 * T; ns = wrap_s; nt = wrap_t; }
-      if (ns != nullptr && cn < sg.c1) {
-        cp_async16(rg.s_slot + stage * 512, ns + (size_t)cn * 8, pol);
-        cp_async16(rg.t_slot + stage * 512, nt + (size_t)cn * 8, pol);
-      }
-      cp_async_commit();
+  for (int i = 0; i < T; ++i, c += 32) {
+    if (i == T - NST) {   // from here on the requests belong to the pass that follows
+      cn = c_first;
+      lim = wrap_s != nullptr ? sg.c1 : -0x7fffffff;
+      ns = (wrap_s != nullptr ? wrap_s : g_s) + (size_t)cn * 8;
+      nt = (wrap_t != nullptr ? wrap_t : g_t) + (size_t)cn * 8;
     }
-    stage = (stage + 1 == NST) ? 0 : stage + 1;
-    body(a, b, c, valid);
-    c += 32;
+    cp_async_wait<NST - 1>();
+    const uint4 a = lds128(slot), b = lds128(slot + T_OFF);
+    if (cn < lim) {
+      cp_async16(slot, ns, pol);
+      cp_async16(slot + T_OFF, nt, pol);
+    } else {
+      sts128(slot, FILLER);
+      sts128(slot + T_OFF, FILLER);
+    }
+    cp_async_commit();
+    cn += 32; ns += 256; nt += 256;
+    slot += 512;
+    if (slot == slot_end) slot = rg.base;
+    body(a, b, c, c < sg.c1);
   }
-  rg.stage = stage;
+  rg.slot = slot;
 }
 
 #ifdef SAKI_PHASE_TIMING
@@ -239,9 +252,13 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
   const int res_chunks = min(sg.c1 - sg.c0, sg.res * 32);          // resident chunks of this warp
   const uint32_t res_bytes = (uint32_t)res_chunks * 16u;
   Ring rg;
-  rg.s_slot = smem_addr(res_s + KS_RES * 32 + lane);
-  rg.t_slot = smem_addr(res_t + KS_RES * 32 + lane);
-  rg.stage = 0;
+  rg.base = smem_addr(res_s + KS_RES * 32 + lane);
+  rg.slot = rg.base;
+  // slots of the resident area that no copy ever writes (a segment that ends inside its last step) hold the filler
+  for (int k = res_chunks + lane; k < RES_CHUNKS; k += 32) {
+    sts128(smem_addr(res_s + k), FILLER);
+    sts128(smem_addr(res_t + k), FILLER);
+  }
 
   const float c32 = (float)(1.4426950408889634 / (double)P.temperature);     // log2(e)/temperature
   Consts K;
@@ -294,6 +311,16 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
   uint32_t phase = 0;
   bool dead = false;
   int rb = 0;
+  // A row that needs no draw leaves its outputs to be written while the next row's sums are gathered
+  // (its broadcast buffer stays intact for one more row); the last one is written after the loop.
+  int64_t pending_row = -1;
+  auto write_pending = [&](int64_t row, const double* bcp) {
+    const __nv_bfloat16 *s, *t;
+    row_ptrs(row, s, t);
+    const int64_t b = row / P.K1;
+    const int xp = P.spec ? P.proposal[b * P.prop_ld + (row - b * P.K1)] : P.proposal[row];
+    write_result(bcp, P.out, !P.spec, row, 0, xp, false, K.c64, s, t);
+  };
 
   for (int64_t row = blockIdx.x; row < P.n_rows; row += gridDim.x, rb ^= 1) {
     double* bc = (double*)(smem + ROFF_BC) + rb * BC_DOUBLES;   // this row's broadcast scalars
@@ -311,14 +338,6 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
     if (next_row < P.n_rows) row_ptrs(next_row, n_s, n_t);
 
     RTS(0);
-    // row scalars that do not depend on the passes
-    if (tid == 32) bc[BC_UACC] = scalar_uniform(P.seed, rid, STAGE_ACCEPT);
-    if (tid == 64) bc[BC_UDRAW] = scalar_uniform(P.seed, rid, bonus ? STAGE_BONUS : STAGE_RESIDUAL);
-    if (tid == 96) {
-      const bool ok = (x >= 0 && x < V);
-      bc[BC_SX] = ok ? (double)__bfloat162float(g_s[x]) : 0.0;
-      bc[BC_TX] = ok ? (double)__bfloat162float(g_t[x]) : 0.0;
-    }
     if (!dead) {
       if (!mbar_wait_bounded(mbar, phase)) dead = true;
       else phase ^= 1u;
@@ -429,7 +448,19 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           }
           if (lane == 0) gat[6] = (double)garg;
         }
+      } else if (lane == 0) {
+        // meanwhile, on warps that would only wait: the row scalars that do not depend on the passes,
+        // and the previous row's outputs
+        if (warp == 8) bc[BC_UACC] = scalar_uniform(P.seed, rid, STAGE_ACCEPT);
+        if (warp == 9) bc[BC_UDRAW] = scalar_uniform(P.seed, rid, bonus ? STAGE_BONUS : STAGE_RESIDUAL);
+        if (warp == 10) {
+          const bool ok = (x >= 0 && x < V);
+          bc[BC_SX] = ok ? (double)__bfloat162float(g_s[x]) : 0.0;
+          bc[BC_TX] = ok ? (double)__bfloat162float(g_t[x]) : 0.0;
+        }
+        if (warp == 11 && pending_row >= 0) write_pending(pending_row, (const double*)(smem + ROFF_BC) + (rb ^ 1) * BC_DOUBLES);
       }
+      pending_row = -1;
       if (any_dead) dead = true;
       __syncthreads();
       RTS(4);
@@ -505,6 +536,9 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
     // ------------------------------------------------ pass "final"
     RTS(10);
     const bool need_draw = bonus || bc[BC_CORR] != 0.0;
+    int d_owner = -1;                    // the draw: owning warp, weight before it, target, "take the last position"
+    double d_before = 0.0, d_target = 0.0;
+    bool d_last = false;
     const float cl = (float)bc[BC_CL], kq = (float)bc[BC_KQ];
     const float iq = (float)bc[BC_IQ], ip = (float)bc[BC_IP];
     const int tok = (int)bc[BC_TOK];
@@ -556,8 +590,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
         }
         if (want_g && valid) st_stream(g_out + (size_t)c * 8, make_uint4(gp[0], gp[1], gp[2], gp[3]), pol_first);
         // once the warp has read its resident part for the last time, the next row's may land there
-        // (a row that still needs its draw may re-read one resident step: its copy is issued after the draw)
-        if (++n_res_done == sg.res && !need_draw) {
+        if (++n_res_done == sg.res) {
           __syncwarp();
           if (lane == 0 && !dead && next_row < P.n_rows) {
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -566,33 +599,56 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           next_issued = true;
         }
       });
-      if (!next_issued && !need_draw && lane == 0 && !dead && next_row < P.n_rows) issue(next_row);   // no elements
+      if (!next_issued && lane == 0 && !dead && next_row < P.n_rows) issue(next_row);   // no elements
       RTS(11);
       const float sq_f = Sq.x + Sq.y, r_f = R.x + R.y;
       double part = 0.0;                               // this warp's draw weight: its step weights, in order
       if (need_draw) {
         __syncwarp();
         const int ns = min(sg.steps, MAX_STEPS);
-        for (int k = 0; k < ns; ++k) part += (double)step_w[k];
+        static_assert(MAX_STEPS <= 64, "two step weights per lane");
+        part = warp_sum_d((lane < ns ? (double)step_w[lane] : 0.0) + (lane + 32 < ns ? (double)step_w[lane + 32] : 0.0));
       }
-      const double v[2] = {warp_sum_d((double)sq_f), warp_sum_d((double)r_f)};
-      if (lane == 0) red[2 * RW + warp] = part;     // ordered per-warp weights of the draw
-      combine(v, 2);
+      const double v0 = warp_sum_d((double)sq_f), v1 = warp_sum_d((double)r_f);
+      if (lane == 0) { red[warp] = v0; red[RW + warp] = v1; red[2 * RW + warp] = part; }   // part: ordered per-warp weights of the draw
+      __syncthreads();
+      if (warp < 2) {
+        const double a = warp_sum_d(lane < RW ? red[warp * RW + lane] : 0.0);
+        if (lane == 0) gat[warp] = a;
+      }
+      if (need_draw) {
+        // every warp finds the warp that owns the inverse-CDF target (ordered scan of the per-warp weights)
+        const double mine = lane < RW ? red[2 * RW + lane] : 0.0;
+        double inc = mine;
+#pragma unroll
+        for (int o = 1; o < RW; o <<= 1) {
+          const double up = __shfl_up_sync(0xffffffffu, inc, o);
+          if (lane >= o) inc += up;
+        }
+        d_target = bc[BC_UDRAW] * __shfl_sync(0xffffffffu, inc, RW - 1);
+        const unsigned cross = __ballot_sync(0xffffffffu, lane < RW && inc > d_target);
+        const unsigned posw = __ballot_sync(0xffffffffu, mine > 0.0);
+        if (cross) {
+          d_owner = __ffs(cross) - 1;
+          d_before = __shfl_sync(0xffffffffu, inc - mine, d_owner);
+        } else {       // rounding left no crossing: the last warp with positive weight, its last position
+          d_owner = posw ? 31 - __clz(posw) : 0;
+          d_before = 0.0;
+          d_last = true;
+        }
+      }
+      __syncthreads();
       RTS(12);
-      if (tid == 0) {
-        bc[BC_TV] = (bc[BC_LAMBDA] > 0.0) ? gat[1] : 0.0;
-        if (!need_draw) write_result(bc, P.out, !P.spec, row, 0, x, false, K.c64, g_s, g_t);
-      }
+      if (tid == 0) bc[BC_TV] = (bc[BC_LAMBDA] > 0.0) ? gat[1] : 0.0;
+      if (!need_draw) pending_row = row;
     }
 
     // ------------------------------------------------ the draw (corrected and bonus rows only)
     if (need_draw) {
-      if (tid == 0) scalar_find_owner(bc, red + 2 * RW, RW);
-      __syncthreads();
-      if (warp == (int)bc[BC_OWNER_WARP]) {
-        const double target = bc[BC_TARGET];
-        bool last_mode = bc[BC_TAKE_LAST] != 0.0;
-        double running = bc[BC_BEFORE];
+      if (warp == d_owner) {
+        const double target = d_target;
+        bool last_mode = d_last;
+        double running = d_before;
         const float* step_w = (const float*)(smem + ROFF_STEP) + warp * MAX_STEPS;
         const int ns = min(sg.steps, MAX_STEPS);
         // the step that holds the target (every lane walks the same few numbers)
@@ -607,10 +663,8 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
         const int c = sg.c0 + ks * 32 + lane;
         const bool valid = c < sg.c1;
         uint4 s4 = make_uint4(0xFF7FFF7Fu, 0xFF7FFF7Fu, 0xFF7FFF7Fu, 0xFF7FFF7Fu), t4 = s4;
-        if (valid) {
-          if (ks < sg.res) { s4 = res_s[ks * 32 + lane]; t4 = res_t[ks * 32 + lane]; }
-          else { s4 = ld_l2(g_s + (size_t)c * 8, pol_last); t4 = ld_l2(g_t + (size_t)c * 8, pol_last); }
-        }
+        // from global memory: the warp's resident area may already be receiving the next row
+        if (valid) { s4 = ld_l2(g_s + (size_t)c * 8, pol_last); t4 = ld_l2(g_t + (size_t)c * 8, pol_last); }
         const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
         float w[8];
 #pragma unroll
@@ -658,12 +712,9 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           y = __shfl_sync(0xffffffffu, lastp, 31 - __clz(posm));
         }
         if (y < 0) y = min(V - 1, max(sg.c0 * 8, sg.c1 * 8 - 1));
-        if (lane == 0) write_result(bc, P.out, !P.spec, row, bonus ? 0 : 1, y, bonus, K.c64, g_s, g_t);
-      }
-      __syncwarp();
-      if (lane == 0 && !dead && next_row < P.n_rows) {
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        issue(next_row);
+        if (lane == 0)
+          write_result_tv(bc, P.out, !P.spec, row, bonus ? 0 : 1, y, bonus, K.c64, g_s, g_t,
+                          (bc[BC_LAMBDA] > 0.0) ? gat[1] : 0.0);
       }
     }
     RTS(13);
@@ -682,6 +733,8 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
            tacc[10] / t_rows, tacc[11] / t_rows, tacc[12] / t_rows, tacc[13] / t_rows);
 #endif
   cp_async_wait<0>();
+  __syncthreads();
+  if (tid == 11 * 32 && pending_row >= 0) write_pending(pending_row, (const double*)(smem + ROFF_BC) + (rb ^ 1) * BC_DOUBLES);
   // a CTA that gave up on a copy still waits (bounded) for what it has in flight before leaving
   if (dead && tid == 0) (void)mbar_wait_bounded(mbar, phase);
 }
