@@ -201,13 +201,20 @@ __device__ __forceinline__ void decide(double* bc, const Consts& K, double lam, 
 }
 
 // after pass "lse": v = {Ss, St, M1, M2, M3, N1, argmax index} on the row's shifts k0, k1
+// e_max: upper bound of the largest term of either sum (1 when the shifts come from the rows' maxima);
+// overflow_redo: shifts that come from an estimate of the maxima can overflow on finite rows, so
+// non-finite sums hand the row to the float64 kernel instead of flagging it.
 static __device__ __noinline__ void scalar_after_lse(double* bc, const double* v, Consts K, float k0f, float k1f, int x,
-                                              bool bonus, bool masked, bool row_timeout) {
+                                              bool bonus, bool masked, bool row_timeout, float e_max = 1.f,
+                                              bool overflow_redo = false) {
   const double SsT = v[0], StT = v[1], eps = K.eps, k0 = (double)k0f, k1 = (double)k1f;
   uint32_t status = 0;
   const double chk = ((v[0] + v[1]) + (v[2] + v[3])) + (v[4] + v[5]);
   if (row_timeout) status = SAKI_ROW_TIMEOUT;
-  else if (!(fabs(chk) < CUDART_INF) || !(SsT > 0.0) || !(StT > 0.0)) status = SAKI_ROW_NONFINITE;
+  else if (!(fabs(chk) < CUDART_INF) || !(SsT > 0.0) || !(StT > 0.0)) {
+    if (overflow_redo) { bc[BC_MODE] = MODE_REDO; return; }
+    status = SAKI_ROW_NONFINITE;
+  }
   else if (!bonus && (x < 0 || x >= K.V)) status = SAKI_ROW_BAD_ID;
   const int vstar = (v[6] >= 0.0 && v[6] < (double)K.V) ? (int)v[6] : 0;
   bc[BC_VSTAR] = (double)vstar;
@@ -215,7 +222,7 @@ static __device__ __noinline__ void scalar_after_lse(double* bc, const double* v
   const double rSs = rcp_fast(SsT), rSt = rcp_fast(StT);
   const double G0 = LN2 * (log2_fast(SsT) - k0), G1 = LN2 * (log2_fast(StT) - k1);
   bc[BC_G0] = G0; bc[BC_G1] = G1; bc[BC_RSS] = rSs;
-  bc[BC_PMAX] = fmax(rSs, rSt);      // upper bound of the largest probability of either row
+  bc[BC_PMAX] = fmin(1.0, (double)e_max * fmax(rSs, rSt));      // upper bound of the largest probability of either row
   if (!(eps > 0.0)) {          // student-only endpoint
     bc[BC_KL] = 0.0;
     decide(bc, K, 0.0, G0, G0, G1, k0, k1, rSs, status | SAKI_ROW_EPS_ZERO, vstar, bonus, masked, x);

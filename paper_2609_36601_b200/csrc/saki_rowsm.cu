@@ -37,19 +37,20 @@ namespace saki {
 #endif
 constexpr int RT = SAKI_ROWSM_THREADS;  // threads per CTA
 constexpr int RW = RT / 32;             // warps per CTA
-constexpr int KS_MAX = RT == 512 ? 13 : RT == 640 ? 10 : RT == 768 ? 8 : 6;  // resident steps per warp (a step = 32 chunks of 8 elements)
+constexpr int KS_MAX = 208 / RW;        // steps per warp that fit in shared memory (a step = 32 chunks of 8 elements = 1 KB of logit pairs)
 constexpr int MAX_STEPS = 64;            // steps per warp the draw bookkeeping can hold (V <= 64*32*8*RW)
 constexpr int RES_CHUNKS = KS_MAX * 32; // resident chunks per warp and row
 constexpr int RNV = 8;                  // doubles per partial vector
 static_assert(RW >= 12, "warps 8-11 do side work while warps 0-6 gather");
+static_assert(KS_MAX - 4 >= 1, "every warp keeps at least its first step resident");
 
 constexpr int ROFF_S = 0;                                        // [RW][RES_CHUNKS] uint4
 constexpr int ROFF_T = RW * RES_CHUNKS * 16;
 constexpr int ROFF_RED = 2 * RW * RES_CHUNKS * 16;               // [RNV][RW] doubles
 constexpr int ROFF_GAT = ROFF_RED + RNV * RW * 8;                // [16] doubles: block totals
 constexpr int ROFF_BC = ROFF_GAT + 16 * 8;                       // [2][BC_DOUBLES] doubles, alternating by row
-constexpr int ROFF_WMAX = ROFF_BC + 2 * BC_DOUBLES * 8;          // [2][RW] floats
-constexpr int ROFF_STEP = ROFF_WMAX + 2 * RW * 4;                // [RW][MAX_STEPS] floats: draw weight of each step
+constexpr int ROFF_WMAX = ROFF_BC + 2 * BC_DOUBLES * 8;          // [3][RW]: teacher maximum, its index, student maximum per warp
+constexpr int ROFF_STEP = ROFF_WMAX + 4 * RW * 4;                // [RW][MAX_STEPS] floats: draw weight of each step
 constexpr int ROFF_MBAR = ROFF_STEP + RW * MAX_STEPS * 4;
 constexpr int RSMEM_BYTES = ROFF_MBAR + 16;
 
@@ -345,38 +346,36 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
     RTS(1);
 
     // ------------------------------------------------ pass "lse" (no separate maximum pass)
-    // Each thread sums under its own running shifts -ceil(c * running max): whole numbers, so that
-    // changing a shift, and later bringing all threads onto the row's shifts, multiplies the sums
-    // by exact powers of two.
+    // The exponent shifts of this pass are fixed before it starts: -ceil(c * m) with m the largest
+    // logit among the first 256 of the warp's segment.  m is an element of the row, so no term that
+    // matters can underflow; a row whose maximum lies more than ~88 nats above m overflows, shows as
+    // a non-finite sum and goes to the float64 kernel.  Shifts are whole numbers, so bringing the
+    // warps onto the row's common shifts multiplies their sums by exact powers of two.  The true
+    // maxima are tracked on the side (packed bf16 for the student, value + chunk for the teacher).
     {
+      float ksw = 1e30f, ktw = 1e30f;            // this warp's shifts (1e30: the warp has no element)
+      {
+        uint4 fs = make_uint4(FILLER, FILLER, FILLER, FILLER), ft = fs;
+        if (sg.c0 + lane < sg.c1) { fs = res_s[lane]; ft = res_t[lane]; }
+        const float2 a = unpack_bf16x2(max_bf16x2(max_bf16x2(fs.x, fs.y), max_bf16x2(fs.z, fs.w)));
+        const float2 b = unpack_bf16x2(max_bf16x2(max_bf16x2(ft.x, ft.y), max_bf16x2(ft.z, ft.w)));
+        const float ms0 = warp_max_f(fmaxf(a.x, a.y)), mt0 = warp_max_f(fmaxf(b.x, b.y));
+        if (sg.c0 < sg.c1) {
+          ksw = -ceilf(c32 * fmaxf(ms0, -1e30f));
+          ktw = -ceilf(c32 * fmaxf(mt0, -1e30f));
+        }
+      }
       float2 Ss = splat(0.f), St = splat(0.f), M1 = splat(0.f), M2 = splat(0.f), M3 = splat(0.f), N1 = splat(0.f);
-      float ms_run = -CUDART_INF_F, mt_run = -CUDART_INF_F, ks = 1e30f, kt = 1e30f;
-      int my_arg = 0x7fffffff;                   // lowest index of this thread's teacher maximum
-      const float2 cc = splat(c32), neg1 = splat(-1.f);
+      uint32_t run_s = FILLER;                   // packed running maxima of the student's even / odd elements
+      float mt_run = -CUDART_INF_F;              // running maximum of the teacher, and the first chunk that reached it
+      int arg_c = -1;
+      const float2 cc = splat(c32), neg1 = splat(-1.f), kk0 = splat(ksw), kk1 = splat(ktw);
       for_each_chunk(sg, lane, res_s, res_t, g_s, g_t, g_s, g_t, pol_last, rg, [&](const uint4& s4, const uint4& t4, int c, bool valid) {
         const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
-        const float2 cms = unpack_bf16x2(max_bf16x2(max_bf16x2(sw[0], sw[1]), max_bf16x2(sw[2], sw[3])));
+        run_s = max_bf16x2(run_s, max_bf16x2(max_bf16x2(sw[0], sw[1]), max_bf16x2(sw[2], sw[3])));
         const float2 cmt = unpack_bf16x2(max_bf16x2(max_bf16x2(tw[0], tw[1]), max_bf16x2(tw[2], tw[3])));
-        const float cm_s = fmaxf(cms.x, cms.y), cm_t = fmaxf(cmt.x, cmt.y);
-        if (valid && cm_s > ms_run) {
-          const float nk = -ceilf(c32 * fmaxf(cm_s, -1e30f));
-          const float2 f = splat(pow2f_exact(nk - ks));
-          Ss = fmul2(Ss, f); M1 = fmul2(M1, f); M2 = fmul2(M2, f); M3 = fmul2(M3, f);
-          ks = nk; ms_run = cm_s;
-        }
-        if (valid && cm_t > mt_run) {
-          const float nk = -ceilf(c32 * fmaxf(cm_t, -1e30f));
-          const float2 f = splat(pow2f_exact(nk - kt));
-          St = fmul2(St, f); N1 = fmul2(N1, f);
-          kt = nk; mt_run = cm_t;
-#pragma unroll
-          for (int i = 3; i >= 0; --i) {
-            const float2 f2 = unpack_bf16x2(tw[i]);
-            if (f2.y == cm_t) my_arg = c * 8 + 2 * i + 1;
-            if (f2.x == cm_t) my_arg = c * 8 + 2 * i;
-          }
-        }
-        const float2 kk0 = splat(ks), kk1 = splat(kt);
+        const float cm_t = fmaxf(cmt.x, cmt.y);
+        if (valid && cm_t > mt_run) { mt_run = cm_t; arg_c = c; }
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const float2 sf = unpack_bf16x2(sw[i]), tf = unpack_bf16x2(tw[i]);
@@ -394,22 +393,33 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
         }
       });
       RTS(2);
-      // warp: common shifts (the smallest), teacher argmax, sums
-      float kws = ks, kwt = kt, wmt = mt_run;
+      // lowest index of this thread's teacher maximum: the first element of chunk arg_c that equals it
+      int my_arg = 0x7fffffff;
+      if (arg_c >= 0) {
+        const int k = (arg_c - sg.c0) >> 5;
+        const uint4 t4 = k < sg.res ? res_t[k * 32 + lane] : ld_l2(g_t + (size_t)arg_c * 8, pol_last);
+        const uint32_t tw[4] = {t4.x, t4.y, t4.z, t4.w};
+#pragma unroll
+        for (int i = 3; i >= 0; --i) {
+          const float2 f2 = unpack_bf16x2(tw[i]);
+          if (f2.y == mt_run) my_arg = arg_c * 8 + 2 * i + 1;
+          if (f2.x == mt_run) my_arg = arg_c * 8 + 2 * i;
+        }
+      }
+      // warp: teacher argmax, student maximum, sums
+      const float2 rs2 = unpack_bf16x2(run_s);
+      const float wms = warp_max_f(fmaxf(rs2.x, rs2.y));
+      float wmt = mt_run;
       int warg = my_arg;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) {
-        kws = fminf(kws, __shfl_xor_sync(0xffffffffu, kws, o));
-        kwt = fminf(kwt, __shfl_xor_sync(0xffffffffu, kwt, o));
         const float om = __shfl_xor_sync(0xffffffffu, wmt, o);
         const int oa = __shfl_xor_sync(0xffffffffu, warg, o);
         if (om > wmt || (om == wmt && oa < warg)) { wmt = om; warg = oa; }
       }
-      const double fs = (double)pow2f_exact(kws - ks), ft = (double)pow2f_exact(kwt - kt);
-      const bool has_s = ks < 1e29f, has_t = kt < 1e29f;
+      const float kws = ksw, kwt = ktw;
       auto tot = [](const float2 a) { return (double)a.x + (double)a.y; };
-      double v[6] = {has_s ? fs * tot(Ss) : 0.0, has_t ? ft * tot(St) : 0.0, has_s ? fs * tot(M1) : 0.0,
-                     has_s ? fs * tot(M2) : 0.0, has_s ? fs * tot(M3) : 0.0, has_t ? ft * tot(N1) : 0.0};
+      double v[6] = {tot(Ss), tot(St), tot(M1), tot(M2), tot(M3), tot(N1)};
 #pragma unroll
       for (int k = 0; k < 6; ++k) v[k] = warp_sum_d(v[k]);
       if (lane == 0) {
@@ -417,7 +427,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
         for (int k = 0; k < 6; ++k) red[k * RW + warp] = v[k];
         red[6 * RW + warp] = (double)kws; red[7 * RW + warp] = (double)kwt;
         float* wm = (float*)(smem + ROFF_WMAX);
-        wm[warp] = wmt; ((int*)wm)[RW + warp] = warg;
+        wm[warp] = wmt; ((int*)wm)[RW + warp] = warg; wm[2 * RW + warp] = wms;
       }
       const int any_dead = __syncthreads_or(dead ? 1 : 0);
       RTS(3);
@@ -446,7 +456,9 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
             const int oa = __shfl_xor_sync(0xffffffffu, garg, o);
             if (om > gmt || (om == gmt && oa < garg)) { gmt = om; garg = oa; }
           }
-          if (lane == 0) gat[6] = (double)garg;
+          float gms = lane < RW ? wm[2 * RW + wl] : -CUDART_INF_F;
+          gms = warp_max_f(gms);
+          if (lane == 0) { gat[6] = (double)garg; gat[9] = (double)gms; gat[10] = (double)gmt; }
         }
       } else if (lane == 0) {
         // meanwhile, on warps that would only wait: the row scalars that do not depend on the passes,
@@ -466,7 +478,9 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       RTS(4);
       if (tid == 0) {
         bc[BC_K0] = gat[7]; bc[BC_K1] = gat[8];
-        scalar_after_lse(bc, gat, K, (float)gat[7], (float)gat[8], x, bonus, masked, any_dead != 0);
+        // largest term of either sum under the row's shifts (the shifts come from estimates of the maxima)
+        const float e_max = fmaxf(ex2f(fmaf(c32, (float)gat[9], (float)gat[7])), ex2f(fmaf(c32, (float)gat[10], (float)gat[8])));
+        scalar_after_lse(bc, gat, K, (float)gat[7], (float)gat[8], x, bonus, masked, any_dead != 0, e_max, true);
       }
       RTS(5);
       __syncthreads();
