@@ -265,6 +265,7 @@ static __device__ __noinline__ void scalar_after_solve(double* bc, const double*
   const double beta = bc[BC_BETA], G0 = bc[BC_G0], kb = bc[BC_KB];
   double lo = bc[BC_LO], hi = bc[BC_HI];
   const int iter = (int)bc[BC_ITER] + 1;
+  if (!(fabs(v[0] + v[1] + v[2]) < CUDART_INF)) { bc[BC_MODE] = MODE_REDO; return; }   // float32 sums overflowed
   const double r0 = rcp_fast(v[0]);
   const double G = LN2 * (log2_fast(v[0]) - kb);
   const double mu = v[1] * r0, var = fmax(v[2] * r0 - mu * mu, 0.0);

@@ -236,6 +236,36 @@ def test_hard_rows(which):
         P.set_kernel(prev)
 
 
+@pytest.mark.parametrize("gap", [30.0, 60.0, 120.0, 400.0])
+def test_wide_range_rows(gap):
+    """Rows whose mass sits on a few positions far above a low plateau.  The row-per-SM kernel fixes the
+    exponent shifts of its first pass from the first 256 logits of each warp's segment: with the plateau
+    `gap` below the peaks its sums grow by up to e^gap, and beyond ~88 nats they overflow, which must
+    hand the row to the float64 kernel, not flag or corrupt it."""
+    prev = P.set_kernel(3)
+    try:
+        V, N = 40000, 12
+        gen = torch.Generator(device=DEV).manual_seed(77)
+        s = torch.full((N, V), -gap, device=DEV) + 0.5 * torch.randn((N, V), generator=gen, device=DEV)
+        t = s + 0.5 * torch.randn((N, V), generator=gen, device=DEV)
+        for i in range(N):
+            # peaks away from the starts of the 16 warp segments (V / 16 = 2500 elements each)
+            pos = torch.randint(400, 2400, (40,), generator=gen, device=DEV) + 2500 * (i % 16)
+            s[i, pos] = 2.0 * torch.randn((40,), generator=gen, device=DEV)
+            t[i, pos] = s[i, pos] + 1.5 * torch.randn((40,), generator=gen, device=DEV)
+        s, t = s.to(torch.bfloat16), t.to(torch.bfloat16)
+        x = torch.argmax(s, dim=1).to(torch.int32)
+        w = synth.Workload("t", N, V, "bf16", 0.1, 1.5, False, 0, 35)
+        _check_fwd_bwd(dict(s=s, t=t, proposal=x, mask=None), w, eps=0.1)
+        assert P.last_kernel() == 3
+        if gap > 100.0:
+            assert P.redo_count() == N      # every row overflowed in float32 and was routed in float64
+        elif gap < 50.0:
+            assert P.redo_count() == 0
+    finally:
+        P.set_kernel(prev)
+
+
 def test_spec_verify_k_limits():
     V = 2048
     for K in (1, 16):
