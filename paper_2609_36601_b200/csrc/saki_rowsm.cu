@@ -188,32 +188,31 @@ __device__ __forceinline__ void for_each_chunk(const Seg& sg, int lane, const ui
   for (int k = 0; k < sg.res; ++k, c += 32) body(res_s[k * 32 + lane], res_t[k * 32 + lane], c, c < sg.c1);
   const int T = sg.steps - sg.res;                  // streamed steps: 0 or more than NST
   if (T <= 0) return;
-  const int c_first = c;
-  int cn = c + 32 * NST;                            // the chunk requested next, and where it comes from
-  int lim = sg.c1;
-  const __nv_bfloat16* ns = g_s + (size_t)cn * 8;
-  const __nv_bfloat16* nt = g_t + (size_t)cn * 8;
+  const uint32_t first_off = (uint32_t)c * 16u;
+  uint32_t off = first_off + 512u * NST;            // byte offset, in either row, of the chunk requested next
+  uint32_t lim = (uint32_t)sg.c1 * 16u;
+  const char* bs = reinterpret_cast<const char*>(g_s);   // (warp-uniform) rows the requests read
+  const char* bt = reinterpret_cast<const char*>(g_t);
   uint32_t slot = rg.slot;
   const uint32_t slot_end = rg.base + NST * 512;
 #pragma unroll 1
   for (int i = 0; i < T; ++i, c += 32) {
     if (i == T - NST) {   // from here on the requests belong to the pass that follows
-      cn = c_first;
-      lim = wrap_s != nullptr ? sg.c1 : -0x7fffffff;
-      ns = (wrap_s != nullptr ? wrap_s : g_s) + (size_t)cn * 8;
-      nt = (wrap_t != nullptr ? wrap_t : g_t) + (size_t)cn * 8;
+      off = first_off;
+      if (wrap_s != nullptr) { bs = reinterpret_cast<const char*>(wrap_s); bt = reinterpret_cast<const char*>(wrap_t); }
+      else lim = 0;
     }
     cp_async_wait<NST - 1>();
     const uint4 a = lds128(slot), b = lds128(slot + T_OFF);
-    if (cn < lim) {
-      cp_async16(slot, ns, pol);
-      cp_async16(slot + T_OFF, nt, pol);
+    if (off < lim) {
+      cp_async16(slot, bs + off, pol);
+      cp_async16(slot + T_OFF, bt + off, pol);
     } else {
       sts128(slot, FILLER);
       sts128(slot + T_OFF, FILLER);
     }
     cp_async_commit();
-    cn += 32; ns += 256; nt += 256;
+    off += 512;
     slot += 512;
     if (slot == slot_end) slot = rg.base;
     body(a, b, c, c < sg.c1);
@@ -235,7 +234,8 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
   int t_rows = 0;
   long long w_solve = 0, w_lse = 0, w_final = 0;
 #endif
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // broadcast: lets the compiler treat it as warp-uniform
   const uint4* res_s = reinterpret_cast<const uint4*>(smem + ROFF_S) + warp * RES_CHUNKS;
   const uint4* res_t = reinterpret_cast<const uint4*>(smem + ROFF_T) + warp * RES_CHUNKS;
   double* red = (double*)(smem + ROFF_RED);
