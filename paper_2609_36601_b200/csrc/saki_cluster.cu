@@ -545,6 +545,7 @@ static int pick_cs(int V) {
 bool cluster_can_serve(const RowParams& p, int dtype) {
   if (dtype != SAKI_BF16) return false;
   if (p.V < 2048 || p.V % 8 != 0 || p.V > MAX_CS * SLICE_CAP) return false;
+  if (p.n_rows > 0x7fffffffLL) return false;     // the redo list keeps row numbers in 32 bits
   auto al16 = [](const void* q) { return ((uintptr_t)q & 15) == 0; };
   if (!al16(p.s) || !al16(p.t)) return false;
   if (p.s_seq % 8 || p.s_pos % 8 || p.t_seq % 8 || p.t_pos % 8) return false;

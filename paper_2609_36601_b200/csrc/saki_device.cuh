@@ -204,9 +204,15 @@ __device__ __forceinline__ void decide(double* bc, const Consts& K, double lam, 
 // e_max: upper bound of the largest term of either sum (1 when the shifts come from the rows' maxima);
 // overflow_redo: shifts that come from an estimate of the maxima can overflow on finite rows, so
 // non-finite sums hand the row to the float64 kernel instead of flagging it.
-static __device__ __noinline__ void scalar_after_lse(double* bc, const double* v, Consts K, float k0f, float k1f, int x,
-                                              bool bonus, bool masked, bool row_timeout, float e_max = 1.f,
-                                              bool overflow_redo = false) {
+// The reciprocal and the log-sum-exp of one row's sum S under shift k: the same instructions for the
+// student and the teacher, so two lanes of a warp can do the two rows at once.
+__device__ __forceinline__ void lse_of_sum(double S, double k, double& rS, double& G) {
+  rS = rcp_fast(S);
+  G = LN2 * (log2_fast(S) - k);
+}
+static __device__ __noinline__ void scalar_after_lse_tail(double* bc, const double* v, Consts K, float k0f, float k1f, int x,
+                                                   bool bonus, bool masked, bool row_timeout, float e_max,
+                                                   bool overflow_redo, double rSs, double rSt, double G0, double G1) {
   const double SsT = v[0], StT = v[1], eps = K.eps, k0 = (double)k0f, k1 = (double)k1f;
   uint32_t status = 0;
   const double chk = ((v[0] + v[1]) + (v[2] + v[3])) + (v[4] + v[5]);
@@ -219,8 +225,6 @@ static __device__ __noinline__ void scalar_after_lse(double* bc, const double* v
   const int vstar = (v[6] >= 0.0 && v[6] < (double)K.V) ? (int)v[6] : 0;
   bc[BC_VSTAR] = (double)vstar;
   if (status) { bc[BC_STATUS] = (double)status; bc[BC_MODE] = MODE_FLAGGED; return; }
-  const double rSs = rcp_fast(SsT), rSt = rcp_fast(StT);
-  const double G0 = LN2 * (log2_fast(SsT) - k0), G1 = LN2 * (log2_fast(StT) - k1);
   bc[BC_G0] = G0; bc[BC_G1] = G1; bc[BC_RSS] = rSs;
   bc[BC_PMAX] = fmin(1.0, (double)e_max * fmax(rSs, rSt));      // upper bound of the largest probability of either row
   if (!(eps > 0.0)) {          // student-only endpoint
@@ -256,6 +260,14 @@ static __device__ __noinline__ void scalar_after_lse(double* bc, const double* v
   bc[BC_KB] = (double)(float)((1.0 - be) * k0 + be * k1);
   bc[BC_LO] = 0.0; bc[BC_HI] = 1.0; bc[BC_ITER] = 0.0;
   bc[BC_MODE] = MODE_SOLVE;
+}
+
+static __device__ __noinline__ void scalar_after_lse(double* bc, const double* v, Consts K, float k0f, float k1f, int x,
+                                              bool bonus, bool masked, bool row_timeout) {
+  double rSs, rSt, G0, G1;
+  lse_of_sum(v[0], (double)k0f, rSs, G0);
+  lse_of_sum(v[1], (double)k1f, rSt, G1);
+  scalar_after_lse_tail(bc, v, K, k0f, k1f, x, bonus, masked, row_timeout, 1.f, false, rSs, rSt, G0, G1);
 }
 
 // after one evaluation of pass "solve": safeguarded Newton step on sqrt(KL); v = {S0, S1, S2}

@@ -267,16 +267,15 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
   K.rc64 = 1.0 / K.c64; K.grad_scale = (double)P.grad_scale; K.sqrt_eps = sqrtf(P.eps); K.V = V;
   const uint64_t pol_last = policy_evict_last(), pol_first = policy_evict_first();
 
+  // rows fit 31 bits (see rowsm_can_serve): 32-bit divisions
   auto row_ptrs = [&](int64_t row, const __nv_bfloat16*& s, const __nv_bfloat16*& t) {
-    const int64_t b = row / P.K1;
+    const int64_t b = P.K1 == 1 ? row : (int64_t)((uint32_t)row / (uint32_t)P.K1);
     const int j = (int)(row - b * P.K1);
     s = (const __nv_bfloat16*)P.s + b * P.s_seq + (int64_t)j * P.s_pos;
     t = (const __nv_bfloat16*)P.t + b * P.t_seq + (int64_t)j * P.t_pos;
   };
   // lane 0 of each warp: fetch the warp's resident part of `row` into shared memory
-  auto issue = [&](int64_t row) {
-    const __nv_bfloat16 *s, *t;
-    row_ptrs(row, s, t);
+  auto issue = [&](const __nv_bfloat16* s, const __nv_bfloat16* t) {
     mbar_expect_tx(mbar, 2u * res_bytes);
     if (res_bytes) {
       bulk_load_hint((void*)res_s, s + (size_t)sg.c0 * 8, res_bytes, mbar, pol_first);
@@ -303,11 +302,11 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
+  const __nv_bfloat16 *n_s = nullptr, *n_t = nullptr;   // the rows of the CTA's next position, if any
   if ((int64_t)blockIdx.x < P.n_rows) {
-    if (lane == 0) issue(blockIdx.x);
-    const __nv_bfloat16 *s0, *t0;
-    row_ptrs(blockIdx.x, s0, t0);
-    ring_prime(rg, sg, lane, s0, t0, pol_last);
+    row_ptrs(blockIdx.x, n_s, n_t);
+    if (lane == 0) issue(n_s, n_t);
+    ring_prime(rg, sg, lane, n_s, n_t, pol_last);
   }
   uint32_t phase = 0;
   bool dead = false;
@@ -318,7 +317,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
   auto write_pending = [&](int64_t row, const double* bcp) {
     const __nv_bfloat16 *s, *t;
     row_ptrs(row, s, t);
-    const int64_t b = row / P.K1;
+    const int64_t b = (int64_t)((uint32_t)row / (uint32_t)P.K1);
     const int xp = P.spec ? P.proposal[b * P.prop_ld + (row - b * P.K1)] : P.proposal[row];
     write_result(bcp, P.out, !P.spec, row, 0, xp, false, K.c64, s, t);
   };
@@ -326,16 +325,15 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
   for (int64_t row = blockIdx.x; row < P.n_rows; row += gridDim.x, rb ^= 1) {
     double* bc = (double*)(smem + ROFF_BC) + rb * BC_DOUBLES;   // this row's broadcast scalars
     const uint64_t rid = P.row_offset + (uint64_t)row;
-    const int64_t seq = row / P.K1;
+    const int64_t seq = P.K1 == 1 ? row : (int64_t)((uint32_t)row / (uint32_t)P.K1);
     const int pos = (int)(row - seq * P.K1);
     const bool bonus = P.spec && (pos == P.K1 - 1);
     const int x = bonus ? 0 : (P.spec ? P.proposal[seq * P.prop_ld + pos] : P.proposal[row]);
     const bool masked = (P.mask != nullptr) && (P.mask[row] == 0);
-    const __nv_bfloat16 *g_s, *g_t;
-    row_ptrs(row, g_s, g_t);
+    const __nv_bfloat16 *g_s = n_s, *g_t = n_t;
     __nv_bfloat16* g_out = P.dlogits ? (__nv_bfloat16*)P.dlogits + row * P.ld_g : nullptr;
     const int64_t next_row = row + gridDim.x;
-    const __nv_bfloat16 *n_s = nullptr, *n_t = nullptr;   // the next row of this CTA, if any
+    n_s = nullptr; n_t = nullptr;
     if (next_row < P.n_rows) row_ptrs(next_row, n_s, n_t);
 
     RTS(0);
@@ -393,24 +391,13 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
         }
       });
       RTS(2);
-      // lowest index of this thread's teacher maximum: the first element of chunk arg_c that equals it
-      int my_arg = 0x7fffffff;
-      if (arg_c >= 0) {
-        const int k = (arg_c - sg.c0) >> 5;
-        const uint4 t4 = k < sg.res ? res_t[k * 32 + lane] : ld_l2(g_t + (size_t)arg_c * 8, pol_last);
-        const uint32_t tw[4] = {t4.x, t4.y, t4.z, t4.w};
-#pragma unroll
-        for (int i = 3; i >= 0; --i) {
-          const float2 f2 = unpack_bf16x2(tw[i]);
-          if (f2.y == mt_run) my_arg = arg_c * 8 + 2 * i + 1;
-          if (f2.x == mt_run) my_arg = arg_c * 8 + 2 * i;
-        }
-      }
-      // warp: teacher argmax, student maximum, sums
+      // warp: teacher maximum with the lowest chunk that holds it (a chunk belongs to one thread, so
+      // chunk order is index order; the element is found once, by the block's winner), student
+      // maximum, sums
       const float2 rs2 = unpack_bf16x2(run_s);
       const float wms = warp_max_f(fmaxf(rs2.x, rs2.y));
       float wmt = mt_run;
-      int warg = my_arg;
+      int warg = arg_c >= 0 ? arg_c : 0x7fffffff;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) {
         const float om = __shfl_xor_sync(0xffffffffu, wmt, o);
@@ -458,7 +445,20 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           }
           float gms = lane < RW ? wm[2 * RW + wl] : -CUDART_INF_F;
           gms = warp_max_f(gms);
-          if (lane == 0) { gat[6] = (double)garg; gat[9] = (double)gms; gat[10] = (double)gmt; }
+          if (lane == 0) {
+            int best = -1;                       // lowest index of the maximum inside the winning chunk
+            if (garg != 0x7fffffff) {
+              const uint4 t4 = ld_l2(g_t + (size_t)garg * 8, pol_last);
+              const uint32_t tw[4] = {t4.x, t4.y, t4.z, t4.w};
+#pragma unroll
+              for (int i = 3; i >= 0; --i) {
+                const float2 f2 = unpack_bf16x2(tw[i]);
+                if (f2.y == gmt) best = garg * 8 + 2 * i + 1;
+                if (f2.x == gmt) best = garg * 8 + 2 * i;
+              }
+            }
+            gat[6] = (double)best; gat[9] = (double)gms; gat[10] = (double)gmt;
+          }
         }
       } else if (lane == 0) {
         // meanwhile, on warps that would only wait: the row scalars that do not depend on the passes,
@@ -476,11 +476,18 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       if (any_dead) dead = true;
       __syncthreads();
       RTS(4);
-      if (tid == 0) {
-        bc[BC_K0] = gat[7]; bc[BC_K1] = gat[8];
-        // largest term of either sum under the row's shifts (the shifts come from estimates of the maxima)
-        const float e_max = fmaxf(ex2f(fmaf(c32, (float)gat[9], (float)gat[7])), ex2f(fmaf(c32, (float)gat[10], (float)gat[8])));
-        scalar_after_lse(bc, gat, K, (float)gat[7], (float)gat[8], x, bonus, masked, any_dead != 0, e_max, true);
+      if (tid < 2) {   // lane 0: the student's sum, lane 1: the teacher's; then lane 0 alone
+        double rS, G;
+        lse_of_sum(gat[lane], gat[7 + lane], rS, G);
+        // largest term of the sum under the row's shift (the shifts come from estimates of the maxima)
+        const float em = ex2f(fmaf(c32, (float)gat[9 + lane], (float)gat[7 + lane]));
+        const double rSt = __shfl_sync(0x3u, rS, 1), G1 = __shfl_sync(0x3u, G, 1);
+        const float e_max = fmaxf(em, __shfl_sync(0x3u, em, 1));
+        if (tid == 0) {
+          bc[BC_K0] = gat[7]; bc[BC_K1] = gat[8];
+          scalar_after_lse_tail(bc, gat, K, (float)gat[7], (float)gat[8], x, bonus, masked, any_dead != 0, e_max, true,
+                                rS, rSt, G, G1);
+        }
       }
       RTS(5);
       __syncthreads();
@@ -541,7 +548,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       __syncwarp();
       if (lane == 0 && !dead && next_row < P.n_rows) {
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        issue(next_row);
+        issue(n_s, n_t);
       }
       ring_prime(rg, sg, lane, n_s, n_t, pol_last);   // the ring holds steps of this row: refill it for the next
       continue;
@@ -608,12 +615,12 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           __syncwarp();
           if (lane == 0 && !dead && next_row < P.n_rows) {
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            issue(next_row);
+            issue(n_s, n_t);
           }
           next_issued = true;
         }
       });
-      if (!next_issued && lane == 0 && !dead && next_row < P.n_rows) issue(next_row);   // no elements
+      if (!next_issued && lane == 0 && !dead && next_row < P.n_rows) issue(n_s, n_t);   // no elements
       RTS(11);
       const float sq_f = Sq.x + Sq.y, r_f = R.x + R.y;
       double part = 0.0;                               // this warp's draw weight: its step weights, in order
@@ -757,6 +764,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
 bool rowsm_can_serve(const RowParams& p, int dtype) {
   if (dtype != SAKI_BF16) return false;
   if (p.V < 2048 || p.V % 8 != 0 || p.V > MAX_STEPS * 32 * 8 * RW) return false;
+  if (p.n_rows > 0x7fffffffLL) return false;     // row numbers are kept in 32 bits (redo list, divisions)
   auto al16 = [](const void* q) { return ((uintptr_t)q & 15) == 0; };
   if (!al16(p.s) || !al16(p.t)) return false;
   if (p.s_seq % 8 || p.s_pos % 8 || p.t_seq % 8 || p.t_pos % 8) return false;
