@@ -316,6 +316,79 @@ static __device__ __noinline__ void scalar_after_solve(double* bc, const double*
   }
 }
 
+// After one evaluation of pass "solve" that also carries the third and fourth moments:
+// v = {S0, S1, S2, S3, S4}, S_k = sum of e_i d_i^k, d = t - s, e_i the shifted terms of q_beta.
+// G(b) = log sum exp((s + b d)/tau) has the derivatives kappa_k(d; q_b) / tau^k, and
+// KL(q_b || p) = b G'(b) - G(b) + G(0)  (Eqs. "bridge", "trust_region").  The fourth-order Taylor model
+// of G around beta gives
+//   KL(beta + h) = KL + h beta G2 + h^2 (beta G3 + G2)/2 + h^3 (beta G4/6 + G3/3) + h^4 G4/8,
+// whose root is lambda up to a fifth-order term: with the initial guess a few percent off that is
+// far below the resolution of the float32 sums, so one evaluation usually settles the row.  The
+// size of the last kept term (with floors against accidentally small cumulants) decides whether
+// another evaluation at the new point is needed.
+static __device__ __noinline__ void scalar_after_solve4(double* bc, const double* v, Consts K, float k0f, float k1f, int x,
+                                                 bool bonus, bool masked) {
+  const double eps = K.eps, rtau = K.rtau;
+  const double beta = bc[BC_BETA], G0 = bc[BC_G0], kb = bc[BC_KB];
+  double lo = bc[BC_LO], hi = bc[BC_HI];
+  const int iter = (int)bc[BC_ITER] + 1;
+  if (!(fabs((v[0] + v[1]) + (v[2] + v[3]) + v[4]) < CUDART_INF)) { bc[BC_MODE] = MODE_REDO; return; }   // float32 sums overflowed
+  const double r0 = rcp_fast(v[0]);
+  const double G = LN2 * (log2_fast(v[0]) - kb);
+  const double m1 = v[1] * r0, m2 = v[2] * r0, m3 = v[3] * r0, m4 = v[4] * r0;   // raw moments of d under q_beta
+  const double m1s = m1 * m1;
+  const double var = fmax(m2 - m1s, 0.0);
+  const double k3 = m3 - 3.0 * m2 * m1 + 2.0 * m1s * m1;
+  const double k4 = m4 - 4.0 * m3 * m1 - 3.0 * m2 * m2 + 12.0 * m2 * m1s - 6.0 * m1s * m1s;
+  const double rt2 = rtau * rtau;
+  const double G1 = m1 * rtau, G2 = var * rt2, G3 = k3 * rt2 * rtau, G4 = k4 * rt2 * rt2;
+  const double kl = beta * G1 - G + G0;                 // KL(q_beta || p)
+  const double slope = beta * G2;                       // d KL / d beta
+  if (kl <= eps) lo = fmax(lo, beta); else hi = fmin(hi, beta);
+  const double c2 = 0.5 * (beta * G3 + G2), c3 = beta * G4 * (1.0 / 6.0) + G3 * (1.0 / 3.0), c4 = 0.125 * G4;
+  double h;
+  float trunc = 0.f;
+  if (slope > 1e-30 && kl > 1e-30 && kl < 1e30) {
+    // the steps are corrections: float32 from here, once eps - KL is formed in float64
+    const float f0 = (float)(eps - kl), a1 = (float)slope, a2 = (float)c2, a3 = (float)c3, a4 = (float)c4;
+    const float rk = sqrtf((float)kl);
+    float hf = __fdividef(f0 * (2.f * rk), (K.sqrt_eps + rk) * a1);     // Newton on sqrt(KL): the starting point
+#pragma unroll
+    for (int it = 0; it < 3; ++it) {
+      const float pv = hf * (a1 + hf * (a2 + hf * (a3 + hf * a4))) - f0;
+      const float dv = a1 + hf * (2.f * a2 + hf * (3.f * a3 + hf * (4.f * a4)));
+      if (dv > 0.25f * a1) hf -= __fdividef(pv, dv);
+    }
+    const float h2 = hf * hf;
+    trunc = fmaxf(fabsf(a4), fmaxf(fabsf(a3), 0.5f * fabsf(a2))) * h2 * h2;
+    h = (double)hf;
+  } else { h = 0.5 * (lo + hi) - beta; trunc = 1e30f; }
+  double nb = beta + h;
+  bool bisected = false;
+  if (!(nb > lo && nb < hi)) { nb = 0.5 * (lo + hi); bisected = true; }
+  const bool done = (!bisected && trunc <= 3e-8f * (float)slope) || iter >= 40 || (hi - lo) < 1e-9;
+  // The float32 sums resolve KL to a few 1e-7 x (largest probability).  Where that would move lambda by
+  // more than the tolerance (a very flat KL: nearly one-hot rows), or the solve did not converge, the row
+  // is handed to the float64 kernel.  (Radii below 5e-3 never reach this kernel: see the dispatcher.)
+  if (done && (3e-7 * bc[BC_PMAX] > 1e-5 * slope || iter >= 40)) { bc[BC_MODE] = MODE_REDO; return; }
+  if (done) {
+    const float cl = (float)(K.c64 * nb);
+    const double lam = (double)cl * K.rc64;
+    const double dl = lam - beta;
+    // the model's predictions at lambda
+    bc[BC_KL] = kl + dl * (slope + dl * (c2 + dl * (c3 + dl * c4)));
+    const double Glam = G + dl * (G1 + dl * (0.5 * G2 + dl * ((1.0 / 6.0) * G3 + dl * (1.0 / 24.0) * G4)));
+    decide(bc, K, lam, Glam, G0, bc[BC_G1], (double)k0f, (double)k1f, bc[BC_RSS], (uint32_t)bc[BC_STATUS],
+           (int)bc[BC_VSTAR], bonus, masked, x);
+  } else {
+    const float cbn = (float)(K.c64 * nb);
+    const double be = (double)cbn * K.rc64;
+    bc[BC_BETA] = be; bc[BC_CB] = (double)cbn;
+    bc[BC_KB] = (double)(float)((1.0 - be) * (double)k0f + be * (double)k1f);
+    bc[BC_LO] = lo; bc[BC_HI] = hi; bc[BC_ITER] = (double)iter;
+  }
+}
+
 // for a draw: the warp that owns the inverse-CDF target (ordered scan of per-warp weights)
 static __device__ __noinline__ void scalar_find_owner(double* bc, const double* warp_part, int n_warps) {
   double total = 0.0;

@@ -115,6 +115,10 @@ __device__ __forceinline__ float pow2f_exact(float n) {   // 2^n for whole n, cl
 #define SAKI_RES_UNROLL 1
 #endif
 constexpr int RES_UNROLL = SAKI_RES_UNROLL;   // unrolling of the resident-part loop
+#ifndef SAKI_RING_UNROLL
+#define SAKI_RING_UNROLL 1
+#endif
+constexpr int RING_UNROLL = SAKI_RING_UNROLL; // unrolling of the streamed-part loop
 #ifndef SAKI_RING
 #define SAKI_RING 4
 #endif
@@ -195,7 +199,7 @@ __device__ __forceinline__ void for_each_chunk(const Seg& sg, int lane, const ui
   const char* bt = reinterpret_cast<const char*>(g_t);
   uint32_t slot = rg.slot;
   const uint32_t slot_end = rg.base + NST * 512;
-#pragma unroll 1
+#pragma unroll RING_UNROLL
   for (int i = 0; i < T; ++i, c += 32) {
     if (i == T - NST) {   // from here on the requests belong to the pass that follows
       off = first_off;
@@ -498,7 +502,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
     while ((int)bc[BC_MODE] == MODE_SOLVE) {
       RTS(6);
       const float cb = (float)bc[BC_CB], kb = (float)bc[BC_KB];
-      float2 S0 = splat(0.f), S1 = splat(0.f), S2 = splat(0.f);
+      float2 S0 = splat(0.f), S1 = splat(0.f), S2 = splat(0.f), S3 = splat(0.f), S4 = splat(0.f);
       const float2 cc = splat(c32), cbb = splat(cb), kbb = splat(kb), neg1 = splat(-1.f);
 #ifdef SAKI_PHASE_TIMING
       const long long w_t0 = clock64();
@@ -513,7 +517,11 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           S0 = fadd2(S0, e);
           const float2 t1 = fmul2(e, d);
           S1 = fadd2(S1, t1);
-          S2 = ffma2(t1, d, S2);
+          const float2 t2 = fmul2(t1, d);
+          S2 = fadd2(S2, t2);
+          const float2 t3 = fmul2(t2, d);
+          S3 = fadd2(S3, t3);
+          S4 = ffma2(t3, d, S4);
         }
       });
 #ifdef SAKI_PHASE_TIMING
@@ -521,10 +529,11 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
 #endif
       RTS(7);
       auto tot = [](const float2 a) { return (double)a.x + (double)a.y; };
-      const double v[3] = {warp_sum_d(tot(S0)), warp_sum_d(tot(S1)), warp_sum_d(tot(S2))};
-      combine(v, 3);
+      const double v[5] = {warp_sum_d(tot(S0)), warp_sum_d(tot(S1)), warp_sum_d(tot(S2)), warp_sum_d(tot(S3)),
+                           warp_sum_d(tot(S4))};
+      combine(v, 5);
       RTS(8);
-      if (tid == 0) scalar_after_solve(bc, gat, K, k0, k1, x, bonus, masked);
+      if (tid == 0) scalar_after_solve4(bc, gat, K, k0, k1, x, bonus, masked);
       RTS(9);
       __syncthreads();
     }
