@@ -366,6 +366,7 @@ static __device__ __noinline__ void scalar_after_solve4(double* bc, const double
   double nb = beta + h;
   bool bisected = false;
   if (!(nb > lo && nb < hi)) { nb = 0.5 * (lo + hi); bisected = true; }
+  // accepted when the bound on the dropped terms moves lambda by less than 3e-8
   const bool done = (!bisected && trunc <= 3e-8f * (float)slope) || iter >= 40 || (hi - lo) < 1e-9;
   // The float32 sums resolve KL to a few 1e-7 x (largest probability).  Where that would move lambda by
   // more than the tolerance (a very flat KL: nearly one-hot rows), or the solve did not converge, the row

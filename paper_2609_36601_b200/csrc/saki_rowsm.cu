@@ -424,21 +424,19 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       RTS(3);
       if (warp < 7) {   // block level: warps 0-5 add up one sum each on the row's shifts, warp 6 finds the argmax
         const int wl = lane < RW ? lane : 0;       // lanes beyond the warp count carry zero weight
-        const double ksw = lane < RW ? red[6 * RW + wl] : 1e30, ktw = lane < RW ? red[7 * RW + wl] : 1e30;
-        double k0d = ksw, k1d = ktw;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          k0d = fmin(k0d, __shfl_xor_sync(0xffffffffu, k0d, o));
-          k1d = fmin(k1d, __shfl_xor_sync(0xffffffffu, k1d, o));
-        }
+        const float* wm = (const float*)(smem + ROFF_WMAX);
         if (warp < 6) {
+          // From here on the row's shifts are those of its true maxima (the largest term of each sum has
+          // its exponent argument in (-1, 0], where float32 resolves it best); a warp's shift came from an
+          // element of the row, so it is never below the row's, and the factor is an exact power of two <= 1.
           const bool teacher = (warp == 1 || warp == 5);
-          const double kw = teacher ? ktw : ksw, kr = teacher ? k1d : k0d;
+          const float mx = warp_max_f(lane < RW ? wm[teacher ? wl : 2 * RW + wl] : -CUDART_INF_F);
+          const double kr = (double)-ceilf(c32 * fmaxf(mx, -1e30f));
+          const double kw = lane < RW ? red[(teacher ? 7 : 6) * RW + wl] : 1e30;
           const double f = kw < 1e29 ? (double)pow2f_exact((float)(kr - kw)) : 0.0;
           const double a = warp_sum_d(f * red[warp * RW + wl]);
-          if (lane == 0) { gat[warp] = a; if (warp == 0) { gat[7] = k0d; gat[8] = k1d; } }
+          if (lane == 0) { gat[warp] = a; if (warp < 2) gat[7 + warp] = kr; }
         } else {
-          const float* wm = (const float*)(smem + ROFF_WMAX);
           float gmt = lane < RW ? wm[wl] : -CUDART_INF_F;
           int garg = ((const int*)wm)[RW + wl];
 #pragma unroll
@@ -447,8 +445,6 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
             const int oa = __shfl_xor_sync(0xffffffffu, garg, o);
             if (om > gmt || (om == gmt && oa < garg)) { gmt = om; garg = oa; }
           }
-          float gms = lane < RW ? wm[2 * RW + wl] : -CUDART_INF_F;
-          gms = warp_max_f(gms);
           if (lane == 0) {
             int best = -1;                       // lowest index of the maximum inside the winning chunk
             if (garg != 0x7fffffff) {
@@ -461,7 +457,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
                 if (f2.x == gmt) best = garg * 8 + 2 * i;
               }
             }
-            gat[6] = (double)best; gat[9] = (double)gms; gat[10] = (double)gmt;
+            gat[6] = (double)best;
           }
         }
       } else if (lane == 0) {
@@ -483,13 +479,10 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       if (tid < 2) {   // lane 0: the student's sum, lane 1: the teacher's; then lane 0 alone
         double rS, G;
         lse_of_sum(gat[lane], gat[7 + lane], rS, G);
-        // largest term of the sum under the row's shift (the shifts come from estimates of the maxima)
-        const float em = ex2f(fmaf(c32, (float)gat[9 + lane], (float)gat[7 + lane]));
         const double rSt = __shfl_sync(0x3u, rS, 1), G1 = __shfl_sync(0x3u, G, 1);
-        const float e_max = fmaxf(em, __shfl_sync(0x3u, em, 1));
         if (tid == 0) {
           bc[BC_K0] = gat[7]; bc[BC_K1] = gat[8];
-          scalar_after_lse_tail(bc, gat, K, (float)gat[7], (float)gat[8], x, bonus, masked, any_dead != 0, e_max, true,
+          scalar_after_lse_tail(bc, gat, K, (float)gat[7], (float)gat[8], x, bonus, masked, any_dead != 0, 1.f, true,
                                 rS, rSt, G, G1);
         }
       }
