@@ -1,25 +1,26 @@
 // One-row-per-SM kernel for bf16 rows.
 //
-// One persistent CTA of 1024 threads per SM routes whole rows, one after the
+// One persistent CTA of 512 threads per SM routes whole rows, one after the
 // other.  A row pair (student + teacher, e.g. 608 KB at V = 151936) does not
-// fit on one SM, so it is kept in two places:
-//   - the leading part of every warp's segment lives in shared memory
-//     (192 KB per CTA), filled by per-warp 1-D bulk async copies that are
-//     issued for the NEXT row as soon as the warp has read its resident part
-//     for the last time;
-//   - the rest is read from global memory in every pass.  Each row is touched
-//     by one SM only, so after the first pass these reads are L2 hits; the
-//     next row's share is pulled into L2 ahead of time with bulk L2 prefetches.
+// fit on one SM.  Every warp owns a contiguous segment of the row and visits
+// it in steps of 32 chunks of 8 elements; it keeps
+//   - the leading steps of its segment resident in shared memory, filled by
+//     per-warp 1-D bulk async copies on an mbarrier, issued for the NEXT row
+//     as soon as the warp has read its resident part for the last time;
+//   - the rest in global memory, streamed in every pass through a small ring
+//     of per-lane cp.async slots.  Each row is touched by one SM only, so
+//     after the first pass these reads are L2 hits.
 // HBM therefore sees each logit row once and the gradient row once.  All
 // reductions stay inside the CTA (warp shuffles + shared memory), so a pass of
 // ~150 k elements per SM amortises them.  Passes:
-//   max      packed bf16 maxima of both rows (first touch of the L2 part)
-//   lse      2 exponentials/element: log-sum-exps, moments of the logit
-//            difference under p (initial guess of lambda), KL(T||p), argmax
-//   solve    1 exponential/element per evaluation of KL(q_beta||p) and its
-//            slope; Newton on sqrt(KL) in a bisection bracket (Eqs. "bridge",
-//            "trust_region")
-//   final    2 exponentials/element: TV = sum [q-p]_+ with per-warp ordered
+//   lse      2 exponentials/element under shifts fixed before the pass:
+//            log-sum-exps, moments of the logit difference under p (initial
+//            guess of lambda), KL(T||p), maxima, teacher argmax
+//   solve    1 exponential/element per evaluation of KL(q_beta||p) and the
+//            first four cumulants of the logit difference under q_beta;
+//            lambda = root of the fourth-order Taylor model in a bisection
+//            bracket (Eqs. "bridge", "trust_region")
+//   final    2 exponentials/element: TV = sum [q-p]_+ with per-step ordered
 //            partial sums for the inverse-CDF residual draw (Eqs. "accept",
 //            "residual"), gradient row streamed out (Eq. "general_objective")
 // Per-element work is float32 (packed f32x2 FMAs, ex2.approx); cross-thread
