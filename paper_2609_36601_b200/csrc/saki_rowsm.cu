@@ -42,7 +42,7 @@ constexpr int KS_MAX = 208 / RW;        // steps per warp that fit in shared mem
 constexpr int MAX_STEPS = 64;            // steps per warp the draw bookkeeping can hold (V <= 64*32*8*RW)
 constexpr int RES_CHUNKS = KS_MAX * 32; // resident chunks per warp and row
 constexpr int RNV = 8;                  // doubles per partial vector
-static_assert(RW >= 12, "warps 8-11 do side work while warps 0-6 gather");
+static_assert(RW >= 13, "warps 8-12 do side work while warps 0-6 gather and thread 0 does the scalars");
 static_assert(KS_MAX - 4 >= 1, "every warp keeps at least its first step resident");
 
 constexpr int ROFF_S = 0;                                        // [RW][RES_CHUNKS] uint4
@@ -181,16 +181,18 @@ __device__ __forceinline__ void ring_prime(Ring& rg, const Seg& sg, int lane, co
 // memory; streamed steps come out of the ring, and each one consumed requests the step NST further
 // on: of this pass, or, past its end, of the next pass, whose rows are wrap_s / wrap_t (the same row
 // again, the next row after the last pass, nullptr if nothing follows).
-template <typename Body>
+// after_resident() runs once the resident steps are done.
+template <typename Body, typename Mid>
 __device__ __forceinline__ void for_each_chunk(const Seg& sg, int lane, const uint4* res_s, const uint4* res_t,
                                                const __nv_bfloat16* g_s, const __nv_bfloat16* g_t,
                                                const __nv_bfloat16* wrap_s, const __nv_bfloat16* wrap_t,
-                                               uint64_t pol, Ring& rg, Body&& body) {
+                                               uint64_t pol, Ring& rg, Body&& body, Mid&& after_resident) {
   // resident part (slots past the end of the segment hold the filler); kept rolled: the pass bodies
   // are large and must stay in the instruction cache
   int c = sg.c0 + lane;
 #pragma unroll RES_UNROLL
   for (int k = 0; k < sg.res; ++k, c += 32) body(res_s[k * 32 + lane], res_t[k * 32 + lane], c, c < sg.c1);
+  after_resident();
   const int T = sg.steps - sg.res;                  // streamed steps: 0 or more than NST
   if (T <= 0) return;
   const uint32_t first_off = (uint32_t)c * 16u;
@@ -394,7 +396,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           M3 = ffma2(t2, d, M3);
           N1 = ffma2(et, d, N1);
         }
-      });
+      }, [] {});
       RTS(2);
       // warp: teacher maximum with the lowest chunk that holds it (a chunk belongs to one thread, so
       // chunk order is index order; the element is found once, by the block's winner), student
@@ -477,6 +479,10 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       if (any_dead) dead = true;
       __syncthreads();
       RTS(4);
+      if (tid == 12 * 32) {   // meanwhile: the student's logit at the teacher's argmax (the supervised token of a corrected row)
+        const int vs = (gat[6] >= 0.0 && gat[6] < (double)V) ? (int)gat[6] : 0;
+        bc[BC_SV] = (double)__bfloat162float(g_s[vs]);
+      }
       if (tid < 2) {   // lane 0: the student's sum, lane 1: the teacher's; then lane 0 alone
         double rS, G;
         lse_of_sum(gat[lane], gat[7 + lane], rS, G);
@@ -508,16 +514,15 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           const float2 sf = unpack_bf16x2(sw[i]), tf = unpack_bf16x2(tw[i]);
           const float2 d = ffma2(sf, neg1, tf);
           const float2 e = ex2f2(ffma2(d, cbb, ffma2(sf, cc, kbb)));
+          const float2 d2 = fmul2(d, d);
           S0 = fadd2(S0, e);
-          const float2 t1 = fmul2(e, d);
-          S1 = fadd2(S1, t1);
-          const float2 t2 = fmul2(t1, d);
-          S2 = fadd2(S2, t2);
-          const float2 t3 = fmul2(t2, d);
-          S3 = fadd2(S3, t3);
-          S4 = ffma2(t3, d, S4);
+          S1 = ffma2(e, d, S1);
+          const float2 u = fmul2(e, d2);
+          S2 = fadd2(S2, u);
+          S3 = ffma2(u, d, S3);
+          S4 = ffma2(u, d2, S4);
         }
-      });
+      }, [] {});
 #ifdef SAKI_PHASE_TIMING
       w_solve += clock64() - w_t0; ++w_lse;
 #endif
@@ -568,14 +573,13 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
     const int tok = (int)bc[BC_TOK];
     const float KGf = (float)bc[BC_KG];
     const float kg = (float)(bc[BC_KG] * (double)ip);     // gradient entry = e_p * kg
+    const float rho = ip / iq;                            // q_i - p_i = iq * (e_q - rho * e_p)
     {
       const bool want_g = (g_out != nullptr);
       float2 Sq = splat(0.f), R = splat(0.f);
       const float2 cc = splat(c32), cll = splat(cl), kqq = splat(kq), kk0 = splat(k0), neg1 = splat(-1.f);
-      const float2 iqq = splat(iq), nip = splat(-ip), kgg = splat(kg);
+      const float2 nrho = splat(-rho), kgg = splat(kg);
       float* step_w = (float*)(smem + ROFF_STEP) + warp * MAX_STEPS;   // draw weight of each of this warp's steps
-      int n_res_done = 0;
-      bool next_issued = false;
       for_each_chunk(sg, lane, res_s, res_t, g_s, g_t, n_s, n_t, pol_last, rg, [&](const uint4& s4, const uint4& t4, int c, bool valid) {
         const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
         uint32_t gp[4];
@@ -587,7 +591,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           const float2 ep = ex2f2(ffma2(sf, cc, kk0));
           const float2 eq = ex2f2(ffma2(d, cll, ffma2(sf, cc, kqq)));
           sqc = fadd2(sqc, eq);
-          float2 r = ffma2(eq, iqq, fmul2(ep, nip));     // q_i - p_i
+          float2 r = ffma2(ep, nrho, eq);                // (q_i - p_i) / iq
           r.x = fmaxf(r.x, 0.f); r.y = fmaxf(r.y, 0.f);
           rc = fadd2(rc, r);
           const float2 gv = fmul2(ep, kgg);
@@ -596,34 +600,21 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
         Sq = fadd2(Sq, sqc);
         R = fadd2(R, rc);
         if (need_draw) {   // ordered bookkeeping for the inverse-CDF draw: the weight of this step of the warp
-          float wsum = bonus ? (sqc.x + sqc.y) * iq : (rc.x + rc.y);
+          float wsum = bonus ? (sqc.x + sqc.y) : (rc.x + rc.y);   // in units of iq, like every draw weight
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
           const int k = (c - sg.c0) >> 5;
           if (lane == 0 && k < MAX_STEPS) step_w[k] = wsum;
         }
-        if ((tok >> 3) == c && tok >= 0) {   // the supervised token is in this chunk: subtract the one-hot part
-          const int e = tok & 7, wi = e >> 1;
-          const uint32_t word = wi == 0 ? sw[0] : wi == 1 ? sw[1] : wi == 2 ? sw[2] : sw[3];
-          const float2 sf = unpack_bf16x2(word);
-          const float ep = ex2f(fmaf((e & 1) ? sf.y : sf.x, c32, k0));
-          const uint32_t g16 = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(fmaf(ep, kg, -KGf)));
-          const uint32_t old = wi == 0 ? gp[0] : wi == 1 ? gp[1] : wi == 2 ? gp[2] : gp[3];
-          const uint32_t neu = (e & 1) ? ((old & 0x0000ffffu) | (g16 << 16)) : ((old & 0xffff0000u) | g16);
-          if (wi == 0) gp[0] = neu; else if (wi == 1) gp[1] = neu; else if (wi == 2) gp[2] = neu; else gp[3] = neu;
-        }
         if (want_g && valid) st_stream(g_out + (size_t)c * 8, make_uint4(gp[0], gp[1], gp[2], gp[3]), pol_first);
-        // once the warp has read its resident part for the last time, the next row's may land there
-        if (++n_res_done == sg.res) {
-          __syncwarp();
-          if (lane == 0 && !dead && next_row < P.n_rows) {
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            issue(n_s, n_t);
-          }
-          next_issued = true;
+      }, [&] {
+        // the warp has read its resident part for the last time: the next row's may land there
+        __syncwarp();
+        if (lane == 0 && !dead && next_row < P.n_rows) {
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          issue(n_s, n_t);
         }
       });
-      if (!next_issued && lane == 0 && !dead && next_row < P.n_rows) issue(n_s, n_t);   // no elements
       RTS(11);
       const float sq_f = Sq.x + Sq.y, r_f = R.x + R.y;
       double part = 0.0;                               // this warp's draw weight: its step weights, in order
@@ -633,7 +624,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
         static_assert(MAX_STEPS <= 64, "two step weights per lane");
         part = warp_sum_d((lane < ns ? (double)step_w[lane] : 0.0) + (lane + 32 < ns ? (double)step_w[lane + 32] : 0.0));
       }
-      const double v0 = warp_sum_d((double)sq_f), v1 = warp_sum_d((double)r_f);
+      const double v0 = warp_sum_d((double)sq_f), v1 = warp_sum_d((double)r_f * (double)iq);
       if (lane == 0) { red[warp] = v0; red[RW + warp] = v1; red[2 * RW + warp] = part; }   // part: ordered per-warp weights of the draw
       __syncthreads();
       if (warp < 2) {
@@ -663,7 +654,14 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       }
       __syncthreads();
       RTS(12);
-      if (tid == 0) bc[BC_TV] = (bc[BC_LAMBDA] > 0.0) ? gat[1] : 0.0;
+      if (tid == 0) {
+        bc[BC_TV] = (bc[BC_LAMBDA] > 0.0) ? gat[1] : 0.0;
+        if (want_g && tok >= 0) {   // the supervised token: gradient KG * (p - 1), over the entry its chunk's owner stored
+          const float s_tok = (float)(tok == x ? bc[BC_SX] : bc[BC_SV]);
+          const float ep = ex2f(fmaf(s_tok, c32, k0));
+          g_out[tok] = __float2bfloat16_rn(fmaf(ep, kg, -KGf));
+        }
+      }
       if (!need_draw) pending_row = row;
     }
 
@@ -697,8 +695,8 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           const float2 d = ffma2(sf, splat(-1.f), tf);
           const float2 ep = ex2f2(ffma2(sf, splat(c32), splat(k0)));
           const float2 eq = ex2f2(ffma2(d, splat(cl), ffma2(sf, splat(c32), splat(kq))));
-          w[2 * i] = bonus ? eq.x * iq : fmaxf(fmaf(eq.x, iq, -(ep.x * ip)), 0.f);
-          w[2 * i + 1] = bonus ? eq.y * iq : fmaxf(fmaf(eq.y, iq, -(ep.y * ip)), 0.f);
+          w[2 * i] = bonus ? eq.x : fmaxf(fmaf(ep.x, -rho, eq.x), 0.f);
+          w[2 * i + 1] = bonus ? eq.y : fmaxf(fmaf(ep.y, -rho, eq.y), 0.f);
         }
         double mine = 0.0;
 #pragma unroll
