@@ -87,6 +87,21 @@ def test_fast_kernel_shapes(V, N, eps, sigma, which):
         P.set_kernel(prev)
 
 
+@pytest.mark.parametrize("V", [53384, 56000, 75008, 262144])
+def test_rowsm_streamed_shapes(V):
+    """Row-per-SM kernel, rows that no longer fit in shared memory: 14 steps per warp (the shortest
+    streamed part), a ragged last step, and the largest V it serves; two rows per block, so the ring
+    of streamed steps runs over from a row's last pass into the next row and ends after the last."""
+    prev = P.set_kernel(3)
+    try:
+        w = synth.Workload("t", 300, V, "bf16", 0.1, 1.5, True, 131, 41)
+        d = synth.generate(w, DEV)
+        _check_fwd_bwd(d, w, rows=range(0, 300, 23), row_offset=3)
+        assert P.last_kernel() == 3
+    finally:
+        P.set_kernel(prev)
+
+
 def test_strided_rows_and_mask(kernel):
     w = synth.Workload("t", 12, 3000, "bf16", 0.05, 1.0, True, 78, 10)
     d = synth.generate(w, DEV)
