@@ -264,6 +264,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
   rg.base = smem_addr(res_s + KS_RES * 32 + lane);
   rg.slot = rg.base;
   // slots of the resident area that no copy ever writes (a segment that ends inside its last step) hold the filler
+#pragma unroll 1
   for (int k = res_chunks + lane; k < RES_CHUNKS; k += 32) {
     sts128(smem_addr(res_s + k), FILLER);
     sts128(smem_addr(res_t + k), FILLER);
@@ -549,6 +550,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
         }
       }
       if (g_out && !redo) {
+#pragma unroll 1
         for (int k = 0; k < sg.steps; ++k) {
           const int c = sg.c0 + k * 32 + lane;
           if (c < sg.c1) st_stream(g_out + (size_t)c * 8, make_uint4(0, 0, 0, 0), pol_first);
@@ -676,6 +678,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
         const int ns = min(sg.steps, MAX_STEPS);
         // the step that holds the target (every lane walks the same few numbers)
         int ks = -1, kpos = -1;
+#pragma unroll 1
         for (int k = 0; k < ns; ++k) {
           const double w = (double)step_w[k];
           if (w > 0.0) kpos = k;
