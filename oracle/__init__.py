@@ -12,4 +12,5 @@ from .saki_oracle import (  # noqa: F401
     log_softmax, bridge_stats, solve_lambda, bridge_distribution,
     total_variation, inverse_cdf_draw, round_to_bf16,
     route_row, route, sample_proposal_row, sample_proposal, spec_verify,
+    bwd_from_meta_row, bwd_from_meta,
 )

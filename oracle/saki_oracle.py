@@ -25,6 +25,10 @@ T = teacher distribution, both full-vocabulary softmaxes of the logit rows):
      objective                                 Eq. "general_objective", Appendix C
   7. block verification: commit the accepted
      prefix, correct at the first rejection    Section 3.5, Appendix I
+  8. the trainer's step: the same loss and
+     gradient for freshly computed student
+     logits, from the rollout's metadata only  Section 3.5; Eqs. "k1_loss_token",
+                                               "teacher_mode_loss"
 
 Readings where the paper is silent are stated next to the code that takes them.
 The random numbers are a counter-based Philox4x32-10 stream keyed by
@@ -37,8 +41,10 @@ root finder, the V=2 closed form, the two endpoints and the monotone-KL
 property; TV by its three equal forms and Pinsker; the coupling by exhaustive
 enumeration and by Monte Carlo over seeds; losses and gradient against
 torch.autograd in float64 and central differences; block verification by the
-product law of the acceptance probabilities.  The paper prints no worked
-numeric example for any of these quantities.
+product law of the acceptance probabilities; the metadata-driven backward
+against torch's cross-entropy (a library routine), central differences, the
+zero row sum of a softmax gradient and route() itself on unchanged logits.  The
+paper prints no worked numeric example for any of these quantities.
 """
 from __future__ import annotations
 
@@ -348,6 +354,76 @@ def route(s, t, proposal, eps, temperature=1.0, seed=0, row_offset=0,
         out["grad"] = np.stack([r["grad"] for r in res]) if res else \
             np.zeros((0, np.asarray(s).shape[1]))
     return out
+
+
+# --------------------------------------------------------------------------
+# The trainer's side: loss and gradient from the routing metadata
+# --------------------------------------------------------------------------
+_ROLLOUT_UNUSABLE = ST_NONFINITE | ST_BAD_ID | ST_TIMEOUT | ST_NOT_COMPUTED
+
+
+def bwd_from_meta_row(s, corrected: int, x: int, v_star: int, advantage: float,
+                      temperature: float, mask: int = 1, rollout_status: int = 0,
+                      grad_scale: float = 1.0, grad_dtype: str = "f32"):
+    """Loss and gradient of one position for the CURRENT student logits `s`,
+    given only what the rollout returned (Section 3.5: the training loop
+    receives token-aligned metadata, not logits): the correction flag C, the
+    proposal x, the teacher mode v* and the stop-gradient advantage
+    A = log T(x) - log p_rollout(x)  (Eq. "k1_advantage_token").
+
+      C = 0:  L = -A log pi(x)          Eq. "k1_loss_token"
+      C = 1:  L = -log pi(v*)           Eq. "teacher_mode_loss"
+      dL/ds_j = coef (pi_j - 1[j = tok]) / temperature, (coef, tok) = (A, x) or (1, v*)
+
+    pi = softmax(s / temperature) of the logits passed here, which need not be
+    the rollout's.  Readings (the paper does not spell this call out): a
+    position that is masked, or whose rollout row was not routed (non-finite
+    logits, bad id, timeout, after the first rejection), contributes nothing
+    and is reported with ST_MASKED resp. ST_NOT_COMPUTED; a non-finite logit
+    or advantage here gives ST_NONFINITE, a supervised token outside [0, V)
+    ST_BAD_ID, both with zero loss and gradient."""
+    s = np.asarray(s, dtype=np.float64)
+    V = s.shape[0]
+    out = dict(loss=0.0, logp_tok=0.0, status=0, grad=np.zeros(V, dtype=np.float64))
+    if mask == 0:
+        out["status"] = ST_MASKED
+        return out
+    if rollout_status & _ROLLOUT_UNUSABLE:
+        out["status"] = ST_NOT_COMPUTED
+        return out
+    tok = int(v_star) if corrected else int(x)
+    coef = 1.0 if corrected else float(advantage)
+    if not (np.all(np.isfinite(s)) and math.isfinite(coef)):
+        out["status"] = ST_NONFINITE
+        return out
+    if not (0 <= tok < V):
+        out["status"] = ST_BAD_ID
+        return out
+    lp = log_softmax(s / temperature)
+    onehot = np.zeros(V, dtype=np.float64)
+    onehot[tok] = 1.0
+    g = grad_scale * coef * (np.exp(lp) - onehot) / temperature
+    g = round_to_bf16(g) if grad_dtype == "bf16" else g.astype(np.float32).astype(np.float64)
+    out.update(loss=float(-coef * lp[tok]), logp_tok=float(lp[tok]), grad=g)
+    return out
+
+
+def bwd_from_meta(s, corrected, proposal, teacher_top1, advantage, temperature=1.0,
+                  mask=None, rollout_status=None, grad_scale=1.0, grad_dtype="f32",
+                  rows=None):
+    """bwd_from_meta_row over the rows `rows` (default: all) of the [N,V] array
+    `s`.  Returns arrays indexed like `rows`; "grad" is [len(rows), V]."""
+    N = len(proposal)
+    rows = range(N) if rows is None else rows
+    res = [bwd_from_meta_row(s[i], int(corrected[i]), int(proposal[i]), int(teacher_top1[i]),
+                             float(advantage[i]), temperature,
+                             1 if mask is None else int(mask[i]),
+                             0 if rollout_status is None else int(rollout_status[i]),
+                             grad_scale, grad_dtype) for i in rows]
+    return dict(loss=np.array([r["loss"] for r in res], dtype=np.float64),
+                logp_tok=np.array([r["logp_tok"] for r in res], dtype=np.float64),
+                status=np.array([r["status"] for r in res], dtype=np.uint32),
+                grad=np.stack([r["grad"] for r in res]) if res else np.zeros((0, np.asarray(s).shape[1])))
 
 
 # --------------------------------------------------------------------------

@@ -394,3 +394,91 @@ def test_spec_verify_semantics():
     # eps = 0: everything accepted, bonus ~ p
     out0 = O.spec_verify(s[:5], t[:5], draft[:5], 0.0, seed=4)
     assert np.all(out0["n_accept"] == K) and np.all(out0["next_is_correction"] == 0)
+
+
+# ---------------------------------------------------------------- metadata-driven backward
+def _meta_case(rng, N, V):
+    s = rng.normal(size=(N, V)) * 2.0
+    C = (rng.random(N) < 0.4).astype(np.uint8)
+    x = rng.integers(0, V, N).astype(np.int32)
+    vs = rng.integers(0, V, N).astype(np.int32)
+    A = rng.normal(size=N)
+    return s, C, x, vs, A
+
+
+def test_meta_backward_matches_torch_cross_entropy_and_autograd():
+    """Corrected rows are a cross-entropy on the teacher mode (Eq. "teacher_mode_loss"): pinned to
+    torch's library routine.  Accepted rows are -A log pi(x) (Eq. "k1_loss_token"): pinned to
+    float64 autograd of that expression written with torch ops."""
+    rng = np.random.default_rng(41)
+    N, V, tau, scale = 12, 57, 0.7, 0.25
+    s, C, x, vs, A = _meta_case(rng, N, V)
+    res = O.bwd_from_meta(s, C, x, vs, A, temperature=tau, grad_scale=scale, grad_dtype="f32")
+    z = torch.tensor(s, dtype=torch.float64, requires_grad=True)
+    ce = torch.nn.functional.cross_entropy(z / tau, torch.tensor(vs, dtype=torch.long), reduction="none")
+    lp = torch.log_softmax(z / tau, dim=1)
+    rkl = -torch.tensor(A) * lp[torch.arange(N), torch.tensor(x, dtype=torch.long)]
+    loss = torch.where(torch.tensor(C.astype(bool)), ce, rkl)
+    (scale * loss.sum()).backward()
+    assert np.allclose(res["loss"], loss.detach().numpy(), rtol=1e-12, atol=1e-12)
+    assert np.allclose(res["grad"], z.grad.numpy().astype(np.float32).astype(np.float64), rtol=0, atol=1e-7)
+    tok = np.where(C == 1, vs, x)
+    assert np.allclose(res["logp_tok"], lp.detach().numpy()[np.arange(N), tok], atol=1e-12)
+    assert np.all(res["status"] == 0)
+
+
+def test_meta_backward_central_differences_and_zero_row_sum():
+    rng = np.random.default_rng(42)
+    N, V, tau = 4, 9, 1.3
+    s, C, x, vs, A = _meta_case(rng, N, V)
+    C[:] = [0, 1, 0, 1]
+    res = O.bwd_from_meta(s, C, x, vs, A, temperature=tau, grad_dtype="f32")
+    # the softmax part sums to one and the one-hot part to one: every gradient row sums to zero
+    assert np.all(np.abs(res["grad"].sum(axis=1)) < 1e-6)
+    h = 1e-6
+    for i in range(N):
+        for j in range(V):
+            sp, sm = s.copy(), s.copy()
+            sp[i, j] += h
+            sm[i, j] -= h
+            lp_ = O.bwd_from_meta(sp, C, x, vs, A, temperature=tau)["loss"][i]
+            lm_ = O.bwd_from_meta(sm, C, x, vs, A, temperature=tau)["loss"][i]
+            assert abs((lp_ - lm_) / (2 * h) - res["grad"][i, j]) < 1e-6
+
+
+def test_meta_backward_on_unchanged_logits_equals_routing():
+    """With the rollout's own logits and its metadata the trainer's call reproduces the loss and the
+    gradient of the routing call (Eq. "general_objective")."""
+    rng = np.random.default_rng(43)
+    N, V, eps, tau = 40, 300, 0.15, 0.9
+    s = rng.normal(size=(N, V)) * 2.0
+    t = s + rng.normal(size=(N, V)) * 1.5
+    x = np.array([O.sample_proposal_row(s[i], tau, 5, i)[0] for i in range(N)], dtype=np.int32)
+    mask = (rng.random(N) < 0.8).astype(np.uint8)
+    r = O.route(s, t, x, eps, tau, seed=5, mask=mask, grad_scale=0.1, want_grad=True, grad_dtype="bf16")
+    assert 0 < r["corrected"].sum() < N
+    A = r["logT_x"] - r["logp_x"]
+    m = O.bwd_from_meta(s, r["corrected"], x, r["teacher_top1"], A, tau, mask=mask, rollout_status=r["status"],
+                        grad_scale=0.1, grad_dtype="bf16")
+    assert np.allclose(m["loss"], r["loss"], rtol=1e-12, atol=1e-14)
+    assert np.array_equal(m["grad"], r["grad"])
+    assert np.all((m["status"] == O.ST_MASKED) == (mask == 0))
+
+
+def test_meta_backward_flags():
+    rng = np.random.default_rng(44)
+    N, V = 6, 33
+    s, C, x, vs, A = _meta_case(rng, N, V)
+    C[:] = [0, 1, 0, 1, 0, 0]
+    s[0, 3] = np.nan
+    vs[1] = V
+    x[2] = -1
+    A[4] = np.inf
+    st = np.zeros(N, dtype=np.uint32)
+    st[3] = O.ST_NOT_COMPUTED
+    mask = np.ones(N, dtype=np.uint8)
+    mask[5] = 0
+    res = O.bwd_from_meta(s, C, x, vs, A, mask=mask, rollout_status=st)
+    assert list(res["status"]) == [O.ST_NONFINITE, O.ST_BAD_ID, O.ST_BAD_ID, O.ST_NOT_COMPUTED, O.ST_NONFINITE,
+                                   O.ST_MASKED]
+    assert np.all(res["grad"] == 0) and np.all(res["loss"] == 0)
