@@ -18,7 +18,10 @@
  *      (Eq. "general_objective"; lambda, q, the coupling outcome and A are
  *      constants of differentiation)
  *   6. for drafted blocks, the left-to-right first-rejection resolve of
- *      Section 3.5 / Appendix I.
+ *      Section 3.5 / Appendix I;
+ *   7. for the training loop, which sees metadata instead of logits, the
+ *      same loss and gradient recomputed from freshly evaluated student
+ *      logits (saki_route_bwd_from_meta).
  *
  * Conventions
  *   - Every pointer in the structs below is a DEVICE pointer owned by the
@@ -145,6 +148,48 @@ SAKI_API int saki_route_fwd_bwd_noalloc(const saki_in* in, const saki_out* out, 
 SAKI_API int saki_route_host(const saki_in* in_host, const saki_out* out_host,
                     void* dlogits_host, int64_t ld_g, float grad_scale);
 
+/* The trainer's step (Section 3.5, Appendix K): the rollout keeps the full-vocabulary rows on its own
+ * GPUs and hands the training loop token-aligned metadata only.  The trainer recomputes the CURRENT
+ * student's logits and needs, per position, the loss of Eq. "general_objective" and its gradient with
+ * respect to those logits:
+ *     C = 0:  L = -A log pi(x),   A = log T(x) - log p_rollout(x)  (Eqs. "k1_loss_token", "k1_advantage_token")
+ *     C = 1:  L = -log pi(v*)                                      (Eq. "teacher_mode_loss")
+ *     dlogits[i,:] = grad_scale * coef * (pi - onehot(tok)) / temperature,  (coef, tok) = (A, x) or (1, v*)
+ * with pi = softmax(student_logits[i,:] / temperature) of the logits passed HERE.  On the rollout's own
+ * logits and metadata this reproduces saki_route_fwd_bwd's loss and gradient. */
+typedef struct {
+  const void* student_logits;   /* [N,V] current student logits, unit stride along V, row stride ld_s elements */
+  int64_t ld_s;                 /* >= V */
+  int64_t N;                    /* >= 0 */
+  int32_t V;                    /* >= 2 */
+  int32_t dtype;                /* saki_dtype of the logits and of dlogits */
+  const uint8_t* corrected;     /* [N] C_t as returned by the routing call. Required */
+  const int32_t* proposal;      /* [N] x_t, the supervised token where C_t = 0. Required */
+  const int32_t* teacher_top1;  /* [N] v*_t, the supervised token where C_t = 1. Required */
+  const float* advantage;       /* [N] A_t = logT_x - logp_x of the routing call (a constant of
+                                   differentiation); read where C_t = 0. Required */
+  const uint8_t* mask;          /* [N] M_t or NULL = all valid */
+  const uint32_t* rollout_status; /* [N] row_status of the routing call, or NULL: rows it flagged NONFINITE,
+                                   BAD_ID, TIMEOUT or NOT_COMPUTED contribute nothing here */
+  float temperature;            /* > 0 */
+} saki_meta_in;
+
+typedef struct {
+  float* loss;          /* [N] un-normalised loss of the position; 0 where it contributes nothing. May be NULL */
+  float* logp_tok;      /* [N] log pi(tok) under the current logits. May be NULL */
+  uint32_t* row_status; /* [N] 0, or SAKI_ROW_MASKED / NOT_COMPUTED (nothing to do), or NONFINITE (a logit or
+                           the advantage is not finite) / BAD_ID (supervised token outside [0,V)): loss 0 and
+                           gradient row 0 in all four cases. May be NULL */
+} saki_meta_out;
+
+/* `in`/`out` are HOST structs read during the call; dlogits [N,V] (required), row stride ld_g >= V
+ * elements, in the logits' dtype (round to nearest even).  Asynchronous on the stream.  bf16 rows with
+ * 16-byte aligned rows, strides and V multiples of 8 and V >= 2048 run on a streaming kernel that reads
+ * each row from HBM once and writes the gradient row once; everything else, and rows whose float32
+ * sums overflow, on a float64 kernel.  Flagged rows count towards saki_check(). */
+SAKI_API int saki_route_bwd_from_meta(const saki_meta_in* in, const saki_meta_out* out, void* dlogits,
+                                      int64_t ld_g, float grad_scale, void* cuda_stream);
+
 /* Block verification (Section 3.5, Appendix I) of B drafted blocks of K tokens. */
 typedef struct {
   const void* student_logits; /* [B,K+1,V]: position j of sequence b at element offset
@@ -199,7 +244,8 @@ SAKI_API int saki_check(void* cuda_stream, uint64_t* n_flagged);
 SAKI_API int saki_set_kernel(int which);
 
 /* Which row kernel the calling thread's last routing call used: 1 general, 2 cluster,
- * 3 row-per-SM, 0 if none yet. */
+ * 3 row-per-SM, 4 the streaming kernel of saki_route_bwd_from_meta (which saki_set_kernel(1) also
+ * turns off), 0 if none yet. */
 SAKI_API int saki_last_kernel(void);
 
 /* Two-tier routing: the float32 kernels (2, 3) hand rows whose KL they cannot resolve to the

@@ -19,7 +19,8 @@ SAKI_F32, SAKI_BF16 = 0, 1
 ROW_SATURATED, ROW_EPS_ZERO, ROW_MASKED, ROW_NONFINITE, ROW_BAD_ID, ROW_TIMEOUT, ROW_NOT_COMPUTED = 1, 2, 4, 8, 16, 32, 64
 
 _FLOAT_FIELDS = ("lambda", "kl", "tv", "accept_prob", "logp_x", "logq_x", "logT_x", "logp_y", "logq_y", "loss")
-EXPORTS = ("saki_route_fwd", "saki_route_fwd_bwd", "saki_route_fwd_bwd_noalloc", "saki_route_host", "saki_spec_verify",
+EXPORTS = ("saki_route_fwd", "saki_route_fwd_bwd", "saki_route_fwd_bwd_noalloc", "saki_route_host",
+           "saki_route_bwd_from_meta", "saki_spec_verify",
            "saki_sample_proposal", "saki_check", "saki_set_kernel", "saki_last_kernel", "saki_redo_count",
            "saki_launch_count",
            "saki_last_error", "saki_version")
@@ -43,6 +44,18 @@ class SakiIn(C.Structure):
 class SakiOut(C.Structure):
     _fields_ = [("corrected", C.c_void_p), ("token", C.c_void_p), ("teacher_top1", C.c_void_p)] + \
                [(f, C.c_void_p) for f in _FLOAT_FIELDS] + [("row_status", C.c_void_p)]
+
+
+class SakiMetaIn(C.Structure):
+    _fields_ = [("student_logits", C.c_void_p), ("ld_s", C.c_int64), ("N", C.c_int64),
+                ("V", C.c_int32), ("dtype", C.c_int32),
+                ("corrected", C.c_void_p), ("proposal", C.c_void_p), ("teacher_top1", C.c_void_p),
+                ("advantage", C.c_void_p), ("mask", C.c_void_p), ("rollout_status", C.c_void_p),
+                ("temperature", C.c_float)]
+
+
+class SakiMetaOut(C.Structure):
+    _fields_ = [("loss", C.c_void_p), ("logp_tok", C.c_void_p), ("row_status", C.c_void_p)]
 
 
 class SakiSpecIn(C.Structure):
@@ -74,6 +87,9 @@ def load_library(path: str | None = None):
     lib.saki_route_fwd_bwd_noalloc.argtypes = lib.saki_route_fwd_bwd.argtypes
     lib.saki_route_fwd_bwd_noalloc.restype = C.c_int
     lib.saki_route_host.argtypes = [C.POINTER(SakiIn), C.POINTER(SakiOut), C.c_void_p, C.c_int64, C.c_float]
+    lib.saki_route_bwd_from_meta.argtypes = [C.POINTER(SakiMetaIn), C.POINTER(SakiMetaOut), C.c_void_p, C.c_int64,
+                                             C.c_float, C.c_void_p]
+    lib.saki_route_bwd_from_meta.restype = C.c_int
     lib.saki_spec_verify.argtypes = [C.POINTER(SakiSpecIn), C.POINTER(SakiSpecOut), C.c_void_p]
     lib.saki_sample_proposal.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_float,
                                          C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p]
@@ -135,6 +151,12 @@ def _out_struct(out: dict) -> SakiOut:
     return so
 
 
+def _vec_check(v, dtype, n, dev, name):
+    if v.dtype != dtype or v.shape != (n,) or v.device != dev or not v.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous {dtype} tensor of length N on the logits' device")
+    return v
+
+
 def _check_rows(s, t):
     if s.dim() != 2 or t.shape != s.shape or t.dtype != s.dtype or s.stride(1) != 1 or t.stride(1) != 1:
         raise SakiError(1, "student/teacher logits must be [N,V] of the same dtype with unit stride along V")
@@ -173,6 +195,42 @@ def route_fwd_bwd(s, t, proposal, eps, temperature=1.0, seed=0, row_offset=0, ma
     si, so = _in_struct(s, t, proposal, mask, eps, temperature, seed, row_offset), _out_struct(out)
     _raise(lib, lib.saki_route_fwd_bwd(C.byref(si), C.byref(so), dlogits.data_ptr(), ld_g, grad_scale,
                                        _stream_ptr(stream)))
+    return out, dlogits
+
+
+def route_bwd_from_meta(s, corrected, proposal, teacher_top1, advantage, temperature=1.0, mask=None,
+                        rollout_status=None, grad_scale=1.0, dlogits=None, stream=None):
+    """saki_route_bwd_from_meta on device tensors: loss and gradient of the routed objective for the
+    current student logits `s`, from the rollout's metadata.  Returns (outputs dict, dlogits)."""
+    lib = load_library()
+    if s.dim() != 2 or s.stride(1) != 1:
+        raise ValueError("logits must be [N,V] with unit stride along V")
+    n, dev = s.shape[0], s.device
+    if dlogits is None:
+        dlogits = torch.empty_like(s)
+    ld_g = dlogits.stride(0) if dlogits.shape[0] > 1 else dlogits.shape[1]
+    out = {"loss": torch.empty(n, dtype=torch.float32, device=dev),
+           "logp_tok": torch.empty(n, dtype=torch.float32, device=dev),
+           "row_status": torch.empty(n, dtype=torch.int32, device=dev)}
+    keep = [_vec_check(corrected, torch.uint8, n, dev, "corrected"),
+            _vec_check(proposal, torch.int32, n, dev, "proposal"),
+            _vec_check(teacher_top1, torch.int32, n, dev, "teacher_top1"),
+            _vec_check(advantage, torch.float32, n, dev, "advantage")]
+    mi = SakiMetaIn()
+    mi.student_logits = s.data_ptr()
+    mi.ld_s = s.stride(0) if n > 1 else s.shape[1]
+    mi.N, mi.V, mi.dtype = n, s.shape[1], _dtype_code(s)
+    mi.corrected, mi.proposal, mi.teacher_top1, mi.advantage = (t.data_ptr() for t in keep)
+    if mask is not None:
+        keep.append(_vec_check(mask, torch.uint8, n, dev, "mask"))
+        mi.mask = keep[-1].data_ptr()
+    if rollout_status is not None:
+        keep.append(_vec_check(rollout_status, torch.int32, n, dev, "rollout_status"))
+        mi.rollout_status = keep[-1].data_ptr()
+    mi.temperature = temperature
+    mo = SakiMetaOut(out["loss"].data_ptr(), out["logp_tok"].data_ptr(), out["row_status"].data_ptr())
+    _raise(lib, lib.saki_route_bwd_from_meta(C.byref(mi), C.byref(mo), dlogits.data_ptr(), ld_g, grad_scale,
+                                             _stream_ptr(stream)))
     return out, dlogits
 
 

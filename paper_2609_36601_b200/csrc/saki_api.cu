@@ -198,6 +198,54 @@ static int route_impl(const saki_in* in, const saki_out* out, void* dlogits, int
   return dispatch_rows(p, in->dtype, (cudaStream_t)stream);
 }
 
+// ---- the trainer's step: loss and gradient from the rollout's metadata (Section 3.5) ----
+static int meta_impl(const saki_meta_in* in, const saki_meta_out* out, void* dlogits, int64_t ld_g, float grad_scale,
+                     void* stream) {
+  g_err[0] = 0;
+  if (!in || !out) return fail(SAKI_ERR_INVALID_ARG, "NULL argument struct");
+  if (in->N < 0) return fail(SAKI_ERR_INVALID_ARG, "negative row count");
+  if (in->V < 2) return fail(SAKI_ERR_INVALID_ARG, "V must be >= 2 (got %d)", in->V);
+  if (in->dtype != SAKI_F32 && in->dtype != SAKI_BF16) return fail(SAKI_ERR_INVALID_ARG, "unknown dtype %d", in->dtype);
+  if (!(in->temperature > 0.f) || std::isinf(in->temperature))
+    return fail(SAKI_ERR_INVALID_ARG, "temperature must be finite and > 0");
+  if (in->ld_s < in->V || ld_g < in->V) return fail(SAKI_ERR_INVALID_ARG, "row stride smaller than V");
+  if (!std::isfinite(grad_scale)) return fail(SAKI_ERR_INVALID_ARG, "grad_scale must be finite");
+  if (in->N == 0) return SAKI_OK;
+  if (!in->student_logits || !dlogits) return fail(SAKI_ERR_INVALID_ARG, "NULL logits or dlogits pointer");
+  if (!in->corrected || !in->proposal || !in->teacher_top1 || !in->advantage)
+    return fail(SAKI_ERR_INVALID_ARG, "corrected, proposal, teacher_top1 and advantage are required");
+  unsigned long long* flagged = nullptr;
+  int rc = device_ready(&flagged);
+  if (rc) return rc;
+  MetaParams p;
+  memset(&p, 0, sizeof(p));
+  p.s = in->student_logits; p.ld_s = in->ld_s; p.n_rows = in->N; p.V = in->V;
+  p.corrected = in->corrected; p.proposal = in->proposal; p.teacher_top1 = in->teacher_top1;
+  p.advantage = in->advantage; p.mask = in->mask; p.rollout_status = in->rollout_status;
+  p.temperature = in->temperature; p.out = *out; p.dlogits = dlogits; p.ld_g = ld_g; p.grad_scale = grad_scale;
+  p.flagged = flagged;
+  cudaStream_t st = (cudaStream_t)stream;
+  int launches = 0;
+  cudaError_t e;
+  bool served = false;
+  int used = 1;
+  if (g_kernel.load() != 1 && meta_stream_can_serve(p, in->dtype)) {
+    rc = redo_scratch(p.n_rows, &p.redo_list, &p.redo_count);
+    if (rc) return rc;
+    e = cudaMemsetAsync(p.redo_count, 0, sizeof(unsigned int), st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+    g_last_redo_count = p.redo_count;
+    e = launch_meta_stream(p, st, &launches, &served);
+    if (e != cudaSuccess) return cuda_fail(e, "streaming backward kernel launch");
+    if (served) { used = 4; p.from_list = 1; }
+  }
+  e = launch_meta_general(p, in->dtype, st, &launches);
+  if (e != cudaSuccess) return cuda_fail(e, "general backward kernel launch");
+  g_launches += (uint64_t)launches;
+  g_last_kernel = used;
+  return SAKI_OK;
+}
+
 // ---- block verification: per-sequence first-rejection resolve (Section 3.5) ----
 __global__ void spec_resolve_kernel(int64_t B, int K, saki_out o, int32_t* n_accept, int32_t* next_token,
                                     uint8_t* next_is_corr) {
@@ -290,6 +338,11 @@ SAKI_API int saki_route_fwd_bwd(const saki_in* in, const saki_out* out, void* dl
 SAKI_API int saki_route_fwd_bwd_noalloc(const saki_in* in, const saki_out* out, void* dlogits, int64_t ld_g,
                                         float grad_scale, void* cuda_stream) {
   return route_impl(in, out, dlogits, ld_g, grad_scale, true, cuda_stream, true);
+}
+
+SAKI_API int saki_route_bwd_from_meta(const saki_meta_in* in, const saki_meta_out* out, void* dlogits, int64_t ld_g,
+                                      float grad_scale, void* cuda_stream) {
+  return meta_impl(in, out, dlogits, ld_g, grad_scale, cuda_stream);
 }
 
 SAKI_API int saki_spec_verify(const saki_spec_in* in, const saki_spec_out* out, void* cuda_stream) {

@@ -37,6 +37,29 @@ struct RowParams {
   int32_t from_list;                   // general kernel only: route the rows of redo_list
 };
 
+// Parameters of the metadata-driven backward kernels (saki_route_bwd_from_meta).
+struct MetaParams {
+  const void* s;                       // current student logits [n_rows, V]
+  int64_t ld_s;
+  int64_t n_rows;
+  int32_t V;
+  const uint8_t* corrected;
+  const int32_t* proposal;
+  const int32_t* teacher_top1;
+  const float* advantage;
+  const uint8_t* mask;                 // may be NULL
+  const uint32_t* rollout_status;      // may be NULL
+  float temperature;
+  saki_meta_out out;
+  void* dlogits;
+  int64_t ld_g;
+  float grad_scale;
+  unsigned long long* flagged;         // device counter of flagged rows
+  int32_t* redo_list;                  // rows the streaming kernel hands to the float64 kernel
+  unsigned int* redo_count;
+  int32_t from_list;                   // general kernel only: take the rows of redo_list
+};
+
 // ---- Philox4x32-10 (Salmon et al., SC'11), written from the published round function ----
 __host__ __device__ inline void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
                                               uint32_t k0, uint32_t k1, uint32_t out[4]) {
@@ -111,5 +134,8 @@ cudaError_t launch_cluster(const RowParams& p, cudaStream_t st, int* n_launches,
 bool cluster_can_serve(const RowParams& p, int dtype);
 cudaError_t launch_rowsm(const RowParams& p, cudaStream_t st, int* n_launches, bool* served);
 bool rowsm_can_serve(const RowParams& p, int dtype);
+cudaError_t launch_meta_general(const MetaParams& p, int dtype, cudaStream_t st, int* n_launches);
+cudaError_t launch_meta_stream(const MetaParams& p, cudaStream_t st, int* n_launches, bool* served);
+bool meta_stream_can_serve(const MetaParams& p, int dtype);
 
 }  // namespace saki
