@@ -42,6 +42,8 @@ FALLBACK_HBM_GBS = 6650.0
 # routed: ncu capture on 2220 rows of the same workload (profiles/rowsm_kernel_cfg3.md); traffic grows
 # in proportion to the rows, so a full launch is this figure times N
 TRAFFIC_BYTES_PER_POSITION = 980210
+# the same for one meta_stream_kernel launch (profiles/meta_stream_kernel_cfg3.md)
+META_TRAFFIC_BYTES_PER_POSITION = 586707
 
 
 def _peaks():
@@ -212,6 +214,31 @@ def run_ours(args):
     n_flagged = P.check()
     kernel_used = P.last_kernel()
 
+    # ---- the step that follows the path: the trainer's loss and gradient from this call's metadata
+    # (saki_route_bwd_from_meta), on the same logits; reported beside the headline, not in it
+    nxt = None
+    if not args.no_next and rank == 0:
+        adv = out["logT_x"] - out["logp_x"]
+        mf = lambda: P.route_bwd_from_meta(s, out["corrected"], x, out["teacher_top1"], adv, w.temperature,
+                                           rollout_status=out["row_status"], grad_scale=1.0 / w.N, dlogits=g,
+                                           stream=stream)
+        for _ in range(3):
+            mf()
+        torch.cuda.synchronize()
+        l1 = P.launch_count()
+        m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        m0.record(stream)
+        for _ in range(args.steps):
+            mf()
+        m1.record(stream)
+        torch.cuda.synchronize()
+        mms = m0.elapsed_time(m1) / args.steps
+        mbytes = 2 * w.V * s.element_size() * w.N
+        nxt = {"call": "saki_route_bwd_from_meta", "value": w.N / (mms * 1e-3), "unit": UNIT, "ms_per_step": mms,
+               "gpu_launches": int(P.launch_count() - l1), "kernel": {4: "saki::meta_stream_kernel"}.get(P.last_kernel(), "saki::meta_general_kernel"),
+               "algorithmic_bytes_per_launch": mbytes, "achieved_gbs": mbytes / (mms * 1e-3) / 1e9,
+               "traffic": META_TRAFFIC_BYTES_PER_POSITION * w.N if META_TRAFFIC_BYTES_PER_POSITION else None}
+
     # ---- end to end: host buffers through saki_route_host
     e2e = None
     if not args.no_e2e:
@@ -281,6 +308,10 @@ def run_ours(args):
                        (s.numel() * s.element_size() / 1e9), "parallelism": f"rows sharded over {world} GPU(s), no collective"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
             "stats": stats, "achieved_gbs": achieved}
+    if nxt is not None:
+        nxt["roofline"] = {"bound": "hbm", "achieved": nxt["achieved_gbs"], "peak": peak, "unit": "GB/s",
+                           "frac": nxt["achieved_gbs"] / peak}
+        line["next_step"] = nxt
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -296,6 +327,7 @@ def main():
     ap.add_argument("--rows", type=int, default=0, help="cut the workload to its first R rows (profiling)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-next", action="store_true", help="skip the metadata-driven backward measurement")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-rows", type=int, default=384)
     ap.add_argument("--ref-rows", type=int, default=32)

@@ -174,44 +174,45 @@ __device__ __forceinline__ float m_pow2(float n) {   // 2^n for whole n, clamped
 // One warp's view of a row: `steps` steps of 32 chunks, the first `res` of them resident.
 struct MSeg { int c0, c1, steps, res; };
 
-// Fills this lane's slot with chunk (c0 + step*32 + lane) of `row_base`, or with the filler where
-// the row has no such chunk (row_base == nullptr: no row).
-__device__ __forceinline__ void m_fill(uint32_t slot, const char* row_base, const MSeg& sg, int step, int lane, uint64_t pol) {
-  const int c = sg.c0 + step * 32 + lane;
-  if (row_base != nullptr && step < sg.steps && c < sg.c1) m_cp_async16(slot, row_base + (size_t)c * 16, pol);
+// Fills this lane's slot with the 16 bytes at byte offset `off` of the row at `row_base`, or with the
+// filler where the row has no such chunk (off >= lim; lim = 0: no row).
+__device__ __forceinline__ void m_fill(uint32_t slot, const char* row_base, uint32_t off, uint32_t lim, uint64_t pol) {
+  if (off < lim) m_cp_async16(slot, row_base + off, pol);
   else m_sts128(slot, M_FILLER);
 }
 
-// Visits the warp's steps in order: body(words, chunk, valid).  Every step commits one cp.async
-// group.  A streamed step, once read, requests the streamed step MNST further on: of this pass, or
-// past its end the first streamed steps of the pass that follows (over `wrap`: the same row again
-// after pass "sum", the next row after pass "grad").  With REFILL, a resident step, once read,
-// requests the same step of `wrap` (the next row).
+// Visits the warp's steps in order: body(words, byte offset of the chunk in its row, valid).  Every
+// step commits one cp.async group.  A streamed step, once read, requests the streamed step MNST
+// further on: of this pass, or past its end the first streamed steps of the pass that follows (over
+// `wrap`: the same row again after pass "sum", the next row after pass "grad"; nullptr: none).  With
+// REFILL, a resident step, once read, requests the same step of `wrap` (the next row).
 template <bool REFILL, typename Body>
 __device__ __forceinline__ void m_visit(const MSeg& sg, int lane, uint32_t base, const char* cur, const char* wrap,
-                                        uint64_t pol_cur, uint64_t pol_wrap, uint32_t& ring_slot, Body&& body) {
-  const int T = sg.steps - sg.res;            // streamed steps: 0 or more than MNST
-  int c = sg.c0 + lane;
+                                        uint64_t pol_cur, uint64_t pol_wrap, uint64_t pol_res, uint32_t& ring_slot,
+                                        Body&& body) {
+  const uint32_t lim = (uint32_t)sg.c1 * 16u;
+  const uint32_t lim_wrap = wrap != nullptr ? lim : 0u;
+  const uint32_t wrap_back = (uint32_t)(MNST - (sg.steps - sg.res)) * 512u;   // (mod 2^32) from a step to the one it requests in the next pass
+  const char* wb = wrap != nullptr ? wrap : cur;
+  uint32_t off = (uint32_t)(sg.c0 + lane) * 16u;
+  uint32_t slot = base;
 #pragma unroll 1
-  for (int k = 0; k < sg.steps; ++k, c += 32) {
+  for (int k = 0; k < sg.steps; ++k, off += 512) {
     uint4 a;
+    m_wait<MNST - 1>();
     if (k < sg.res) {
-      const uint32_t slot = base + k * 512;
-      m_wait<MNST - 1>();
       a = m_lds128(slot);
-      if (REFILL) m_fill(slot, wrap, sg, k, lane, m_policy_first());
-      m_commit();
+      if (REFILL) m_fill(slot, wb, off, lim_wrap, pol_res);
+      slot += 512;
     } else {
-      m_wait<MNST - 1>();
       a = m_lds128(ring_slot);
-      const int kn = k + MNST;                // the step requested now
-      if (kn < sg.steps) m_fill(ring_slot, cur, sg, kn, lane, pol_cur);
-      else m_fill(ring_slot, wrap, sg, kn - T, lane, pol_wrap);
-      m_commit();
+      if (k + MNST < sg.steps) m_fill(ring_slot, cur, off + MNST * 512u, lim, pol_cur);
+      else m_fill(ring_slot, wb, off + wrap_back, lim_wrap, pol_wrap);
       ring_slot += 512;
       if (ring_slot == base + MKS * 512) ring_slot = base + MRES * 512;
     }
-    body(a, c, c < sg.c1);
+    m_commit();
+    body(a, off, off < lim);
   }
 }
 
@@ -239,9 +240,13 @@ __global__ void __launch_bounds__(MT, 1) meta_stream_kernel(const MetaParams P) 
   // first row of this CTA: request its resident steps and the first ring steps, one group per step
   if ((int64_t)blockIdx.x < P.n_rows) {
     const char* b0 = row_base(blockIdx.x);
-    for (int k = 0; k < sg.res; ++k) { m_fill(base + k * 512, b0, sg, k, lane, pol_first); m_commit(); }
+    const uint32_t lim = (uint32_t)sg.c1 * 16u, off0 = (uint32_t)(sg.c0 + lane) * 16u;
+    for (int k = 0; k < sg.res; ++k) { m_fill(base + k * 512, b0, off0 + k * 512u, lim, pol_first); m_commit(); }
     if (sg.res < sg.steps)
-      for (int j = 0; j < MNST; ++j) { m_fill(ring_slot + j * 512, b0, sg, sg.res + j, lane, pol_last); m_commit(); }
+      for (int j = 0; j < MNST; ++j) {
+        m_fill(ring_slot + j * 512, b0, off0 + (uint32_t)(sg.res + j) * 512u, lim, pol_last);
+        m_commit();
+      }
   }
 
   int rb = 0;
@@ -280,7 +285,7 @@ __global__ void __launch_bounds__(MT, 1) meta_stream_kernel(const MetaParams P) 
     uint32_t run = M_FILLER;
     {
       const float2 cc = splat(c32), kk = splat(ksw);
-      m_visit<false>(sg, lane, base, cur, cur, pol_last, pol_first, ring_slot, [&](const uint4& w, int, bool) {
+      m_visit<false>(sg, lane, base, cur, cur, pol_last, pol_first, pol_first, ring_slot, [&](const uint4& w, uint32_t, bool) {
         run = max_bf16x2(run, max_bf16x2(max_bf16x2(w.x, w.y), max_bf16x2(w.z, w.w)));
         S0 = fadd2(S0, ex2f2(ffma2(unpack_bf16x2(w.x), cc, kk)));
         S1 = fadd2(S1, ex2f2(ffma2(unpack_bf16x2(w.y), cc, kk)));
@@ -339,8 +344,10 @@ __global__ void __launch_bounds__(MT, 1) meta_stream_kernel(const MetaParams P) 
     {
       const float kr = bc[0], scale = bc[1], kg = bc[2];
       const int tok = __float_as_int(bc[3]);
+      const uint32_t tok_off = tok >= 0 ? (uint32_t)(tok >> 3) * 16u : 0xffffffffu;   // byte offset of the supervised token's chunk
       const float2 cc = splat(c32), kk = splat(kr), sc = splat(scale);
-      m_visit<true>(sg, lane, base, cur, nxt, pol_first, pol_last, ring_slot, [&](const uint4& w, int c, bool valid) {
+      char* g_bytes = reinterpret_cast<char*>(g_out);
+      m_visit<true>(sg, lane, base, cur, nxt, pol_first, pol_last, pol_first, ring_slot, [&](const uint4& w, uint32_t off, bool valid) {
         uint4 g = make_uint4(0u, 0u, 0u, 0u);
         if (tok >= 0) {    // a row that contributes nothing gets exact zeros, whatever its logits
           const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
@@ -350,7 +357,7 @@ __global__ void __launch_bounds__(MT, 1) meta_stream_kernel(const MetaParams P) 
             const float2 e = fmul2(ex2f2(ffma2(unpack_bf16x2(ww[i]), cc, kk)), sc);
             gp[i] = pack_bf16x2(e.x, e.y);
           }
-          if ((tok >> 3) == c) {   // the supervised token: subtract the one-hot part
+          if (off == tok_off) {   // the supervised token: subtract the one-hot part
             const int el = tok & 7, wi = el >> 1;
             const uint32_t word = wi == 0 ? ww[0] : wi == 1 ? ww[1] : wi == 2 ? ww[2] : ww[3];
             const float2 sf = unpack_bf16x2(word);
@@ -362,7 +369,7 @@ __global__ void __launch_bounds__(MT, 1) meta_stream_kernel(const MetaParams P) 
           }
           g = make_uint4(gp[0], gp[1], gp[2], gp[3]);
         }
-        if (valid) m_st_stream(g_out + (size_t)c * 8, g, pol_first);
+        if (valid) m_st_stream(g_bytes + off, g, pol_first);
       });
     }
   }
