@@ -68,9 +68,6 @@ __device__ __forceinline__ uint64_t policy_evict_first() {
   asm("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
   return p;
 }
-__device__ __forceinline__ void prefetch_l2(const void* src, uint32_t bytes, uint64_t pol) {
-  asm volatile("cp.async.bulk.prefetch.L2.global.L2::cache_hint [%0], %1, %2;" ::"l"(src), "r"(bytes), "l"(pol) : "memory");
-}
 __device__ __forceinline__ void bulk_load_hint(void* dst_smem, const void* src, uint32_t bytes, uint64_t* bar, uint64_t pol) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
                ::"r"(smem_addr(dst_smem)), "l"(src), "r"(bytes), "r"(smem_addr(bar)), "l"(pol) : "memory");
@@ -89,11 +86,6 @@ __device__ __forceinline__ void st_stream(__nv_bfloat16* p, uint4 v, uint64_t po
 __device__ __forceinline__ double warp_sum_d(double a) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-  return a;
-}
-__device__ __forceinline__ double warp_min_d(double a) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) a = fmin(a, __shfl_xor_sync(0xffffffffu, a, o));
   return a;
 }
 __device__ __forceinline__ float warp_max_f(float a) {
@@ -240,7 +232,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
   long long tacc[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
   long long tlast = clock64();
   int t_rows = 0;
-  long long w_solve = 0, w_lse = 0, w_final = 0;
+  long long w_solve = 0, w_evals = 0;
 #endif
   const int tid = threadIdx.x, lane = tid & 31;
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // broadcast: lets the compiler treat it as warp-uniform
@@ -526,7 +518,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
         }
       }, [] {});
 #ifdef SAKI_PHASE_TIMING
-      w_solve += clock64() - w_t0; ++w_lse;
+      w_solve += clock64() - w_t0; ++w_evals;
 #endif
       RTS(7);
       auto tot = [](const float2 a) { return (double)a.x + (double)a.y; };
@@ -750,8 +742,8 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
 
 #ifdef SAKI_PHASE_TIMING
   for (int64_t row = blockIdx.x; row < P.n_rows; row += gridDim.x) ++t_rows;
-  if (lane == 0 && blockIdx.x == 5 && t_rows > 0) printf("warp %d solve loop %lld cycles per row, %lld evaluations in %d rows, %d steps\n", warp, w_solve / t_rows, w_lse, t_rows, sg.steps);
-  if ((tid == 0 || tid == 1023) && (blockIdx.x == 0 || blockIdx.x == 77) && t_rows > 0)
+  if (lane == 0 && blockIdx.x == 5 && t_rows > 0) printf("warp %d solve loop %lld cycles per row, %lld evaluations in %d rows, %d steps\n", warp, w_solve / t_rows, w_evals, t_rows, sg.steps);
+  if (tid == 0 && (blockIdx.x == 0 || blockIdx.x == 77) && t_rows > 0)
     printf("blk %d tid %d rows %d | endbar %lld copy-wait %lld | lse %lld warp+bar %lld gather %lld scalar %lld | "
            "bar %lld solve %lld combine %lld scalar %lld | bar %lld final %lld combine %lld tail %lld (cycles per row)\n",
            (int)blockIdx.x, tid, t_rows, tacc[0] / t_rows, tacc[1] / t_rows, tacc[2] / t_rows, tacc[3] / t_rows,
