@@ -250,7 +250,8 @@ SAKI_API int saki_last_kernel(void);
 
 /* Two-tier routing: the float32 kernels (2, 3) hand rows whose KL they cannot resolve to the
  * tolerance (very small eps, nearly one-hot rows) to the float64 kernel, through a row list in device
- * memory that the library allocates once per device and keeps.  Synchronises the stream and returns
+ * memory that the library allocates once per device and stream and keeps (calls on different streams
+ * may overlap; calls on one stream are ordered by it).  Synchronises the stream and returns
  * how many rows of the calling thread's last routing call took that second tier. */
 SAKI_API int saki_redo_count(void* cuda_stream, uint64_t* n_rows);
 

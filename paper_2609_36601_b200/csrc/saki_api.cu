@@ -7,7 +7,10 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <iterator>
+#include <map>
 #include <mutex>
+#include <utility>
 #include <vector>
 #include <algorithm>
 
@@ -46,30 +49,37 @@ static int device_ready(unsigned long long** flagged) {
 }
 
 // Scratch of the two-tier routing: the float32 kernels append the rows they cannot resolve to a list
-// that the float64 kernel then routes.  One buffer per device, grown on demand, kept until exit.
-struct RedoScratch {
-  std::mutex mu;
-  int dev = -1;
+// that the float64 kernel then routes.  One buffer per (device, stream), so that calls on different
+// streams do not share a list; grown on demand, kept until exit.  (Calls on one stream are ordered by the
+// stream, so they may share.)
+struct RedoBuf {
   int32_t* list = nullptr;       // [cap] rows, followed by the counter
   int64_t cap = 0;
 };
-static RedoScratch g_redo;
+static std::mutex g_redo_mu;
+static std::map<std::pair<int, cudaStream_t>, RedoBuf> g_redo;
 static thread_local unsigned int* g_last_redo_count = nullptr;
 
-static int redo_scratch(int64_t n_rows, int32_t** list, unsigned int** count) {
-  std::lock_guard<std::mutex> lock(g_redo.mu);
+static int redo_scratch(int64_t n_rows, cudaStream_t st, int32_t** list, unsigned int** count) {
+  std::lock_guard<std::mutex> lock(g_redo_mu);
   int dev = 0;
   cudaGetDevice(&dev);
-  if (g_redo.dev != dev || g_redo.cap < n_rows) {
-    if (g_redo.list && g_redo.dev == dev) cudaFree(g_redo.list);
-    g_redo.list = nullptr; g_redo.cap = 0; g_redo.dev = dev;
-    const int64_t cap = std::max<int64_t>(n_rows, 1 << 16);
-    cudaError_t e = cudaMalloc((void**)&g_redo.list, (size_t)(cap + 64) * sizeof(int32_t));
-    if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc (redo list)");
-    g_redo.cap = cap;
+  if (g_redo.size() > 256) {   // many short-lived streams: start over (cudaFree waits for work in flight)
+    for (auto& kv : g_redo)
+      if (kv.first.first == dev && kv.second.list) { cudaFree(kv.second.list); kv.second = RedoBuf(); }
+    for (auto it = g_redo.begin(); it != g_redo.end();) it = it->second.list ? std::next(it) : g_redo.erase(it);
   }
-  *list = g_redo.list;
-  *count = (unsigned int*)(g_redo.list + g_redo.cap);
+  RedoBuf& b = g_redo[std::make_pair(dev, st)];
+  if (b.cap < n_rows) {
+    if (b.list) cudaFree(b.list);
+    b = RedoBuf();
+    const int64_t cap = std::max<int64_t>(n_rows, 1 << 16);
+    cudaError_t e = cudaMalloc((void**)&b.list, (size_t)(cap + 64) * sizeof(int32_t));
+    if (e != cudaSuccess) { b = RedoBuf(); return cuda_fail(e, "cudaMalloc (redo list)"); }
+    b.cap = cap;
+  }
+  *list = b.list;
+  *count = (unsigned int*)(b.list + b.cap);
   return SAKI_OK;
 }
 
@@ -127,7 +137,7 @@ static int dispatch_rows(RowParams p, int dtype, cudaStream_t st, int32_t* scrat
   if (fast) {
     if (scratch_list) { p.redo_list = scratch_list; p.redo_count = scratch_count; }
     else {
-      const int rc = redo_scratch(p.n_rows, &p.redo_list, &p.redo_count);
+      const int rc = redo_scratch(p.n_rows, st, &p.redo_list, &p.redo_count);
       if (rc) return rc;
     }
     e = cudaMemsetAsync(p.redo_count, 0, sizeof(unsigned int), st);
@@ -230,7 +240,7 @@ static int meta_impl(const saki_meta_in* in, const saki_meta_out* out, void* dlo
   bool served = false;
   int used = 1;
   if (g_kernel.load() != 1 && meta_stream_can_serve(p, in->dtype)) {
-    rc = redo_scratch(p.n_rows, &p.redo_list, &p.redo_count);
+    rc = redo_scratch(p.n_rows, st, &p.redo_list, &p.redo_count);
     if (rc) return rc;
     e = cudaMemsetAsync(p.redo_count, 0, sizeof(unsigned int), st);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");

@@ -281,6 +281,34 @@ def test_wide_range_rows(gap):
         P.set_kernel(prev)
 
 
+def test_calls_on_two_streams_do_not_share_scratch():
+    """The row list of the two-tier routing is kept per stream: two calls whose kernels may overlap on
+    the GPU give what each gives alone."""
+    prev = P.set_kernel(0)
+    try:
+        ws = [synth.Workload("a", 1500, 32000, "bf16", 0.005, 1.0, True, 1002, 2),
+              synth.Workload("b", 1200, 8192, "bf16", 0.005, 0.5, True, 99, 18)]
+        ds = [synth.generate(w, DEV) for w in ws]
+        alone = []
+        for w, d in zip(ws, ds):
+            alone.append(P.route_fwd_bwd(d["s"], d["t"], d["proposal"], w.eps, seed=w.seed))
+            torch.cuda.synchronize()
+            assert P.redo_count() > 0, "the workloads should put rows on the list"
+        streams = [torch.cuda.Stream(device=DEV) for _ in ws]
+        for rep in range(3):
+            res = []
+            for w, d, st in zip(ws, ds, streams):
+                with torch.cuda.stream(st):
+                    res.append(P.route_fwd_bwd(d["s"], d["t"], d["proposal"], w.eps, seed=w.seed, stream=st))
+            torch.cuda.synchronize()
+            for (o, g), (ro, rg) in zip(res, alone):
+                for k in o:
+                    assert torch.equal(o[k], ro[k]), (rep, k)
+                assert torch.equal(g, rg), rep
+    finally:
+        P.set_kernel(prev)
+
+
 def test_spec_verify_k_limits():
     V = 2048
     for K in (1, 16):
