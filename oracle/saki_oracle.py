@@ -427,6 +427,67 @@ def bwd_from_meta(s, corrected, proposal, teacher_top1, advantage, temperature=1
 
 
 # --------------------------------------------------------------------------
+# Placement controls: where teacher-mode supervision goes (Appendix "placement_control")
+# --------------------------------------------------------------------------
+STAGE_SELECT = 4     # the uniform of a position's exponential-race key
+SELECT_RANDOM = 0
+SELECT_TV_WEIGHTED = 1
+
+
+def select_tm(seq_start, corrected, tv, mode: int, seed=0, row_offset=0, mask=None,
+              rollout_status=None):
+    """For every trajectory b (positions seq_start[b] .. seq_start[b+1]-1) choose
+    m_b = number of corrected valid positions of b, valid positions to receive
+    the teacher-mode loss instead of the coupling's own corrections:
+
+      Random-TM        m_b valid positions uniformly at random (count-matched
+                       random locations);
+      TV-Weighted-TM   m_b valid positions without replacement with weights
+                       d_t = TV(p_t, q_t), by exponential-race keys
+                       -log U_t / d_t, the m_b smallest; if fewer than m_b
+                       valid positions have positive TV the rest is filled
+                       uniformly.
+
+    Readings: U_t is the (seed, row, STAGE_SELECT) uniform of the position; a
+    position is valid if its mask is 1 and the rollout routed it; "uniformly"
+    = the smallest U_t among the positions not yet chosen; ties go to the
+    lower index.  Returns (selected [N] uint8, m [B] int32, margin [B]: the
+    relative gap between the last chosen and the first rejected key, inf if
+    there is no choice to make)."""
+    seq_start = np.asarray(seq_start, dtype=np.int64)
+    N = int(seq_start[-1])
+    B = len(seq_start) - 1
+    selected = np.zeros(N, dtype=np.uint8)
+    m_out = np.zeros(B, dtype=np.int32)
+    margin = np.full(B, np.inf)
+    for b in range(B):
+        lo, hi = int(seq_start[b]), int(seq_start[b + 1])
+        keys = []
+        m = 0
+        for i in range(lo, hi):
+            ok = (mask is None or mask[i] != 0) and \
+                 (rollout_status is None or not (int(rollout_status[i]) & _ROLLOUT_UNUSABLE))
+            if not ok:
+                continue
+            m += int(corrected[i] != 0)
+            u = scalar_uniform(seed, row_offset + i, STAGE_SELECT)
+            d = float(tv[i]) if mode == SELECT_TV_WEIGHTED else 0.0
+            if mode == SELECT_TV_WEIGHTED and d > 0.0 and math.isfinite(d):
+                keys.append((0, -math.log(u) / d, i))
+            else:
+                keys.append((1 if mode == SELECT_TV_WEIGHTED else 0, u, i))
+        keys.sort()
+        m_out[b] = m
+        for k in keys[:m]:
+            selected[k[2]] = 1
+        if 0 < m < len(keys):
+            a, c = keys[m - 1], keys[m]
+            if a[0] == c[0]:
+                margin[b] = abs(c[1] - a[1]) / max(abs(c[1]), 1e-300)
+    return selected, m_out, margin
+
+
+# --------------------------------------------------------------------------
 # Proposal utility: x ~ softmax(s / temperature) by Gumbel-max
 # --------------------------------------------------------------------------
 def sample_proposal_row(s, temperature: float, seed: int, row: int):

@@ -482,3 +482,58 @@ def test_meta_backward_flags():
     assert list(res["status"]) == [O.ST_NONFINITE, O.ST_BAD_ID, O.ST_BAD_ID, O.ST_NOT_COMPUTED, O.ST_NONFINITE,
                                    O.ST_MASKED]
     assert np.all(res["grad"] == 0) and np.all(res["loss"] == 0)
+
+
+# ---------------------------------------------------------------- placement controls
+def test_select_tm_counts_and_validity():
+    rng = np.random.default_rng(50)
+    lens = [7, 1, 0, 30, 12]
+    seq = np.concatenate([[0], np.cumsum(lens)])
+    N = int(seq[-1])
+    C = (rng.random(N) < 0.4).astype(np.uint8)
+    tv = rng.random(N) * (rng.random(N) < 0.7)
+    mask = (rng.random(N) < 0.8).astype(np.uint8)
+    st = np.where(rng.random(N) < 0.1, O.ST_NOT_COMPUTED, 0).astype(np.uint32)
+    valid = (mask != 0) & (st == 0)
+    for mode in (O.SELECT_RANDOM, O.SELECT_TV_WEIGHTED):
+        sel, m, _ = O.select_tm(seq, C, tv, mode, seed=3, mask=mask, rollout_status=st)
+        assert np.all(sel[~valid] == 0)
+        for b in range(len(lens)):
+            lo, hi = seq[b], seq[b + 1]
+            assert m[b] == int((C[lo:hi] != 0)[valid[lo:hi]].sum()) == int(sel[lo:hi].sum())
+
+
+def test_select_tm_laws():
+    """Exponential race: with one pick the chance of position t is d_t / sum d; with two picks the
+    successive-sampling law (closed forms).  Random-TM: every subset of the right size equally likely."""
+    d = np.array([0.5, 0.2, 0.3])
+    seq = np.array([0, 3])
+    trials = 6000
+    first = np.zeros(3)
+    pairs = {}
+    uni = np.zeros(3)
+    for sd in range(trials):
+        sel, _, _ = O.select_tm(seq, np.array([1, 0, 0]), d, O.SELECT_TV_WEIGHTED, seed=sd)
+        first += sel
+        sel2, _, _ = O.select_tm(seq, np.array([1, 1, 0]), d, O.SELECT_TV_WEIGHTED, seed=sd)
+        pairs[tuple(sel2)] = pairs.get(tuple(sel2), 0) + 1
+        selr, _, _ = O.select_tm(seq, np.array([0, 1, 0]), d, O.SELECT_RANDOM, seed=sd)
+        uni += selr
+    assert np.all(np.abs(first / trials - d / d.sum()) < 0.025)
+    assert np.all(np.abs(uni / trials - 1 / 3) < 0.025)
+    D = d.sum()
+    for (i, j), key in (((0, 1), (1, 1, 0)), ((0, 2), (1, 0, 1)), ((1, 2), (0, 1, 1))):
+        want = d[i] / D * d[j] / (D - d[i]) + d[j] / D * d[i] / (D - d[j])
+        assert abs(pairs.get(key, 0) / trials - want) < 0.025
+
+
+def test_select_tm_uniform_fill_when_too_few_positive():
+    tv = np.array([0.0, 0.3, 0.0, 0.0, 0.1, 0.0])
+    C = np.array([1, 1, 1, 0, 1, 0])              # m = 4 > 2 positions with positive TV
+    hits = np.zeros(6)
+    for sd in range(3000):
+        sel, m, _ = O.select_tm(np.array([0, 6]), C, tv, O.SELECT_TV_WEIGHTED, seed=sd)
+        assert m[0] == 4 and sel[1] == 1 and sel[4] == 1 and sel.sum() == 4
+        hits += sel
+    zeros = [0, 2, 3, 5]                            # two of the four zero-TV positions, uniformly
+    assert np.all(np.abs(hits[zeros] / 3000 - 0.5) < 0.03)
