@@ -248,7 +248,7 @@ def run_ours(args):
         hout = None
         esz = s.element_size()
         h2d = 2 * s.numel() * esz + hx.numel() * 4
-        d2h = s.numel() * esz + w.N * (1 + 4 * 13)
+        d2h = s.numel() * esz + w.N * (1 + 4 * 14)
         n_e2e = max(1, min(args.steps, args.e2e_steps))
         hout, _ = P.route_host(hs, ht, hx, w.eps, w.temperature, w.seed, row_offset, grad_scale=1.0 / w.N,
                                out=hout, dlogits=hg)      # warm-up: staging buffers get allocated

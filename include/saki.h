@@ -37,8 +37,8 @@
  *     ids to -1.
  *   - Random numbers: Philox4x32-10, key = (seed lo, seed hi), counter =
  *     (row lo, row hi, stage, block); stage 0 proposal Gumbel noise (word
- *     v%4 of block v/4), 1 acceptance uniform, 2 residual draw, 3 bonus draw
- *     (word 0 of block 0).  A word w gives the uniform ((w>>9)+0.5) 2^-23.
+ *     v%4 of block v/4), 1 acceptance uniform, 2 residual draw, 3 bonus draw,
+ *     4 placement-control key (word 0 of block 0).  A word w gives the uniform ((w>>9)+0.5) 2^-23.
  *     `row` is the GLOBAL row id row_offset + i, so results do not depend on
  *     how a batch is chunked or sharded.
  *   - Results are deterministic: same inputs, same GPU model, same outputs.
@@ -110,6 +110,7 @@ typedef struct {
   float* logT_x;
   float* logp_y;         /* log p(y), log q(y) at the committed token */
   float* logq_y;
+  float* logT_y;         /* log T(y): with logp_y, the advantage at the committed token */
   float* loss;           /* routed loss of the position, NOT scaled by grad_scale; 0 where masked */
   uint32_t* row_status;  /* SAKI_ROW_* bits */
 } saki_out;
@@ -189,6 +190,35 @@ typedef struct {
  * sums overflow, on a float64 kernel.  Flagged rows count towards saki_check(). */
 SAKI_API int saki_route_bwd_from_meta(const saki_meta_in* in, const saki_meta_out* out, void* dlogits,
                                       int64_t ld_g, float grad_scale, void* cuda_stream);
+
+/* Placement controls of the paper's ablation (Appendix "placement_control"): for every trajectory b
+ * (positions seq_start[b] .. seq_start[b+1]-1) choose m_b = number of its corrected valid positions,
+ * valid positions that receive the teacher-mode loss INSTEAD of the coupling's own corrections:
+ *   SAKI_SELECT_RANDOM       m_b valid positions uniformly at random;
+ *   SAKI_SELECT_TV_WEIGHTED  m_b valid positions without replacement with weights tv[t], by
+ *                            exponential-race keys -log(U_t)/tv[t], the m_b smallest; if fewer than m_b
+ *                            valid positions have positive TV, the rest is filled uniformly (smallest U_t).
+ * U_t is the uniform of (seed, row_offset + t, stage 4); a position is valid if mask[t] != 0 and the
+ * rollout routed it; ties go to the lower index.  Keys are formed in float64.  Feed `selected` to
+ * saki_route_bwd_from_meta as its `corrected`.  (Teacher-sampled supervision, the other ablation,
+ * needs no call of its own: draw the target with saki_sample_proposal on the teacher's logits under
+ * another seed and pass it as `teacher_top1`.) */
+typedef enum { SAKI_SELECT_RANDOM = 0, SAKI_SELECT_TV_WEIGHTED = 1 } saki_select_mode;
+typedef struct {
+  int64_t N;                      /* positions, = seq_start[B] */
+  int64_t B;                      /* trajectories */
+  const int64_t* seq_start;       /* [B+1] DEVICE, non-decreasing, seq_start[0] = 0 */
+  const uint8_t* corrected;       /* [N] C_t of the routing call. Required */
+  const float* tv;                /* [N] TV(p_t, q_t) of the routing call. Required in TV-weighted mode */
+  const uint8_t* mask;            /* [N] or NULL */
+  const uint32_t* rollout_status; /* [N] or NULL */
+  int32_t mode;                   /* saki_select_mode */
+  uint64_t seed;
+  uint64_t row_offset;            /* global id of position 0 */
+} saki_select_in;
+
+/* selected: [N] uint8 (required); m: [B] int32 or NULL.  Asynchronous on the stream. */
+SAKI_API int saki_select_tm(const saki_select_in* in, uint8_t* selected, int32_t* m, void* cuda_stream);
 
 /* Block verification (Section 3.5, Appendix I) of B drafted blocks of K tokens. */
 typedef struct {

@@ -230,7 +230,7 @@ def round_to_bf16(x):
 # --------------------------------------------------------------------------
 _ZERO_ROW = dict(corrected=0, token=-1, teacher_top1=-1, lam=0.0, kl=0.0,
                  tv=0.0, accept_prob=0.0, logp_x=0.0, logq_x=0.0, logT_x=0.0,
-                 logp_y=0.0, logq_y=0.0, loss=0.0, margin_accept=math.inf,
+                 logp_y=0.0, logq_y=0.0, logT_y=0.0, loss=0.0, margin_accept=math.inf,
                  margin_draw=math.inf)
 
 
@@ -305,7 +305,7 @@ def route_row(s, t, x: int, eps: float, temperature: float, seed: int,
     out.update(corrected=corrected, token=y, teacher_top1=v_star, lam=lam,
                kl=kl, tv=tv, accept_prob=accept_prob, logp_x=float(lp[x]),
                logq_x=float(lq[x]), logT_x=float(lT[x]), logp_y=float(lp[y]),
-               logq_y=float(lq[y]), loss=float(loss), status=status,
+               logq_y=float(lq[y]), logT_y=float(lT[y]), loss=float(loss), status=status,
                margin_accept=abs(u_acc - accept_prob) if lam > 0.0 else math.inf,
                margin_draw=margin_draw)
 
@@ -330,7 +330,7 @@ def route_row(s, t, x: int, eps: float, temperature: float, seed: int,
 
 
 _FIELDS = ("corrected", "token", "teacher_top1", "lam", "kl", "tv",
-           "accept_prob", "logp_x", "logq_x", "logT_x", "logp_y", "logq_y",
+           "accept_prob", "logp_x", "logq_x", "logT_x", "logp_y", "logq_y", "logT_y",
            "loss", "status", "margin_accept", "margin_draw")
 _INT_FIELDS = {"corrected": np.uint8, "token": np.int32,
                "teacher_top1": np.int32, "status": np.uint32}
@@ -580,7 +580,7 @@ def spec_verify(s, t, draft, eps, temperature=1.0, seed=0, seq_offset=0):
                 bonus.update(token=y, teacher_top1=int(np.argmax(tk)), lam=lam,
                              kl=kl if lam > 0 else 0.0,
                              tv=total_variation(np.exp(lp), q) if lam > 0 else 0.0,
-                             logp_y=float(lp[y]), logq_y=float(lq[y]),
+                             logp_y=float(lp[y]), logq_y=float(lq[y]), logT_y=float(lT[y]),
                              margin_draw=m)
                 if not (eps > 0):
                     bonus["status"] |= ST_EPS_ZERO

@@ -18,9 +18,9 @@ _lib = None
 SAKI_F32, SAKI_BF16 = 0, 1
 ROW_SATURATED, ROW_EPS_ZERO, ROW_MASKED, ROW_NONFINITE, ROW_BAD_ID, ROW_TIMEOUT, ROW_NOT_COMPUTED = 1, 2, 4, 8, 16, 32, 64
 
-_FLOAT_FIELDS = ("lambda", "kl", "tv", "accept_prob", "logp_x", "logq_x", "logT_x", "logp_y", "logq_y", "loss")
+_FLOAT_FIELDS = ("lambda", "kl", "tv", "accept_prob", "logp_x", "logq_x", "logT_x", "logp_y", "logq_y", "logT_y", "loss")
 EXPORTS = ("saki_route_fwd", "saki_route_fwd_bwd", "saki_route_fwd_bwd_noalloc", "saki_route_host",
-           "saki_route_bwd_from_meta", "saki_spec_verify",
+           "saki_route_bwd_from_meta", "saki_select_tm", "saki_spec_verify",
            "saki_sample_proposal", "saki_check", "saki_set_kernel", "saki_last_kernel", "saki_redo_count",
            "saki_launch_count",
            "saki_last_error", "saki_version")
@@ -58,6 +58,12 @@ class SakiMetaOut(C.Structure):
     _fields_ = [("loss", C.c_void_p), ("logp_tok", C.c_void_p), ("row_status", C.c_void_p)]
 
 
+class SakiSelectIn(C.Structure):
+    _fields_ = [("N", C.c_int64), ("B", C.c_int64), ("seq_start", C.c_void_p), ("corrected", C.c_void_p),
+                ("tv", C.c_void_p), ("mask", C.c_void_p), ("rollout_status", C.c_void_p), ("mode", C.c_int32),
+                ("seed", C.c_uint64), ("row_offset", C.c_uint64)]
+
+
 class SakiSpecIn(C.Structure):
     _fields_ = [("student_logits", C.c_void_p), ("teacher_logits", C.c_void_p),
                 ("ss_seq", C.c_int64), ("ss_pos", C.c_int64), ("ts_seq", C.c_int64), ("ts_pos", C.c_int64),
@@ -90,6 +96,8 @@ def load_library(path: str | None = None):
     lib.saki_route_bwd_from_meta.argtypes = [C.POINTER(SakiMetaIn), C.POINTER(SakiMetaOut), C.c_void_p, C.c_int64,
                                              C.c_float, C.c_void_p]
     lib.saki_route_bwd_from_meta.restype = C.c_int
+    lib.saki_select_tm.argtypes = [C.POINTER(SakiSelectIn), C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.saki_select_tm.restype = C.c_int
     lib.saki_spec_verify.argtypes = [C.POINTER(SakiSpecIn), C.POINTER(SakiSpecOut), C.c_void_p]
     lib.saki_sample_proposal.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_float,
                                          C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p]
@@ -232,6 +240,36 @@ def route_bwd_from_meta(s, corrected, proposal, teacher_top1, advantage, tempera
     _raise(lib, lib.saki_route_bwd_from_meta(C.byref(mi), C.byref(mo), dlogits.data_ptr(), ld_g, grad_scale,
                                              _stream_ptr(stream)))
     return out, dlogits
+
+
+SELECT_RANDOM, SELECT_TV_WEIGHTED = 0, 1
+
+
+def select_tm(seq_start, corrected, tv, mode, seed=0, row_offset=0, mask=None, rollout_status=None, stream=None):
+    """saki_select_tm on device tensors: the placement controls (Random-TM, TV-Weighted-TM).  `seq_start`
+    is the int64 [B+1] tensor of trajectory boundaries.  Returns (selected uint8 [N], m int32 [B])."""
+    lib = load_library()
+    dev = corrected.device
+    n, nb = corrected.shape[0], seq_start.shape[0] - 1
+    if seq_start.dtype != torch.int64 or seq_start.device != dev or not seq_start.is_contiguous():
+        raise ValueError("seq_start must be a contiguous int64 tensor on the same device")
+    keep = [_vec_check(corrected, torch.uint8, n, dev, "corrected")]
+    si = SakiSelectIn()
+    si.N, si.B, si.seq_start, si.corrected = n, nb, seq_start.data_ptr(), corrected.data_ptr()
+    if tv is not None:
+        keep.append(_vec_check(tv, torch.float32, n, dev, "tv"))
+        si.tv = tv.data_ptr()
+    if mask is not None:
+        keep.append(_vec_check(mask, torch.uint8, n, dev, "mask"))
+        si.mask = mask.data_ptr()
+    if rollout_status is not None:
+        keep.append(_vec_check(rollout_status, torch.int32, n, dev, "rollout_status"))
+        si.rollout_status = rollout_status.data_ptr()
+    si.mode, si.seed, si.row_offset = mode, seed, row_offset
+    selected = torch.empty(n, dtype=torch.uint8, device=dev)
+    m = torch.empty(max(nb, 0), dtype=torch.int32, device=dev)
+    _raise(lib, lib.saki_select_tm(C.byref(si), selected.data_ptr(), m.data_ptr(), _stream_ptr(stream)))
+    return selected, m
 
 
 def route_fwd_bwd_noalloc(s, t, proposal, eps, out, dlogits, temperature=1.0, seed=0, row_offset=0, mask=None,

@@ -355,6 +355,30 @@ SAKI_API int saki_route_bwd_from_meta(const saki_meta_in* in, const saki_meta_ou
   return meta_impl(in, out, dlogits, ld_g, grad_scale, cuda_stream);
 }
 
+SAKI_API int saki_select_tm(const saki_select_in* in, uint8_t* selected, int32_t* m, void* cuda_stream) {
+  g_err[0] = 0;
+  if (!in) return fail(SAKI_ERR_INVALID_ARG, "NULL argument struct");
+  if (in->N < 0 || in->B < 0) return fail(SAKI_ERR_INVALID_ARG, "negative size");
+  if (in->mode != SAKI_SELECT_RANDOM && in->mode != SAKI_SELECT_TV_WEIGHTED)
+    return fail(SAKI_ERR_INVALID_ARG, "unknown selection mode %d", in->mode);
+  if (in->B == 0 || in->N == 0) return SAKI_OK;
+  if (!in->seq_start || !in->corrected || !selected) return fail(SAKI_ERR_INVALID_ARG, "seq_start, corrected and selected are required");
+  if (in->mode == SAKI_SELECT_TV_WEIGHTED && !in->tv) return fail(SAKI_ERR_INVALID_ARG, "tv is required in TV-weighted mode");
+  unsigned long long* flagged = nullptr;
+  int rc = device_ready(&flagged);
+  if (rc) return rc;
+  SelectParams p;
+  memset(&p, 0, sizeof(p));
+  p.N = in->N; p.B = in->B; p.seq_start = in->seq_start; p.corrected = in->corrected; p.tv = in->tv;
+  p.mask = in->mask; p.rollout_status = in->rollout_status; p.mode = in->mode; p.seed = in->seed;
+  p.row_offset = in->row_offset; p.selected = selected; p.m = m;
+  int launches = 0;
+  cudaError_t e = launch_select(p, (cudaStream_t)cuda_stream, &launches);
+  if (e != cudaSuccess) return cuda_fail(e, "selection kernel launch");
+  g_launches += (uint64_t)launches;
+  return SAKI_OK;
+}
+
 SAKI_API int saki_spec_verify(const saki_spec_in* in, const saki_spec_out* out, void* cuda_stream) {
   g_err[0] = 0;
   if (!in || !out) return fail(SAKI_ERR_INVALID_ARG, "NULL argument struct");
@@ -477,8 +501,8 @@ SAKI_API int saki_route_host(const saki_in* in, const saki_out* out, void* dlogi
   const size_t o_g = dlogits ? take(chunk * row_bytes) : 0;
   const size_t o_prop = take(chunk * 4), o_mask = take(chunk);
   const size_t o_corr = take(chunk), o_tok = take(chunk * 4), o_top = take(chunk * 4), o_stat = take(chunk * 4);
-  size_t o_f[10];
-  for (int k = 0; k < 10; ++k) o_f[k] = take(chunk * 4);
+  size_t o_f[11];
+  for (int k = 0; k < 11; ++k) o_f[k] = take(chunk * 4);
   const size_t total = off;
   for (int k = 0; k < 2; ++k) {
     if (g_stage.cap[k] < total) {
@@ -489,8 +513,8 @@ SAKI_API int saki_route_host(const saki_in* in, const saki_out* out, void* dlogi
       g_stage.cap[k] = total;
     }
   }
-  float* const host_f[10] = {out->lambda, out->kl, out->tv, out->accept_prob, out->logp_x,
-                             out->logq_x, out->logT_x, out->logp_y, out->logq_y, out->loss};
+  float* const host_f[11] = {out->lambda, out->kl, out->tv, out->accept_prob, out->logp_x,
+                             out->logq_x, out->logT_x, out->logp_y, out->logq_y, out->logT_y, out->loss};
   int result = SAKI_OK;
   int k = 0;
   for (int64_t r0 = 0; r0 < in->N && result == SAKI_OK; r0 += chunk, k ^= 1) {
@@ -514,9 +538,9 @@ SAKI_API int saki_route_host(const saki_in* in, const saki_out* out, void* dlogi
     saki_out dout;
     dout.corrected = (uint8_t*)(base + o_corr); dout.token = (int32_t*)(base + o_tok);
     dout.teacher_top1 = (int32_t*)(base + o_top); dout.row_status = (uint32_t*)(base + o_stat);
-    float** df[10] = {&dout.lambda, &dout.kl, &dout.tv, &dout.accept_prob, &dout.logp_x,
-                      &dout.logq_x, &dout.logT_x, &dout.logp_y, &dout.logq_y, &dout.loss};
-    for (int q = 0; q < 10; ++q) *df[q] = (float*)(base + o_f[q]);
+    float** df[11] = {&dout.lambda, &dout.kl, &dout.tv, &dout.accept_prob, &dout.logp_x,
+                      &dout.logq_x, &dout.logT_x, &dout.logp_y, &dout.logq_y, &dout.logT_y, &dout.loss};
+    for (int q = 0; q < 11; ++q) *df[q] = (float*)(base + o_f[q]);
     result = route_impl(&din, &dout, dlogits ? base + o_g : nullptr, (int64_t)Vp, grad_scale, dlogits != nullptr, st);
     if (result != SAKI_OK) break;
     e = cudaMemcpyAsync(out->corrected + r0, dout.corrected, n, cudaMemcpyDeviceToHost, st);
@@ -525,7 +549,7 @@ SAKI_API int saki_route_host(const saki_in* in, const saki_out* out, void* dlogi
       e = cudaMemcpyAsync(out->teacher_top1 + r0, dout.teacher_top1, n * 4, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess && out->row_status)
       e = cudaMemcpyAsync(out->row_status + r0, dout.row_status, n * 4, cudaMemcpyDeviceToHost, st);
-    for (int q = 0; q < 10 && e == cudaSuccess; ++q)
+    for (int q = 0; q < 11 && e == cudaSuccess; ++q)
       if (host_f[q]) e = cudaMemcpyAsync(host_f[q] + r0, *df[q], n * 4, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess && dlogits)
       e = cudaMemcpy2DAsync((char*)dlogits + (size_t)r0 * ld_g * es, ld_g * es, base + o_g, row_bytes, in->V * es, n,

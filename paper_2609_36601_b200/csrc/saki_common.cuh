@@ -7,7 +7,7 @@
 
 namespace saki {
 
-enum { STAGE_PROPOSE = 0, STAGE_ACCEPT = 1, STAGE_RESIDUAL = 2, STAGE_BONUS = 3 };
+enum { STAGE_PROPOSE = 0, STAGE_ACCEPT = 1, STAGE_RESIDUAL = 2, STAGE_BONUS = 3, STAGE_SELECT = 4 };
 
 // Everything a row kernel needs; passed by value as the kernel parameter.
 // Plain routing and block verification share it: row i is position
@@ -60,6 +60,20 @@ struct MetaParams {
   int32_t from_list;                   // general kernel only: take the rows of redo_list
 };
 
+// Parameters of the placement-control kernel (saki_select_tm).
+struct SelectParams {
+  int64_t N, B;
+  const int64_t* seq_start;
+  const uint8_t* corrected;
+  const float* tv;
+  const uint8_t* mask;
+  const uint32_t* rollout_status;
+  int32_t mode;
+  uint64_t seed, row_offset;
+  uint8_t* selected;
+  int32_t* m;
+};
+
 // ---- Philox4x32-10 (Salmon et al., SC'11), written from the published round function ----
 __host__ __device__ inline void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
                                               uint32_t k0, uint32_t k1, uint32_t out[4]) {
@@ -99,7 +113,7 @@ template <> __device__ __forceinline__ void st_from_float<__nv_bfloat16>(__nv_bf
 // Per-row scalar results, written by one thread.
 struct RowResult {
   int corrected, token, vstar;
-  float lambda, kl, tv, accept, logp_x, logq_x, logT_x, logp_y, logq_y, loss;
+  float lambda, kl, tv, accept, logp_x, logq_x, logT_x, logp_y, logq_y, logT_y, loss;
   uint32_t status;
 };
 
@@ -116,6 +130,7 @@ __device__ inline void write_row(const saki_out& o, int64_t i, const RowResult& 
   if (o.logT_x) o.logT_x[i] = r.logT_x;
   if (o.logp_y) o.logp_y[i] = r.logp_y;
   if (o.logq_y) o.logq_y[i] = r.logq_y;
+  if (o.logT_y) o.logT_y[i] = r.logT_y;
   if (o.loss && write_loss) o.loss[i] = r.loss;
   if (o.row_status) o.row_status[i] = r.status;
 }
@@ -123,7 +138,7 @@ __device__ inline void write_row(const saki_out& o, int64_t i, const RowResult& 
 __device__ inline RowResult zero_row(uint32_t status) {
   RowResult r;
   r.corrected = 0; r.token = -1; r.vstar = -1;
-  r.lambda = r.kl = r.tv = r.accept = r.logp_x = r.logq_x = r.logT_x = r.logp_y = r.logq_y = r.loss = 0.f;
+  r.lambda = r.kl = r.tv = r.accept = r.logp_x = r.logq_x = r.logT_x = r.logp_y = r.logq_y = r.logT_y = r.loss = 0.f;
   r.status = status;
   return r;
 }
@@ -137,5 +152,6 @@ bool rowsm_can_serve(const RowParams& p, int dtype);
 cudaError_t launch_meta_general(const MetaParams& p, int dtype, cudaStream_t st, int* n_launches);
 cudaError_t launch_meta_stream(const MetaParams& p, cudaStream_t st, int* n_launches, bool* served);
 bool meta_stream_can_serve(const MetaParams& p, int dtype);
+cudaError_t launch_select(const SelectParams& p, cudaStream_t st, int* n_launches);
 
 }  // namespace saki

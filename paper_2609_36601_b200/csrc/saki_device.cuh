@@ -428,10 +428,10 @@ static __device__ __noinline__ void write_result_tv(const double* bc, saki_out o
   if (corrected || bonus) {
     const double lp_y = LN2 * (c64 * (double)__bfloat162float(g_s[y])) - G0;
     const double lT_y = LN2 * (c64 * (double)__bfloat162float(g_t[y])) - G1;
-    r.logp_y = (float)lp_y; r.logq_y = (float)(lp_y + lam * (lT_y - lp_y) - Lam);
+    r.logp_y = (float)lp_y; r.logq_y = (float)(lp_y + lam * (lT_y - lp_y) - Lam); r.logT_y = (float)lT_y;
     if (corrected && !(status & SAKI_ROW_MASKED))   // teacher-mode loss: -log p(v*)
       r.loss = (float)-(LN2 * (c64 * (double)__bfloat162float(g_s[r.vstar])) - G0);
-  } else { r.logp_y = r.logp_x; r.logq_y = r.logq_x; }
+  } else { r.logp_y = r.logp_x; r.logq_y = r.logq_x; r.logT_y = r.logT_x; }
   r.status = status;
   write_row(out, row, r, write_loss);
 }

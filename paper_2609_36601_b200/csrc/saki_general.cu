@@ -291,6 +291,7 @@ __global__ void __launch_bounds__(GT) general_kernel(const RowParams P) {
       const double lT_y = (double)ld_as_float(t, y) / tau - lse_t;
       r.logp_y = (float)lp_y;
       r.logq_y = (float)(lp_y + lam * (lT_y - lp_y) - Lam);
+      r.logT_y = (float)lT_y;
       r.loss = (float)loss;
       r.status = status;
       write_row(P.out, row, r, !P.spec);

@@ -79,7 +79,7 @@ def compare_rows(gpu: dict, ref: dict, rows=None, check_loss=True):
         d = np.abs(g[name].astype(np.float64) - ref[key])
         assert np.all(d <= tol), f"{name}: max error {d.max():.3e}"
     same = ok & (g["corrected"] == ref["corrected"]) & (g["token"] == ref["token"])
-    for name in ("logp_x", "logq_x", "logT_x", "logp_y", "logq_y"):
+    for name in ("logp_x", "logq_x", "logT_x", "logp_y", "logq_y", "logT_y"):
         d = np.abs(g[name].astype(np.float64) - ref[name])[same]
         assert np.all(d <= 1e-5 * (1 + np.abs(ref[name][same]))), f"{name}: max error {d.max():.3e}"
     if check_loss:

@@ -33,7 +33,7 @@ def test_version_and_error_text_without_a_gpu():
 def test_struct_layouts_match_the_header():
     # sizes that the C compiler gives the same structs (checked with a tiny C program)
     import subprocess, tempfile
-    src = '#include <stdio.h>\n#include "saki.h"\nint main(){printf("%zu %zu %zu %zu %zu %zu\\n",sizeof(saki_in),sizeof(saki_out),sizeof(saki_spec_in),sizeof(saki_spec_out),sizeof(saki_meta_in),sizeof(saki_meta_out));return 0;}\n'
+    src = '#include <stdio.h>\n#include "saki.h"\nint main(){printf("%zu %zu %zu %zu %zu %zu %zu\\n",sizeof(saki_in),sizeof(saki_out),sizeof(saki_spec_in),sizeof(saki_spec_out),sizeof(saki_meta_in),sizeof(saki_meta_out),sizeof(saki_select_in));return 0;}\n'
     with tempfile.TemporaryDirectory() as td:
         c = os.path.join(td, "a.c")
         open(c, "w").write(src)
@@ -42,4 +42,5 @@ def test_struct_layouts_match_the_header():
         sizes = [int(v) for v in subprocess.check_output([exe]).split()]
     assert sizes == [ctypes.sizeof(binding.SakiIn), ctypes.sizeof(binding.SakiOut),
                      ctypes.sizeof(binding.SakiSpecIn), ctypes.sizeof(binding.SakiSpecOut),
-                     ctypes.sizeof(binding.SakiMetaIn), ctypes.sizeof(binding.SakiMetaOut)]
+                     ctypes.sizeof(binding.SakiMetaIn), ctypes.sizeof(binding.SakiMetaOut),
+                     ctypes.sizeof(binding.SakiSelectIn)]

@@ -194,7 +194,7 @@ def test_spec_verify_small(kernel):
             assert per["token"][b, j] == r["token"] and per["corrected"][b, j] == r["corrected"]
             for name, key in (("lambda", "lam"), ("tv", "tv"), ("kl", "kl"), ("accept_prob", "accept_prob")):
                 assert abs(per[name][b, j] - r[key]) <= 1e-5, (name, b, j)
-            for name in ("logp_y", "logq_y", "logp_x", "logq_x"):
+            for name in ("logp_y", "logq_y", "logT_y", "logp_x", "logq_x"):
                 assert abs(per[name][b, j] - r[name]) <= 1e-5 * (1 + abs(r[name])), (name, b, j)
     assert ref["n_accept"][5] <= 1 and res["next_token"][5].item() == ref["next_token"][5]
 
