@@ -283,9 +283,14 @@ __global__ void __launch_bounds__(MT, 1) meta_stream_kernel(const MetaParams P) 
     }
     float2 S0 = splat(0.f), S1 = splat(0.f);
     uint32_t run = M_FILLER;
+    const char* pf = sg.steps == sg.res ? nxt : nullptr;
     {
       const float2 cc = splat(c32), kk = splat(ksw);
-      m_visit<false>(sg, lane, base, cur, cur, pol_last, pol_first, pol_first, ring_slot, [&](const uint4& w, uint32_t, bool) {
+      m_visit<false>(sg, lane, base, cur, cur, pol_last, pol_first, pol_first, ring_slot, [&](const uint4& w, uint32_t off, bool valid) {
+        // a row that is entirely resident leaves L2 free: the next row's bytes of this step are sent on
+        // their way into L2 (one lane per 128-byte line), so that HBM stays busy during this pass.  With
+        // a streamed part kept in L2 between the passes the same prefetch evicts it (measured: -17 %).
+        if (pf != nullptr && valid && (lane & 7) == 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(pf + off));
         run = max_bf16x2(run, max_bf16x2(max_bf16x2(w.x, w.y), max_bf16x2(w.z, w.w)));
         S0 = fadd2(S0, ex2f2(ffma2(unpack_bf16x2(w.x), cc, kk)));
         S1 = fadd2(S1, ex2f2(ffma2(unpack_bf16x2(w.y), cc, kk)));
