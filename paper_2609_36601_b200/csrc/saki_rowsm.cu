@@ -42,7 +42,7 @@ constexpr int KS_MAX = 208 / RW;        // steps per warp that fit in shared mem
 constexpr int MAX_STEPS = 64;            // steps per warp the draw bookkeeping can hold (V <= 64*32*8*RW)
 constexpr int RES_CHUNKS = KS_MAX * 32; // resident chunks per warp and row
 constexpr int RNV = 8;                  // doubles per partial vector
-static_assert(RW >= 13, "warps 8-12 do side work while warps 0-6 gather and thread 0 does the scalars");
+static_assert(RW >= 14, "warps 8-13 do side work while warps 0-6 gather and thread 0 does the scalars");
 static_assert(KS_MAX - 4 >= 1, "every warp keeps at least its first step resident");
 
 constexpr int ROFF_S = 0;                                        // [RW][RES_CHUNKS] uint4
@@ -52,7 +52,9 @@ constexpr int ROFF_GAT = ROFF_RED + RNV * RW * 8;                // [16] doubles
 constexpr int ROFF_BC = ROFF_GAT + 16 * 8;                       // [2][BC_DOUBLES] doubles, alternating by row
 constexpr int ROFF_WMAX = ROFF_BC + 2 * BC_DOUBLES * 8;          // [3][RW]: teacher maximum, its index, student maximum per warp
 constexpr int ROFF_STEP = ROFF_WMAX + 4 * RW * 4;                // [RW][MAX_STEPS] floats: draw weight of each step
-constexpr int ROFF_MBAR = ROFF_STEP + RW * MAX_STEPS * 4;
+constexpr int ROFF_FIN = ROFF_STEP + RW * MAX_STEPS * 4;          // [2][2][RW] doubles: what pass "final" leaves per warp, by row parity
+constexpr int ROFF_MBAR = ROFF_FIN + 2 * 2 * RW * 8;
+constexpr int FIN_WARP = 12;            // the warp that finishes the previous row
 constexpr int RSMEM_BYTES = ROFF_MBAR + 16;
 
 // L2 residency hints: the part of a row that is re-read from L2 in every pass is marked
@@ -312,15 +314,128 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
   uint32_t phase = 0;
   bool dead = false;
   int rb = 0;
-  // A row that needs no draw leaves its outputs to be written while the next row's sums are gathered
-  // (its broadcast buffer stays intact for one more row); the last one is written after the loop.
+  // Pass "final" ends without a barrier.  What is left of a row after it (the total variation, the
+  // one-hot entry of the gradient, the residual draw, the outputs) is done one row later by warp
+  // FIN_WARP while thread 0 does the next row's scalars: the row's broadcast buffer, the per-warp sums
+  // of its last pass and the step weights of the draw stay intact until then.  The last row of the
+  // CTA is finished after the loop.  `pb`: the row's buffer parity; all 32 lanes call.
   int64_t pending_row = -1;
-  auto write_pending = [&](int64_t row, const double* bcp) {
-    const __nv_bfloat16 *s, *t;
-    row_ptrs(row, s, t);
-    const int64_t b = (int64_t)((uint32_t)row / (uint32_t)P.K1);
-    const int xp = P.spec ? P.proposal[b * P.prop_ld + (row - b * P.K1)] : P.proposal[row];
-    write_result(bcp, P.out, !P.spec, row, 0, xp, false, K.c64, s, t);
+  auto finish_row = [&](int64_t prow, int pb) {
+    const double* bcp = (const double*)(smem + ROFF_BC) + pb * BC_DOUBLES;
+    const double* fin = (const double*)(smem + ROFF_FIN) + pb * 2 * RW;
+    const __nv_bfloat16 *ps, *pt;
+    row_ptrs(prow, ps, pt);
+    const int64_t pseq = P.K1 == 1 ? prow : (int64_t)((uint32_t)prow / (uint32_t)P.K1);
+    const int ppos = (int)(prow - pseq * P.K1);
+    const bool pbonus = P.spec && (ppos == P.K1 - 1);
+    const int xp = pbonus ? 0 : (P.spec ? P.proposal[pseq * P.prop_ld + ppos] : P.proposal[prow]);
+    const double tv_sum = warp_sum_d(lane < RW ? fin[lane] : 0.0);
+    const double tv = (bcp[BC_LAMBDA] > 0.0) ? tv_sum : 0.0;
+    const float k0p = (float)bcp[BC_K0];
+    const int tok = (int)bcp[BC_TOK];
+    if (lane == 0 && P.dlogits && tok >= 0) {   // the supervised token: gradient KG * (p - 1), over the entry its chunk's owner stored
+      const float ipf = (float)bcp[BC_IP];
+      const float kgf = (float)(bcp[BC_KG] * (double)ipf);
+      const float s_tok = (float)(tok == xp ? bcp[BC_SX] : bcp[BC_SV]);
+      const float ep = ex2f(fmaf(s_tok, c32, k0p));
+      ((__nv_bfloat16*)P.dlogits + prow * P.ld_g)[tok] = __float2bfloat16_rn(fmaf(ep, kgf, -(float)bcp[BC_KG]));
+    }
+    if (!(pbonus || bcp[BC_CORR] != 0.0)) {
+      if (lane == 0) write_result_tv(bcp, P.out, !P.spec, prow, 0, xp, false, K.c64, ps, pt, tv);
+      return;
+    }
+    // ---- the draw (corrected and bonus rows): the warp that owns the inverse-CDF target, by an
+    // ordered scan of the per-warp weights
+    const double mine_w = lane < RW ? fin[RW + lane] : 0.0;
+    double inc_w = mine_w;
+#pragma unroll
+    for (int o = 1; o < RW; o <<= 1) {
+      const double up = __shfl_up_sync(0xffffffffu, inc_w, o);
+      if (lane >= o) inc_w += up;
+    }
+    const double target = bcp[BC_UDRAW] * __shfl_sync(0xffffffffu, inc_w, RW - 1);
+    const unsigned cross = __ballot_sync(0xffffffffu, lane < RW && inc_w > target);
+    const unsigned posw = __ballot_sync(0xffffffffu, mine_w > 0.0);
+    int owner;
+    double running = 0.0;
+    bool last_mode = false;
+    if (cross) {
+      owner = __ffs(cross) - 1;
+      running = __shfl_sync(0xffffffffu, inc_w - mine_w, owner);
+    } else {       // rounding left no crossing: the last warp with positive weight, its last position
+      owner = posw ? 31 - __clz(posw) : 0;
+      last_mode = true;
+    }
+    Seg so;          // the owner's segment
+    so.c0 = min(n_chunks, owner * cpw);
+    so.c1 = min(n_chunks, so.c0 + cpw);
+    so.steps = (so.c1 - so.c0 + 31) / 32;
+    const float* step_w = (const float*)(smem + ROFF_STEP) + owner * MAX_STEPS;
+    const int ns = min(so.steps, MAX_STEPS);
+    // the step that holds the target (every lane walks the same few numbers)
+    int ks = -1, kpos = -1;
+#pragma unroll 1
+    for (int k = 0; k < ns; ++k) {
+      const double w = (double)step_w[k];
+      if (w > 0.0) kpos = k;
+      if (!last_mode && running + w > target) { ks = k; break; }
+      running += w;
+    }
+    if (ks < 0) { last_mode = true; ks = max(kpos, 0); }   // rounding: last step with positive weight
+    const int c = so.c0 + ks * 32 + lane;
+    const bool valid = c < so.c1;
+    uint4 s4 = make_uint4(FILLER, FILLER, FILLER, FILLER), t4 = s4;
+    if (valid) { s4 = ld_l2(ps + (size_t)c * 8, pol_last); t4 = ld_l2(pt + (size_t)c * 8, pol_last); }
+    const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
+    const float clp = (float)bcp[BC_CL], kqp = (float)bcp[BC_KQ];
+    const float rhop = (float)bcp[BC_IP] / (float)bcp[BC_IQ];     // as in pass "final": weights in units of iq
+    float w[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 sf = unpack_bf16x2(sw[i]), tf = unpack_bf16x2(tw[i]);
+      const float2 d = ffma2(sf, splat(-1.f), tf);
+      const float2 ep = ex2f2(ffma2(sf, splat(c32), splat(k0p)));
+      const float2 eq = ex2f2(ffma2(d, splat(clp), ffma2(sf, splat(c32), splat(kqp))));
+      w[2 * i] = pbonus ? eq.x : fmaxf(fmaf(ep.x, -rhop, eq.x), 0.f);
+      w[2 * i + 1] = pbonus ? eq.y : fmaxf(fmaf(ep.y, -rhop, eq.y), 0.f);
+    }
+    double mine = 0.0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) mine += (double)w[i];
+    double inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const double up = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += up;
+    }
+    const unsigned posm = __ballot_sync(0xffffffffu, mine > 0.0);
+    const unsigned hit = last_mode ? 0u : __ballot_sync(0xffffffffu, running + inc > target);
+    int y = -1;
+    if (hit) {
+      int found = -1;
+      if (lane == __ffs(hit) - 1) {                   // walk the 8 elements of the crossing chunk
+        double run = running + inc - mine;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          run += (double)w[i];
+          if (found < 0 && run > target) found = c * 8 + i;
+        }
+        if (found < 0) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) if (w[i] > 0.f) found = c * 8 + i;
+        }
+      }
+      y = __shfl_sync(0xffffffffu, found, __ffs(hit) - 1);
+    } else if (posm) {                                // rounding: last positive element of the step
+      int lastp = -1;
+      if (lane == 31 - __clz(posm)) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) if (w[i] > 0.f) lastp = c * 8 + i;
+      }
+      y = __shfl_sync(0xffffffffu, lastp, 31 - __clz(posm));
+    }
+    if (y < 0) y = min(V - 1, max(so.c0 * 8, so.c1 * 8 - 1));
+    if (lane == 0) write_result_tv(bcp, P.out, !P.spec, prow, pbonus ? 0 : 1, y, pbonus, K.c64, ps, pt, tv);
   };
 
   for (int64_t row = blockIdx.x; row < P.n_rows; row += gridDim.x, rb ^= 1) {
@@ -458,8 +573,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           }
         }
       } else if (lane == 0) {
-        // meanwhile, on warps that would only wait: the row scalars that do not depend on the passes,
-        // and the previous row's outputs
+        // meanwhile, on warps that would only wait: the row scalars that do not depend on the passes
         if (warp == 8) bc[BC_UACC] = scalar_uniform(P.seed, rid, STAGE_ACCEPT);
         if (warp == 9) bc[BC_UDRAW] = scalar_uniform(P.seed, rid, bonus ? STAGE_BONUS : STAGE_RESIDUAL);
         if (warp == 10) {
@@ -467,13 +581,13 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           bc[BC_SX] = ok ? (double)__bfloat162float(g_s[x]) : 0.0;
           bc[BC_TX] = ok ? (double)__bfloat162float(g_t[x]) : 0.0;
         }
-        if (warp == 11 && pending_row >= 0) write_pending(pending_row, (const double*)(smem + ROFF_BC) + (rb ^ 1) * BC_DOUBLES);
       }
-      pending_row = -1;
       if (any_dead) dead = true;
       __syncthreads();
       RTS(4);
-      if (tid == 12 * 32) {   // meanwhile: the student's logit at the teacher's argmax (the supervised token of a corrected row)
+      if (warp == FIN_WARP && pending_row >= 0) finish_row(pending_row, rb ^ 1);   // meanwhile: the previous row's draw and outputs
+      pending_row = -1;
+      if (tid == 13 * 32) {   // and the student's logit at the teacher's argmax (the supervised token of a corrected row)
         const int vs = (gat[6] >= 0.0 && gat[6] < (double)V) ? (int)gat[6] : 0;
         bc[BC_SV] = (double)__bfloat162float(g_s[vs]);
       }
@@ -560,18 +674,13 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
     // ------------------------------------------------ pass "final"
     RTS(10);
     const bool need_draw = bonus || bc[BC_CORR] != 0.0;
-    int d_owner = -1;                    // the draw: owning warp, weight before it, target, "take the last position"
-    double d_before = 0.0, d_target = 0.0;
-    bool d_last = false;
     const float cl = (float)bc[BC_CL], kq = (float)bc[BC_KQ];
     const float iq = (float)bc[BC_IQ], ip = (float)bc[BC_IP];
-    const int tok = (int)bc[BC_TOK];
-    const float KGf = (float)bc[BC_KG];
     const float kg = (float)(bc[BC_KG] * (double)ip);     // gradient entry = e_p * kg
     const float rho = ip / iq;                            // q_i - p_i = iq * (e_q - rho * e_p)
     {
       const bool want_g = (g_out != nullptr);
-      float2 Sq = splat(0.f), R = splat(0.f);
+      float2 R = splat(0.f);
       const float2 cc = splat(c32), cll = splat(cl), kqq = splat(kq), kk0 = splat(k0), neg1 = splat(-1.f);
       const float2 nrho = splat(-rho), kgg = splat(kg);
       float* step_w = (float*)(smem + ROFF_STEP) + warp * MAX_STEPS;   // draw weight of each of this warp's steps
@@ -592,7 +701,6 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           const float2 gv = fmul2(ep, kgg);
           gp[i] = pack_bf16x2(gv.x, gv.y);
         }
-        Sq = fadd2(Sq, sqc);
         R = fadd2(R, rc);
         if (need_draw) {   // ordered bookkeeping for the inverse-CDF draw: the weight of this step of the warp
           float wsum = bonus ? (sqc.x + sqc.y) : (rc.x + rc.y);   // in units of iq, like every draw weight
@@ -611,129 +719,21 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
         }
       });
       RTS(11);
-      const float sq_f = Sq.x + Sq.y, r_f = R.x + R.y;
-      double part = 0.0;                               // this warp's draw weight: its step weights, in order
+      // no barrier: each warp leaves its share of the total variation and its draw weight (its step
+      // weights, in order) for finish_row
+      double part = 0.0;
       if (need_draw) {
         __syncwarp();
         const int ns = min(sg.steps, MAX_STEPS);
         static_assert(MAX_STEPS <= 64, "two step weights per lane");
         part = warp_sum_d((lane < ns ? (double)step_w[lane] : 0.0) + (lane + 32 < ns ? (double)step_w[lane + 32] : 0.0));
       }
-      const double v0 = warp_sum_d((double)sq_f), v1 = warp_sum_d((double)r_f * (double)iq);
-      if (lane == 0) { red[warp] = v0; red[RW + warp] = v1; red[2 * RW + warp] = part; }   // part: ordered per-warp weights of the draw
-      __syncthreads();
-      if (warp < 2) {
-        const double a = warp_sum_d(lane < RW ? red[warp * RW + lane] : 0.0);
-        if (lane == 0) gat[warp] = a;
+      const double v1 = warp_sum_d((double)(R.x + R.y) * (double)iq);
+      if (lane == 0) {
+        double* fin = (double*)(smem + ROFF_FIN) + rb * 2 * RW;
+        fin[warp] = v1; fin[RW + warp] = part;
       }
-      if (need_draw) {
-        // every warp finds the warp that owns the inverse-CDF target (ordered scan of the per-warp weights)
-        const double mine = lane < RW ? red[2 * RW + lane] : 0.0;
-        double inc = mine;
-#pragma unroll
-        for (int o = 1; o < RW; o <<= 1) {
-          const double up = __shfl_up_sync(0xffffffffu, inc, o);
-          if (lane >= o) inc += up;
-        }
-        d_target = bc[BC_UDRAW] * __shfl_sync(0xffffffffu, inc, RW - 1);
-        const unsigned cross = __ballot_sync(0xffffffffu, lane < RW && inc > d_target);
-        const unsigned posw = __ballot_sync(0xffffffffu, mine > 0.0);
-        if (cross) {
-          d_owner = __ffs(cross) - 1;
-          d_before = __shfl_sync(0xffffffffu, inc - mine, d_owner);
-        } else {       // rounding left no crossing: the last warp with positive weight, its last position
-          d_owner = posw ? 31 - __clz(posw) : 0;
-          d_before = 0.0;
-          d_last = true;
-        }
-      }
-      __syncthreads();
-      RTS(12);
-      if (tid == 0) {
-        bc[BC_TV] = (bc[BC_LAMBDA] > 0.0) ? gat[1] : 0.0;
-        if (want_g && tok >= 0) {   // the supervised token: gradient KG * (p - 1), over the entry its chunk's owner stored
-          const float s_tok = (float)(tok == x ? bc[BC_SX] : bc[BC_SV]);
-          const float ep = ex2f(fmaf(s_tok, c32, k0));
-          g_out[tok] = __float2bfloat16_rn(fmaf(ep, kg, -KGf));
-        }
-      }
-      if (!need_draw) pending_row = row;
-    }
-
-    // ------------------------------------------------ the draw (corrected and bonus rows only)
-    if (need_draw) {
-      if (warp == d_owner) {
-        const double target = d_target;
-        bool last_mode = d_last;
-        double running = d_before;
-        const float* step_w = (const float*)(smem + ROFF_STEP) + warp * MAX_STEPS;
-        const int ns = min(sg.steps, MAX_STEPS);
-        // the step that holds the target (every lane walks the same few numbers)
-        int ks = -1, kpos = -1;
-#pragma unroll 1
-        for (int k = 0; k < ns; ++k) {
-          const double w = (double)step_w[k];
-          if (w > 0.0) kpos = k;
-          if (!last_mode && running + w > target) { ks = k; break; }
-          running += w;
-        }
-        if (ks < 0) { last_mode = true; ks = max(kpos, 0); }   // rounding: last step with positive weight
-        const int c = sg.c0 + ks * 32 + lane;
-        const bool valid = c < sg.c1;
-        uint4 s4 = make_uint4(0xFF7FFF7Fu, 0xFF7FFF7Fu, 0xFF7FFF7Fu, 0xFF7FFF7Fu), t4 = s4;
-        // from global memory: the warp's resident area may already be receiving the next row
-        if (valid) { s4 = ld_l2(g_s + (size_t)c * 8, pol_last); t4 = ld_l2(g_t + (size_t)c * 8, pol_last); }
-        const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
-        float w[8];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float2 sf = unpack_bf16x2(sw[i]), tf = unpack_bf16x2(tw[i]);
-          const float2 d = ffma2(sf, splat(-1.f), tf);
-          const float2 ep = ex2f2(ffma2(sf, splat(c32), splat(k0)));
-          const float2 eq = ex2f2(ffma2(d, splat(cl), ffma2(sf, splat(c32), splat(kq))));
-          w[2 * i] = bonus ? eq.x : fmaxf(fmaf(ep.x, -rho, eq.x), 0.f);
-          w[2 * i + 1] = bonus ? eq.y : fmaxf(fmaf(ep.y, -rho, eq.y), 0.f);
-        }
-        double mine = 0.0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) mine += (double)w[i];
-        double inc = mine;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const double up = __shfl_up_sync(0xffffffffu, inc, o);
-          if (lane >= o) inc += up;
-        }
-        const unsigned posm = __ballot_sync(0xffffffffu, mine > 0.0);
-        const unsigned hit = last_mode ? 0u : __ballot_sync(0xffffffffu, running + inc > target);
-        int y = -1;
-        if (hit) {
-          int found = -1;
-          if (lane == __ffs(hit) - 1) {                   // walk the 8 elements of the crossing chunk
-            double run = running + inc - mine;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              run += (double)w[i];
-              if (found < 0 && run > target) found = c * 8 + i;
-            }
-            if (found < 0) {
-#pragma unroll
-              for (int i = 0; i < 8; ++i) if (w[i] > 0.f) found = c * 8 + i;
-            }
-          }
-          y = __shfl_sync(0xffffffffu, found, __ffs(hit) - 1);
-        } else if (posm) {                                // rounding: last positive element of the step
-          int lastp = -1;
-          if (lane == 31 - __clz(posm)) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) if (w[i] > 0.f) lastp = c * 8 + i;
-          }
-          y = __shfl_sync(0xffffffffu, lastp, 31 - __clz(posm));
-        }
-        if (y < 0) y = min(V - 1, max(sg.c0 * 8, sg.c1 * 8 - 1));
-        if (lane == 0)
-          write_result_tv(bc, P.out, !P.spec, row, bonus ? 0 : 1, y, bonus, K.c64, g_s, g_t,
-                          (bc[BC_LAMBDA] > 0.0) ? gat[1] : 0.0);
-      }
+      pending_row = row;
     }
     RTS(13);
     // no barrier here: the next row uses the other broadcast buffer, and every other shared area is
@@ -752,7 +752,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
 #endif
   cp_async_wait<0>();
   __syncthreads();
-  if (tid == 11 * 32 && pending_row >= 0) write_pending(pending_row, (const double*)(smem + ROFF_BC) + (rb ^ 1) * BC_DOUBLES);
+  if (warp == FIN_WARP && pending_row >= 0) finish_row(pending_row, rb ^ 1);
   // a CTA that gave up on a copy still waits (bounded) for what it has in flight before leaving
   if (dead && tid == 0) (void)mbar_wait_bounded(mbar, phase);
 }
