@@ -44,3 +44,39 @@ def test_struct_layouts_match_the_header():
                      ctypes.sizeof(binding.SakiSpecIn), ctypes.sizeof(binding.SakiSpecOut),
                      ctypes.sizeof(binding.SakiMetaIn), ctypes.sizeof(binding.SakiMetaOut),
                      ctypes.sizeof(binding.SakiSelectIn)]
+
+
+def test_argument_validation_returns_codes_before_any_device_work():
+    """Bad arguments are rejected, and empty batches accepted, on the host: these calls return before the
+    library touches a device, so they behave the same on a machine without a GPU."""
+    lib = binding.load_library()
+    C = ctypes
+    null = C.c_void_p(None)
+    assert lib.saki_route_fwd(None, None, null) == 1
+    si, so = binding.SakiIn(), binding.SakiOut()
+    si.N, si.V, si.dtype, si.eps, si.temperature = 4, 1, 1, 0.1, 1.0          # V < 2
+    assert lib.saki_route_fwd(C.byref(si), C.byref(so), null) == 1 and "V" in P.last_error()
+    si.V, si.eps = 128, float("nan")
+    assert lib.saki_route_fwd(C.byref(si), C.byref(so), null) == 1
+    si.eps, si.temperature = 0.1, 0.0
+    assert lib.saki_route_fwd(C.byref(si), C.byref(so), null) == 1
+    si.temperature, si.dtype = 1.0, 7
+    assert lib.saki_route_fwd(C.byref(si), C.byref(so), null) == 1
+    si.dtype, si.N, si.ld_s, si.ld_t = 1, 0, 128, 128                          # empty batch: a no-op
+    assert lib.saki_route_fwd(C.byref(si), C.byref(so), null) == 0
+    assert lib.saki_route_fwd_bwd(C.byref(si), C.byref(so), null, 128, 1.0, null) == 0
+    assert lib.saki_route_fwd_bwd(C.byref(si), C.byref(so), null, 64, 1.0, null) == 1      # ld_g < V
+    assert lib.saki_route_fwd_bwd_noalloc(C.byref(si), C.byref(so), null, 128, float("inf"), null) == 1
+    mi, mo = binding.SakiMetaIn(), binding.SakiMetaOut()
+    mi.N, mi.V, mi.dtype, mi.ld_s, mi.temperature = 0, 128, 1, 128, 1.0
+    assert lib.saki_route_bwd_from_meta(C.byref(mi), C.byref(mo), null, 128, 1.0, null) == 0
+    mi.temperature = -1.0
+    assert lib.saki_route_bwd_from_meta(C.byref(mi), C.byref(mo), null, 128, 1.0, null) == 1
+    sel = binding.SakiSelectIn()
+    sel.N, sel.B, sel.mode = 0, 0, 1
+    assert lib.saki_select_tm(C.byref(sel), null, null, null) == 0
+    sel.mode = 9
+    assert lib.saki_select_tm(C.byref(sel), null, null, null) == 1
+    sp, spo = binding.SakiSpecIn(), binding.SakiSpecOut()
+    sp.B, sp.K, sp.V, sp.dtype, sp.eps, sp.temperature = 2, 17, 128, 1, 0.1, 1.0           # K outside [1,16]
+    assert lib.saki_spec_verify(C.byref(sp), C.byref(spo), null) == 1
