@@ -166,6 +166,8 @@ def run_ours(args):
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
     torch.cuda.set_device(local)
+    if args.kernel:
+        P.set_kernel(args.kernel)
     dev = f"cuda:{local}"
     P.load_library()
 
@@ -283,7 +285,7 @@ def run_ours(args):
                 "peak_kind": f"of {peak_kind} (device-to-device copy, MEASURED_PEAKS.json)"
                 if peak_kind == "measured" else "of fallback",
                 "traffic": (TRAFFIC_BYTES_PER_POSITION * w.N) if TRAFFIC_BYTES_PER_POSITION else None,
-                "algorithmic_bytes_per_launch": bpp * w.N, "kernel": {3: "saki::rowsm_kernel", 2: "saki::cluster_kernel<8>"}.get(kernel_used, "saki::general_kernel"),
+                "algorithmic_bytes_per_launch": bpp * w.N, "kernel": {3: "saki::rowsm_kernel", 2: "saki::cluster_kernel"}.get(kernel_used, "saki::general_kernel"),
                 "kernel_ms": kern_ms,
                 "frac_of_nominal_8TBs": achieved / 8000.0}
 
@@ -325,6 +327,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg3")
     ap.add_argument("--rows", type=int, default=0, help="cut the workload to its first R rows (profiling)")
+    ap.add_argument("--kernel", type=int, default=0, choices=[0, 1, 2, 3],
+                    help="row kernel (saki_set_kernel): 0 automatic, 1 general, 2 cluster, 3 row-per-SM (profiling)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-next", action="store_true", help="skip the metadata-driven backward measurement")
