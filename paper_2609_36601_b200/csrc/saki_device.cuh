@@ -7,7 +7,7 @@
 
 namespace saki {
 
-constexpr int BC_DOUBLES = 40;             // doubles of one broadcast area
+constexpr int BC_DOUBLES = 48;             // doubles of one broadcast area
 constexpr double LN2 = 0.693147180559945309417232121458;
 constexpr double INV_LN2 = 1.44269504088896340735992468100;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // ~2 s: give up on a wait
@@ -18,7 +18,7 @@ enum { BC_MODE = 0, BC_BETA, BC_CB, BC_KB, BC_LO, BC_HI, BC_ITER,               
        BC_CL, BC_KQ, BC_IQ, BC_IP, BC_KG, BC_TOK, BC_STATUS, BC_CORR, BC_LAMBDA,    // final pass
        BC_GLAM, BC_G0, BC_G1, BC_ACC, BC_LPX, BC_LTX, BC_LOSS, BC_VSTAR, BC_KL, BC_TV,
        BC_OWNER_WARP, BC_BEFORE, BC_TARGET, BC_TAKE_LAST, BC_RSS,
-       BC_UACC, BC_UDRAW, BC_SX, BC_TX, BC_K0, BC_K1, BC_PMAX, BC_SV, BC_COUNT };
+       BC_UACC, BC_UDRAW, BC_SX, BC_TX, BC_K0, BC_K1, BC_PMAX, BC_SV, BC_P2, BC_P3, BC_P4, BC_COUNT };
 static_assert(BC_COUNT <= BC_DOUBLES, "broadcast area too small");
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -212,7 +212,8 @@ __device__ __forceinline__ void lse_of_sum(double S, double k, double& rS, doubl
 }
 static __device__ __noinline__ void scalar_after_lse_tail(double* bc, const double* v, Consts K, float k0f, float k1f, int x,
                                                    bool bonus, bool masked, bool row_timeout, float e_max,
-                                                   bool overflow_redo, double rSs, double rSt, double G0, double G1) {
+                                                   bool overflow_redo, double rSs, double rSt, double G0, double G1,
+                                                   const double* m4_raw = nullptr) {
   const double SsT = v[0], StT = v[1], eps = K.eps, k0 = (double)k0f, k1 = (double)k1f;
   uint32_t status = 0;
   const double chk = ((v[0] + v[1]) + (v[2] + v[3])) + (v[4] + v[5]);
@@ -240,15 +241,31 @@ static __device__ __noinline__ void scalar_after_lse_tail(double* bc, const doub
     decide(bc, K, 1.0, G1, G0, G1, k0, k1, rSs, status | SAKI_ROW_SATURATED, vstar, bonus, masked, x);
     return;
   }
-  // initial guess from KL(beta) ~ beta^2/2 Var_p(d) + beta^3/3 kappa3_p(d); float32 is plenty
+  // initial guess from KL(beta) ~ beta^2/2 Var_p(d) + beta^3/3 kappa3_p(d) (+ beta^4/8 kappa4_p(d) where the
+  // fourth moment is at hand); float32 is plenty
   const float rt = (float)rtau;
-  const float vd = fmaxf((float)(m2 - m1 * m1) * rt * rt, 1e-30f);
-  const float k3 = (float)(m3 - 3.0 * m1 * m2 + 2.0 * m1 * m1 * m1) * rt * rt * rt;
+  const double var_p = m2 - m1 * m1, k3_p = m3 - 3.0 * m1 * m2 + 2.0 * m1 * m1 * m1;
+  const float vd = fmaxf((float)var_p * rt * rt, 1e-30f);
+  const float k3 = (float)k3_p * rt * rt * rt;
+  double k4_p = 0.0;
+  if (m4_raw) {
+    const double m4 = *m4_raw * rSs, m1s = m1 * m1;
+    k4_p = m4 - 4.0 * m3 * m1 - 3.0 * m2 * m2 + 12.0 * m2 * m1s - 6.0 * m1s * m1s;
+  }
+  const float k4 = (float)k4_p * (rt * rt) * (rt * rt);
+  // second to fourth derivative of G at 0: they fix the slope b G2(b) of KL at the student's end, for
+  // the quadrature of scalar_after_solve4
+  const double rt2 = rtau * rtau;
+  // (the cumulants come from raw moments: where the mean of d dwarfs its spread they have lost their
+  // digits to cancellation, and a negative entry tells the quadrature to stand aside)
+  bc[BC_P2] = (m1 * m1 <= 100.0 * var_p) ? var_p * rt2 : -1.0;
+  bc[BC_P3] = k3_p * rt2 * rtau; bc[BC_P4] = k4_p * rt2 * rt2;
   const float e2 = 2.f * (float)eps;
   float b = sqrtf(__fdividef(e2, vd));
 #pragma unroll
   for (int it = 0; it < 3; ++it) {
-    const float den = vd + (2.f / 3.f) * fminf(b, 1.f) * k3;
+    const float bb = fminf(b, 1.f);
+    const float den = vd + (2.f / 3.f) * bb * k3 + 0.25f * bb * bb * k4;
     if (den > 0.25f * vd) b = sqrtf(__fdividef(e2, den));
   }
   if (!(b > 1e-7f)) b = 1e-7f;
@@ -342,8 +359,27 @@ static __device__ __noinline__ void scalar_after_solve4(double* bc, const double
   const double k4 = m4 - 4.0 * m3 * m1 - 3.0 * m2 * m2 + 12.0 * m2 * m1s - 6.0 * m1s * m1s;
   const double rt2 = rtau * rtau;
   const double G1 = m1 * rtau, G2 = var * rt2, G3 = k3 * rt2 * rtau, G4 = k4 * rt2 * rt2;
-  const double kl = beta * G1 - G + G0;                 // KL(q_beta || p)
   const double slope = beta * G2;                       // d KL / d beta
+  // KL(q_beta || p).  Directly, beta G1 - G + G(0) is a difference of O(1) numbers known to a few 1e-7
+  // x (largest probability) from float32 sums: good for radii of 1e-2 and more, useless for 1e-4.  But
+  // KL(beta) is also the integral of its slope f(b) = b G2(b) from 0, and f and its first two
+  // derivatives are known at both ends (cumulants of d under p from pass "lse", under q_beta from this
+  // evaluation; at 0 also the third), each to ~1e-6 RELATIVE: two-point Hermite quadrature.  The rule
+  // with three derivatives at 0 and two at beta (exact for degree 6) is taken for small radii when the
+  // symmetric rule with two derivatives at each end (exact for degree 5) agrees with it to 2e-6.
+  const double kl_direct = beta * G1 - G + G0;
+  double kl = kl_direct;
+  bool by_quadrature = false;
+  if (eps < 0.02 && bc[BC_P2] >= 0.0 && m1s <= 100.0 * var) {
+    const double f1 = slope, f1p = G2 + beta * G3, f1pp = 2.0 * G3 + beta * G4;
+    const double f0p = bc[BC_P2], f0pp = 2.0 * bc[BC_P3], f0ppp = 3.0 * bc[BC_P4];
+    const double h2 = beta * beta, h3 = h2 * beta;
+    const double i6 = 0.5 * beta * f1 + h2 * 0.1 * (f0p - f1p) + h3 * (1.0 / 120.0) * (f0pp + f1pp);
+    const double i7 = (3.0 / 7.0) * beta * f1 + h2 * ((1.0 / 7.0) * f0p - (1.0 / 14.0) * f1p) +
+                      h3 * ((2.0 / 105.0) * f0pp + (1.0 / 210.0) * f1pp) + h2 * h2 * (1.0 / 840.0) * f0ppp;
+    if (i7 > 0.0 && fabs(i7 - i6) <= 2e-6 * i7) { kl = i7; by_quadrature = true; }
+  }
+  const double Gq = by_quadrature ? beta * G1 + G0 - kl : G;   // log-partition consistent with the KL used
   if (kl <= eps) lo = fmax(lo, beta); else hi = fmin(hi, beta);
   const double c2 = 0.5 * (beta * G3 + G2), c3 = beta * G4 * (1.0 / 6.0) + G3 * (1.0 / 3.0), c4 = 0.125 * G4;
   double h;
@@ -371,14 +407,19 @@ static __device__ __noinline__ void scalar_after_solve4(double* bc, const double
   // The float32 sums resolve KL to a few 1e-7 x (largest probability).  Where that would move lambda by
   // more than the tolerance (a very flat KL: nearly one-hot rows), or the solve did not converge, the row
   // is handed to the float64 kernel.  (Radii below 5e-3 never reach this kernel: see the dispatcher.)
-  if (done && (3e-7 * bc[BC_PMAX] > 1e-5 * slope || iter >= 40)) { bc[BC_MODE] = MODE_REDO; return; }
+  // Below 5e-3 the direct value, where the quadrature was not taken, is held to a fifth of the tolerance
+  // and to the worst case of its error: 3e-7 absolute (a flat row, where ex2.approx errs the same way on
+  // every element).
+  const double kl_tol = (eps < 5e-3 ? 2e-6 : 1e-5) * slope;
+  const double kl_err = 3e-7 * (eps < 5e-3 ? 1.0 : bc[BC_PMAX]);
+  if (done && ((!by_quadrature && kl_err > kl_tol) || iter >= 40)) { bc[BC_MODE] = MODE_REDO; return; }
   if (done) {
     const float cl = (float)(K.c64 * nb);
     const double lam = (double)cl * K.rc64;
     const double dl = lam - beta;
     // the model's predictions at lambda
     bc[BC_KL] = kl + dl * (slope + dl * (c2 + dl * (c3 + dl * c4)));
-    const double Glam = G + dl * (G1 + dl * (0.5 * G2 + dl * ((1.0 / 6.0) * G3 + dl * (1.0 / 24.0) * G4)));
+    const double Glam = Gq + dl * (G1 + dl * (0.5 * G2 + dl * ((1.0 / 6.0) * G3 + dl * (1.0 / 24.0) * G4)));
     decide(bc, K, lam, Glam, G0, bc[BC_G1], (double)k0f, (double)k1f, bc[BC_RSS], (uint32_t)bc[BC_STATUS],
            (int)bc[BC_VSTAR], bonus, masked, x);
   } else {

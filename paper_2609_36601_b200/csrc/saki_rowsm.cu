@@ -41,8 +41,8 @@ constexpr int RW = RT / 32;             // warps per CTA
 constexpr int KS_MAX = 208 / RW;        // steps per warp that fit in shared memory (a step = 32 chunks of 8 elements = 1 KB of logit pairs)
 constexpr int MAX_STEPS = 64;            // steps per warp the draw bookkeeping can hold (V <= 64*32*8*RW)
 constexpr int RES_CHUNKS = KS_MAX * 32; // resident chunks per warp and row
-constexpr int RNV = 8;                  // doubles per partial vector
-static_assert(RW >= 14, "warps 8-13 do side work while warps 0-6 gather and thread 0 does the scalars");
+constexpr int RNV = 9;                  // doubles per partial vector
+static_assert(RW >= 14, "warps 8-13 do side work while warps 0-7 gather and thread 0 does the scalars");
 static_assert(KS_MAX - 4 >= 1, "every warp keeps at least its first step resident");
 
 constexpr int ROFF_S = 0;                                        // [RW][RES_CHUNKS] uint4
@@ -479,7 +479,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           ktw = -ceilf(c32 * fmaxf(mt0, -1e30f));
         }
       }
-      float2 Ss = splat(0.f), St = splat(0.f), M1 = splat(0.f), M2 = splat(0.f), M3 = splat(0.f), N1 = splat(0.f);
+      float2 Ss = splat(0.f), St = splat(0.f), M1 = splat(0.f), M2 = splat(0.f), M3 = splat(0.f), M4 = splat(0.f), N1 = splat(0.f);
       uint32_t run_s = FILLER;                   // packed running maxima of the student's even / odd elements
       float mt_run = -CUDART_INF_F;              // running maximum of the teacher, and the first chunk that reached it
       int arg_c = -1;
@@ -498,11 +498,12 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           const float2 et = ex2f2(ffma2(tf, cc, kk1));
           Ss = fadd2(Ss, es);
           St = fadd2(St, et);
-          const float2 t1 = fmul2(es, d);
-          M1 = fadd2(M1, t1);
-          const float2 t2 = fmul2(t1, d);
-          M2 = fadd2(M2, t2);
-          M3 = ffma2(t2, d, M3);
+          const float2 d2 = fmul2(d, d);
+          M1 = ffma2(es, d, M1);
+          const float2 u = fmul2(es, d2);
+          M2 = fadd2(M2, u);
+          M3 = ffma2(u, d, M3);
+          M4 = ffma2(u, d2, M4);
           N1 = ffma2(et, d, N1);
         }
       }, [] {});
@@ -522,32 +523,32 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       }
       const float kws = ksw, kwt = ktw;
       auto tot = [](const float2 a) { return (double)a.x + (double)a.y; };
-      double v[6] = {tot(Ss), tot(St), tot(M1), tot(M2), tot(M3), tot(N1)};
+      double v[7] = {tot(Ss), tot(St), tot(M1), tot(M2), tot(M3), tot(N1), tot(M4)};
 #pragma unroll
-      for (int k = 0; k < 6; ++k) v[k] = warp_sum_d(v[k]);
+      for (int k = 0; k < 7; ++k) v[k] = warp_sum_d(v[k]);
       if (lane == 0) {
 #pragma unroll
-        for (int k = 0; k < 6; ++k) red[k * RW + warp] = v[k];
-        red[6 * RW + warp] = (double)kws; red[7 * RW + warp] = (double)kwt;
+        for (int k = 0; k < 7; ++k) red[k * RW + warp] = v[k];
+        red[7 * RW + warp] = (double)kws; red[8 * RW + warp] = (double)kwt;
         float* wm = (float*)(smem + ROFF_WMAX);
         wm[warp] = wmt; ((int*)wm)[RW + warp] = warg; wm[2 * RW + warp] = wms;
       }
       const int any_dead = __syncthreads_or(dead ? 1 : 0);
       RTS(3);
-      if (warp < 7) {   // block level: warps 0-5 add up one sum each on the row's shifts, warp 6 finds the argmax
+      if (warp < 8) {   // block level: warps 0-6 add up one sum each on the row's shifts, warp 7 finds the argmax
         const int wl = lane < RW ? lane : 0;       // lanes beyond the warp count carry zero weight
         const float* wm = (const float*)(smem + ROFF_WMAX);
-        if (warp < 6) {
+        if (warp < 7) {
           // From here on the row's shifts are those of its true maxima (the largest term of each sum has
           // its exponent argument in (-1, 0], where float32 resolves it best); a warp's shift came from an
           // element of the row, so it is never below the row's, and the factor is an exact power of two <= 1.
           const bool teacher = (warp == 1 || warp == 5);
           const float mx = warp_max_f(lane < RW ? wm[teacher ? wl : 2 * RW + wl] : -CUDART_INF_F);
           const double kr = (double)-ceilf(c32 * fmaxf(mx, -1e30f));
-          const double kw = lane < RW ? red[(teacher ? 7 : 6) * RW + wl] : 1e30;
+          const double kw = lane < RW ? red[(teacher ? 8 : 7) * RW + wl] : 1e30;
           const double f = kw < 1e29 ? (double)pow2f_exact((float)(kr - kw)) : 0.0;
           const double a = warp_sum_d(f * red[warp * RW + wl]);
-          if (lane == 0) { gat[warp] = a; if (warp < 2) gat[7 + warp] = kr; }
+          if (lane == 0) { gat[warp < 6 ? warp : 9] = a; if (warp < 2) gat[7 + warp] = kr; }   // gat[9]: the fourth moment
         } else {
           float gmt = lane < RW ? wm[wl] : -CUDART_INF_F;
           int garg = ((const int*)wm)[RW + wl];
@@ -598,7 +599,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
         if (tid == 0) {
           bc[BC_K0] = gat[7]; bc[BC_K1] = gat[8];
           scalar_after_lse_tail(bc, gat, K, (float)gat[7], (float)gat[8], x, bonus, masked, any_dead != 0, 1.f, true,
-                                rS, rSt, G, G1);
+                                rS, rSt, G, G1, gat + 9);
         }
       }
       RTS(5);
