@@ -129,10 +129,10 @@ static int dispatch_rows(RowParams p, int dtype, cudaStream_t st, int32_t* scrat
   bool served = false;
   const int which = g_kernel.load();
   int used = 1;
-  // The float32 kernels resolve KL(q||p) to a few 1e-7 absolute: enough for |d lambda| <= 1e-5 when
-  // eps >= 5e-3 (measured), not below.  Smaller positive radii run on the float64 kernel.
-  // The row-per-SM kernel gets KL for small radii from a quadrature of its slope instead (relative, not
-  // absolute, accuracy) and takes every radius.
+  // Directly, float32 sums resolve KL(q||p) to a few 1e-7 absolute: enough for |d lambda| <= 1e-5 when
+  // eps >= 5e-3 (measured), not below: for the cluster kernel smaller positive radii run on the float64
+  // kernel.  The row-per-SM kernel gets KL for small radii from a quadrature of its slope instead
+  // (relative, not absolute, accuracy) and takes every radius.
   const bool eps_ok = !(p.eps > 0.f) || p.eps >= 5e-3f;
   const bool rowsm_ok = (which == 0 || which == 3) && rowsm_can_serve(p, dtype);
   const bool fast = (which != 1) && (rowsm_ok || (eps_ok && cluster_can_serve(p, dtype)));

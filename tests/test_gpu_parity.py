@@ -281,6 +281,25 @@ def test_wide_range_rows(gap):
         P.set_kernel(prev)
 
 
+@pytest.mark.parametrize("eps", [1e-6, 1e-4, 2e-3, 4.9e-3, 0.015])
+def test_small_radii_on_the_row_per_sm_kernel(eps):
+    """Radii of the paper's late schedule (eps -> 0): the row-per-SM kernel forms KL by quadrature of its
+    slope there, which keeps lambda accurate relatively, not just absolutely."""
+    prev = P.set_kernel(3)
+    try:
+        w = synth.Workload("t", 400, 32000, "bf16", eps, 1.0, True, 1002, 2)
+        d = synth.generate(w, DEV)
+        rows = range(0, 400, 9)
+        out, ref, _, _ = _check_fwd_bwd(d, w, rows=rows, row_offset=5)
+        assert P.last_kernel() == 3
+        assert P.redo_count() <= 20
+        lam = out["lambda"].cpu().numpy()[list(rows)].astype(np.float64)
+        # below 5e-3 every row is settled by the quadrature or by the float64 kernel
+        assert np.max(np.abs(lam - ref["lam"])) <= (5e-7 if eps < 5e-3 else 1e-5)
+    finally:
+        P.set_kernel(prev)
+
+
 def test_calls_on_two_streams_do_not_share_scratch():
     """The row list of the two-tier routing is kept per stream: two calls whose kernels may overlap on
     the GPU give what each gives alone."""
