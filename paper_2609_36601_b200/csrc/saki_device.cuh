@@ -7,7 +7,7 @@
 
 namespace saki {
 
-constexpr int BC_DOUBLES = 48;             // doubles of one broadcast area
+constexpr int BC_DOUBLES = 56;             // doubles of one broadcast area
 constexpr double LN2 = 0.693147180559945309417232121458;
 constexpr double INV_LN2 = 1.44269504088896340735992468100;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // ~2 s: give up on a wait
@@ -18,7 +18,9 @@ enum { BC_MODE = 0, BC_BETA, BC_CB, BC_KB, BC_LO, BC_HI, BC_ITER,               
        BC_CL, BC_KQ, BC_IQ, BC_IP, BC_KG, BC_TOK, BC_STATUS, BC_CORR, BC_LAMBDA,    // final pass
        BC_GLAM, BC_G0, BC_G1, BC_ACC, BC_LPX, BC_LTX, BC_LOSS, BC_VSTAR, BC_KL, BC_TV,
        BC_OWNER_WARP, BC_BEFORE, BC_TARGET, BC_TAKE_LAST, BC_RSS,
-       BC_UACC, BC_UDRAW, BC_SX, BC_TX, BC_K0, BC_K1, BC_PMAX, BC_SV, BC_P2, BC_P3, BC_P4, BC_COUNT };
+       BC_UACC, BC_UDRAW, BC_SX, BC_TX, BC_K0, BC_K1, BC_PMAX, BC_SV, BC_P2, BC_P3, BC_P4,
+       BC_QSTATE, BC_E_BETA, BC_E_G, BC_E_G1, BC_E_G2, BC_E_G3, BC_E_G4, BC_E_I7,   // an evaluation waiting for its midpoint
+       BC_COUNT };
 static_assert(BC_COUNT <= BC_DOUBLES, "broadcast area too small");
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -275,7 +277,7 @@ static __device__ __noinline__ void scalar_after_lse_tail(double* bc, const doub
   bc[BC_STATUS] = (double)status;
   bc[BC_BETA] = be; bc[BC_CB] = (double)cb;
   bc[BC_KB] = (double)(float)((1.0 - be) * k0 + be * k1);
-  bc[BC_LO] = 0.0; bc[BC_HI] = 1.0; bc[BC_ITER] = 0.0;
+  bc[BC_LO] = 0.0; bc[BC_HI] = 1.0; bc[BC_ITER] = 0.0; bc[BC_QSTATE] = 0.0;
   bc[BC_MODE] = MODE_SOLVE;
 }
 
@@ -314,7 +316,7 @@ static __device__ __noinline__ void scalar_after_solve(double* bc, const double*
   const bool done = (!bisected && fabs(nb - beta) <= 2e-4 * beta) || iter >= 40 || (hi - lo) < 1e-9;
   // The float32 sums resolve KL to a few 1e-7 x (largest probability).  Where that would move lambda by
   // more than the tolerance (a very flat KL: nearly one-hot rows), or the solve did not converge, the row
-  // is handed to the float64 kernel.  (Radii below 5e-3 never reach this kernel: see the dispatcher.)
+  // is handed to the float64 kernel.
   if (done && (3e-7 * bc[BC_PMAX] > 1e-5 * slope || iter >= 40)) { bc[BC_MODE] = MODE_REDO; return; }
   if (done) {
     const float cl = (float)(K.c64 * nb);
@@ -346,39 +348,80 @@ static __device__ __noinline__ void scalar_after_solve(double* bc, const double*
 static __device__ __noinline__ void scalar_after_solve4(double* bc, const double* v, Consts K, float k0f, float k1f, int x,
                                                  bool bonus, bool masked) {
   const double eps = K.eps, rtau = K.rtau;
-  const double beta = bc[BC_BETA], G0 = bc[BC_G0], kb = bc[BC_KB];
+  const double G0 = bc[BC_G0], kb = bc[BC_KB];
   double lo = bc[BC_LO], hi = bc[BC_HI];
   const int iter = (int)bc[BC_ITER] + 1;
   if (!(fabs((v[0] + v[1]) + (v[2] + v[3]) + v[4]) < CUDART_INF)) { bc[BC_MODE] = MODE_REDO; return; }   // float32 sums overflowed
-  const double r0 = rcp_fast(v[0]);
-  const double G = LN2 * (log2_fast(v[0]) - kb);
-  const double m1 = v[1] * r0, m2 = v[2] * r0, m3 = v[3] * r0, m4 = v[4] * r0;   // raw moments of d under q_beta
-  const double m1s = m1 * m1;
-  const double var = fmax(m2 - m1s, 0.0);
-  const double k3 = m3 - 3.0 * m2 * m1 + 2.0 * m1s * m1;
-  const double k4 = m4 - 4.0 * m3 * m1 - 3.0 * m2 * m2 + 12.0 * m2 * m1s - 6.0 * m1s * m1s;
-  const double rt2 = rtau * rtau;
-  const double G1 = m1 * rtau, G2 = var * rt2, G3 = k3 * rt2 * rtau, G4 = k4 * rt2 * rt2;
-  const double slope = beta * G2;                       // d KL / d beta
+  // this evaluation: log-partition and cumulants of d under q at bc[BC_BETA]
+  double beta = bc[BC_BETA], G, G1, G2, G3, G4;
+  bool well_conditioned;
+  {
+    const double r0 = rcp_fast(v[0]);
+    G = LN2 * (log2_fast(v[0]) - kb);
+    const double m1 = v[1] * r0, m2 = v[2] * r0, m3 = v[3] * r0, m4 = v[4] * r0;   // raw moments of d under q_beta
+    const double m1s = m1 * m1;
+    const double var = fmax(m2 - m1s, 0.0);
+    const double k3 = m3 - 3.0 * m2 * m1 + 2.0 * m1s * m1;
+    const double k4 = m4 - 4.0 * m3 * m1 - 3.0 * m2 * m2 + 12.0 * m2 * m1s - 6.0 * m1s * m1s;
+    const double rt2 = rtau * rtau;
+    G1 = m1 * rtau; G2 = var * rt2; G3 = k3 * rt2 * rtau; G4 = k4 * rt2 * rt2;
+    well_conditioned = m1s <= 100.0 * var;      // else the cumulants have lost their digits to cancellation
+  }
   // KL(q_beta || p).  Directly, beta G1 - G + G(0) is a difference of O(1) numbers known to a few 1e-7
   // x (largest probability) from float32 sums: good for radii of 1e-2 and more, useless for 1e-4.  But
   // KL(beta) is also the integral of its slope f(b) = b G2(b) from 0, and f and its first two
   // derivatives are known at both ends (cumulants of d under p from pass "lse", under q_beta from this
   // evaluation; at 0 also the third), each to ~1e-6 RELATIVE: two-point Hermite quadrature.  The rule
   // with three derivatives at 0 and two at beta (exact for degree 6) is taken for small radii when the
-  // symmetric rule with two derivatives at each end (exact for degree 5) agrees with it to 2e-6.
-  const double kl_direct = beta * G1 - G + G0;
-  double kl = kl_direct;
+  // symmetric rule with two derivatives at each end (exact for degree 5) agrees with it to 2e-6.  Where
+  // it does not (heavy tails of d: the integrand is no polynomial of that degree over [0, beta]) and
+  // the direct value cannot do either, one more evaluation at beta/2 splits the integral in two panels.
+  double kl;
   bool by_quadrature = false;
-  if (eps < 0.02 && bc[BC_P2] >= 0.0 && m1s <= 100.0 * var) {
-    const double f1 = slope, f1p = G2 + beta * G3, f1pp = 2.0 * G3 + beta * G4;
-    const double f0p = bc[BC_P2], f0pp = 2.0 * bc[BC_P3], f0ppp = 3.0 * bc[BC_P4];
-    const double h2 = beta * beta, h3 = h2 * beta;
-    const double i6 = 0.5 * beta * f1 + h2 * 0.1 * (f0p - f1p) + h3 * (1.0 / 120.0) * (f0pp + f1pp);
-    const double i7 = (3.0 / 7.0) * beta * f1 + h2 * ((1.0 / 7.0) * f0p - (1.0 / 14.0) * f1p) +
-                      h3 * ((2.0 / 105.0) * f0pp + (1.0 / 210.0) * f1pp) + h2 * h2 * (1.0 / 840.0) * f0ppp;
-    if (i7 > 0.0 && fabs(i7 - i6) <= 2e-6 * i7) { kl = i7; by_quadrature = true; }
+  const bool quad_ok = eps < 0.02 && bc[BC_P2] >= 0.0;
+  const double f0p = bc[BC_P2], f0pp = 2.0 * bc[BC_P3], f0ppp = 3.0 * bc[BC_P4];
+  auto rule7 = [&](double b, double g2, double g3, double g4) {   // integral over [0, b], three derivatives known at 0
+    const double f1 = b * g2, f1p = g2 + b * g3, f1pp = 2.0 * g3 + b * g4, h2 = b * b;
+    return (3.0 / 7.0) * b * f1 + h2 * ((1.0 / 7.0) * f0p - (1.0 / 14.0) * f1p) +
+           h2 * b * ((2.0 / 105.0) * f0pp + (1.0 / 210.0) * f1pp) + h2 * h2 * (1.0 / 840.0) * f0ppp;
+  };
+  if ((int)bc[BC_QSTATE] == 1) {
+    // this was the midpoint: panel [0, m] by the rule above, panel [m, beta] by the symmetric rule
+    const double m = beta, mG2 = G2, mG3 = G3, mG4 = G4;
+    const bool m_ok = well_conditioned;
+    beta = bc[BC_E_BETA]; G = bc[BC_E_G]; G1 = bc[BC_E_G1]; G2 = bc[BC_E_G2]; G3 = bc[BC_E_G3]; G4 = bc[BC_E_G4];
+    bc[BC_QSTATE] = 0.0;
+    const double fa = m * mG2, fap = mG2 + m * mG3, fapp = 2.0 * mG3 + m * mG4;
+    const double fb = beta * G2, fbp = G2 + beta * G3, fbpp = 2.0 * G3 + beta * G4;
+    const double h = beta - m;
+    const double two = rule7(m, mG2, mG3, mG4) + 0.5 * h * (fa + fb) + h * h * 0.1 * (fap - fbp) +
+                       h * h * h * (1.0 / 120.0) * (fapp + fbpp);
+    kl = beta * G1 - G + G0;
+    // one panel was off by about |two - one|; two panels are closer by the seventh power of two or so
+    if (m_ok && two > 0.0 && fabs(two - bc[BC_E_I7]) <= 1e-4 * two) { kl = two; by_quadrature = true; }
+  } else {
+    kl = beta * G1 - G + G0;
+    if (quad_ok && well_conditioned) {
+      const double f1 = beta * G2, f1p = G2 + beta * G3, f1pp = 2.0 * G3 + beta * G4;
+      const double h2 = beta * beta;
+      const double i6 = 0.5 * beta * f1 + h2 * 0.1 * (f0p - f1p) + h2 * beta * (1.0 / 120.0) * (f0pp + f1pp);
+      const double i7 = rule7(beta, G2, G3, G4);
+      if (i7 > 0.0 && fabs(i7 - i6) <= 2e-6 * i7) { kl = i7; by_quadrature = true; }
+      else if (i7 > 0.0 && 3e-7 * (eps < 5e-3 ? 1.0 : bc[BC_PMAX]) > (eps < 5e-3 ? 2e-6 : 1e-5) * beta * G2 && iter < 38) {
+        // neither form will do (see the second-tier test below): evaluate at beta/2 first
+        bc[BC_QSTATE] = 1.0;
+        bc[BC_E_BETA] = beta; bc[BC_E_G] = G; bc[BC_E_G1] = G1; bc[BC_E_G2] = G2; bc[BC_E_G3] = G3; bc[BC_E_G4] = G4;
+        bc[BC_E_I7] = i7;
+        const float cbm = (float)(K.c64 * 0.5 * beta);
+        const double bm = (double)cbm * K.rc64;
+        bc[BC_BETA] = bm; bc[BC_CB] = (double)cbm;
+        bc[BC_KB] = (double)(float)((1.0 - bm) * (double)k0f + bm * (double)k1f);
+        bc[BC_ITER] = (double)iter;
+        return;
+      }
+    }
   }
+  const double slope = beta * G2;                       // d KL / d beta
   const double Gq = by_quadrature ? beta * G1 + G0 - kl : G;   // log-partition consistent with the KL used
   if (kl <= eps) lo = fmax(lo, beta); else hi = fmin(hi, beta);
   const double c2 = 0.5 * (beta * G3 + G2), c3 = beta * G4 * (1.0 / 6.0) + G3 * (1.0 / 3.0), c4 = 0.125 * G4;
@@ -406,7 +449,7 @@ static __device__ __noinline__ void scalar_after_solve4(double* bc, const double
   const bool done = (!bisected && trunc <= 3e-8f * (float)slope) || iter >= 40 || (hi - lo) < 1e-9;
   // The float32 sums resolve KL to a few 1e-7 x (largest probability).  Where that would move lambda by
   // more than the tolerance (a very flat KL: nearly one-hot rows), or the solve did not converge, the row
-  // is handed to the float64 kernel.  (Radii below 5e-3 never reach this kernel: see the dispatcher.)
+  // is handed to the float64 kernel.
   // Below 5e-3 the direct value, where the quadrature was not taken, is held to a fifth of the tolerance
   // and to the worst case of its error: 3e-7 absolute (a flat row, where ex2.approx errs the same way on
   // every element).

@@ -104,3 +104,20 @@ def oracle_inputs(d: dict, rows=None):
         idx = torch.as_tensor(list(rows), device=s.device)
         s, t = s[idx], t[idx]
     return to_np64(s), to_np64(t)
+
+
+def force_second_tier(d, rows):
+    """Rewrites the given rows of a generated bf16 workload so that the row-per-SM kernel must hand them to
+    the float64 kernel: a plateau 400 nats below a few peaks that sit away from the first 256 logits of
+    every warp segment, so the float32 sums of its first pass overflow."""
+    V = d["s"].shape[1]
+    seg = ((V // 8 + 15) // 16) * 8                      # elements per warp segment (16 warps)
+    g = torch.Generator(device=d["s"].device).manual_seed(1234)
+    for r in rows:
+        s = torch.full((V,), -400.0, device=d["s"].device) + 0.5 * torch.randn(V, generator=g, device=d["s"].device)
+        pos = (torch.randint(300, max(301, seg - 8), (24,), generator=g, device=d["s"].device) + seg * (r % 16)).clamp(max=V - 1)
+        s[pos] = 2.0 * torch.randn(24, generator=g, device=d["s"].device)
+        t = s + 0.7 * torch.randn(V, generator=g, device=d["s"].device)
+        d["s"][r] = s.to(d["s"].dtype)
+        d["t"][r] = t.to(d["t"].dtype)
+        d["proposal"][r] = int(pos[0])

@@ -6,7 +6,7 @@ import torch
 import oracle as O
 import paper_2609_36601_b200 as P
 from paper_2609_36601_b200 import synth
-from parity import compare_rows, grad_check, oracle_inputs, to_np64
+from parity import compare_rows, force_second_tier, grad_check, oracle_inputs, to_np64
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -308,6 +308,8 @@ def test_calls_on_two_streams_do_not_share_scratch():
         ws = [synth.Workload("a", 1500, 32000, "bf16", 0.005, 1.0, True, 1002, 2),
               synth.Workload("b", 1200, 8192, "bf16", 0.005, 0.5, True, 99, 18)]
         ds = [synth.generate(w, DEV) for w in ws]
+        force_second_tier(ds[0], [5, 6, 900, 1499])
+        force_second_tier(ds[1], [0, 77, 1199])
         alone = []
         for w, d in zip(ws, ds):
             alone.append(P.route_fwd_bwd(d["s"], d["t"], d["proposal"], w.eps, seed=w.seed))

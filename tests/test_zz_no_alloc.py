@@ -7,6 +7,7 @@ import torch
 
 import paper_2609_36601_b200 as P
 from paper_2609_36601_b200 import synth
+from parity import force_second_tier
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -15,11 +16,11 @@ DEV = "cuda:0"
 def test_noalloc_entry_matches_regular_entry_twice_in_a_row():
     prev = P.set_kernel(0)
     try:
-        # a small radius on the V = 32000 workload: a few rows have a KL curve too flat for float32 sums and
-        # are handed to the float64 kernel, so the fixed scratch really carries a list
+        # the V = 32000 workload with some rows that overflow the float32 sums and are handed to the float64
+        # kernel, so the fixed scratch really carries a list
         w = synth.shrink(synth.WORKLOADS["cfg2"], 2048)
-        w = synth.Workload(w.name, w.N, w.V, w.dtype, 0.005, w.sigma, w.zipf, w.gen_seed, w.seed)
         d = synth.generate(w, DEV)
+        force_second_tier(d, [3, 700, 701, 1999])
         ref_out, ref_g = P.route_fwd_bwd(d["s"], d["t"], d["proposal"], w.eps, seed=w.seed, grad_scale=0.5)
         torch.cuda.synchronize()
         n_redo = P.redo_count()
@@ -36,6 +37,7 @@ def test_noalloc_entry_matches_regular_entry_twice_in_a_row():
         # a second workload right after, with different rows on the list: stale list contents must not matter
         w2 = synth.Workload("noalloc2", 300, 8192, "bf16", 0.005, 0.5, True, 99, 18)
         d2 = synth.generate(w2, DEV)
+        force_second_tier(d2, [0, 150, 299])
         r2, g2 = P.route_fwd_bwd(d2["s"], d2["t"], d2["proposal"], w2.eps, seed=w2.seed)
         out2 = P.alloc_outputs(w2.N, DEV)
         gg2 = torch.empty_like(d2["s"])
