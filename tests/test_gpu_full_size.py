@@ -4,7 +4,8 @@ selection, one call over the whole batch), on sampled rows the oracle computes o
 cfg1 runs in test_gpu_parity.py (all 64 rows).  cfg2, cfg3 and cfg5 run at full size here.  The
 throughput sweep (cfg4) keeps its full vocabulary and all 9 regime x radius cells but routes the
 first 2368 positions of each regime (16 rows per SM) instead of 65536: the per-row work and the launch shape
-per SM are the same, only the row loop is shorter."""
+per SM are the same, only the row loop is shorter; one cell (the mixed one) also runs at the full
+65536 positions in one call when the device has room for it."""
 import numpy as np
 import pytest
 import torch
@@ -81,6 +82,24 @@ def test_cfg4_cells(regime):
         assert saturated[1.0] > 0.99 and 0.0 < saturated[0.1] < 0.99   # an (almost) saturated and a mixed cell
     if regime == "ind":
         assert saturated[1.0] == 0.0
+
+
+def test_cfg4_one_cell_at_65536_positions():
+    w = synth.WORKLOADS["cfg4_s05_e0.1"]
+    need = 3 * w.N * w.V * 2 + (4 << 30)                          # s, t, gradient and slack
+    if torch.cuda.mem_get_info(0)[0] < need:
+        pytest.skip("needs %.0f GB of free device memory" % (need / 1e9))
+    d = synth.generate(w, DEV)
+    rows = list(range(11, w.N, 2731))                             # 24 rows over the whole batch
+    out, ref, n_exempt = _sampled(w, d, rows)
+    assert P.last_kernel() == 3 and n_exempt <= 1
+    st = out["row_status"]
+    assert int((st & ~1).max().item()) == 0                       # no status bit but "saturated" on any of the rows
+    tv = out["tv"].cpu().numpy()
+    assert np.all(tv <= np.sqrt(w.eps / 2) + 1e-5)
+    assert abs(out["corrected"].float().mean().item() - tv.mean()) < 4 * np.sqrt(0.25 / w.N)
+    del d, out
+    torch.cuda.empty_cache()
 
 
 def test_cfg5_full():
