@@ -285,6 +285,19 @@ SAKI_API int saki_last_kernel(void);
  * how many rows of the calling thread's last routing call took that second tier. */
 SAKI_API int saki_redo_count(void* cuda_stream, uint64_t* n_rows);
 
+/* Block verification, early out (Section 3.5: what follows a sequence's first rejected position is
+ * discarded).  When on (the default), the row-per-SM kernel hands out whole sequences to its blocks
+ * from a device counter; a block walks a sequence position by position and leaves it at the first
+ * position that is rejected or flagged, so the positions behind it are never read.  Which block routes
+ * which sequence varies from run to run; the outputs do not (every random number is keyed by the
+ * position).  Off: every position of every sequence is routed, then resolved (what the other kernels
+ * always do).  Process-wide; returns the previous value. */
+SAKI_API int saki_set_spec_early_out(int on);
+
+/* Synchronises the stream and returns how many positions the calling thread's last saki_spec_verify
+ * actually routed when it ran with early out (0 otherwise); B * (K + 1) minus this were skipped. */
+SAKI_API int saki_spec_positions_routed(void* cuda_stream, uint64_t* n_positions);
+
 /* Number of kernels this library has launched in this process (all threads). */
 SAKI_API uint64_t saki_launch_count(void);
 

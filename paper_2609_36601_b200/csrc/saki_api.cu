@@ -19,6 +19,7 @@ namespace saki {
 static thread_local char g_err[512] = "";
 static std::atomic<uint64_t> g_launches{0};
 static std::atomic<int> g_kernel{0};
+static std::atomic<int> g_spec_early_out{1};
 static thread_local int g_last_kernel = 0;
 
 static int fail(int code, const char* fmt, ...) {
@@ -143,12 +144,14 @@ static int dispatch_rows(RowParams p, int dtype, cudaStream_t st, int32_t* scrat
       const int rc = redo_scratch(p.n_rows, st, &p.redo_list, &p.redo_count);
       if (rc) return rc;
     }
-    e = cudaMemsetAsync(p.redo_count, 0, sizeof(unsigned int), st);
+    e = cudaMemsetAsync(p.redo_count, 0, 4 * sizeof(unsigned int), st);   // the counter and the three words after it
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
     g_last_redo_count = p.redo_count;
   }
   if (fast && (which == 0 || which == 3) && rowsm_can_serve(p, dtype)) {
+    p.seq_next = (p.spec && g_spec_early_out.load()) ? p.redo_count + 1 : nullptr;   // block verification: sequences handed out, early out
     e = launch_rowsm(p, st, &launches, &served);
+    p.seq_next = nullptr;
     if (e != cudaSuccess) return cuda_fail(e, "row-per-SM kernel launch");
     if (served) used = 3;
   }
@@ -589,6 +592,22 @@ SAKI_API int saki_redo_count(void* cuda_stream, uint64_t* n_rows) {
   e = cudaMemcpy(&h, g_last_redo_count, sizeof(h), cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy");
   *n_rows = h;
+  return SAKI_OK;
+}
+
+SAKI_API int saki_set_spec_early_out(int on) { return g_spec_early_out.exchange(on ? 1 : 0); }
+
+SAKI_API int saki_spec_positions_routed(void* cuda_stream, uint64_t* n_positions) {
+  g_err[0] = 0;
+  if (!n_positions) return fail(SAKI_ERR_INVALID_ARG, "NULL output pointer");
+  *n_positions = 0;
+  if (!g_last_redo_count) return SAKI_OK;
+  cudaError_t e = cudaStreamSynchronize((cudaStream_t)cuda_stream);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+  unsigned int h = 0;
+  e = cudaMemcpy(&h, g_last_redo_count + 2, sizeof(h), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy");
+  *n_positions = h;
   return SAKI_OK;
 }
 

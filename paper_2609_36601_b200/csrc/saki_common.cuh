@@ -35,6 +35,8 @@ struct RowParams {
   int32_t* redo_list;                  // scratch: rows the float32 kernels hand to the float64 kernel
   unsigned int* redo_count;            // scratch: their number (zeroed before the launch)
   int32_t from_list;                   // general kernel only: route the rows of redo_list
+  unsigned int* seq_next;              // row-per-SM kernel, block verification: [0] sequence counter, [1] positions
+                                       // routed (both zeroed before the launch); NULL: rows in static order
 };
 
 // Parameters of the metadata-driven backward kernels (saki_route_bwd_from_meta).

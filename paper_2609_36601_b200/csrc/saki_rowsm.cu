@@ -300,14 +300,23 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
     __syncthreads();
   };
 
+  // Block verification hands out whole sequences: a CTA walks one sequence position by position, leaves
+  // it at the first position that is not accepted (what lies behind it is never computed: Section 3.5
+  // discards it) and takes the next sequence from a device counter.  `seqres`: [0] a sequence reserved
+  // for this CTA ahead of time (n_seq: none left), [1] 1 once thread 0 has taken it.
+  const bool dyn = P.seq_next != nullptr;
+  const int n_seq = dyn ? (int)(P.n_rows / P.K1) : 0;
+  int* seqres = (int*)(smem + ROFF_MBAR + 8);
   if (tid == 0) {
     mbar_init(mbar, RW);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    seqres[0] = 0; seqres[1] = 1;
   }
   __syncthreads();
   const __nv_bfloat16 *n_s = nullptr, *n_t = nullptr;   // the rows of the CTA's next position, if any
-  if ((int64_t)blockIdx.x < P.n_rows) {
-    row_ptrs(blockIdx.x, n_s, n_t);
+  const int64_t first_row = dyn ? (int64_t)blockIdx.x * P.K1 : (int64_t)blockIdx.x;
+  if (first_row < P.n_rows) {
+    row_ptrs(first_row, n_s, n_t);
     if (lane == 0) issue(n_s, n_t);
     ring_prime(rg, sg, lane, n_s, n_t, pol_last);
   }
@@ -438,7 +447,8 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
     if (lane == 0) write_result_tv(bcp, P.out, !P.spec, prow, pbonus ? 0 : 1, y, pbonus, K.c64, ps, pt, tv);
   };
 
-  for (int64_t row = blockIdx.x; row < P.n_rows; row += gridDim.x, rb ^= 1) {
+  int64_t next_row_c = P.n_rows;
+  for (int64_t row = first_row; row < P.n_rows; row = next_row_c, rb ^= 1) {
     double* bc = (double*)(smem + ROFF_BC) + rb * BC_DOUBLES;   // this row's broadcast scalars
     const uint64_t rid = P.row_offset + (uint64_t)row;
     const int64_t seq = P.K1 == 1 ? row : (int64_t)((uint32_t)row / (uint32_t)P.K1);
@@ -448,9 +458,19 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
     const bool masked = (P.mask != nullptr) && (P.mask[row] == 0);
     const __nv_bfloat16 *g_s = n_s, *g_t = n_t;
     __nv_bfloat16* g_out = P.dlogits ? (__nv_bfloat16*)P.dlogits + row * P.ld_g : nullptr;
-    const int64_t next_row = row + gridDim.x;
-    n_s = nullptr; n_t = nullptr;
-    if (next_row < P.n_rows) row_ptrs(next_row, n_s, n_t);
+    // thread 0, once the row's decision is known: where the CTA goes next when sequences are handed out
+    auto plan_next = [&] {
+      const int mode = (int)bc[BC_MODE];
+      if (!dyn || mode == MODE_SOLVE) return;
+      const bool stop = bonus || mode == MODE_FLAGGED || (mode == MODE_FINAL && bc[BC_CORR] != 0.0);
+      int64_t nx = row + 1;
+      if (stop) { nx = (int64_t)seqres[0] * P.K1; seqres[1] = 1; }
+      bc[BC_NEXT] = (double)nx;
+      atomicAdd(P.seq_next + 1, 1u);             // statistic: positions routed
+    };
+#ifdef SAKI_PHASE_TIMING
+    ++t_rows;
+#endif
 
     RTS(0);
     if (!dead) {
@@ -582,6 +602,11 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           bc[BC_SX] = ok ? (double)__bfloat162float(g_s[x]) : 0.0;
           bc[BC_TX] = ok ? (double)__bfloat162float(g_t[x]) : 0.0;
         }
+        if (warp == 11 && dyn && seqres[1] != 0 && seqres[0] < n_seq) {   // reserve the CTA's next sequence
+          const unsigned int nxt = gridDim.x + atomicAdd(P.seq_next, 1u);
+          seqres[0] = (int)min(nxt, (unsigned int)n_seq);
+          seqres[1] = 0;
+        }
       }
       if (any_dead) dead = true;
       __syncthreads();
@@ -600,6 +625,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           bc[BC_K0] = gat[7]; bc[BC_K1] = gat[8];
           scalar_after_lse_tail(bc, gat, K, (float)gat[7], (float)gat[8], x, bonus, masked, any_dead != 0, 1.f, true,
                                 rS, rSt, G, G1, gat + 9);
+          plan_next();
         }
       }
       RTS(5);
@@ -641,10 +667,14 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
                            warp_sum_d(tot(S4))};
       combine(v, 5);
       RTS(8);
-      if (tid == 0) scalar_after_solve4(bc, gat, K, k0, k1, x, bonus, masked);
+      if (tid == 0) { scalar_after_solve4(bc, gat, K, k0, k1, x, bonus, masked); plan_next(); }
       RTS(9);
       __syncthreads();
     }
+    const int64_t next_row = dyn ? (int64_t)bc[BC_NEXT] : row + gridDim.x;
+    next_row_c = next_row;
+    n_s = nullptr; n_t = nullptr;
+    if (next_row < P.n_rows) row_ptrs(next_row, n_s, n_t);
 
     // ------------------------------------------------ flagged row: zero outputs, zero gradient
     if ((int)bc[BC_MODE] == MODE_FLAGGED || (int)bc[BC_MODE] == MODE_REDO) {
@@ -742,7 +772,6 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
   }
 
 #ifdef SAKI_PHASE_TIMING
-  for (int64_t row = blockIdx.x; row < P.n_rows; row += gridDim.x) ++t_rows;
   if (lane == 0 && blockIdx.x == 5 && t_rows > 0) printf("warp %d solve loop %lld cycles per row, %lld evaluations in %d rows, %d steps\n", warp, w_solve / t_rows, w_evals, t_rows, sg.steps);
   if (tid == 0 && (blockIdx.x == 0 || blockIdx.x == 77) && t_rows > 0)
     printf("blk %d tid %d rows %d | endbar %lld copy-wait %lld | lse %lld warp+bar %lld gather %lld scalar %lld | "
@@ -787,7 +816,8 @@ cudaError_t launch_rowsm(const RowParams& p, cudaStream_t st, int* n_launches, b
       cached_dev = dev;
     }
   }
-  const int grid = (int)(p.n_rows < cached_sms ? p.n_rows : cached_sms);
+  const int64_t units = p.seq_next ? p.n_rows / p.K1 : p.n_rows;   // sequences when they are handed out, else rows
+  const int grid = (int)(units < cached_sms ? units : cached_sms);
   rowsm_kernel<<<grid, RT, RSMEM_BYTES, st>>>(p);
   cudaError_t e = cudaGetLastError();
   if (e == cudaSuccess) { *served = true; if (n_launches) *n_launches += 1; }

@@ -108,6 +108,7 @@ def test_cfg5_full():
     d = synth.generate(w, DEV)
     s3, t3 = d["s"].view(B, K + 1, V), d["t"].view(B, K + 1, V)
     draft = d["proposal"].view(B, K + 1)[:, :K].contiguous()
+    P.check()                                                     # clears what earlier tests may have left
     res = P.spec_verify(s3, t3, draft, w.eps, seed=w.seed)
     torch.cuda.synchronize()
     assert P.check() == 0 and P.last_kernel() == 3
