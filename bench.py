@@ -15,6 +15,10 @@ positions: one saki_route_fwd_bwd call.  Prints ONE JSON line.
             gradient row once) / measured kernel time, against the measured
             copy bandwidth of this machine's B200s
   cpu_baseline  the float64 test oracle, as it stands, on a bounded sample
+  next_step, spec_verify  (rank 0, unless --no-next) two further calls timed the
+            same way beside the headline: saki_route_bwd_from_meta on the same
+            logits, and saki_spec_verify on its own workload with and without
+            early out
 
 With N > 1 (under torchrun) every rank routes its own batch of the same
 shape (rows are independent: no collective on the data path); the time is
@@ -241,6 +245,38 @@ def run_ours(args):
                "algorithmic_bytes_per_launch": mbytes, "achieved_gbs": mbytes / (mms * 1e-3) / 1e9,
                "traffic": META_TRAFFIC_BYTES_PER_POSITION * w.N if META_TRAFFIC_BYTES_PER_POSITION else None}
 
+    # ---- block verification (saki_spec_verify) on its own workload, with and without early out; beside the
+    # headline like the step above
+    spec = None
+    if not args.no_next and rank == 0 and "cfg5" in synth.WORKLOADS:
+        w5 = synth.WORKLOADS["cfg5"]
+        d5 = synth.generate(w5, dev)
+        s5, t5 = d5["s"].view(w5.B, w5.K + 1, w5.V), d5["t"].view(w5.B, w5.K + 1, w5.V)
+        draft = d5["proposal"].view(w5.B, w5.K + 1)[:, :w5.K].contiguous()
+        spec = {"call": "saki_spec_verify", "workload": "cfg5: B=%d sequences, K=%d draft tokens, V=%d, bf16, eps=%g" %
+                (w5.B, w5.K, w5.V, w5.eps), "positions": w5.N}
+        prev = P.set_spec_early_out(True)
+        for on in (False, True):
+            P.set_spec_early_out(on)
+            for _ in range(3):
+                r5 = P.spec_verify(s5, t5, draft, w5.eps, seed=w5.seed, stream=stream)
+            torch.cuda.synchronize()
+            c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            c0.record(stream)
+            for _ in range(args.steps):
+                r5 = P.spec_verify(s5, t5, draft, w5.eps, seed=w5.seed, stream=stream)
+            c1.record(stream)
+            torch.cuda.synchronize()
+            ms5 = c0.elapsed_time(c1) / args.steps
+            if on:
+                spec.update({"ms_per_call": ms5, "value": w5.B / (ms5 * 1e-3), "unit": "sequences/s",
+                             "positions_routed": P.spec_positions_routed(stream),
+                             "mean_accepted": float(r5["n_accept"].float().mean().item())})
+            else:
+                spec["ms_per_call_all_positions"] = ms5
+        P.set_spec_early_out(prev)
+        del d5, s5, t5
+
     # ---- end to end: host buffers through saki_route_host
     e2e = None
     if not args.no_e2e:
@@ -314,6 +350,8 @@ def run_ours(args):
         nxt["roofline"] = {"bound": "hbm", "achieved": nxt["achieved_gbs"], "peak": peak, "unit": "GB/s",
                            "frac": nxt["achieved_gbs"] / peak}
         line["next_step"] = nxt
+    if spec is not None:
+        line["spec_verify"] = spec
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -149,7 +149,9 @@ static int dispatch_rows(RowParams p, int dtype, cudaStream_t st, int32_t* scrat
     g_last_redo_count = p.redo_count;
   }
   if (fast && (which == 0 || which == 3) && rowsm_can_serve(p, dtype)) {
-    p.seq_next = (p.spec && g_spec_early_out.load()) ? p.redo_count + 1 : nullptr;   // block verification: sequences handed out, early out
+    // block verification: sequences handed out, early out.  A block walks its sequence serially, so with
+    // few sequences (under two per SM) routing every position in static order keeps more SMs busy.
+    p.seq_next = (p.spec && g_spec_early_out.load() && p.n_rows / p.K1 >= 2 * rowsm_sm_count()) ? p.redo_count + 1 : nullptr;
     e = launch_rowsm(p, st, &launches, &served);
     p.seq_next = nullptr;
     if (e != cudaSuccess) return cuda_fail(e, "row-per-SM kernel launch");

@@ -151,6 +151,7 @@ cudaError_t launch_cluster(const RowParams& p, cudaStream_t st, int* n_launches,
 bool cluster_can_serve(const RowParams& p, int dtype);
 cudaError_t launch_rowsm(const RowParams& p, cudaStream_t st, int* n_launches, bool* served);
 bool rowsm_can_serve(const RowParams& p, int dtype);
+int rowsm_sm_count();                 // SMs of the current device (0 if the query fails)
 cudaError_t launch_meta_general(const MetaParams& p, int dtype, cudaStream_t st, int* n_launches);
 cudaError_t launch_meta_stream(const MetaParams& p, cudaStream_t st, int* n_launches, bool* served);
 bool meta_stream_can_serve(const MetaParams& p, int dtype);

@@ -799,6 +799,12 @@ bool rowsm_can_serve(const RowParams& p, int dtype) {
   return true;
 }
 
+int rowsm_sm_count() {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+  return sms;
+}
+
 cudaError_t launch_rowsm(const RowParams& p, cudaStream_t st, int* n_launches, bool* served) {
   *served = false;
   if (p.n_rows <= 0) { *served = true; return cudaSuccess; }

@@ -1,7 +1,9 @@
 """Block verification with early out (Section 3.5: positions behind a sequence's first rejection are
 discarded).  The row-per-SM kernel hands out whole sequences and never routes the discarded positions;
 every output must be the one the call gives when it routes all positions and resolves afterwards, and
-the number of positions routed must be exactly the number that verification needs."""
+the number of positions routed must be exactly the number that verification needs.  With fewer than two
+sequences per SM the library routes every position in static order instead (a block walks its sequence
+serially, so few sequences would leave SMs idle)."""
 import numpy as np
 import pytest
 import torch
@@ -49,7 +51,11 @@ def _same(a, b):
         assert torch.equal(x, y), k          # bit-identical, floats included
 
 
-@pytest.mark.parametrize("B,K,V", [(300, 6, 4096), (7, 16, 8192), (149, 1, 2048), (1, 5, 32000)])
+def _sms():
+    return torch.cuda.get_device_properties(0).multi_processor_count
+
+
+@pytest.mark.parametrize("B,K,V", [(300, 6, 4096), (640, 16, 2048), (1500, 1, 2048), (7, 16, 8192), (149, 1, 2048), (1, 5, 32000)])
 def test_outputs_do_not_depend_on_early_out(B, K, V):
     w, d, s3, t3, draft = _case(B, K, V)
     out = _both(s3, t3, draft, w.eps, w.seed)
@@ -57,15 +63,18 @@ def test_outputs_do_not_depend_on_early_out(B, K, V):
     n_acc = out[True][0]["n_accept"].cpu().numpy()
     st = out[True][0]["per_pos"]["row_status"].view(B, K + 1).cpu().numpy()
     assert out[False][1] == 0
-    # a sequence needs its first n_accept + 1 positions (all K + 1 if every draft token was accepted)
-    assert out[True][1] == int(np.minimum(n_acc + 1, K + 1).sum())
+    if B >= 2 * _sms():
+        # a sequence needs its first n_accept + 1 positions (all K + 1 if every draft token was accepted)
+        assert out[True][1] == int(np.minimum(n_acc + 1, K + 1).sum())
+    else:
+        assert out[True][1] == 0           # few sequences: every position routed, in static order
     for b in range(B):
         assert np.all(st[b, n_acc[b] + 1:] == P.binding.ROW_NOT_COMPUTED)
         assert np.all(st[b, :n_acc[b] + 1] & P.binding.ROW_NOT_COMPUTED == 0)
 
 
 def test_early_out_against_the_oracle():
-    B, K, V = 40, 5, 4096
+    B, K, V = 2 * _sms() + 5, 5, 4096
     w, d, s3, t3, draft = _case(B, K, V, eps=0.1, gen_seed=92, seed=22)
     res = P.spec_verify(s3, t3, draft, w.eps, seed=w.seed)
     torch.cuda.synchronize()
@@ -78,7 +87,7 @@ def test_early_out_against_the_oracle():
 
 
 def test_flagged_and_second_tier_positions_inside_sequences():
-    B, K, V = 64, 4, 8192
+    B, K, V = 2 * _sms() + 4, 4, 8192
     w, d, s3, t3, draft = _case(B, K, V, gen_seed=93, seed=23)
     s3[3, 1, 17] = float("nan")            # flagged position: verification of sequence 3 stops there
     s3[9, 0, 5] = float("inf")
@@ -100,7 +109,7 @@ def test_flagged_and_second_tier_positions_inside_sequences():
 
 
 def test_strided_sequences_and_a_second_stream():
-    B, K, V = 33, 3, 2048
+    B, K, V = 2 * _sms() + 14, 3, 2048
     w, d, s3, t3, draft = _case(B, K, V, gen_seed=94, seed=24)
     pad_s = torch.zeros((B, K + 3, V + 64), dtype=torch.bfloat16, device=DEV)
     pad_t = torch.zeros_like(pad_s)
@@ -113,3 +122,4 @@ def test_strided_sequences_and_a_second_stream():
         b = P.spec_verify(pad_s[:, 1:K + 2, :V], pad_t[:, 1:K + 2, :V], draft, w.eps, seed=w.seed, stream=st)
     torch.cuda.synchronize()
     _same(a, b)
+    assert P.spec_positions_routed(st) > 0
