@@ -219,6 +219,7 @@ def run_ours(args):
     value = world * w.N / (ms_per_step * 1e-3)
     n_flagged = P.check()
     kernel_used = P.last_kernel()
+    evals_last_step = P.solve_evaluations(stream) if kernel_used == 3 else 0   # of the last timed launch
 
     # ---- the step that follows the path: the trainer's loss and gradient from this call's metadata
     # (saki_route_bwd_from_meta), on the same logits; reported beside the headline, not in it
@@ -324,6 +325,19 @@ def run_ours(args):
                 "algorithmic_bytes_per_launch": bpp * w.N, "kernel": {3: "saki::rowsm_kernel", 2: "saki::cluster_kernel"}.get(kernel_used, "saki::general_kernel"),
                 "kernel_ms": kern_ms,
                 "frac_of_nominal_8TBs": achieved / 8000.0}
+    if kernel_used == 3:
+        # What the kernel is actually bound by: exponentials on the special-function pipe.  Per vocabulary
+        # element 2 in pass lse (student, teacher), 2 in pass final (p, q) and 1 per evaluation pass, the
+        # evaluation passes counted by the kernel itself; peak = 16 ex2 per clock per SM (the throughput of
+        # base-2 exponentials on this architecture) x SMs x the SM clock sampled during the timed region.
+        evals = evals_last_step / max(1, w.N)
+        sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
+        mhz = (clocks or {}).get("sm_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0
+        xu_peak = 16.0 * sm_count * mhz * 1e6 / 1e9
+        xu_ach = (4.0 + evals) * w.V * w.N / (kern_ms * 1e-3) / 1e9
+        roofline["special_function_pipe"] = {"achieved": xu_ach, "peak": xu_peak, "unit": "G ex2/s",
+                                             "frac": xu_ach / xu_peak, "evaluation_passes_per_row": evals,
+                                             "ex2_per_element": 4.0 + evals}
 
     stats = {"correction_rate": float(out["corrected"].float().mean().item()),
              "median_tv": float(out["tv"].median().item()), "mean_lambda": float(out["lambda"].mean().item()),

@@ -285,6 +285,12 @@ SAKI_API int saki_last_kernel(void);
  * how many rows of the calling thread's last routing call took that second tier. */
 SAKI_API int saki_redo_count(void* cuda_stream, uint64_t* n_rows);
 
+/* Synchronises the stream and returns how many evaluation passes (one pass over a row at a trial
+ * beta, Section 3.2's boundary search) the row-per-SM kernel ran in the calling thread's last routing
+ * call, summed over its rows; 0 if another kernel served the call.  Every row also takes the two fixed
+ * passes (log-sum-exp with moments, final). */
+SAKI_API int saki_solve_evaluations(void* cuda_stream, uint64_t* n_passes);
+
 /* Block verification, early out (Section 3.5: what follows a sequence's first rejected position is
  * discarded).  When on (the default), the row-per-SM kernel hands out whole sequences to its blocks
  * from a device counter; a block walks a sequence position by position and leaves it at the first

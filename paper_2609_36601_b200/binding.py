@@ -22,7 +22,7 @@ _FLOAT_FIELDS = ("lambda", "kl", "tv", "accept_prob", "logp_x", "logq_x", "logT_
 EXPORTS = ("saki_route_fwd", "saki_route_fwd_bwd", "saki_route_fwd_bwd_noalloc", "saki_route_host",
            "saki_route_bwd_from_meta", "saki_select_tm", "saki_spec_verify",
            "saki_sample_proposal", "saki_check", "saki_set_kernel", "saki_last_kernel", "saki_redo_count",
-           "saki_set_spec_early_out", "saki_spec_positions_routed", "saki_launch_count",
+           "saki_set_spec_early_out", "saki_spec_positions_routed", "saki_solve_evaluations", "saki_launch_count",
            "saki_last_error", "saki_version")
 
 
@@ -108,6 +108,8 @@ def load_library(path: str | None = None):
     lib.saki_set_spec_early_out.restype = C.c_int
     lib.saki_spec_positions_routed.argtypes = [C.c_void_p, C.POINTER(C.c_uint64)]
     lib.saki_spec_positions_routed.restype = C.c_int
+    lib.saki_solve_evaluations.argtypes = [C.c_void_p, C.POINTER(C.c_uint64)]
+    lib.saki_solve_evaluations.restype = C.c_int
     lib.saki_launch_count.restype = C.c_uint64
     lib.saki_last_error.restype = C.c_char_p
     for f in ("saki_route_fwd", "saki_route_fwd_bwd", "saki_route_host", "saki_spec_verify",
@@ -366,6 +368,14 @@ def redo_count(stream=None) -> int:
     lib = load_library()
     n = C.c_uint64(0)
     _raise(lib, lib.saki_redo_count(_stream_ptr(stream), C.byref(n)))
+    return int(n.value)
+
+
+def solve_evaluations(stream=None) -> int:
+    """Evaluation passes of the row-per-SM kernel in the last routing call, over all rows (synchronises)."""
+    lib = load_library()
+    n = C.c_uint64(0)
+    _raise(lib, lib.saki_solve_evaluations(_stream_ptr(stream), C.byref(n)))
     return int(n.value)
 
 

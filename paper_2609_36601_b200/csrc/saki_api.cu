@@ -138,6 +138,7 @@ static int dispatch_rows(RowParams p, int dtype, cudaStream_t st, int32_t* scrat
   const bool rowsm_ok = (which == 0 || which == 3) && rowsm_can_serve(p, dtype);
   const bool fast = (which != 1) && (rowsm_ok || (eps_ok && cluster_can_serve(p, dtype)));
   p.redo_list = nullptr; p.redo_count = nullptr; p.from_list = 0;
+  g_last_redo_count = nullptr;          // the counters below describe this call only
   if (fast) {
     if (scratch_list) { p.redo_list = scratch_list; p.redo_count = scratch_count; }
     else {
@@ -247,10 +248,11 @@ static int meta_impl(const saki_meta_in* in, const saki_meta_out* out, void* dlo
   cudaError_t e;
   bool served = false;
   int used = 1;
+  g_last_redo_count = nullptr;
   if (g_kernel.load() != 1 && meta_stream_can_serve(p, in->dtype)) {
     rc = redo_scratch(p.n_rows, st, &p.redo_list, &p.redo_count);
     if (rc) return rc;
-    e = cudaMemsetAsync(p.redo_count, 0, sizeof(unsigned int), st);
+    e = cudaMemsetAsync(p.redo_count, 0, 4 * sizeof(unsigned int), st);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
     g_last_redo_count = p.redo_count;
     e = launch_meta_stream(p, st, &launches, &served);
@@ -594,6 +596,20 @@ SAKI_API int saki_redo_count(void* cuda_stream, uint64_t* n_rows) {
   e = cudaMemcpy(&h, g_last_redo_count, sizeof(h), cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy");
   *n_rows = h;
+  return SAKI_OK;
+}
+
+SAKI_API int saki_solve_evaluations(void* cuda_stream, uint64_t* n_passes) {
+  g_err[0] = 0;
+  if (!n_passes) return fail(SAKI_ERR_INVALID_ARG, "NULL output pointer");
+  *n_passes = 0;
+  if (!g_last_redo_count) return SAKI_OK;
+  cudaError_t e = cudaStreamSynchronize((cudaStream_t)cuda_stream);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+  unsigned int h = 0;
+  e = cudaMemcpy(&h, g_last_redo_count + 3, sizeof(h), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy");
+  *n_passes = h;
   return SAKI_OK;
 }
 

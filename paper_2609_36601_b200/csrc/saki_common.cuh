@@ -33,7 +33,8 @@ struct RowParams {
   float grad_scale;
   unsigned long long* flagged;         // device counter of flagged rows
   int32_t* redo_list;                  // scratch: rows the float32 kernels hand to the float64 kernel
-  unsigned int* redo_count;            // scratch: their number (zeroed before the launch)
+  unsigned int* redo_count;            // scratch: their number (zeroed before the launch, with the three words
+                                       // after it: [1], [2] see seq_next; [3] evaluation passes of the row-per-SM kernel)
   int32_t from_list;                   // general kernel only: route the rows of redo_list
   unsigned int* seq_next;              // row-per-SM kernel, block verification: [0] sequence counter, [1] positions
                                        // routed (both zeroed before the launch); NULL: rows in static order

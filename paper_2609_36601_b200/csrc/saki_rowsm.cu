@@ -667,7 +667,11 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
                            warp_sum_d(tot(S4))};
       combine(v, 5);
       RTS(8);
-      if (tid == 0) { scalar_after_solve4(bc, gat, K, k0, k1, x, bonus, masked); plan_next(); }
+      if (tid == 0) {
+        scalar_after_solve4(bc, gat, K, k0, k1, x, bonus, masked);
+        plan_next();
+        atomicAdd(P.redo_count + 3, 1u);         // statistic: evaluation passes
+      }
       RTS(9);
       __syncthreads();
     }

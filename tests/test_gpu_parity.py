@@ -346,3 +346,20 @@ def test_spec_verify_k_limits():
     with pytest.raises(P.SakiError):
         bad = torch.zeros((2, 18, V), dtype=torch.bfloat16, device=DEV)
         P.spec_verify(bad, bad, torch.zeros((2, 17), dtype=torch.int32, device=DEV), 0.1)
+
+
+def test_evaluation_pass_counter():
+    """The row-per-SM kernel counts its evaluation passes: none at eps = 0, about one per unsaturated row otherwise."""
+    w = synth.shrink(synth.WORKLOADS["cfg2"], 600)
+    d = synth.generate(w, DEV)
+    out = P.route_fwd(d["s"], d["t"], d["proposal"], 0.0, seed=w.seed)
+    assert P.last_kernel() == 3 and P.solve_evaluations() == 0
+    out = P.route_fwd(d["s"], d["t"], d["proposal"], w.eps, seed=w.seed)
+    n_solved = int(((out["row_status"] & 1) == 0).sum().item())
+    assert n_solved <= P.solve_evaluations() <= int(1.2 * n_solved)
+    prev = P.set_kernel(1)
+    try:
+        P.route_fwd(d["s"], d["t"], d["proposal"], w.eps, seed=w.seed)
+        assert P.solve_evaluations() == 0      # another kernel served the call
+    finally:
+        P.set_kernel(prev)
