@@ -292,12 +292,13 @@ SAKI_API int saki_redo_count(void* cuda_stream, uint64_t* n_rows);
 SAKI_API int saki_solve_evaluations(void* cuda_stream, uint64_t* n_passes);
 
 /* Block verification, early out (Section 3.5: what follows a sequence's first rejected position is
- * discarded).  When on (the default), the row-per-SM kernel hands out whole sequences to its blocks
- * from a device counter; a block walks a sequence position by position and leaves it at the first
- * position that is rejected or flagged, so the positions behind it are never read.  Which block routes
- * which sequence varies from run to run; the outputs do not (every random number is keyed by the
- * position).  Off: every position of every sequence is routed, then resolved (what the other kernels
- * always do).  Process-wide; returns the previous value. */
+ * discarded).  When on (the default) and the call has at least two sequences per SM, the row-per-SM
+ * kernel hands out positions from a device counter in position-major order and passes over a position
+ * once an earlier position of its sequence is known to be rejected or flagged, so most discarded
+ * positions are never read; nothing waits, a position whose predecessor is still undecided is routed.
+ * Which block routes which position varies from run to run; the outputs do not (every random number is
+ * keyed by the position).  Off, or with fewer sequences: every position of every sequence is routed,
+ * then resolved (what the other kernels always do).  Process-wide; returns the previous value. */
 SAKI_API int saki_set_spec_early_out(int on);
 
 /* Synchronises the stream and returns how many positions the calling thread's last saki_spec_verify

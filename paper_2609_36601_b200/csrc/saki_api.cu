@@ -75,7 +75,8 @@ static int redo_scratch(int64_t n_rows, cudaStream_t st, int32_t** list, unsigne
     if (b.list) cudaFree(b.list);
     b = RedoBuf();
     const int64_t cap = std::max<int64_t>(n_rows, 1 << 16);
-    cudaError_t e = cudaMalloc((void**)&b.list, (size_t)(cap + 64) * sizeof(int32_t));
+    // row ids, 64 words of counters, and as many words again (block verification: one per sequence)
+    cudaError_t e = cudaMalloc((void**)&b.list, (size_t)(2 * cap + 64) * sizeof(int32_t));
     if (e != cudaSuccess) { b = RedoBuf(); return cuda_fail(e, "cudaMalloc (redo list)"); }
     b.cap = cap;
   }
@@ -150,11 +151,20 @@ static int dispatch_rows(RowParams p, int dtype, cudaStream_t st, int32_t* scrat
     g_last_redo_count = p.redo_count;
   }
   if (fast && (which == 0 || which == 3) && rowsm_can_serve(p, dtype)) {
-    // block verification: sequences handed out, early out.  A block walks its sequence serially, so with
-    // few sequences (under two per SM) routing every position in static order keeps more SMs busy.
-    p.seq_next = (p.spec && g_spec_early_out.load() && p.n_rows / p.K1 >= 2 * rowsm_sm_count()) ? p.redo_count + 1 : nullptr;
+    // Block verification with early out: positions handed out as tickets, sequences record their first stop.
+    // Only with two or more sequences per SM: with fewer, most positions are handed out before their
+    // predecessor's decision is known, and the bookkeeping costs more than the few skipped rows save.
+    int sms = 0, dev_now = 0;
+    if (p.spec && (cudaGetDevice(&dev_now) != cudaSuccess ||
+                   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev_now) != cudaSuccess)) sms = 0;
+    if (p.spec && g_spec_early_out.load() && !scratch_list && sms > 0 && p.n_rows / p.K1 >= 2 * (int64_t)sms) {
+      p.seq_next = p.redo_count + 1;
+      p.seq_stop = (int*)(p.redo_count + 64);
+      e = cudaMemsetAsync(p.seq_stop, 0x7f, (size_t)(p.n_rows / p.K1) * sizeof(int), st);   // "no stop yet": above any position
+      if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+    }
     e = launch_rowsm(p, st, &launches, &served);
-    p.seq_next = nullptr;
+    p.seq_next = nullptr; p.seq_stop = nullptr;
     if (e != cudaSuccess) return cuda_fail(e, "row-per-SM kernel launch");
     if (served) used = 3;
   }

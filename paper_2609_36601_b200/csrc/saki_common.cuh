@@ -36,8 +36,9 @@ struct RowParams {
   unsigned int* redo_count;            // scratch: their number (zeroed before the launch, with the three words
                                        // after it: [1], [2] see seq_next; [3] evaluation passes of the row-per-SM kernel)
   int32_t from_list;                   // general kernel only: route the rows of redo_list
-  unsigned int* seq_next;              // row-per-SM kernel, block verification: [0] sequence counter, [1] positions
-                                       // routed (both zeroed before the launch); NULL: rows in static order
+  unsigned int* seq_next;              // row-per-SM kernel, block verification with early out: [0] ticket counter,
+                                       // [1] positions routed (both zeroed before the launch); NULL: rows in static order
+  int* seq_stop;                       // [n_rows / K1] position of each sequence's first stop (>= K1 before the launch)
 };
 
 // Parameters of the metadata-driven backward kernels (saki_route_bwd_from_meta).
@@ -152,7 +153,6 @@ cudaError_t launch_cluster(const RowParams& p, cudaStream_t st, int* n_launches,
 bool cluster_can_serve(const RowParams& p, int dtype);
 cudaError_t launch_rowsm(const RowParams& p, cudaStream_t st, int* n_launches, bool* served);
 bool rowsm_can_serve(const RowParams& p, int dtype);
-int rowsm_sm_count();                 // SMs of the current device (0 if the query fails)
 cudaError_t launch_meta_general(const MetaParams& p, int dtype, cudaStream_t st, int* n_launches);
 cudaError_t launch_meta_stream(const MetaParams& p, cudaStream_t st, int* n_launches, bool* served);
 bool meta_stream_can_serve(const MetaParams& p, int dtype);

@@ -20,7 +20,6 @@ enum { BC_MODE = 0, BC_BETA, BC_CB, BC_KB, BC_LO, BC_HI, BC_ITER,               
        BC_OWNER_WARP, BC_BEFORE, BC_TARGET, BC_TAKE_LAST, BC_RSS,
        BC_UACC, BC_UDRAW, BC_SX, BC_TX, BC_K0, BC_K1, BC_PMAX, BC_SV, BC_P2, BC_P3, BC_P4,
        BC_QSTATE, BC_E_BETA, BC_E_G, BC_E_G1, BC_E_G2, BC_E_G3, BC_E_G4, BC_E_I7,   // an evaluation waiting for its midpoint
-       BC_NEXT,                                                                      // block verification: the CTA's next row
        BC_COUNT };
 static_assert(BC_COUNT <= BC_DOUBLES, "broadcast area too small");
 

@@ -55,7 +55,8 @@ constexpr int ROFF_STEP = ROFF_WMAX + 4 * RW * 4;                // [RW][MAX_STE
 constexpr int ROFF_FIN = ROFF_STEP + RW * MAX_STEPS * 4;          // [2][2][RW] doubles: what pass "final" leaves per warp, by row parity
 constexpr int ROFF_MBAR = ROFF_FIN + 2 * 2 * RW * 8;
 constexpr int FIN_WARP = 12;            // the warp that finishes the previous row
-constexpr int RSMEM_BYTES = ROFF_MBAR + 16;
+constexpr int ROFF_SEQ = ROFF_MBAR + 16;   // [4] ints: block verification, the CTA's reservation state
+constexpr int RSMEM_BYTES = ROFF_SEQ + 16;
 
 // L2 residency hints: the part of a row that is re-read from L2 in every pass is marked
 // evict-last; everything that passes through L2 once (the shared-memory resident part, the
@@ -300,21 +301,58 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
     __syncthreads();
   };
 
-  // Block verification hands out whole sequences: a CTA walks one sequence position by position, leaves
-  // it at the first position that is not accepted (what lies behind it is never computed: Section 3.5
-  // discards it) and takes the next sequence from a device counter.  `seqres`: [0] a sequence reserved
-  // for this CTA ahead of time (n_seq: none left), [1] 1 once thread 0 has taken it.
+  // Block verification with early out (Section 3.5 discards what lies behind a sequence's first
+  // rejection).  Positions are handed out as tickets from a device counter in position-major order
+  // (ticket = position * n_seq + sequence: all first positions, then all second ones, ...).  A row whose
+  // draft token is rejected, or that is flagged, records its position in seq_stop[sequence] (atomicMin)
+  // as soon as its decision is known; a ticket whose sequence has stopped before its position is passed
+  // over.  Nothing waits: a ticket whose predecessor is still undecided is routed anyway (the resolve
+  // step discards it if it was not needed).  `seqres`: [0] the row reserved for this CTA's next turn
+  // (n_rows: none left), [1], [2] the rest of a ticket range this CTA holds, [3] how many tickets it takes
+  // at a time: it aims at one live ticket per range (doubles after a range without one, halves after a
+  // range with several), so late positions, where most sequences have stopped, cost few round trips.
   const bool dyn = P.seq_next != nullptr;
-  const int n_seq = dyn ? (int)(P.n_rows / P.K1) : 0;
-  int* seqres = (int*)(smem + ROFF_MBAR + 8);
+  const int n_seq = dyn ? (int)(P.n_rows / P.K1) : 1;
+  const int n_tickets = (int)P.n_rows;
+  int* seqres = (int*)(smem + ROFF_SEQ);
+  auto ticket_row = [&](int tk) { const int j = tk / n_seq; return (int64_t)(tk - j * n_seq) * P.K1 + j; };
+  auto ticket_live = [&](int tk, int hi) {   // not known to lie behind its sequence's first stop
+    if (tk >= hi) return false;
+    const int j = tk / n_seq;
+    return *(volatile const int*)(P.seq_stop + (tk - j * n_seq)) >= j;
+  };
+  // warp-wide, all 32 lanes: find this CTA's next row.  Each turn of the loop takes tickets from the
+  // device counter or uses up tickets the CTA holds, so it ends without depending on any other CTA.
+  auto reserve_next = [&] {
+    int blo = seqres[1], bhi = seqres[2], n = seqres[3], res = n_tickets;
+    while (res == n_tickets) {
+      bool fresh = false;
+      if (blo >= bhi) {
+        int old = 0;
+        if (lane == 0) old = (int)min((unsigned int)n_tickets, gridDim.x + atomicAdd(P.seq_next, (unsigned int)n));
+        old = __shfl_sync(0xffffffffu, old, 0);
+        blo = old; bhi = min(old + n, n_tickets);
+        if (blo >= bhi) break;
+        fresh = true;
+      }
+      const unsigned m = __ballot_sync(0xffffffffu, ticket_live(blo + lane, bhi));   // a range is at most 32 tickets
+      if (fresh) n = m == 0 ? min(32, 2 * n) : (__popc(m) > 1 ? max(1, n / 2) : n);
+      if (m) { res = blo + __ffs(m) - 1; blo = res + 1; }
+      else blo = bhi;
+    }
+    if (lane == 0) {
+      seqres[0] = res < n_tickets ? (int)ticket_row(res) : n_tickets;
+      seqres[1] = blo; seqres[2] = bhi; seqres[3] = n;
+    }
+  };
   if (tid == 0) {
     mbar_init(mbar, RW);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    seqres[0] = 0; seqres[1] = 1;
+    seqres[0] = n_tickets; seqres[1] = 0; seqres[2] = 0; seqres[3] = 1;
   }
   __syncthreads();
   const __nv_bfloat16 *n_s = nullptr, *n_t = nullptr;   // the rows of the CTA's next position, if any
-  const int64_t first_row = dyn ? (int64_t)blockIdx.x * P.K1 : (int64_t)blockIdx.x;
+  const int64_t first_row = dyn ? ticket_row((int)blockIdx.x) : (int64_t)blockIdx.x;   // grid <= n_rows
   if (first_row < P.n_rows) {
     row_ptrs(first_row, n_s, n_t);
     if (lane == 0) issue(n_s, n_t);
@@ -462,10 +500,8 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
     auto plan_next = [&] {
       const int mode = (int)bc[BC_MODE];
       if (!dyn || mode == MODE_SOLVE) return;
-      const bool stop = bonus || mode == MODE_FLAGGED || (mode == MODE_FINAL && bc[BC_CORR] != 0.0);
-      int64_t nx = row + 1;
-      if (stop) { nx = (int64_t)seqres[0] * P.K1; seqres[1] = 1; }
-      bc[BC_NEXT] = (double)nx;
+      if (!bonus && (mode == MODE_FLAGGED || (mode == MODE_FINAL && bc[BC_CORR] != 0.0)))
+        atomicMin(P.seq_stop + seq, pos);        // verification of this sequence ends here
       atomicAdd(P.seq_next + 1, 1u);             // statistic: positions routed
     };
 #ifdef SAKI_PHASE_TIMING
@@ -602,16 +638,12 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
           bc[BC_SX] = ok ? (double)__bfloat162float(g_s[x]) : 0.0;
           bc[BC_TX] = ok ? (double)__bfloat162float(g_t[x]) : 0.0;
         }
-        if (warp == 11 && dyn && seqres[1] != 0 && seqres[0] < n_seq) {   // reserve the CTA's next sequence
-          const unsigned int nxt = gridDim.x + atomicAdd(P.seq_next, 1u);
-          seqres[0] = (int)min(nxt, (unsigned int)n_seq);
-          seqres[1] = 0;
-        }
       }
       if (any_dead) dead = true;
       __syncthreads();
       RTS(4);
       if (warp == FIN_WARP && pending_row >= 0) finish_row(pending_row, rb ^ 1);   // meanwhile: the previous row's draw and outputs
+      if (dyn && warp == 11) reserve_next();     // and the CTA's next row (block verification), while thread 0 does the scalars
       pending_row = -1;
       if (tid == 13 * 32) {   // and the student's logit at the teacher's argmax (the supervised token of a corrected row)
         const int vs = (gat[6] >= 0.0 && gat[6] < (double)V) ? (int)gat[6] : 0;
@@ -675,7 +707,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       RTS(9);
       __syncthreads();
     }
-    const int64_t next_row = dyn ? (int64_t)bc[BC_NEXT] : row + gridDim.x;
+    const int64_t next_row = dyn ? (int64_t)seqres[0] : row + gridDim.x;
     next_row_c = next_row;
     n_s = nullptr; n_t = nullptr;
     if (next_row < P.n_rows) row_ptrs(next_row, n_s, n_t);
@@ -803,12 +835,6 @@ bool rowsm_can_serve(const RowParams& p, int dtype) {
   return true;
 }
 
-int rowsm_sm_count() {
-  int dev = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-  return sms;
-}
-
 cudaError_t launch_rowsm(const RowParams& p, cudaStream_t st, int* n_launches, bool* served) {
   *served = false;
   if (p.n_rows <= 0) { *served = true; return cudaSuccess; }
@@ -826,8 +852,7 @@ cudaError_t launch_rowsm(const RowParams& p, cudaStream_t st, int* n_launches, b
       cached_dev = dev;
     }
   }
-  const int64_t units = p.seq_next ? p.n_rows / p.K1 : p.n_rows;   // sequences when they are handed out, else rows
-  const int grid = (int)(units < cached_sms ? units : cached_sms);
+  const int grid = (int)(p.n_rows < cached_sms ? p.n_rows : cached_sms);
   rowsm_kernel<<<grid, RT, RSMEM_BYTES, st>>>(p);
   cudaError_t e = cudaGetLastError();
   if (e == cudaSuccess) { *served = true; if (n_launches) *n_launches += 1; }

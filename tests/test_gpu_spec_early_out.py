@@ -1,9 +1,10 @@
 """Block verification with early out (Section 3.5: positions behind a sequence's first rejection are
-discarded).  The row-per-SM kernel hands out whole sequences and never routes the discarded positions;
-every output must be the one the call gives when it routes all positions and resolves afterwards, and
-the number of positions routed must be exactly the number that verification needs.  With fewer than two
-sequences per SM the library routes every position in static order instead (a block walks its sequence
-serially, so few sequences would leave SMs idle)."""
+discarded).  The row-per-SM kernel hands out positions in position-major order and passes over those
+whose sequence is known to have stopped; every output must be the one the call gives when it routes all
+positions and resolves afterwards, and the positions routed must cover the ones verification needs (a
+position whose predecessor was still undecided when it was handed out is routed without need: with many
+sequences per SM that is rare; with fewer than two per SM the library routes every position in static
+order instead)."""
 import numpy as np
 import pytest
 import torch
@@ -63,11 +64,14 @@ def test_outputs_do_not_depend_on_early_out(B, K, V):
     n_acc = out[True][0]["n_accept"].cpu().numpy()
     st = out[True][0]["per_pos"]["row_status"].view(B, K + 1).cpu().numpy()
     assert out[False][1] == 0
-    if B >= 2 * _sms():
-        # a sequence needs its first n_accept + 1 positions (all K + 1 if every draft token was accepted)
-        assert out[True][1] == int(np.minimum(n_acc + 1, K + 1).sum())
-    else:
+    # a sequence needs its first n_accept + 1 positions (all K + 1 if every draft token was accepted)
+    needed = int(np.minimum(n_acc + 1, K + 1).sum())
+    if B < 2 * _sms():
         assert out[True][1] == 0           # few sequences: every position routed, in static order
+        return
+    assert needed <= out[True][1] <= B * (K + 1)
+    if B >= 4 * _sms():
+        assert out[True][1] <= needed + (B * (K + 1) - needed) // 4, (needed, out[True][1])   # most of the rest is skipped
     for b in range(B):
         assert np.all(st[b, n_acc[b] + 1:] == P.binding.ROW_NOT_COMPUTED)
         assert np.all(st[b, :n_acc[b] + 1] & P.binding.ROW_NOT_COMPUTED == 0)
