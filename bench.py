@@ -45,7 +45,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one rowsm_kernel launch divided by the positions it
 # routed: ncu capture on 2220 rows of the same workload (profiles/rowsm_kernel_cfg3.md); traffic grows
 # in proportion to the rows, so a full launch is this figure times N
-TRAFFIC_BYTES_PER_POSITION = 954671
+TRAFFIC_BYTES_PER_POSITION = 953372
 # the same for one meta_stream_kernel launch (profiles/meta_stream_kernel_cfg3.md)
 META_TRAFFIC_BYTES_PER_POSITION = 586707
 
