@@ -222,11 +222,13 @@ __global__ void __launch_bounds__(MT, 1) meta_stream_kernel(const MetaParams P) 
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
   double* red = (double*)(msm + MOFF_RED);
   const int V = P.V, n_chunks = V / 8;
-  const int cpw = (n_chunks + MW - 1) / MW;
+  // whole steps of 32 chunks, dealt out in order: steps_q to every warp, one more to the first steps_r
+  // (a segment that ended inside a step would cost its warp a partly empty step in both passes)
+  const int steps_all = (n_chunks + 31) / 32, steps_q = steps_all / MW, steps_r = steps_all - steps_q * MW;
   MSeg sg;
-  sg.c0 = min(n_chunks, warp * cpw);
-  sg.c1 = min(n_chunks, sg.c0 + cpw);
-  sg.steps = (sg.c1 - sg.c0 + 31) / 32;
+  sg.steps = steps_q + (warp < steps_r ? 1 : 0);
+  sg.c0 = min(n_chunks, 32 * (warp * steps_q + min(warp, steps_r)));
+  sg.c1 = min(n_chunks, sg.c0 + 32 * sg.steps);
   sg.res = sg.steps <= MKS ? sg.steps : MRES;
   const uint32_t base = smem_addr(msm) + (uint32_t)warp * (MKS * 512) + (uint32_t)lane * 16;   // this lane's slot of step 0
   uint32_t ring_slot = base + MRES * 512;

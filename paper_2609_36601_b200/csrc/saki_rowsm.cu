@@ -267,11 +267,17 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
 
   const int V = P.V;
   const int n_chunks = V / 8;
-  const int cpw = (n_chunks + RW - 1) / RW;
+  // A row is cut into steps of 32 chunks (256 elements) and the steps are dealt out in order: every warp
+  // gets steps_q of them, the first steps_r warps one more.  Whole steps: a segment that ended inside a
+  // step would cost its warp a nearly empty step in every pass.
+  const int steps_all = (n_chunks + 31) / 32, steps_q = steps_all / RW, steps_r = steps_all - steps_q * RW;
+  auto seg_of = [&](int w, Seg& g) {
+    g.steps = steps_q + (w < steps_r ? 1 : 0);
+    g.c0 = min(n_chunks, 32 * (w * steps_q + min(w, steps_r)));
+    g.c1 = min(n_chunks, g.c0 + 32 * g.steps);
+  };
   Seg sg;
-  sg.c0 = min(n_chunks, warp * cpw);
-  sg.c1 = min(n_chunks, sg.c0 + cpw);
-  sg.steps = (sg.c1 - sg.c0 + 31) / 32;
+  seg_of(warp, sg);
   sg.res = sg.steps <= KS_MAX ? sg.steps : KS_RES;   // a segment that does not fit leaves NST steps to the ring
   const int res_chunks = min(sg.c1 - sg.c0, sg.res * 32);          // resident chunks of this warp
   const uint32_t res_bytes = (uint32_t)res_chunks * 16u;
@@ -434,9 +440,7 @@ __global__ void __launch_bounds__(RT, 1) rowsm_kernel(const RowParams P) {
       last_mode = true;
     }
     Seg so;          // the owner's segment
-    so.c0 = min(n_chunks, owner * cpw);
-    so.c1 = min(n_chunks, so.c0 + cpw);
-    so.steps = (so.c1 - so.c0 + 31) / 32;
+    seg_of(owner, so);
     const float* step_w = (const float*)(smem + ROFF_STEP) + owner * MAX_STEPS;
     const int ns = min(so.steps, MAX_STEPS);
     // the step that holds the target (every lane walks the same few numbers)

@@ -109,13 +109,20 @@ def oracle_inputs(d: dict, rows=None):
 def force_second_tier(d, rows):
     """Rewrites the given rows of a generated bf16 workload so that the row-per-SM kernel must hand them to
     the float64 kernel: a plateau 400 nats below a few peaks that sit away from the first 256 logits of
-    every warp segment, so the float32 sums of its first pass overflow."""
+    a warp's segment (steps of 256 elements dealt out in order to 16 warps), so the float32 sums of that
+    warp's first pass overflow."""
     V = d["s"].shape[1]
-    seg = ((V // 8 + 15) // 16) * 8                      # elements per warp segment (16 warps)
+    steps = (V + 255) // 256
+    q, rem = divmod(steps, 16)
+    assert q + (1 if rem else 0) >= 2, "the rows need a warp segment of two steps or more"
     g = torch.Generator(device=d["s"].device).manual_seed(1234)
     for r in rows:
+        w = (r % rem) if (rem and q < 2) else (r % 16)             # a warp whose segment has at least two steps
+        n = q + (1 if w < rem else 0)
+        lo = 256 * (w * q + min(w, rem))
+        hi = min(V, lo + 256 * n)
         s = torch.full((V,), -400.0, device=d["s"].device) + 0.5 * torch.randn(V, generator=g, device=d["s"].device)
-        pos = (torch.randint(300, max(301, seg - 8), (24,), generator=g, device=d["s"].device) + seg * (r % 16)).clamp(max=V - 1)
+        pos = torch.randint(lo + 300, max(lo + 301, hi - 8), (24,), generator=g, device=d["s"].device).clamp(max=V - 1)
         s[pos] = 2.0 * torch.randn(24, generator=g, device=d["s"].device)
         t = s + 0.7 * torch.randn(V, generator=g, device=d["s"].device)
         d["s"][r] = s.to(d["s"].dtype)

@@ -118,9 +118,12 @@ def test_wide_range_rows_take_the_float64_kernel():
     N, V = 6, 40000
     g = torch.Generator(device=DEV).manual_seed(9)
     s = torch.full((N, V), -400.0, device=DEV) + 0.5 * torch.randn((N, V), generator=g, device=DEV)
-    seg = ((V // 8 + 31) // 32) * 8        # elements per warp segment of the streaming kernel (32 warps)
-    for i in range(N):                     # peaks away from the first 256 logits of every segment
-        pos = torch.randint(400, 1200, (30,), generator=g, device=DEV) + seg * (5 * i)
+    # the streaming kernel deals the row's 157 steps of 256 elements out in order to its 32 warps: 5 steps each
+    # to the first 29, 4 to the others
+    for i in range(N):                     # peaks away from the first 256 logits of a warp's segment
+        wi = 5 * i
+        start = 256 * (4 * wi + min(wi, 29))
+        pos = torch.randint(400, 1000, (30,), generator=g, device=DEV) + start
         s[i, pos] = 2.0 * torch.randn((30,), generator=g, device=DEV)
     s = s.to(torch.bfloat16)
     C, x, vs, A = _meta(N, V, 13)

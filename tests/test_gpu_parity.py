@@ -264,8 +264,11 @@ def test_wide_range_rows(gap):
         s = torch.full((N, V), -gap, device=DEV) + 0.5 * torch.randn((N, V), generator=gen, device=DEV)
         t = s + 0.5 * torch.randn((N, V), generator=gen, device=DEV)
         for i in range(N):
-            # peaks away from the starts of the 16 warp segments (V / 16 = 2500 elements each)
-            pos = torch.randint(400, 2400, (40,), generator=gen, device=DEV) + 2500 * (i % 16)
+            # peaks away from the start of a warp's segment (157 steps of 256 elements dealt out in order:
+            # 10 steps each to the first 13 warps, 9 to the others)
+            wi = i % 16
+            start = 256 * (9 * wi + min(wi, 13))
+            pos = (torch.randint(400, 2200, (40,), generator=gen, device=DEV) + start).clamp(max=V - 1)
             s[i, pos] = 2.0 * torch.randn((40,), generator=gen, device=DEV)
             t[i, pos] = s[i, pos] + 1.5 * torch.randn((40,), generator=gen, device=DEV)
         s, t = s.to(torch.bfloat16), t.to(torch.bfloat16)
