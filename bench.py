@@ -45,9 +45,9 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one rowsm_kernel launch divided by the positions it
 # routed: ncu capture on 2220 rows of the same workload (profiles/rowsm_kernel_cfg3.md); traffic grows
 # in proportion to the rows, so a full launch is this figure times N
-TRAFFIC_BYTES_PER_POSITION = 953372
+TRAFFIC_BYTES_PER_POSITION = 946367
 # the same for one meta_stream_kernel launch (profiles/meta_stream_kernel_cfg3.md)
-META_TRAFFIC_BYTES_PER_POSITION = 586707
+META_TRAFFIC_BYTES_PER_POSITION = 581514
 
 
 def _peaks():
