@@ -106,20 +106,26 @@ def oracle_inputs(d: dict, rows=None):
     return to_np64(s), to_np64(t)
 
 
+def warp_segments(V):
+    """How the row-per-SM kernel deals a row of V elements out to its warps: steps of 256 elements in order,
+    steps // W to every warp and one more to the first steps % W; W = 8 warps (two CTAs per SM) up to
+    V = 98304, 16 beyond.  Returns [(first element, number of steps)] per warp."""
+    W = 8 if V <= 98304 else 16
+    steps = (V + 255) // 256
+    q, rem = divmod(steps, W)
+    return [(256 * (w * q + min(w, rem)), q + (1 if w < rem else 0)) for w in range(W)]
+
+
 def force_second_tier(d, rows):
     """Rewrites the given rows of a generated bf16 workload so that the row-per-SM kernel must hand them to
     the float64 kernel: a plateau 400 nats below a few peaks that sit away from the first 256 logits of
-    a warp's segment (steps of 256 elements dealt out in order to 16 warps), so the float32 sums of that
-    warp's first pass overflow."""
+    a warp's segment, so the float32 sums of that warp's first pass overflow."""
     V = d["s"].shape[1]
-    steps = (V + 255) // 256
-    q, rem = divmod(steps, 16)
-    assert q + (1 if rem else 0) >= 2, "the rows need a warp segment of two steps or more"
+    segs = [sg for sg in warp_segments(V) if sg[1] >= 2]
+    assert segs, "the rows need a warp segment of two steps or more"
     g = torch.Generator(device=d["s"].device).manual_seed(1234)
     for r in rows:
-        w = (r % rem) if (rem and q < 2) else (r % 16)             # a warp whose segment has at least two steps
-        n = q + (1 if w < rem else 0)
-        lo = 256 * (w * q + min(w, rem))
+        lo, n = segs[r % len(segs)]
         hi = min(V, lo + 256 * n)
         s = torch.full((V,), -400.0, device=d["s"].device) + 0.5 * torch.randn(V, generator=g, device=d["s"].device)
         pos = torch.randint(lo + 300, max(lo + 301, hi - 8), (24,), generator=g, device=d["s"].device).clamp(max=V - 1)

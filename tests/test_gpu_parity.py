@@ -6,7 +6,7 @@ import torch
 import oracle as O
 import paper_2609_36601_b200 as P
 from paper_2609_36601_b200 import synth
-from parity import compare_rows, force_second_tier, grad_check, oracle_inputs, to_np64
+from parity import compare_rows, force_second_tier, grad_check, oracle_inputs, to_np64, warp_segments
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -264,11 +264,10 @@ def test_wide_range_rows(gap):
         s = torch.full((N, V), -gap, device=DEV) + 0.5 * torch.randn((N, V), generator=gen, device=DEV)
         t = s + 0.5 * torch.randn((N, V), generator=gen, device=DEV)
         for i in range(N):
-            # peaks away from the start of a warp's segment (157 steps of 256 elements dealt out in order:
-            # 10 steps each to the first 13 warps, 9 to the others)
-            wi = i % 16
-            start = 256 * (9 * wi + min(wi, 13))
-            pos = (torch.randint(400, 2200, (40,), generator=gen, device=DEV) + start).clamp(max=V - 1)
+            # peaks away from the first 256 logits of a warp's segment
+            segs = warp_segments(V)
+            start, nsteps = segs[i % len(segs)]
+            pos = (torch.randint(400, 256 * nsteps - 100, (40,), generator=gen, device=DEV) + start).clamp(max=V - 1)
             s[i, pos] = 2.0 * torch.randn((40,), generator=gen, device=DEV)
             t[i, pos] = s[i, pos] + 1.5 * torch.randn((40,), generator=gen, device=DEV)
         s, t = s.to(torch.bfloat16), t.to(torch.bfloat16)
