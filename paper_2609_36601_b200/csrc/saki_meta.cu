@@ -127,15 +127,21 @@ cudaError_t launch_meta_general(const MetaParams& p, int dtype, cudaStream_t st,
 }
 
 // ---------------------------------------------------------------- streaming kernel (bf16)
-constexpr int MT = 1024;                 // threads per CTA
-constexpr int MW = MT / 32;              // warps
+// The kernel is instantiated for 32 warps (one CTA per SM) and for 16 warps (two CTAs per SM, for short
+// rows: one CTA's block barriers and scalar step run under the other's passes).
+constexpr int MW_FULL = 32, MW_HALF = 16;
+#ifndef SAKI_META_HALF_MAX_V
+#define SAKI_META_HALF_MAX_V 98304   /* M positions/s, one / two CTAs per SM: V = 8192 52 / 77, 32000 30.8 / 37.5,
+                                        50048 23.2 / 27.0, 65536 19.5 / 19.9, 131072 10.5 / 10.6, 151936 9.1 / 8.8 */
+#endif
+constexpr int M_HALF_MAX_V = SAKI_META_HALF_MAX_V;   // rows up to this length take the 16-warp instance
 constexpr int MKS = 13;                  // 512-byte steps of shared memory per warp (a step = 32 chunks of 8 elements)
 constexpr int MNST = 5;                  // ring stages of a warp whose segment does not fit
 constexpr int MRES = MKS - MNST;         // resident steps of such a warp
 constexpr int M_MAX_STEPS = 64;          // V <= 64 * 32 * 8 * MW
-constexpr int MOFF_RED = MW * MKS * 512; // [3][MW] doubles: per-warp sum, shift, maximum
-constexpr int MOFF_BC = MOFF_RED + 3 * MW * 8;       // [2][8] floats: the row's broadcast scalars, by row parity
-constexpr int MSMEM_BYTES = MOFF_BC + 2 * 8 * 4;
+__host__ __device__ constexpr int moff_red(int MW) { return MW * MKS * 512; }              // [3][MW] doubles: per-warp sum, shift, maximum
+__host__ __device__ constexpr int moff_bc(int MW) { return moff_red(MW) + 3 * MW * 8; }    // [2][8] floats: the row's broadcast scalars, by row parity
+__host__ __device__ constexpr int msmem_bytes(int MW) { return moff_bc(MW) + 2 * 8 * 4; }
 constexpr uint32_t M_FILLER = 0xFF7FFF7Fu;           // two bf16 of the most negative finite value: exp -> 0
 
 __device__ __forceinline__ void m_cp_async16(uint32_t dst, const void* src, uint64_t pol) {
@@ -216,7 +222,9 @@ __device__ __forceinline__ void m_visit(const MSeg& sg, int lane, uint32_t base,
   }
 }
 
-__global__ void __launch_bounds__(MT, 1) meta_stream_kernel(const MetaParams P) {
+template <int MW>
+__global__ void __launch_bounds__(MW * 32, MW_FULL / MW) meta_stream_kernel(const MetaParams P) {
+  constexpr int MOFF_RED = moff_red(MW), MOFF_BC = moff_bc(MW);
   extern __shared__ __align__(128) unsigned char msm[];
   const int tid = threadIdx.x, lane = tid & 31;
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
@@ -315,12 +323,13 @@ __global__ void __launch_bounds__(MT, 1) meta_stream_kernel(const MetaParams P) 
     if (warp == 0) {
       // the row's shift is that of its true maximum; a warp's shift came from an element of the row, so
       // it is never below the row's and the factors are exact powers of two <= 1
-      float mx = (float)red[2 * MW + lane];
+      const int wl = lane < MW ? lane : 0;        // lanes beyond the warp count carry nothing
+      float mx = lane < MW ? (float)red[2 * MW + wl] : -CUDART_INF_F;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
       const float kr = -ceilf(c32 * fmaxf(mx, -1e30f));
-      const double kw = red[MW + lane];
-      double sum = kw < 1e29 ? red[lane] * (double)m_pow2(kr - (float)kw) : 0.0;
+      const double kw = lane < MW ? red[MW + wl] : 1e30;
+      double sum = kw < 1e29 ? red[wl] * (double)m_pow2(kr - (float)kw) : 0.0;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
       if (lane == 0) {
@@ -385,7 +394,7 @@ __global__ void __launch_bounds__(MT, 1) meta_stream_kernel(const MetaParams P) 
 
 bool meta_stream_can_serve(const MetaParams& p, int dtype) {
   if (dtype != SAKI_BF16) return false;
-  if (p.V < 2048 || p.V % 8 != 0 || p.V > M_MAX_STEPS * 32 * 8 * MW) return false;
+  if (p.V < 2048 || p.V % 8 != 0 || p.V > M_MAX_STEPS * 32 * 8 * MW_FULL) return false;
   if (p.n_rows > 0x7fffffffLL) return false;
   auto al16 = [](const void* q) { return ((uintptr_t)q & 15) == 0; };
   if (!al16(p.s) || !al16(p.dlogits)) return false;
@@ -393,9 +402,8 @@ bool meta_stream_can_serve(const MetaParams& p, int dtype) {
   return true;
 }
 
-cudaError_t launch_meta_stream(const MetaParams& p, cudaStream_t st, int* n_launches, bool* served) {
-  *served = false;
-  if (p.n_rows <= 0) { *served = true; return cudaSuccess; }
+template <int MW>
+static cudaError_t launch_meta_stream_as(const MetaParams& p, cudaStream_t st) {
   static std::mutex mu;
   static int cached_dev = -1, cached_sms = 0;
   int dev = 0;
@@ -403,18 +411,25 @@ cudaError_t launch_meta_stream(const MetaParams& p, cudaStream_t st, int* n_laun
   {
     std::lock_guard<std::mutex> lock(mu);
     if (cached_dev != dev) {
-      cudaError_t e = cudaFuncSetAttribute(meta_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MSMEM_BYTES);
+      cudaError_t e = cudaFuncSetAttribute(meta_stream_kernel<MW>, cudaFuncAttributeMaxDynamicSharedMemorySize, msmem_bytes(MW));
       if (e != cudaSuccess) return e;
       e = cudaDeviceGetAttribute(&cached_sms, cudaDevAttrMultiProcessorCount, dev);
       if (e != cudaSuccess) return e;
       cached_dev = dev;
     }
   }
-  const int grid = (int)std::min<int64_t>(p.n_rows, cached_sms);
-  meta_stream_kernel<<<grid, MT, MSMEM_BYTES, st>>>(p);
+  const int grid = (int)std::min<int64_t>(p.n_rows, (int64_t)cached_sms * (MW_FULL / MW));
+  meta_stream_kernel<MW><<<grid, MW * 32, msmem_bytes(MW), st>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_meta_stream(const MetaParams& p, cudaStream_t st, int* n_launches, bool* served) {
+  *served = false;
+  if (p.n_rows <= 0) { *served = true; return cudaSuccess; }
+  const cudaError_t e = p.V <= M_HALF_MAX_V ? launch_meta_stream_as<MW_HALF>(p, st) : launch_meta_stream_as<MW_FULL>(p, st);
   ++*n_launches;
   *served = true;
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace saki

@@ -118,12 +118,14 @@ def test_wide_range_rows_take_the_float64_kernel():
     N, V = 6, 40000
     g = torch.Generator(device=DEV).manual_seed(9)
     s = torch.full((N, V), -400.0, device=DEV) + 0.5 * torch.randn((N, V), generator=g, device=DEV)
-    # the streaming kernel deals the row's 157 steps of 256 elements out in order to its 32 warps: 5 steps each
-    # to the first 29, 4 to the others
+    # the streaming kernel deals the row's steps of 256 elements out in order to its warps (16 per block up to
+    # V = 98304, 32 beyond): steps // W each, one more to the first steps % W
+    W = 16 if V <= 98304 else 32
+    q, rem = divmod((V + 255) // 256, W)
     for i in range(N):                     # peaks away from the first 256 logits of a warp's segment
-        wi = 5 * i
-        start = 256 * (4 * wi + min(wi, 29))
-        pos = torch.randint(400, 1000, (30,), generator=g, device=DEV) + start
+        wi = (5 * i) % W
+        start = 256 * (q * wi + min(wi, rem))
+        pos = (torch.randint(400, 256 * q - 50, (30,), generator=g, device=DEV) + start).clamp(max=V - 1)
         s[i, pos] = 2.0 * torch.randn((30,), generator=g, device=DEV)
     s = s.to(torch.bfloat16)
     C, x, vs, A = _meta(N, V, 13)
