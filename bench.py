@@ -46,6 +46,9 @@ FALLBACK_HBM_GBS = 6650.0
 # routed: ncu capture on 2220 rows of the same workload (profiles/rowsm_kernel_cfg3.md); traffic grows
 # in proportion to the rows, so a full launch is this figure times N
 TRAFFIC_BYTES_PER_POSITION = 946367
+# rows up to this length are served by the instances of the two streaming kernels that run two CTAs per SM
+# (namespace half_sm, meta_stream_kernel<16>); the names below are the ones a profiler shows
+TWO_CTA_MAX_V = 98304
 # the same for one meta_stream_kernel launch (profiles/meta_stream_kernel_cfg3.md)
 META_TRAFFIC_BYTES_PER_POSITION = 581514
 
@@ -242,7 +245,7 @@ def run_ours(args):
         mms = m0.elapsed_time(m1) / args.steps
         mbytes = 2 * w.V * s.element_size() * w.N
         nxt = {"call": "saki_route_bwd_from_meta", "value": w.N / (mms * 1e-3), "unit": UNIT, "ms_per_step": mms,
-               "gpu_launches": int(P.launch_count() - l1), "kernel": {4: "saki::meta_stream_kernel"}.get(P.last_kernel(), "saki::meta_general_kernel"),
+               "gpu_launches": int(P.launch_count() - l1), "kernel": {4: "saki::meta_stream_kernel<%d>" % (16 if w.V <= TWO_CTA_MAX_V else 32)}.get(P.last_kernel(), "saki::meta_general_kernel"),
                "algorithmic_bytes_per_launch": mbytes, "achieved_gbs": mbytes / (mms * 1e-3) / 1e9,
                "traffic": META_TRAFFIC_BYTES_PER_POSITION * w.N if META_TRAFFIC_BYTES_PER_POSITION else None}
 
@@ -322,7 +325,8 @@ def run_ours(args):
                 "peak_kind": f"of {peak_kind} (device-to-device copy, MEASURED_PEAKS.json)"
                 if peak_kind == "measured" else "of fallback",
                 "traffic": (TRAFFIC_BYTES_PER_POSITION * w.N) if TRAFFIC_BYTES_PER_POSITION else None,
-                "algorithmic_bytes_per_launch": bpp * w.N, "kernel": {3: "saki::rowsm_kernel", 2: "saki::cluster_kernel"}.get(kernel_used, "saki::general_kernel"),
+                "algorithmic_bytes_per_launch": bpp * w.N, "kernel": {3: "saki::%s::rowsm_kernel" % ("half_sm" if w.V <= TWO_CTA_MAX_V else "full_sm"),
+                           2: "saki::cluster_kernel"}.get(kernel_used, "saki::general_kernel"),
                 "kernel_ms": kern_ms,
                 "frac_of_nominal_8TBs": achieved / 8000.0}
     if kernel_used == 3:
