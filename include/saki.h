@@ -266,7 +266,8 @@ SAKI_API int saki_check(void* cuda_stream, uint64_t* n_flagged);
 /* Selects the row kernel: 0 = automatic, 1 = the general kernel (one block per
  * row, float64, any V, dtype and layout), 2 = the register-resident cluster
  * kernel (one row per cluster of up to 8 blocks), 3 = the row-per-SM kernel
- * (one row per block; shared memory plus L2).  2 and 3 serve bf16 rows with
+ * (one row per block; shared memory plus L2; one block of 512 threads per SM for
+ * V > 98304, two of 256 for shorter rows).  2 and 3 serve bf16 rows with
  * 16-byte aligned rows and V a multiple of 8, V >= 2048 (2: V <= 163840; and
  * eps = 0 or eps >= 5e-3: its float32 sums cannot resolve smaller radii to the
  * tolerance, whereas 3 takes every radius); other inputs fall back to 1.  Automatic prefers 3.  Process-wide; meant for
