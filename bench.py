@@ -45,12 +45,12 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one rowsm_kernel launch divided by the positions it
 # routed: ncu capture on 2220 rows of the same workload (profiles/rowsm_kernel_cfg3.md); traffic grows
 # in proportion to the rows, so a full launch is this figure times N
-TRAFFIC_BYTES_PER_POSITION = 946367
+TRAFFIC_BYTES_PER_POSITION = 945005
 # rows up to this length are served by the instances of the two streaming kernels that run two CTAs per SM
 # (namespace half_sm, meta_stream_kernel<16>); the names below are the ones a profiler shows
 TWO_CTA_MAX_V = 98304
 # the same for one meta_stream_kernel launch (profiles/meta_stream_kernel_cfg3.md)
-META_TRAFFIC_BYTES_PER_POSITION = 581514
+META_TRAFFIC_BYTES_PER_POSITION = 581046
 
 
 def _peaks():
