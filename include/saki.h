@@ -270,7 +270,9 @@ SAKI_API int saki_check(void* cuda_stream, uint64_t* n_flagged);
  * V > 98304, two of 256 for shorter rows).  2 and 3 serve bf16 rows with
  * 16-byte aligned rows and V a multiple of 8, V >= 2048 (2: V <= 163840; and
  * eps = 0 or eps >= 5e-3: its float32 sums cannot resolve smaller radii to the
- * tolerance, whereas 3 takes every radius); other inputs fall back to 1.  Automatic prefers 3.  Process-wide; meant for
+ * tolerance, whereas 3 takes every radius); other inputs fall back to 1.  Automatic prefers 3,
+ * except for calls of at most 32 rows with V >= 65536 that 2 can serve: a few long rows finish sooner
+ * spread over the whole GPU.  Process-wide; meant for
  * tests and benchmarks.  Returns the previous value. */
 SAKI_API int saki_set_kernel(int which);
 

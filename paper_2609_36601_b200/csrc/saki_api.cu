@@ -150,7 +150,16 @@ static int dispatch_rows(RowParams p, int dtype, cudaStream_t st, int32_t* scrat
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
     g_last_redo_count = p.redo_count;
   }
-  if (fast && (which == 0 || which == 3) && rowsm_can_serve(p, dtype)) {
+  // A handful of long rows (a decoding step of a small batch) finish sooner spread over the whole GPU, one
+  // row per cluster of 8 blocks, than on one SM each: 32 clusters fit at once, and at V = 151936 a call of
+  // up to 32 rows takes 32 to 40 us there against 62 us (V = 65536: 28 to 34 against 33 to 39; at V = 32000
+  // the row-per-SM kernel is the faster one at every size).
+  if (fast && which == 0 && p.n_rows <= 32 && p.V >= 65536 && eps_ok && cluster_can_serve(p, dtype)) {
+    e = launch_cluster(p, st, &launches, &served);
+    if (e != cudaSuccess) return cuda_fail(e, "cluster kernel launch");
+    if (served) used = 2;
+  }
+  if (fast && !served && (which == 0 || which == 3) && rowsm_can_serve(p, dtype)) {
     // Block verification with early out: positions handed out as tickets, sequences record their first stop.
     // Only with two or more sequences per SM: with fewer, most positions are handed out before their
     // predecessor's decision is known, and the bookkeeping costs more than the few skipped rows save.

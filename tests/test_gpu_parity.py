@@ -365,3 +365,26 @@ def test_evaluation_pass_counter():
         assert P.solve_evaluations() == 0      # another kernel served the call
     finally:
         P.set_kernel(prev)
+
+
+def test_small_batches_of_long_rows_take_the_cluster_kernel():
+    """Automatic dispatch: up to 32 rows with V >= 65536 go one row per cluster (lower latency for a decoding
+    step of a small batch); more rows, shorter rows or a radius the cluster kernel cannot resolve do not."""
+    prev = P.set_kernel(0)
+    try:
+        w = synth.Workload("t", 12, 65536, "bf16", 0.1, 1.5, True, 611, 41)
+        d = synth.generate(w, DEV)
+        _check_fwd_bwd(d, w)
+        assert P.last_kernel() == 2
+        _check_fwd_bwd(d, w, eps=1e-3)               # below the cluster kernel's smallest radius
+        assert P.last_kernel() == 3
+        w2 = synth.Workload("t", 33, 65536, "bf16", 0.1, 1.5, True, 612, 42)
+        d2 = synth.generate(w2, DEV)
+        P.route_fwd(d2["s"], d2["t"], d2["proposal"], w2.eps, seed=w2.seed)
+        assert P.last_kernel() == 3
+        w3 = synth.Workload("t", 12, 32000, "bf16", 0.1, 1.5, True, 613, 43)
+        d3 = synth.generate(w3, DEV)
+        P.route_fwd(d3["s"], d3["t"], d3["proposal"], w3.eps, seed=w3.seed)
+        assert P.last_kernel() == 3
+    finally:
+        P.set_kernel(prev)
