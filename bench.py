@@ -15,10 +15,10 @@ positions: one saki_route_fwd_bwd call.  Prints ONE JSON line.
             gradient row once) / measured kernel time, against the measured
             copy bandwidth of this machine's B200s
   cpu_baseline  the float64 test oracle, as it stands, on a bounded sample
-  next_step, spec_verify  (rank 0, unless --no-next) two further calls timed the
-            same way beside the headline: saki_route_bwd_from_meta on the same
-            logits, and saki_spec_verify on its own workload with and without
-            early out
+  next_step, spec_verify, small_batch  (rank 0, unless --no-next) further calls
+            timed the same way beside the headline: saki_route_bwd_from_meta on
+            the same logits, saki_spec_verify on its own workload with and
+            without early out, and the latency of saki_route_fwd on 8 rows
 
 With N > 1 (under torchrun) every rank routes its own batch of the same
 shape (rows are independent: no collective on the data path); the time is
@@ -281,6 +281,24 @@ def run_ours(args):
         P.set_spec_early_out(prev)
         del d5, s5, t5
 
+    # ---- latency of a decoding step of a small batch: saki_route_fwd on the first 8 rows (forward only, as
+    # at rollout time); automatic dispatch sends so few long rows to the cluster kernel
+    small = None
+    if not args.no_next and rank == 0 and w.N >= 8:
+        s8, t8, x8 = s[:8], t[:8], x[:8]
+        o8 = None
+        for _ in range(5):
+            o8 = P.route_fwd(s8, t8, x8, w.eps, w.temperature, w.seed, row_offset, out=o8, stream=stream)
+        torch.cuda.synchronize()
+        q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        q0.record(stream)
+        for _ in range(50):
+            P.route_fwd(s8, t8, x8, w.eps, w.temperature, w.seed, row_offset, out=o8, stream=stream)
+        q1.record(stream)
+        torch.cuda.synchronize()
+        small = {"call": "saki_route_fwd", "rows": 8, "us_per_call": q0.elapsed_time(q1) / 50 * 1e3,
+                 "kernel": {2: "saki::cluster_kernel", 3: "saki::rowsm_kernel"}.get(P.last_kernel(), "saki::general_kernel")}
+
     # ---- end to end: host buffers through saki_route_host
     e2e = None
     if not args.no_e2e:
@@ -370,6 +388,8 @@ def run_ours(args):
         line["next_step"] = nxt
     if spec is not None:
         line["spec_verify"] = spec
+    if small is not None:
+        line["small_batch"] = small
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
