@@ -215,7 +215,7 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
         issue(next);
       }
       mbar_expect_tx(&mbar[3 + rb], (uint32_t)(CS * 16));          // maxima of all CTAs
-      mbar_expect_tx(&mbar[1 + parity], (uint32_t)(CS * CW * 7 * 8));   // partials of pass "lse"
+      mbar_expect_tx(&mbar[1 + parity], (uint32_t)(CS * CW * 8 * 8));   // partials of pass "lse"
     }
     float ms_r = wmax[(rb * 2 + 0) * CW], mt_r = wmax[(rb * 2 + 1) * CW];
 #pragma unroll
@@ -263,7 +263,8 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
     float k0, k1;        // the row's shifts
     bool row_timeout;
     {
-      float2 Ss = splat(0.f), St = splat(0.f), M1 = splat(0.f), M2 = splat(0.f), M3 = splat(0.f), N1 = splat(0.f);
+      float2 Ss = splat(0.f), St = splat(0.f), M1 = splat(0.f), M2 = splat(0.f), M3 = splat(0.f), M4 = splat(0.f),
+             N1 = splat(0.f);
       const float2 cc = splat(c32), kk0 = splat(k0r), kk1 = splat(k1r), neg1 = splat(-1.f);
 #pragma unroll
       for (int i = 0; i < NPAIR; ++i) {
@@ -278,6 +279,7 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
         const float2 t2 = fmul2(t1, d);
         M2 = fadd2(M2, t2);
         M3 = ffma2(t2, d, M3);
+        M4 = ffma2(t2, fmul2(d, d), M4);
         N1 = ffma2(et, d, N1);
       }
       // the row's maxima have arrived meanwhile: move the partial sums onto the row's shifts
@@ -298,14 +300,15 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
       k0 = -ceilf(c32 * fmaxf(gms, -1e30f)); k1 = -ceilf(c32 * fmaxf(gmt, -1e30f));
       const double fs = pow2_exact((int)(k0 - k0r)), ft = pow2_exact((int)(k1 - k1r));
       auto tot = [](const float2 a) { return (double)a.x + (double)a.y; };
-      double v[7] = {fs * tot(Ss), ft * tot(St), fs * tot(M1), fs * tot(M2), fs * tot(M3), ft * tot(N1),
-                     (mt_r == gmt) ? cand : CUDART_INF};
+      double v[8] = {fs * tot(Ss), ft * tot(St), fs * tot(M1), fs * tot(M2), fs * tot(M3), ft * tot(N1),
+                     (mt_r == gmt) ? cand : CUDART_INF, fs * tot(M4)};
 #pragma unroll
       for (int k = 0; k < 6; ++k) v[k] = warp_sum(v[k]);
       v[6] = warp_min(v[6]);
-      push(v, 7, parity);
+      v[7] = warp_sum(v[7]);
+      push(v, 8, parity);
       TS(5);
-      if (warp < 7) {
+      if (warp < 8) {
         if (!mbar_wait_bounded(&mbar[1 + parity], parity ? xph1 : xph0)) dead = true;
         TS(6);
         const double g = gather(parity, warp, warp == 6);
@@ -316,8 +319,8 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
       __syncthreads();
       TS(7);
       if (tid == 0) {
-        scalar_after_lse(bc, gat, K, k0, k1, x, bonus, masked, row_timeout);
-        if ((int)bc[BC_MODE] == MODE_SOLVE) mbar_expect_tx(&mbar[1 + parity], (uint32_t)(CS * CW * 3 * 8));
+        scalar_after_lse(bc, gat, K, k0, k1, x, bonus, masked, row_timeout, gat + 7);
+        if ((int)bc[BC_MODE] == MODE_SOLVE) mbar_expect_tx(&mbar[1 + parity], (uint32_t)(CS * CW * 5 * 8));
         else if ((int)bc[BC_MODE] == MODE_FINAL) mbar_expect_tx(&mbar[1 + parity], (uint32_t)(CS * CW * 3 * 8));
       }
       TS(8);
@@ -327,7 +330,8 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
     // ------------------------------------------------ pass "solve" (repeated)
     while ((int)bc[BC_MODE] == MODE_SOLVE) {
       const float cb = (float)bc[BC_CB], kb = (float)bc[BC_KB];
-      float2 S0[2] = {splat(0.f), splat(0.f)}, S1[2] = {splat(0.f), splat(0.f)}, S2[2] = {splat(0.f), splat(0.f)};
+      float2 S0[2] = {splat(0.f), splat(0.f)}, S1[2] = {splat(0.f), splat(0.f)}, S2[2] = {splat(0.f), splat(0.f)},
+             S3[2] = {splat(0.f), splat(0.f)}, S4[2] = {splat(0.f), splat(0.f)};
       const float2 cc = splat(c32), cbb = splat(cb), kbb = splat(kb), neg1 = splat(-1.f);
 #pragma unroll
       for (int i = 0; i < NPAIR; ++i) {
@@ -338,13 +342,16 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
         S0[h] = fadd2(S0[h], e);
         const float2 t1 = fmul2(e, d);
         S1[h] = fadd2(S1[h], t1);
-        S2[h] = ffma2(t1, d, S2[h]);
+        const float2 t2 = fmul2(t1, d);
+        S2[h] = fadd2(S2[h], t2);
+        S3[h] = ffma2(t2, d, S3[h]);
+        S4[h] = ffma2(t2, fmul2(d, d), S4[h]);
       }
       auto tot = [](const float2 (&a)[2]) { return ((double)a[0].x + (double)a[0].y) + ((double)a[1].x + (double)a[1].y); };
       TS(9);
-      double v[3] = {warp_sum(tot(S0)), warp_sum(tot(S1)), warp_sum(tot(S2))};
-      push(v, 3, parity);
-      if (warp < 3) {
+      double v[5] = {warp_sum(tot(S0)), warp_sum(tot(S1)), warp_sum(tot(S2)), warp_sum(tot(S3)), warp_sum(tot(S4))};
+      push(v, 5, parity);
+      if (warp < 5) {
         if (!mbar_wait_bounded(&mbar[1 + parity], parity ? xph1 : xph0)) dead = true;
         TS(10);
         const double g = gather(parity, warp, false);
@@ -355,9 +362,9 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
       __syncthreads();
       TS(11);
       if (tid == 0) {
-        scalar_after_solve(bc, gat, K, k0, k1, x, bonus, masked);
-        if ((int)bc[BC_MODE] == MODE_SOLVE || (int)bc[BC_MODE] == MODE_FINAL)
-          mbar_expect_tx(&mbar[1 + parity], (uint32_t)(CS * CW * 3 * 8));   // next evaluation, or pass "final"
+        scalar_after_solve4(bc, gat, K, k0, k1, x, bonus, masked);
+        if ((int)bc[BC_MODE] == MODE_SOLVE) mbar_expect_tx(&mbar[1 + parity], (uint32_t)(CS * CW * 5 * 8));   // next evaluation
+        else if ((int)bc[BC_MODE] == MODE_FINAL) mbar_expect_tx(&mbar[1 + parity], (uint32_t)(CS * CW * 3 * 8));   // pass "final"
       }
       TS(12);
       __syncthreads();

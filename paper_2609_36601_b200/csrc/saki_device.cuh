@@ -282,57 +282,11 @@ static __device__ __noinline__ void scalar_after_lse_tail(double* bc, const doub
 }
 
 static __device__ __noinline__ void scalar_after_lse(double* bc, const double* v, Consts K, float k0f, float k1f, int x,
-                                              bool bonus, bool masked, bool row_timeout) {
+                                              bool bonus, bool masked, bool row_timeout, const double* m4_raw = nullptr) {
   double rSs, rSt, G0, G1;
   lse_of_sum(v[0], (double)k0f, rSs, G0);
   lse_of_sum(v[1], (double)k1f, rSt, G1);
-  scalar_after_lse_tail(bc, v, K, k0f, k1f, x, bonus, masked, row_timeout, 1.f, false, rSs, rSt, G0, G1);
-}
-
-// after one evaluation of pass "solve": safeguarded Newton step on sqrt(KL); v = {S0, S1, S2}
-static __device__ __noinline__ void scalar_after_solve(double* bc, const double* v, Consts K, float k0f, float k1f, int x,
-                                                bool bonus, bool masked) {
-  const double eps = K.eps, rtau = K.rtau;
-  const double beta = bc[BC_BETA], G0 = bc[BC_G0], kb = bc[BC_KB];
-  double lo = bc[BC_LO], hi = bc[BC_HI];
-  const int iter = (int)bc[BC_ITER] + 1;
-  if (!(fabs(v[0] + v[1] + v[2]) < CUDART_INF)) { bc[BC_MODE] = MODE_REDO; return; }   // float32 sums overflowed
-  const double r0 = rcp_fast(v[0]);
-  const double G = LN2 * (log2_fast(v[0]) - kb);
-  const double mu = v[1] * r0, var = fmax(v[2] * r0 - mu * mu, 0.0);
-  const double kl = beta * mu * rtau - G + G0;          // KL(q_beta || p)
-  const double slope = beta * var * rtau * rtau;        // d KL / d beta
-  if (kl <= eps) lo = fmax(lo, beta); else hi = fmin(hi, beta);
-  // KL is nearly quadratic in beta, so its square root is nearly linear: Newton on sqrt(KL).
-  // The step is a correction, so float32 suffices for it once eps - KL is formed in float64.
-  double step;
-  if (slope > 1e-30 && kl > 1e-30 && kl < 1e30) {
-    const float rk = sqrtf((float)kl);
-    step = (double)__fdividef((float)(eps - kl) * (2.f * rk), (K.sqrt_eps + rk) * (float)slope);
-  } else step = 0.5 * (lo + hi) - beta;
-  double nb = beta + step;
-  bool bisected = false;
-  if (!(nb > lo && nb < hi)) { nb = 0.5 * (lo + hi); bisected = true; }
-  const bool done = (!bisected && fabs(nb - beta) <= 2e-4 * beta) || iter >= 40 || (hi - lo) < 1e-9;
-  // The float32 sums resolve KL to a few 1e-7 x (largest probability).  Where that would move lambda by
-  // more than the tolerance (a very flat KL: nearly one-hot rows), or the solve did not converge, the row
-  // is handed to the float64 kernel.
-  if (done && (3e-7 * bc[BC_PMAX] > 1e-5 * slope || iter >= 40)) { bc[BC_MODE] = MODE_REDO; return; }
-  if (done) {
-    const float cl = (float)(K.c64 * nb);
-    const double lam = (double)cl * K.rc64;
-    const double dle = lam - beta;
-    // second-order predictions at lambda from this evaluation
-    bc[BC_KL] = kl + dle * slope;
-    decide(bc, K, lam, G + dle * mu * rtau + 0.5 * dle * dle * var * rtau * rtau, G0, bc[BC_G1], (double)k0f,
-           (double)k1f, bc[BC_RSS], (uint32_t)bc[BC_STATUS], (int)bc[BC_VSTAR], bonus, masked, x);
-  } else {
-    const float cbn = (float)(K.c64 * nb);
-    const double be = (double)cbn * K.rc64;
-    bc[BC_BETA] = be; bc[BC_CB] = (double)cbn;
-    bc[BC_KB] = (double)(float)((1.0 - be) * (double)k0f + be * (double)k1f);
-    bc[BC_LO] = lo; bc[BC_HI] = hi; bc[BC_ITER] = (double)iter;
-  }
+  scalar_after_lse_tail(bc, v, K, k0f, k1f, x, bonus, masked, row_timeout, 1.f, false, rSs, rSt, G0, G1, m4_raw);
 }
 
 // After one evaluation of pass "solve" that also carries the third and fourth moments:
