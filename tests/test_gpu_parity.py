@@ -386,5 +386,18 @@ def test_small_batches_of_long_rows_take_the_cluster_kernel():
         d3 = synth.generate(w3, DEV)
         P.route_fwd(d3["s"], d3["t"], d3["proposal"], w3.eps, seed=w3.seed)
         assert P.last_kernel() == 3
+        # a block verification of few positions goes the same way
+        B, K, V = 4, 6, 65536
+        w4 = synth.Workload("t", B * (K + 1), V, "bf16", 0.2, 1.5, True, 614, 44, K=K)
+        d4 = synth.generate(w4, DEV)
+        s3, t3 = d4["s"].view(B, K + 1, V), d4["t"].view(B, K + 1, V)
+        draft = d4["proposal"].view(B, K + 1)[:, :K].contiguous()
+        res = P.spec_verify(s3, t3, draft, w4.eps, seed=w4.seed)
+        torch.cuda.synchronize()
+        assert P.last_kernel() == 2
+        ref = O.spec_verify(to_np64(s3), to_np64(t3), draft.cpu().numpy(), w4.eps, seed=w4.seed)
+        ok = ref["margin"] >= 1e-6
+        assert np.array_equal(res["n_accept"].cpu().numpy()[ok], ref["n_accept"][ok])
+        assert np.array_equal(res["next_token"].cpu().numpy()[ok], ref["next_token"][ok])
     finally:
         P.set_kernel(prev)
