@@ -294,6 +294,21 @@ SAKI_API int saki_redo_count(void* cuda_stream, uint64_t* n_rows);
  * passes (log-sum-exp with moments, final). */
 SAKI_API int saki_solve_evaluations(void* cuda_stream, uint64_t* n_passes);
 
+/* Where the row-per-SM kernel's time goes (no counterpart in the paper: a measurement aid, off by
+ * default; it costs the kernel about 1.5 %).  saki_set_phase_clock(1) makes the routing calls that follow,
+ * from any thread, carry the clock (returns the previous setting).  With it, thread 0 of
+ * every thread block reads the SM's cycle counter at fixed marks of its row loop and adds the differences
+ * up per phase; saki_phase_cycles synchronises the stream and copies the SAKI_PHASE_COUNTERS sums (over all thread
+ * blocks) of the calling thread's last routing call into cycles[] (HOST memory, caller-owned): in order,
+ * the top of the row loop, the wait for the row's bulk copy, pass "lse", its warp reductions up to the
+ * first block barrier, the block-level gather, the float64 scalar step, the top of an evaluation, pass
+ * "solve", its block combine, its scalar step, the top of pass "final", pass "final", the end of the row
+ * loop, the kernel's tail, one spare word, and last the number of rows behind the sums.  Divide by that
+ * number for cycles per row.  All zero if the clock was off or another kernel served the call. */
+#define SAKI_PHASE_COUNTERS 16
+SAKI_API int saki_set_phase_clock(int on);
+SAKI_API int saki_phase_cycles(void* cuda_stream, uint64_t* cycles);
+
 /* Block verification, early out (Section 3.5: what follows a sequence's first rejected position is
  * discarded).  When on (the default) and the call has at least two sequences per SM, the row-per-SM
  * kernel hands out positions from a device counter in position-major order and passes over a position

@@ -22,7 +22,8 @@ _FLOAT_FIELDS = ("lambda", "kl", "tv", "accept_prob", "logp_x", "logq_x", "logT_
 EXPORTS = ("saki_route_fwd", "saki_route_fwd_bwd", "saki_route_fwd_bwd_noalloc", "saki_route_host",
            "saki_route_bwd_from_meta", "saki_select_tm", "saki_spec_verify",
            "saki_sample_proposal", "saki_check", "saki_set_kernel", "saki_last_kernel", "saki_redo_count",
-           "saki_set_spec_early_out", "saki_spec_positions_routed", "saki_solve_evaluations", "saki_launch_count",
+           "saki_set_spec_early_out", "saki_spec_positions_routed", "saki_solve_evaluations", "saki_set_phase_clock", "saki_phase_cycles",
+           "saki_launch_count",
            "saki_last_error", "saki_version")
 
 
@@ -110,6 +111,10 @@ def load_library(path: str | None = None):
     lib.saki_spec_positions_routed.restype = C.c_int
     lib.saki_solve_evaluations.argtypes = [C.c_void_p, C.POINTER(C.c_uint64)]
     lib.saki_solve_evaluations.restype = C.c_int
+    lib.saki_set_phase_clock.argtypes = [C.c_int]
+    lib.saki_set_phase_clock.restype = C.c_int
+    lib.saki_phase_cycles.argtypes = [C.c_void_p, C.POINTER(C.c_uint64)]
+    lib.saki_phase_cycles.restype = C.c_int
     lib.saki_launch_count.restype = C.c_uint64
     lib.saki_last_error.restype = C.c_char_p
     for f in ("saki_route_fwd", "saki_route_fwd_bwd", "saki_route_host", "saki_spec_verify",
@@ -377,6 +382,24 @@ def solve_evaluations(stream=None) -> int:
     n = C.c_uint64(0)
     _raise(lib, lib.saki_solve_evaluations(_stream_ptr(stream), C.byref(n)))
     return int(n.value)
+
+
+PHASES = ("row_top", "copy_wait", "lse", "lse_reduce", "lse_gather", "lse_scalar", "solve_top", "solve",
+          "solve_combine", "solve_scalar", "final_top", "final", "row_end", "tail", "spare", "rows")
+
+
+def set_phase_clock(on: bool) -> bool:
+    """Phase clock of the row-per-SM kernel for the calls that follow (default off); returns the previous setting."""
+    return bool(load_library().saki_set_phase_clock(1 if on else 0))
+
+
+def phase_cycles(stream=None) -> dict:
+    """SM cycles per phase of the row-per-SM kernel's row loop in the last routing call, summed over thread
+    blocks, and the number of rows behind them (synchronises)."""
+    lib = load_library()
+    buf = (C.c_uint64 * len(PHASES))()
+    _raise(lib, lib.saki_phase_cycles(_stream_ptr(stream), buf))
+    return {k: int(v) for k, v in zip(PHASES, buf)}
 
 
 def set_spec_early_out(on: bool) -> bool:

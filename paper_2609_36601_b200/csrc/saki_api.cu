@@ -20,6 +20,7 @@ static thread_local char g_err[512] = "";
 static std::atomic<uint64_t> g_launches{0};
 static std::atomic<int> g_kernel{0};
 static std::atomic<int> g_spec_early_out{1};
+static std::atomic<int> g_phase_clock{0};
 static thread_local int g_last_kernel = 0;
 
 static int fail(int code, const char* fmt, ...) {
@@ -146,8 +147,10 @@ static int dispatch_rows(RowParams p, int dtype, cudaStream_t st, int32_t* scrat
       const int rc = redo_scratch(p.n_rows, st, &p.redo_list, &p.redo_count);
       if (rc) return rc;
     }
-    e = cudaMemsetAsync(p.redo_count, 0, 4 * sizeof(unsigned int), st);   // the counter and the three words after it
+    // the counter, the three statistics words after it, and the phase clock's sums
+    e = cudaMemsetAsync(p.redo_count, 0, (8 + 2 * SAKI_PHASE_COUNTERS) * sizeof(unsigned int), st);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+    p.phase_cycles = g_phase_clock.load() ? (unsigned long long*)(p.redo_count + 8) : nullptr;
     g_last_redo_count = p.redo_count;
   }
   // A handful of long rows (a decoding step of a small batch) finish sooner spread over the whole GPU, one
@@ -271,7 +274,7 @@ static int meta_impl(const saki_meta_in* in, const saki_meta_out* out, void* dlo
   if (g_kernel.load() != 1 && meta_stream_can_serve(p, in->dtype)) {
     rc = redo_scratch(p.n_rows, st, &p.redo_list, &p.redo_count);
     if (rc) return rc;
-    e = cudaMemsetAsync(p.redo_count, 0, 4 * sizeof(unsigned int), st);
+    e = cudaMemsetAsync(p.redo_count, 0, (8 + 2 * SAKI_PHASE_COUNTERS) * sizeof(unsigned int), st);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
     g_last_redo_count = p.redo_count;
     e = launch_meta_stream(p, st, &launches, &served);
@@ -629,6 +632,20 @@ SAKI_API int saki_solve_evaluations(void* cuda_stream, uint64_t* n_passes) {
   e = cudaMemcpy(&h, g_last_redo_count + 3, sizeof(h), cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy");
   *n_passes = h;
+  return SAKI_OK;
+}
+
+SAKI_API int saki_set_phase_clock(int on) { return g_phase_clock.exchange(on ? 1 : 0); }
+
+SAKI_API int saki_phase_cycles(void* cuda_stream, uint64_t* cycles) {
+  g_err[0] = 0;
+  if (!cycles) return fail(SAKI_ERR_INVALID_ARG, "NULL output pointer");
+  memset(cycles, 0, SAKI_PHASE_COUNTERS * sizeof(uint64_t));
+  if (!g_last_redo_count) return SAKI_OK;
+  cudaError_t e = cudaStreamSynchronize((cudaStream_t)cuda_stream);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+  e = cudaMemcpy(cycles, g_last_redo_count + 8, SAKI_PHASE_COUNTERS * sizeof(uint64_t), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy");
   return SAKI_OK;
 }
 

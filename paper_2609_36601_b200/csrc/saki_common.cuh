@@ -7,6 +7,13 @@
 
 namespace saki {
 
+// Phases of the row-per-SM kernel's row loop, as timed by thread 0 of every CTA (saki_phase_cycles):
+// the three passes, the waits and block reductions around them, the float64 scalar steps between them.
+enum { PH_ROW_TOP = 0, PH_COPY_WAIT, PH_LSE, PH_LSE_REDUCE, PH_LSE_GATHER, PH_LSE_SCALAR, PH_SOLVE_TOP, PH_SOLVE,
+       PH_SOLVE_COMBINE, PH_SOLVE_SCALAR, PH_FINAL_TOP, PH_FINAL, PH_ROW_END, PH_TAIL, PH_SPARE, PH_ROWS,
+       PH_LAST /* shared memory only: the last mark */, PH_WORDS };
+static_assert(PH_LAST == SAKI_PHASE_COUNTERS, "saki.h publishes the number of phase counters");
+
 enum { STAGE_PROPOSE = 0, STAGE_ACCEPT = 1, STAGE_RESIDUAL = 2, STAGE_BONUS = 3, STAGE_SELECT = 4 };
 
 // Everything a row kernel needs; passed by value as the kernel parameter.
@@ -36,6 +43,8 @@ struct RowParams {
   unsigned int* redo_count;            // scratch: their number (zeroed before the launch, with the three words
                                        // after it: [1], [2] see seq_next; [3] evaluation passes of the row-per-SM kernel)
   int32_t from_list;                   // general kernel only: route the rows of redo_list
+  unsigned long long* phase_cycles;    // row-per-SM kernel: [SAKI_PHASE_COUNTERS] cycle sums per phase (zeroed before
+                                       // the launch); NULL: not wanted
   unsigned int* seq_next;              // row-per-SM kernel, block verification with early out: [0] ticket counter,
                                        // [1] positions routed (both zeroed before the launch); NULL: rows in static order
   int* seq_stop;                       // [n_rows / K1] position of each sequence's first stop (>= K1 before the launch)

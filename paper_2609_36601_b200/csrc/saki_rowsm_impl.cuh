@@ -31,9 +31,6 @@
 // combinations and per-row scalars are float64.
 #include "saki_device.cuh"
 #include <mutex>
-#ifdef SAKI_PHASE_TIMING
-#include <cstdio>
-#endif
 
 #ifdef SAKI_ROWSM_HALF
 #define SAKI_ROWSM_NS half_sm
@@ -79,7 +76,8 @@ constexpr int ROFF_FIN = ROFF_STEP + RW * MAX_STEPS * 4;          // [2][2][RW] 
 constexpr int ROFF_MBAR = ROFF_FIN + 2 * 2 * RW * 8;
 constexpr int FIN_WARP = SIDE_WARPS ? 12 : 4;   // the warp that finishes the previous row
 constexpr int ROFF_SEQ = ROFF_MBAR + 16;   // [4] ints: block verification, the CTA's reservation state
-constexpr int RSMEM_BYTES = ROFF_SEQ + 16;
+constexpr int ROFF_PH = ROFF_SEQ + 16;     // [PH_WORDS] 64-bit words: the phase clock of thread 0
+constexpr int RSMEM_BYTES = ROFF_PH + PH_WORDS * 8;
 
 // L2 residency hints: the part of a row that is re-read from L2 in every pass is marked
 // evict-last; everything that passes through L2 once (the shared-memory resident part, the
@@ -266,21 +264,26 @@ __device__ __forceinline__ void for_each_chunk(const Seg& sg, int lane, const ui
   rg.slot = slot;
 }
 
-#ifdef SAKI_PHASE_TIMING
-#define RTS(i) do { const long long _n = clock64(); tacc[i] += _n - tlast; tlast = _n; } while (0)
-#else
-#define RTS(i) do { } while (0)
-#endif
+// Phase clock (only when the call asks for it): thread 0 of every CTA adds the cycles between two marks
+// to phase i of a small table in shared memory; at the end of the kernel the table goes to the device
+// counters that saki_phase_cycles() reads (sums over CTAs; PH_ROWS counts the rows behind them).
+#define RTS(i) do { if (timing && tid == 0) { const long long _n = clock64(); ph[i] += _n - ph[PH_LAST]; ph[PH_LAST] = _n; } } while (0)
 
+// SPEC: the instance that serves block verification (bonus rows, positions handed out as tickets); plain
+// routing runs an instance without that code.
+template <bool SPEC>
 __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams P) {
   extern __shared__ __align__(128) unsigned char smem[];
-#ifdef SAKI_PHASE_TIMING
-  long long tacc[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
-  long long tlast = clock64();
-  int t_rows = 0;
-  long long w_solve = 0, w_evals = 0;
-#endif
   const int tid = threadIdx.x, lane = tid & 31;
+  const bool spec = SPEC && P.spec != 0;
+  const int K1c = SPEC ? P.K1 : 1;             // positions per sequence
+  const bool timing = P.phase_cycles != nullptr;
+  long long* ph = (long long*)(smem + ROFF_PH);
+  if (timing && tid == 0) {
+#pragma unroll 1
+    for (int i = 0; i < PH_WORDS; ++i) ph[i] = 0;
+    ph[PH_LAST] = clock64();
+  }
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // broadcast: lets the compiler treat it as warp-uniform
   const uint4* res_s = reinterpret_cast<const uint4*>(smem + ROFF_S) + warp * RES_CHUNKS;
   const uint4* res_t = reinterpret_cast<const uint4*>(smem + ROFF_T) + warp * RES_CHUNKS;
@@ -322,8 +325,8 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
 
   // rows fit 31 bits (see rowsm_can_serve): 32-bit divisions
   auto row_ptrs = [&](int64_t row, const __nv_bfloat16*& s, const __nv_bfloat16*& t) {
-    const int64_t b = P.K1 == 1 ? row : (int64_t)((uint32_t)row / (uint32_t)P.K1);
-    const int j = (int)(row - b * P.K1);
+    const int64_t b = K1c == 1 ? row : (int64_t)((uint32_t)row / (uint32_t)K1c);
+    const int j = (int)(row - b * K1c);
     s = (const __nv_bfloat16*)P.s + b * P.s_seq + (int64_t)j * P.s_pos;
     t = (const __nv_bfloat16*)P.t + b * P.t_seq + (int64_t)j * P.t_pos;
   };
@@ -360,11 +363,11 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
   // (n_rows: none left), [1], [2] the rest of a ticket range this CTA holds, [3] how many tickets it takes
   // at a time: it aims at one live ticket per range (doubles after a range without one, halves after a
   // range with several), so late positions, where most sequences have stopped, cost few round trips.
-  const bool dyn = P.seq_next != nullptr;
-  const int n_seq = dyn ? (int)(P.n_rows / P.K1) : 1;
+  const bool dyn = SPEC && P.seq_next != nullptr;
+  const int n_seq = dyn ? (int)(P.n_rows / K1c) : 1;
   const int n_tickets = (int)P.n_rows;
   int* seqres = (int*)(smem + ROFF_SEQ);
-  auto ticket_row = [&](int tk) { const int j = tk / n_seq; return (int64_t)(tk - j * n_seq) * P.K1 + j; };
+  auto ticket_row = [&](int tk) { const int j = tk / n_seq; return (int64_t)(tk - j * n_seq) * K1c + j; };
   auto ticket_live = [&](int tk, int hi) {   // not known to lie behind its sequence's first stop
     if (tk >= hi) return false;
     const int j = tk / n_seq;
@@ -421,10 +424,10 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
     const double* fin = (const double*)(smem + ROFF_FIN) + pb * 2 * RW;
     const __nv_bfloat16 *ps, *pt;
     row_ptrs(prow, ps, pt);
-    const int64_t pseq = P.K1 == 1 ? prow : (int64_t)((uint32_t)prow / (uint32_t)P.K1);
-    const int ppos = (int)(prow - pseq * P.K1);
-    const bool pbonus = P.spec && (ppos == P.K1 - 1);
-    const int xp = pbonus ? 0 : (P.spec ? P.proposal[pseq * P.prop_ld + ppos] : P.proposal[prow]);
+    const int64_t pseq = K1c == 1 ? prow : (int64_t)((uint32_t)prow / (uint32_t)K1c);
+    const int ppos = (int)(prow - pseq * K1c);
+    const bool pbonus = spec && (ppos == K1c - 1);
+    const int xp = pbonus ? 0 : (spec ? P.proposal[pseq * P.prop_ld + ppos] : P.proposal[prow]);
     const double tv_sum = warp_sum_d(lane < RW ? fin[lane] : 0.0);
     const double tv = (bcp[BC_LAMBDA] > 0.0) ? tv_sum : 0.0;
     const float k0p = (float)bcp[BC_K0];
@@ -437,7 +440,7 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
       ((__nv_bfloat16*)P.dlogits + prow * P.ld_g)[tok] = __float2bfloat16_rn(fmaf(ep, kgf, -(float)bcp[BC_KG]));
     }
     if (!(pbonus || bcp[BC_CORR] != 0.0)) {
-      if (lane == 0) write_result_tv(bcp, P.out, !P.spec, prow, 0, xp, false, K.c64, ps, pt, tv);
+      if (lane == 0) write_result_tv(bcp, P.out, !spec, prow, 0, xp, false, K.c64, ps, pt, tv);
       return;
     }
     // ---- the draw (corrected and bonus rows): the warp that owns the inverse-CDF target, by an
@@ -529,17 +532,17 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
       y = __shfl_sync(0xffffffffu, lastp, 31 - __clz(posm));
     }
     if (y < 0) y = min(V - 1, max(so.c0 * 8, so.c1 * 8 - 1));
-    if (lane == 0) write_result_tv(bcp, P.out, !P.spec, prow, pbonus ? 0 : 1, y, pbonus, K.c64, ps, pt, tv);
+    if (lane == 0) write_result_tv(bcp, P.out, !spec, prow, pbonus ? 0 : 1, y, pbonus, K.c64, ps, pt, tv);
   };
 
   int64_t next_row_c = P.n_rows;
   for (int64_t row = first_row; row < P.n_rows; row = next_row_c, rb ^= 1) {
     double* bc = (double*)(smem + ROFF_BC) + rb * BC_DOUBLES;   // this row's broadcast scalars
     const uint64_t rid = P.row_offset + (uint64_t)row;
-    const int64_t seq = P.K1 == 1 ? row : (int64_t)((uint32_t)row / (uint32_t)P.K1);
-    const int pos = (int)(row - seq * P.K1);
-    const bool bonus = P.spec && (pos == P.K1 - 1);
-    const int x = bonus ? 0 : (P.spec ? P.proposal[seq * P.prop_ld + pos] : P.proposal[row]);
+    const int64_t seq = K1c == 1 ? row : (int64_t)((uint32_t)row / (uint32_t)K1c);
+    const int pos = (int)(row - seq * K1c);
+    const bool bonus = spec && (pos == K1c - 1);
+    const int x = bonus ? 0 : (spec ? P.proposal[seq * P.prop_ld + pos] : P.proposal[row]);
     const bool masked = (P.mask != nullptr) && (P.mask[row] == 0);
     const __nv_bfloat16 *g_s = n_s, *g_t = n_t;
     __nv_bfloat16* g_out = P.dlogits ? (__nv_bfloat16*)P.dlogits + row * P.ld_g : nullptr;
@@ -551,16 +554,13 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
         atomicMin(P.seq_stop + seq, pos);        // verification of this sequence ends here
       atomicAdd(P.seq_next + 1, 1u);             // statistic: positions routed
     };
-#ifdef SAKI_PHASE_TIMING
-    ++t_rows;
-#endif
-
-    RTS(0);
+    if (timing && tid == 0) ph[PH_ROWS] += 1;
+    RTS(PH_ROW_TOP);
     if (!dead) {
       if (!mbar_wait_bounded(mbar, phase)) dead = true;
       else phase ^= 1u;
     }
-    RTS(1);
+    RTS(PH_COPY_WAIT);
 
     // ------------------------------------------------ pass "lse" (no separate maximum pass)
     // The exponent shifts of this pass are fixed before it starts: -ceil(c * m) with m the largest
@@ -610,7 +610,7 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
           N1 = ffma2(et, d, N1);
         }
       }, [] {});
-      RTS(2);
+      RTS(PH_LSE);
       // warp: teacher maximum with the lowest chunk that holds it (a chunk belongs to one thread, so
       // chunk order is index order; the element is found once, by the block's winner), student
       // maximum, sums
@@ -648,7 +648,7 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
       };
       if (!SIDE_WARPS && lane == 0) side_work();
       const int any_dead = __syncthreads_or(dead ? 1 : 0);
-      RTS(3);
+      RTS(PH_LSE_REDUCE);
       if (warp < 8) {   // block level: warps 0-6 add up one sum each on the row's shifts, warp 7 finds the argmax
         const int wl = lane < RW ? lane : 0;       // lanes beyond the warp count carry zero weight
         const float* wm = (const float*)(smem + ROFF_WMAX);
@@ -692,7 +692,7 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
       }
       if (any_dead) dead = true;
       __syncthreads();
-      RTS(4);
+      RTS(PH_LSE_GATHER);
       if (warp == FIN_WARP && pending_row >= 0) finish_row(pending_row, rb ^ 1);   // meanwhile: the previous row's draw and outputs
       if (dyn && warp == RES_WARP) reserve_next();     // and the CTA's next row (block verification), while thread 0 does the scalars
       pending_row = -1;
@@ -711,20 +711,17 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
           plan_next();
         }
       }
-      RTS(5);
+      RTS(PH_LSE_SCALAR);
       __syncthreads();
     }
     const float k0 = (float)bc[BC_K0], k1 = (float)bc[BC_K1];   // the row's shifts: exponent arguments <= 0
 
     // ------------------------------------------------ pass "solve" (repeated)
     while ((int)bc[BC_MODE] == MODE_SOLVE) {
-      RTS(6);
+      RTS(PH_SOLVE_TOP);
       const float cb = (float)bc[BC_CB], kb = (float)bc[BC_KB];
       float2 S0 = splat(0.f), S1 = splat(0.f), S2 = splat(0.f), S3 = splat(0.f), S4 = splat(0.f);
       const float2 cc = splat(c32), cbb = splat(cb), kbb = splat(kb), neg1 = splat(-1.f);
-#ifdef SAKI_PHASE_TIMING
-      const long long w_t0 = clock64();
-#endif
       for_each_chunk(sg, lane, res_s, res_t, g_s, g_t, g_s, g_t, pol_last, rg, [&](const uint4& s4, const uint4& t4, int, bool) {
         const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
 #pragma unroll
@@ -741,21 +738,18 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
           S4 = ffma2(u, d2, S4);
         }
       }, [] {});
-#ifdef SAKI_PHASE_TIMING
-      w_solve += clock64() - w_t0; ++w_evals;
-#endif
-      RTS(7);
+      RTS(PH_SOLVE);
       auto tot = [](const float2 a) { return (double)a.x + (double)a.y; };
       const double v[5] = {warp_sum_d(tot(S0)), warp_sum_d(tot(S1)), warp_sum_d(tot(S2)), warp_sum_d(tot(S3)),
                            warp_sum_d(tot(S4))};
       combine(v, 5);
-      RTS(8);
+      RTS(PH_SOLVE_COMBINE);
       if (tid == 0) {
         scalar_after_solve4(bc, gat, K, k0, k1, x, bonus, masked);
         plan_next();
         atomicAdd(P.redo_count + 3, 1u);         // statistic: evaluation passes
       }
-      RTS(9);
+      RTS(PH_SOLVE_SCALAR);
       __syncthreads();
     }
     const int64_t next_row = dyn ? (int64_t)seqres[0] : row + gridDim.x;
@@ -769,7 +763,7 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
       if (tid == 0) {
         if (redo) P.redo_list[atomicAdd(P.redo_count, 1u)] = (int32_t)row;
         else {
-          write_row(P.out, row, zero_row((uint32_t)bc[BC_STATUS]), !P.spec);
+          write_row(P.out, row, zero_row((uint32_t)bc[BC_STATUS]), !spec);
           atomicAdd(P.flagged, 1ull);
         }
       }
@@ -790,7 +784,7 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
     }
 
     // ------------------------------------------------ pass "final"
-    RTS(10);
+    RTS(PH_FINAL_TOP);
     const bool need_draw = bonus || bc[BC_CORR] != 0.0;
     const float cl = (float)bc[BC_CL], kq = (float)bc[BC_KQ];
     const float iq = (float)bc[BC_IQ], ip = (float)bc[BC_IP];
@@ -836,7 +830,7 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
           issue(n_s, n_t);
         }
       });
-      RTS(11);
+      RTS(PH_FINAL);
       // no barrier: each warp leaves its share of the total variation and its draw weight (its step
       // weights, in order) for finish_row
       double part = 0.0;
@@ -853,25 +847,21 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
       }
       pending_row = row;
     }
-    RTS(13);
+    RTS(PH_ROW_END);
     // no barrier here: the next row uses the other broadcast buffer, and every other shared area is
     // rewritten only after the next row's first block barrier
   }
 
-#ifdef SAKI_PHASE_TIMING
-  if (lane == 0 && blockIdx.x == 5 && t_rows > 0) printf("warp %d solve loop %lld cycles per row, %lld evaluations in %d rows, %d steps\n", warp, w_solve / t_rows, w_evals, t_rows, sg.steps);
-  if (tid == 0 && (blockIdx.x == 0 || blockIdx.x == 77) && t_rows > 0)
-    printf("blk %d tid %d rows %d | endbar %lld copy-wait %lld | lse %lld warp+bar %lld gather %lld scalar %lld | "
-           "bar %lld solve %lld combine %lld scalar %lld | bar %lld final %lld combine %lld tail %lld (cycles per row)\n",
-           (int)blockIdx.x, tid, t_rows, tacc[0] / t_rows, tacc[1] / t_rows, tacc[2] / t_rows, tacc[3] / t_rows,
-           tacc[4] / t_rows, tacc[5] / t_rows, tacc[6] / t_rows, tacc[7] / t_rows, tacc[8] / t_rows, tacc[9] / t_rows,
-           tacc[10] / t_rows, tacc[11] / t_rows, tacc[12] / t_rows, tacc[13] / t_rows);
-#endif
   cp_async_wait<0>();
   __syncthreads();
   if (warp == FIN_WARP && pending_row >= 0) finish_row(pending_row, rb ^ 1);
   // a CTA that gave up on a copy still waits (bounded) for what it has in flight before leaving
   if (dead && tid == 0) (void)mbar_wait_bounded(mbar, phase);
+  if (timing && tid == 0) {
+    RTS(PH_TAIL);
+#pragma unroll 1
+    for (int i = 0; i < PH_LAST; ++i) atomicAdd(P.phase_cycles + i, (unsigned long long)ph[i]);
+  }
 }
 
 // ---------------------------------------------------------------- host side
@@ -885,7 +875,9 @@ cudaError_t launch(const RowParams& p, cudaStream_t st, int* n_launches, bool* s
   {
     std::lock_guard<std::mutex> lock(mu);
     if (cached_dev != dev) {
-      cudaError_t e = cudaFuncSetAttribute(rowsm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, RSMEM_BYTES);
+      cudaError_t e = cudaFuncSetAttribute(rowsm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, RSMEM_BYTES);
+      if (e != cudaSuccess) return e;
+      e = cudaFuncSetAttribute(rowsm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, RSMEM_BYTES);
       if (e != cudaSuccess) return e;
       e = cudaDeviceGetAttribute(&cached_sms, cudaDevAttrMultiProcessorCount, dev);
       if (e != cudaSuccess) return e;
@@ -894,7 +886,8 @@ cudaError_t launch(const RowParams& p, cudaStream_t st, int* n_launches, bool* s
   }
   const int64_t ctas = (int64_t)cached_sms * CTAS_PER_SM;
   const int grid = (int)(p.n_rows < ctas ? p.n_rows : ctas);
-  rowsm_kernel<<<grid, RT, RSMEM_BYTES, st>>>(p);
+  if (p.spec) rowsm_kernel<true><<<grid, RT, RSMEM_BYTES, st>>>(p);
+  else rowsm_kernel<false><<<grid, RT, RSMEM_BYTES, st>>>(p);
   cudaError_t e = cudaGetLastError();
   if (e == cudaSuccess) { *served = true; if (n_launches) *n_launches += 1; }
   return e;
