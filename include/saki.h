@@ -294,6 +294,16 @@ SAKI_API int saki_redo_count(void* cuda_stream, uint64_t* n_rows);
  * passes (log-sum-exp with moments, final). */
 SAKI_API int saki_solve_evaluations(void* cuda_stream, uint64_t* n_passes);
 
+/* Failure behaviour of the row-per-SM kernel (no counterpart in the paper).  A thread block waits for a
+ * row's bulk copy from global memory for a bounded number of SM cycles (about two seconds' worth by
+ * default).  If the wait runs out the block stops fetching, flags that row and every row it still owns
+ * SAKI_ROW_TIMEOUT with zero outputs, waits (full limit) for the copy it has in flight, and returns: the
+ * kernel always terminates, saki_check() counts the flagged rows and later calls are unaffected.  This
+ * call sets the limit for the routing calls that follow, from any thread (0: the default), and returns
+ * the previous value; tests use a limit of a few cycles to exercise that path without withholding
+ * anything. */
+SAKI_API int64_t saki_set_wait_limit(int64_t cycles);
+
 /* Where the row-per-SM kernel's time goes (no counterpart in the paper: a measurement aid, off by
  * default; it costs the kernel about 1.5 %).  saki_set_phase_clock(1) makes the routing calls that follow,
  * from any thread, carry the clock (returns the previous setting).  With it, thread 0 of

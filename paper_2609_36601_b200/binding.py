@@ -22,7 +22,7 @@ _FLOAT_FIELDS = ("lambda", "kl", "tv", "accept_prob", "logp_x", "logq_x", "logT_
 EXPORTS = ("saki_route_fwd", "saki_route_fwd_bwd", "saki_route_fwd_bwd_noalloc", "saki_route_host",
            "saki_route_bwd_from_meta", "saki_select_tm", "saki_spec_verify",
            "saki_sample_proposal", "saki_check", "saki_set_kernel", "saki_last_kernel", "saki_redo_count",
-           "saki_set_spec_early_out", "saki_spec_positions_routed", "saki_solve_evaluations", "saki_set_phase_clock", "saki_phase_cycles",
+           "saki_set_spec_early_out", "saki_spec_positions_routed", "saki_solve_evaluations", "saki_set_wait_limit", "saki_set_phase_clock", "saki_phase_cycles",
            "saki_launch_count",
            "saki_last_error", "saki_version")
 
@@ -111,6 +111,8 @@ def load_library(path: str | None = None):
     lib.saki_spec_positions_routed.restype = C.c_int
     lib.saki_solve_evaluations.argtypes = [C.c_void_p, C.POINTER(C.c_uint64)]
     lib.saki_solve_evaluations.restype = C.c_int
+    lib.saki_set_wait_limit.argtypes = [C.c_int64]
+    lib.saki_set_wait_limit.restype = C.c_int64
     lib.saki_set_phase_clock.argtypes = [C.c_int]
     lib.saki_set_phase_clock.restype = C.c_int
     lib.saki_phase_cycles.argtypes = [C.c_void_p, C.POINTER(C.c_uint64)]
@@ -386,6 +388,12 @@ def solve_evaluations(stream=None) -> int:
 
 PHASES = ("row_top", "copy_wait", "lse", "lse_reduce", "lse_gather", "lse_scalar", "solve_top", "solve",
           "solve_combine", "solve_scalar", "final_top", "final", "row_end", "tail", "spare", "rows")
+
+
+def set_wait_limit(cycles: int) -> int:
+    """SM cycles a block of the row-per-SM kernel waits for a row's bulk copy before it flags its rows TIMEOUT
+    (0: the default of about two seconds); returns the previous setting."""
+    return int(load_library().saki_set_wait_limit(int(cycles)))
 
 
 def set_phase_clock(on: bool) -> bool:

@@ -21,6 +21,7 @@ static std::atomic<uint64_t> g_launches{0};
 static std::atomic<int> g_kernel{0};
 static std::atomic<int> g_spec_early_out{1};
 static std::atomic<int> g_phase_clock{0};
+static std::atomic<long long> g_wait_limit{0};
 static thread_local int g_last_kernel = 0;
 
 static int fail(int code, const char* fmt, ...) {
@@ -140,6 +141,7 @@ static int dispatch_rows(RowParams p, int dtype, cudaStream_t st, int32_t* scrat
   const bool rowsm_ok = (which == 0 || which == 3) && rowsm_can_serve(p, dtype);
   const bool fast = (which != 1) && (rowsm_ok || (eps_ok && cluster_can_serve(p, dtype)));
   p.redo_list = nullptr; p.redo_count = nullptr; p.from_list = 0;
+  p.wait_limit = g_wait_limit.load();
   g_last_redo_count = nullptr;          // the counters below describe this call only
   if (fast) {
     if (scratch_list) { p.redo_list = scratch_list; p.redo_count = scratch_count; }
@@ -634,6 +636,8 @@ SAKI_API int saki_solve_evaluations(void* cuda_stream, uint64_t* n_passes) {
   *n_passes = h;
   return SAKI_OK;
 }
+
+SAKI_API int64_t saki_set_wait_limit(int64_t cycles) { return (int64_t)g_wait_limit.exchange(cycles > 0 ? (long long)cycles : 0); }
 
 SAKI_API int saki_set_phase_clock(int on) { return g_phase_clock.exchange(on ? 1 : 0); }
 

@@ -32,9 +32,6 @@
 #include <cooperative_groups.h>
 #include <math_constants.h>
 #include <mutex>
-#ifdef SAKI_PHASE_TIMING
-#include <cstdio>
-#endif
 
 namespace cg = cooperative_groups;
 
@@ -63,21 +60,9 @@ constexpr int OFF_MBAR = OFF_SCR + 2 * EPT * 2;                 // copy barrier,
 constexpr int SMEM_BYTES = OFF_MBAR + 5 * 8 + 8;
 static_assert(OFF_MBAR % 8 == 0 && OFF_SCR % 16 == 0, "alignment");
 
-// Optional per-phase cycle counters of thread 0 (compile with -DSAKI_PHASE_TIMING; printed at kernel end).
-#ifdef SAKI_PHASE_TIMING
-#define TS(i) do { const long long _n = clock64(); tacc[i] += _n - tlast; tlast = _n; } while (0)
-#else
-#define TS(i) do { } while (0)
-#endif
-
 template <int CS>
 __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const int n_clusters) {
   extern __shared__ __align__(128) unsigned char smem[];
-#ifdef SAKI_PHASE_TIMING
-  long long tacc[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
-  long long tlast = clock64();
-  int t_rows = 0, t_solves = 0;
-#endif
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const unsigned rank = cg::this_cluster().block_rank();
   const int cluster_id = blockIdx.x / CS;
@@ -161,13 +146,11 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
     __nv_bfloat16* g_out = P.dlogits ? (__nv_bfloat16*)P.dlogits + row * P.ld_g : nullptr;
 
     // ------------------------------------------------ stage: shared slot -> registers
-    TS(0);
     bool timed_out = dead;
     if (!dead) {
       if (!mbar_wait_bounded(&mbar[0], phase)) timed_out = true;
       else phase ^= 1u;
     }
-    TS(1);
     uint32_t sr[NPAIR], tr[NPAIR];
 #pragma unroll
     for (int j = 0; j < CHUNKS; ++j) {
@@ -204,9 +187,7 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
         wmax[(rb * 2 + 1) * CW + warp] = fmaxf(fb.x, fb.y);
       }
     }
-    TS(2);
     const int any_timeout = __syncthreads_or(timed_out ? 1 : 0);   // also: every thread has drained the slot
-    TS(3);
     if (any_timeout) dead = true;
     if (tid == 0) {
       const int64_t next = row + n_clusters;
@@ -283,7 +264,6 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
         N1 = ffma2(et, d, N1);
       }
       // the row's maxima have arrived meanwhile: move the partial sums onto the row's shifts
-      TS(4);
       bool mx_timeout = false;
       if (!mbar_wait_bounded(&mbar[3 + rb], rb ? mph1 : mph0)) mx_timeout = true;
       if (rb) mph1 ^= 1u; else mph0 ^= 1u;
@@ -307,23 +287,19 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
       v[6] = warp_min(v[6]);
       v[7] = warp_sum(v[7]);
       push(v, 8, parity);
-      TS(5);
       if (warp < 8) {
         if (!mbar_wait_bounded(&mbar[1 + parity], parity ? xph1 : xph0)) dead = true;
-        TS(6);
         const double g = gather(parity, warp, warp == 6);
         if (lane == 0) gat[warp] = g;
       }
       if (parity) xph1 ^= 1u; else xph0 ^= 1u;
       parity ^= 1;
       __syncthreads();
-      TS(7);
       if (tid == 0) {
         scalar_after_lse(bc, gat, K, k0, k1, x, bonus, masked, row_timeout, gat + 7);
         if ((int)bc[BC_MODE] == MODE_SOLVE) mbar_expect_tx(&mbar[1 + parity], (uint32_t)(CS * CW * 5 * 8));
         else if ((int)bc[BC_MODE] == MODE_FINAL) mbar_expect_tx(&mbar[1 + parity], (uint32_t)(CS * CW * 3 * 8));
       }
-      TS(8);
       __syncthreads();
     }
 
@@ -348,29 +324,22 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
         S4[h] = ffma2(t2, fmul2(d, d), S4[h]);
       }
       auto tot = [](const float2 (&a)[2]) { return ((double)a[0].x + (double)a[0].y) + ((double)a[1].x + (double)a[1].y); };
-      TS(9);
       double v[5] = {warp_sum(tot(S0)), warp_sum(tot(S1)), warp_sum(tot(S2)), warp_sum(tot(S3)), warp_sum(tot(S4))};
       push(v, 5, parity);
       if (warp < 5) {
         if (!mbar_wait_bounded(&mbar[1 + parity], parity ? xph1 : xph0)) dead = true;
-        TS(10);
         const double g = gather(parity, warp, false);
         if (lane == 0) gat[warp] = g;
       }
       if (parity) xph1 ^= 1u; else xph0 ^= 1u;
       parity ^= 1;
       __syncthreads();
-      TS(11);
       if (tid == 0) {
         scalar_after_solve4(bc, gat, K, k0, k1, x, bonus, masked);
         if ((int)bc[BC_MODE] == MODE_SOLVE) mbar_expect_tx(&mbar[1 + parity], (uint32_t)(CS * CW * 5 * 8));   // next evaluation
         else if ((int)bc[BC_MODE] == MODE_FINAL) mbar_expect_tx(&mbar[1 + parity], (uint32_t)(CS * CW * 3 * 8));   // pass "final"
       }
-      TS(12);
       __syncthreads();
-#ifdef SAKI_PHASE_TIMING
-      ++t_solves;
-#endif
     }
 
     // ------------------------------------------------ flagged row: zero outputs, zero gradient
@@ -395,7 +364,6 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
       continue;
     }
 
-    TS(15);
     // ------------------------------------------------ pass "final"
     const bool need_draw = bonus || bc[BC_CORR] != 0.0;
     float my_part;       // this thread's ordered weight for the inverse-CDF draw
@@ -444,12 +412,10 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
           g_out[tok] = __float2bfloat16_rn(fmaf(ep, kg, -KGf));
         }
       }
-      TS(13);
       double v[3] = {warp_sum((double)sq_f), warp_sum((double)r_f), warp_sum((double)my_part)};
       push(v, 3, parity);
       if (warp == 0) {
         if (!mbar_wait_bounded(&mbar[1 + parity], parity ? xph1 : xph0)) dead = true;
-        TS(14);
         const double tv = gather(parity, 1, false);
         if (lane == 0) {
           bc[BC_TV] = (bc[BC_LAMBDA] > 0.0) ? tv : 0.0;
@@ -527,16 +493,6 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
     }
   }
 
-#ifdef SAKI_PHASE_TIMING
-  for (int64_t row = cluster_id; row < P.n_rows; row += n_clusters) ++t_rows;
-  if (tid == 0 && (blockIdx.x == 0 || blockIdx.x == 77) && t_rows > 0)
-    printf("blk %d rows %d solves %d | tail %lld copy-wait %lld stage %lld sync %lld | lse %lld mx+push %lld xwait %lld "
-           "gather+bar %lld scalar %lld bar %lld | solve %lld xwait %lld gather+bar %lld scalar %lld | final %lld "
-           "xwait %lld (cycles per row)\n", (int)blockIdx.x, t_rows, t_solves, tacc[0] / t_rows, tacc[1] / t_rows,
-           tacc[2] / t_rows, tacc[3] / t_rows, tacc[4] / t_rows, tacc[5] / t_rows, tacc[6] / t_rows, tacc[7] / t_rows,
-           tacc[8] / t_rows, (tacc[15]) / t_rows, tacc[9] / t_rows, tacc[10] / t_rows, tacc[11] / t_rows,
-           tacc[12] / t_rows, tacc[13] / t_rows, tacc[14] / t_rows);
-#endif
   // a CTA that gave up on a copy still waits (bounded) for what it has in flight before leaving
   if (dead && tid == 0) (void)mbar_wait_bounded(&mbar[0], phase);
   cg::this_cluster().sync();   // no CTA leaves while a peer may still write its shared memory

@@ -130,11 +130,9 @@ cudaError_t launch_meta_general(const MetaParams& p, int dtype, cudaStream_t st,
 // The kernel is instantiated for 32 warps (one CTA per SM) and for 16 warps (two CTAs per SM, for short
 // rows: one CTA's block barriers and scalar step run under the other's passes).
 constexpr int MW_FULL = 32, MW_HALF = 16;
-#ifndef SAKI_META_HALF_MAX_V
-#define SAKI_META_HALF_MAX_V 98304   /* M positions/s, one / two CTAs per SM: V = 8192 52 / 77, 32000 30.8 / 37.5,
-                                        50048 23.2 / 27.0, 65536 19.5 / 19.9, 131072 10.5 / 10.6, 151936 9.1 / 8.8 */
-#endif
-constexpr int M_HALF_MAX_V = SAKI_META_HALF_MAX_V;   // rows up to this length take the 16-warp instance
+// rows up to this length take the 16-warp instance (M positions/s, one / two CTAs per SM: V = 8192 52 / 77,
+// 32000 30.8 / 37.5, 50048 23.2 / 27.0, 65536 19.5 / 19.9, 131072 10.5 / 10.6, 151936 9.1 / 8.8)
+constexpr int M_HALF_MAX_V = 98304;
 constexpr int MKS = 13;                  // 512-byte steps of shared memory per warp (a step = 32 chunks of 8 elements)
 constexpr int MNST = 5;                  // ring stages of a warp whose segment does not fit
 constexpr int MRES = MKS - MNST;         // resident steps of such a warp

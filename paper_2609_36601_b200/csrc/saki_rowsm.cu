@@ -10,10 +10,7 @@ namespace saki {
 // the streamed parts of all rows no longer stay in L2 between the passes.  Measured (fwd+bwd, M rows/s,
 // one / two CTAs per SM): V = 8192 15.9 / 25.3, 32000 9.9 / 12.7, 65536 6.5 / 7.5, 81920 5.6 / 6.3,
 // 100000 4.85 / 5.06, 131072 3.95 / 3.76.
-#ifndef SAKI_HALF_MAX_V
-#define SAKI_HALF_MAX_V 98304
-#endif
-constexpr int HALF_MAX_V = SAKI_HALF_MAX_V;
+constexpr int HALF_MAX_V = 98304;
 
 bool rowsm_can_serve(const RowParams& p, int dtype) {
   if (dtype != SAKI_BF16) return false;

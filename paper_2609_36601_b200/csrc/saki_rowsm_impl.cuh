@@ -38,9 +38,7 @@
 #define SAKI_ROWSM_CTAS 2
 #else
 #define SAKI_ROWSM_NS full_sm
-#ifndef SAKI_ROWSM_THREADS
 #define SAKI_ROWSM_THREADS 512
-#endif
 #define SAKI_ROWSM_CTAS 1
 #endif
 
@@ -128,22 +126,7 @@ __device__ __forceinline__ float pow2f_exact(float n) {   // 2^n for whole n, cl
   return __uint_as_float((uint32_t)(127 + i) << 23);
 }
 
-#ifndef SAKI_RES_UNROLL
-#define SAKI_RES_UNROLL 1
-#endif
-constexpr int RES_UNROLL = SAKI_RES_UNROLL;   // unrolling of the resident-part loop
-#ifndef SAKI_RING_UNROLL
-#define SAKI_RING_UNROLL 1
-#endif
-constexpr int RING_UNROLL = SAKI_RING_UNROLL; // unrolling of the streamed-part loop
-#ifndef SAKI_FAST_UNROLL
-#define SAKI_FAST_UNROLL 1
-#endif
-constexpr int FAST_UNROLL = SAKI_FAST_UNROLL; // unrolling of its check-free copy
-#ifndef SAKI_RING
-#define SAKI_RING 4
-#endif
-constexpr int NST = SAKI_RING;          // ring stages: steps of the streamed part in flight per warp
+constexpr int NST = 4;                  // ring stages: steps of the streamed part in flight per warp
 constexpr int KS_RES = KS_MAX - NST;    // resident steps of a warp whose segment does not fit entirely
 
 // 16-byte asynchronous copy global -> shared (through L2 only), grouped per thread
@@ -211,7 +194,7 @@ __device__ __forceinline__ void for_each_chunk(const Seg& sg, int lane, const ui
   // resident part (slots past the end of the segment hold the filler); kept rolled: the pass bodies
   // are large and must stay in the instruction cache
   int c = sg.c0 + lane;
-#pragma unroll RES_UNROLL
+#pragma unroll 1
   for (int k = 0; k < sg.res; ++k, c += 32) body(res_s[k * 32 + lane], res_t[k * 32 + lane], c, c < sg.c1);
   after_resident();
   const int T = sg.steps - sg.res;                  // streamed steps: 0 or more than NST
@@ -227,7 +210,7 @@ __device__ __forceinline__ void for_each_chunk(const Seg& sg, int lane, const ui
   // all but the last NST + 1 steps: the chunk consumed and the chunk requested exist for every lane, and
   // the requests stay inside this pass, so this copy of the loop carries none of the checks below (the
   // body is instantiated twice; 1.7 % faster on V = 151936 in spite of the larger code)
-#pragma unroll FAST_UNROLL
+#pragma unroll 1
   for (; i < T - NST - 1; ++i, c += 32) {
     cp_async_wait<NST - 1>();
     const uint4 a = lds128(slot), b = lds128(slot + T_OFF);
@@ -239,7 +222,7 @@ __device__ __forceinline__ void for_each_chunk(const Seg& sg, int lane, const ui
     if (slot == slot_end) slot = rg.base;
     body(a, b, c, true);
   }
-#pragma unroll RING_UNROLL
+#pragma unroll 1
   for (; i < T; ++i, c += 32) {
     if (i == T - NST) {   // from here on the requests belong to the pass that follows
       off = first_off;
@@ -278,6 +261,9 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
   const bool spec = SPEC && P.spec != 0;
   const int K1c = SPEC ? P.K1 : 1;             // positions per sequence
   const bool timing = P.phase_cycles != nullptr;
+  // how long a thread waits for a row's bulk copy before the block gives up on its rows (the drain at
+  // the end of the kernel always takes the full limit: no copy is in flight when a block leaves)
+  const long long wait_limit = P.wait_limit > 0 ? P.wait_limit : WAIT_LIMIT_CYCLES;
   long long* ph = (long long*)(smem + ROFF_PH);
   if (timing && tid == 0) {
 #pragma unroll 1
@@ -412,6 +398,7 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
   }
   uint32_t phase = 0;
   bool dead = false;
+  bool undrained = false;   // this thread gave up on a copy that may still be in flight
   int rb = 0;
   // Pass "final" ends without a barrier.  What is left of a row after it (the total variation, the
   // one-hot entry of the gradient, the residual draw, the outputs) is done one row later by warp
@@ -557,7 +544,7 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
     if (timing && tid == 0) ph[PH_ROWS] += 1;
     RTS(PH_ROW_TOP);
     if (!dead) {
-      if (!mbar_wait_bounded(mbar, phase)) dead = true;
+      if (!mbar_wait_bounded(mbar, phase, wait_limit)) { dead = true; undrained = true; }
       else phase ^= 1u;
     }
     RTS(PH_COPY_WAIT);
@@ -856,7 +843,7 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
   __syncthreads();
   if (warp == FIN_WARP && pending_row >= 0) finish_row(pending_row, rb ^ 1);
   // a CTA that gave up on a copy still waits (bounded) for what it has in flight before leaving
-  if (dead && tid == 0) (void)mbar_wait_bounded(mbar, phase);
+  if (undrained && tid == 0) (void)mbar_wait_bounded(mbar, phase);
   if (timing && tid == 0) {
     RTS(PH_TAIL);
 #pragma unroll 1

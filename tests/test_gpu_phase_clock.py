@@ -22,7 +22,7 @@ def test_phase_clock_counts_rows_and_leaves_results_alone():
         out1, g1 = P.route_fwd_bwd(d["s"], d["t"], d["proposal"], w.eps, seed=w.seed)
         on = P.phase_cycles()
         P.set_phase_clock(False)
-        out2, _ = P.route_fwd(d["s"], d["t"], d["proposal"], w.eps, seed=w.seed)
+        out2 = P.route_fwd(d["s"], d["t"], d["proposal"], w.eps, seed=w.seed)
         assert all(v == 0 for v in P.phase_cycles().values())
     finally:
         P.set_phase_clock(False)
