@@ -2,7 +2,7 @@
 """Benchmark of the SAKI routing hot path on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload cfg3] [--rows R] [--no-e2e] [--no-cpu]
+                    [--workload cfg3] [--rows R] [--no-e2e] [--no-cpu] [--no-next] [--no-sweep]
 
 One "step" is one pass of the whole hot path (log-softmax x2, lambda solve,
 coupling + TV, routed loss, fused gradient) over one batch of synthetic
@@ -14,15 +14,22 @@ positions: one saki_route_fwd_bwd call.  Prints ONE JSON line.
   roofline  algorithmic HBM bytes (read both logit rows once, write the
             gradient row once) / measured kernel time, against the measured
             copy bandwidth of this machine's B200s
-  cpu_baseline  the float64 test oracle, as it stands, on a bounded sample
+  cpu_baseline  the float64 test oracle, as it stands, on a bounded sample:
+            on one host core, and on all host cores (a process pool over rows)
   next_step, spec_verify, small_batch  (rank 0, unless --no-next) further calls
             timed the same way beside the headline: saki_route_bwd_from_meta on
             the same logits, saki_spec_verify on its own workload with and
             without early out, and the latency of saki_route_fwd on 8 rows
+  sweep     (rank 0, unless --no-sweep) the throughput sweep at its full size
+            (65536 positions, three disagreement regimes x three radii) and the
+            V = 32000 workload: positions/s, fraction of the copy bandwidth,
+            evaluation passes per row, saturated fraction, second-tier rows
+  phase_cycles_per_row  where the row-per-SM kernel's cycles go (its phase
+            clock, on one extra untimed call)
 
-With N > 1 (under torchrun) every rank routes its own batch of the same
-shape (rows are independent: no collective on the data path); the time is
-the maximum over ranks.
+With N > 1 every rank routes its own batch of the same shape (rows are
+independent: no collective on the data path); the time is the maximum over
+ranks.  `--gpus N` without a torchrun environment starts the N ranks itself.
 """
 from __future__ import annotations
 
@@ -43,13 +50,13 @@ METRIC = "routed positions/sec (fwd+bwd, V=151936 bf16)"
 UNIT = "positions/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one rowsm_kernel launch divided by the positions it
-# routed: ncu capture on 2220 rows of the same workload (profiles/rowsm_kernel_cfg3.md); traffic grows
-# in proportion to the rows, so a full launch is this figure times N
+# routed, from an ncu capture on 2220 rows of the same workload (the kernel's ncu summary gives the
+# command); traffic grows in proportion to the rows, so a full launch is this figure times N
 TRAFFIC_BYTES_PER_POSITION = 945005
 # rows up to this length are served by the instances of the two streaming kernels that run two CTAs per SM
 # (namespace half_sm, meta_stream_kernel<16>); the names below are the ones a profiler shows
 TWO_CTA_MAX_V = 98304
-# the same for one meta_stream_kernel launch (profiles/meta_stream_kernel_cfg3.md)
+# the same for one meta_stream_kernel launch
 META_TRAFFIC_BYTES_PER_POSITION = 581046
 
 
@@ -111,19 +118,65 @@ class ClockSampler:
         return out
 
 
-def _oracle_sample(w, d, rows, grad=True):
-    """Times the float64 oracle on `rows` rows of the workload (host cores)."""
-    import numpy as np
+def _bf16_bits(x):
+    """Host copy of logits as raw 16-bit words (bf16) or float32 values: small to ship to worker processes."""
     import torch
+    return x.cpu().view(torch.int16).numpy() if x.dtype == torch.bfloat16 else x.cpu().numpy()
+
+
+def _to_f64(a):
+    """float64 array of what _bf16_bits shipped (bf16 -> float64 is exact)."""
+    import numpy as np
+    if a.dtype == np.int16:
+        return (a.astype(np.int32) << 16).view(np.float32).astype(np.float64)
+    return a.astype(np.float64)
+
+
+def _oracle_rows(job):
+    """Worker of the all-cores baseline: routes a block of rows with the oracle; returns seconds spent."""
     import oracle as O
-    idx = torch.arange(rows)
-    s = d["s"][idx.to(d["s"].device)].to("cpu").to(torch.float64).numpy()
-    t = d["t"][idx.to(d["t"].device)].to("cpu").to(torch.float64).numpy()
+    sb, tb, x, eps, tau, seed, row0, dtype = job
+    t0 = time.perf_counter()
+    O.route(_to_f64(sb), _to_f64(tb), x, eps, tau, seed, row0, want_grad=True, grad_dtype=dtype)
+    return time.perf_counter() - t0
+
+
+def _oracle_sample(w, d, rows, grad=True):
+    """Times the float64 oracle on `rows` rows of the workload (one host core)."""
+    import oracle as O
+    s = _to_f64(_bf16_bits(d["s"][:rows]))
+    t = _to_f64(_bf16_bits(d["t"][:rows]))
     x = d["proposal"][:rows].to("cpu").numpy()
     t0 = time.perf_counter()
     ref = O.route(s, t, x, w.eps, w.temperature, w.seed, 0, want_grad=grad, grad_dtype=w.dtype)
     dt = time.perf_counter() - t0
     return rows / dt, dt, ref
+
+
+def _oracle_all_cores(w, d, rows_per_core):
+    """The same oracle on every host core at once: a pool of processes, each with its own block of rows
+    (the rows that follow the one-core sample).  Returns positions/s over the wall time of the pool."""
+    import multiprocessing as mp
+    cores = os.cpu_count() or 1
+    first = rows_per_core                      # do not reuse the one-core sample's rows
+    jobs = []
+    for c in range(cores):
+        a, b = first + c * rows_per_core, first + (c + 1) * rows_per_core
+        if b > w.N:
+            break
+        jobs.append((_bf16_bits(d["s"][a:b]), _bf16_bits(d["t"][a:b]), d["proposal"][a:b].cpu().numpy(), w.eps,
+                     w.temperature, w.seed, a, w.dtype))
+    if not jobs:
+        return None
+    with mp.get_context("spawn").Pool(len(jobs)) as pool:
+        pool.map(_oracle_rows, [(j[0][:1], j[1][:1], j[2][:1]) + j[3:] for j in jobs])     # start-up and imports
+        t0 = time.perf_counter()
+        pool.map(_oracle_rows, jobs, chunksize=1)
+        dt = time.perf_counter() - t0
+    n = len(jobs) * rows_per_core
+    return {"value": n / dt, "unit": UNIT, "cores": len(jobs), "kind": "oracle",
+            "sample": f"{n} rows of {w.name} after the one-core sample, {rows_per_core} per process, forward + "
+                      f"gradient, {dt:.1f} s wall on {len(jobs)} processes (os.cpu_count() = {cores})"}
 
 
 def run_reference(args):
@@ -147,17 +200,73 @@ def run_reference(args):
     line = {"metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": 1e3 * tot_t / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "impl": "reference",
-            "config": {"workload": _describe(w), "sample": f"{rows} rows per step"},
+            "config": _config(w, args.gpus),
             "cpu_baseline": {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
-                             "sample": f"first {rows} rows of {w.name}, forward + gradient, {args.steps} steps"},
+                             "sample": f"first {rows} rows of {w.name} per step, forward + gradient, {args.steps} steps"},
             "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
 
 
+def _config(w, world):
+    esz = 4 if w.dtype == "f32" else 2
+    return {"workload": _describe(w),
+            "l2": "inputs (2 x %.1f GB) exceed L2; no flush needed" % (w.N * w.V * esz / 1e9),
+            "parallelism": f"rows sharded over {world} GPU(s), no collective"}
+
+
 def _describe(w):
     return (f"{w.name}: N={w.N} positions, V={w.V}, {w.dtype} logits, eps={w.eps}, temperature={w.temperature}, "
             f"teacher noise sigma={w.sigma}, fused fwd+bwd with {w.dtype} dlogits")
+
+
+def _sweep(P, synth, dev, stream, peak, args):
+    """positions/s of saki_route_fwd_bwd on every cell of the throughput sweep at its full size (one input set
+    per disagreement regime, three radii each) and on the V = 32000 workload; timed like the headline."""
+    import torch
+    cells = []
+    groups = [[n for n in synth.WORKLOADS if n.startswith("cfg4_" + r + "_")] for r in ("s05", "s20", "ind")]
+    groups.append(["cfg2"])
+    for names in groups:
+        w0 = synth.WORKLOADS[names[0]]
+        d = synth.generate(w0, dev)
+        g = torch.empty_like(d["s"])
+        out = None
+        for name in names:
+            w = synth.WORKLOADS[name]
+            n_steps = 3 if w.N * w.V > (1 << 32) else 20
+
+            def call():
+                nonlocal out
+                out, _ = P.route_fwd_bwd(d["s"], d["t"], d["proposal"], w.eps, w.temperature, w.seed, 0,
+                                         grad_scale=1.0 / w.N, out=out, dlogits=g, stream=stream)
+            for _ in range(3):
+                call()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(n_steps):
+                call()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / n_steps
+            gbs = synth.bytes_per_position(w, True) * w.N / (ms * 1e-3) / 1e9
+            st = out["row_status"]
+            cells.append({"workload": name, "N": w.N, "V": w.V, "eps": w.eps,
+                          "teacher": "independent" if w.sigma < 0 else f"sigma={w.sigma:g}",
+                          "value": w.N / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "achieved_gbs": gbs,
+                          "frac": gbs / peak, "kernel": P.last_kernel(),
+                          "evaluation_passes_per_row": P.solve_evaluations(stream) / w.N,
+                          "frac_saturated": float(((st & 1) != 0).float().mean().item()),
+                          "second_tier_rows": int(P.redo_count(stream)),
+                          "correction_rate": float(out["corrected"].float().mean().item()),
+                          "mean_lambda": float(out["lambda"].mean().item()),
+                          "rows_flagged": int(P.check())})
+        del d, g, out
+        torch.cuda.empty_cache()
+    return {"call": "saki_route_fwd_bwd", "timing": "3 warm-up calls, then 3 timed calls per cell (20 for the short "
+            "workload), CUDA events; inputs exceed L2", "frac": "of the same copy bandwidth as roofline.peak",
+            "cells": cells}
 
 
 def run_ours(args):
@@ -223,6 +332,17 @@ def run_ours(args):
     n_flagged = P.check()
     kernel_used = P.last_kernel()
     evals_last_step = P.solve_evaluations(stream) if kernel_used == 3 else 0   # of the last timed launch
+    redo_last_step = P.redo_count(stream)
+    phases = None
+    if kernel_used == 3 and rank == 0:        # one more call, untimed, with the kernel's phase clock on
+        P.set_phase_clock(True)
+        step()
+        ph = P.phase_cycles(stream)
+        P.set_phase_clock(False)
+        rows_ph = max(1, ph.pop("rows"))
+        ph.pop("spare", None)
+        phases = {k: round(v / rows_ph, 1) for k, v in ph.items()}
+        phases["total"] = round(sum(ph.values()) / rows_ph, 1)
 
     # ---- the step that follows the path: the trainer's loss and gradient from this call's metadata
     # (saki_route_bwd_from_meta), on the same logits; reported beside the headline, not in it
@@ -343,7 +463,7 @@ def run_ours(args):
                 "peak_kind": f"of {peak_kind} (device-to-device copy, MEASURED_PEAKS.json)"
                 if peak_kind == "measured" else "of fallback",
                 "traffic": (TRAFFIC_BYTES_PER_POSITION * w.N) if TRAFFIC_BYTES_PER_POSITION else None,
-                "algorithmic_bytes_per_launch": bpp * w.N, "kernel": {3: "saki::%s::rowsm_kernel" % ("half_sm" if w.V <= TWO_CTA_MAX_V else "full_sm"),
+                "algorithmic_bytes_per_launch": bpp * w.N, "kernel": {3: "saki::%s::rowsm_kernel<false>" % ("half_sm" if w.V <= TWO_CTA_MAX_V else "full_sm"),
                            2: "saki::cluster_kernel"}.get(kernel_used, "saki::general_kernel"),
                 "kernel_ms": kern_ms,
                 "frac_of_nominal_8TBs": achieved / 8000.0}
@@ -364,24 +484,55 @@ def run_ours(args):
     stats = {"correction_rate": float(out["corrected"].float().mean().item()),
              "median_tv": float(out["tv"].median().item()), "mean_lambda": float(out["lambda"].mean().item()),
              "frac_saturated": float(((out["row_status"] & 1) != 0).float().mean().item()),
-             "rows_flagged": n_flagged}
+             "rows_flagged": n_flagged, "second_tier_rows": int(redo_last_step)}
 
     cpu = None
     if not args.no_cpu:
-        v, dt, ref = _oracle_sample(w, d, args.cpu_rows)
         import numpy as np
-        agree = int(np.sum(out["corrected"][:args.cpu_rows].cpu().numpy() == ref["corrected"]))
+        n1 = min(args.cpu_rows, w.N)
+        v, dt, ref = _oracle_sample(w, d, n1)
+        got = {k: out[k][:n1].cpu().numpy() for k in ("corrected", "token", "teacher_top1", "lambda", "tv", "loss")}
+        margin = np.minimum(ref["margin_accept"], ref["margin_draw"])
+        exempt = margin < 1e-6            # decisions too close to call: counted, not compared
+        ok = ~exempt
+        flags_agree = int(np.sum(got["corrected"][ok] == ref["corrected"][ok]))
+        tokens_agree = int(np.sum(got["token"][ok] == ref["token"][ok]))
+        loss_err = np.abs(got["loss"] - ref["loss"])
+        stats["oracle_sample"] = {
+            "rows": int(n1), "margin_exempt": int(exempt.sum()),
+            "margin_exempt_accept": int(np.sum(ref["margin_accept"] < 1e-6)),
+            "margin_exempt_draw": int(np.sum(ref["margin_draw"] < 1e-6)),
+            "flags_agree": f"{flags_agree}/{int(ok.sum())}", "tokens_agree": f"{tokens_agree}/{int(ok.sum())}",
+            "teacher_top1_agree": f"{int(np.sum(got['teacher_top1'] == ref['teacher_top1']))}/{int(n1)}",
+            "max_abs_dlambda": float(np.max(np.abs(got["lambda"] - ref["lam"]))),
+            "max_abs_dtv": float(np.max(np.abs(got["tv"] - ref["tv"]))),
+            "loss_beyond_1e-4_relative": int(np.sum(loss_err[ok] > 1e-4 * np.abs(ref["loss"][ok])))}
         cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
-               "sample": f"first {args.cpu_rows} rows of {w.name}, forward + gradient, {dt:.1f} s on one host core "
-                         f"(of {os.cpu_count()}); accept/correct flags agree with the GPU on {agree}/{args.cpu_rows}"}
+               "sample": f"first {n1} rows of {w.name}, forward + gradient, {dt:.1f} s on one host core "
+                         f"(of {os.cpu_count()})"}
+        if w.N >= 2 * n1:
+            allc = _oracle_all_cores(w, d, max(8, n1 // 4))
+            if allc:
+                cpu["all_cores"] = allc
+
+    # ---- the throughput sweep at its full size and the V = 32000 workload: beside the headline
+    sweep = None
+    if not args.no_sweep and not args.rows and rank == 0:
+        del s, t, g, x, d
+        out = None
+        torch.cuda.empty_cache()
+        sweep = _sweep(P, synth, dev, stream, peak, args)
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": _describe(w), "l2": "inputs (2 x %.1f GB) exceed L2; no flush needed" %
-                       (s.numel() * s.element_size() / 1e9), "parallelism": f"rows sharded over {world} GPU(s), no collective"},
+            "config": _config(w, world),
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
             "stats": stats, "achieved_gbs": achieved}
+    if phases is not None:
+        line["phase_cycles_per_row"] = phases
+    if sweep is not None:
+        line["sweep"] = sweep
     if nxt is not None:
         nxt["roofline"] = {"bound": "hbm", "achieved": nxt["achieved_gbs"], "peak": peak, "unit": "GB/s",
                            "frac": nxt["achieved_gbs"] / peak}
@@ -393,6 +544,20 @@ def run_ours(args):
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def _spawn_ranks(n):
+    """`--gpus N` outside a torchrun environment: start N ranks of this command, one GPU each, on this node."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")                       # NCCL's own log stays on, in a file per rank:
+    env.setdefault("NCCL_DEBUG_FILE", os.path.join(tempfile.gettempdir(), "saki_bench_nccl.%h.%p.log"))   # stdout carries the JSON line
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd, env=env)
 
 
 def main():
@@ -408,10 +573,13 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-next", action="store_true", help="skip the metadata-driven backward measurement")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the throughput sweep and the V = 32000 workload")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-rows", type=int, default=384)
     ap.add_argument("--ref-rows", type=int, default=32)
     args = ap.parse_args()
+    if args.gpus > 1 and "RANK" not in os.environ:
+        sys.exit(_spawn_ranks(args.gpus))
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -54,27 +54,40 @@ static int device_ready(unsigned long long** flagged) {
 // Scratch of the two-tier routing: the float32 kernels append the rows they cannot resolve to a list
 // that the float64 kernel then routes.  One buffer per (device, stream), so that calls on different
 // streams do not share a list; grown on demand, kept until exit.  (Calls on one stream are ordered by the
-// stream, so they may share.)
+// stream, so they may share.)  A caller holds g_redo_mu from the hand-out until its kernels are launched,
+// and nothing is freed while work that may use it is in flight: a buffer that was outgrown is retired,
+// not freed, and the sweep that follows many short-lived streams first waits for the device.  Every
+// free bumps g_redo_generation, which the counter readers check before they follow g_last_redo_count.
 struct RedoBuf {
   int32_t* list = nullptr;       // [cap] rows, followed by the counter
   int64_t cap = 0;
 };
 static std::mutex g_redo_mu;
 static std::map<std::pair<int, cudaStream_t>, RedoBuf> g_redo;
+static std::vector<std::pair<int, int32_t*>> g_retired;          // (device, buffer) outgrown, still possibly in use
+static std::atomic<uint64_t> g_redo_generation{0};
 static thread_local unsigned int* g_last_redo_count = nullptr;
+static thread_local uint64_t g_last_redo_generation = 0;
 
+// g_redo_mu held by the caller
 static int redo_scratch(int64_t n_rows, cudaStream_t st, int32_t** list, unsigned int** count) {
-  std::lock_guard<std::mutex> lock(g_redo_mu);
   int dev = 0;
   cudaGetDevice(&dev);
-  if (g_redo.size() > 256) {   // many short-lived streams: start over (cudaFree waits for work in flight)
+  if (g_redo.size() > 256) {   // many short-lived streams: start over, once nothing on the device can still use a list
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceSynchronize (scratch sweep)");
     for (auto& kv : g_redo)
       if (kv.first.first == dev && kv.second.list) { cudaFree(kv.second.list); kv.second = RedoBuf(); }
     for (auto it = g_redo.begin(); it != g_redo.end();) it = it->second.list ? std::next(it) : g_redo.erase(it);
+    for (auto& r : g_retired)
+      if (r.first == dev && r.second) { cudaFree(r.second); r.second = nullptr; }
+    g_retired.erase(std::remove_if(g_retired.begin(), g_retired.end(), [](const std::pair<int, int32_t*>& r) { return !r.second; }),
+                    g_retired.end());
+    g_redo_generation.fetch_add(1);
   }
   RedoBuf& b = g_redo[std::make_pair(dev, st)];
   if (b.cap < n_rows) {
-    if (b.list) cudaFree(b.list);
+    if (b.list) g_retired.emplace_back(dev, b.list);   // an earlier call on this stream may still be running on it
     b = RedoBuf();
     const int64_t cap = std::max<int64_t>(n_rows, 1 << 16);
     // row ids, 64 words of counters, and as many words again (block verification: one per sequence)
@@ -85,6 +98,10 @@ static int redo_scratch(int64_t n_rows, cudaStream_t st, int32_t** list, unsigne
   *list = b.list;
   *count = (unsigned int*)(b.list + b.cap);
   return SAKI_OK;
+}
+// the calling thread's last routing call's counters, or NULL if there are none (any more)
+static unsigned int* last_counters() {
+  return g_last_redo_generation == g_redo_generation.load() ? g_last_redo_count : nullptr;
 }
 
 // Fixed scratch of saki_route_fwd_bwd_noalloc: the redo list of the two-tier routing for callers that must
@@ -143,9 +160,11 @@ static int dispatch_rows(RowParams p, int dtype, cudaStream_t st, int32_t* scrat
   p.redo_list = nullptr; p.redo_count = nullptr; p.from_list = 0;
   p.wait_limit = g_wait_limit.load();
   g_last_redo_count = nullptr;          // the counters below describe this call only
+  std::unique_lock<std::mutex> scratch_lock(g_redo_mu, std::defer_lock);
   if (fast) {
     if (scratch_list) { p.redo_list = scratch_list; p.redo_count = scratch_count; }
     else {
+      scratch_lock.lock();       // until the kernels that use the list are launched
       const int rc = redo_scratch(p.n_rows, st, &p.redo_list, &p.redo_count);
       if (rc) return rc;
     }
@@ -154,6 +173,7 @@ static int dispatch_rows(RowParams p, int dtype, cudaStream_t st, int32_t* scrat
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
     p.phase_cycles = g_phase_clock.load() ? (unsigned long long*)(p.redo_count + 8) : nullptr;
     g_last_redo_count = p.redo_count;
+    g_last_redo_generation = g_redo_generation.load();
   }
   // A handful of long rows (a decoding step of a small batch) finish sooner spread over the whole GPU, one
   // row per cluster of 8 blocks, than on one SM each: 32 clusters fit at once, and at V = 151936 a call of
@@ -273,12 +293,15 @@ static int meta_impl(const saki_meta_in* in, const saki_meta_out* out, void* dlo
   bool served = false;
   int used = 1;
   g_last_redo_count = nullptr;
+  std::unique_lock<std::mutex> scratch_lock(g_redo_mu, std::defer_lock);
   if (g_kernel.load() != 1 && meta_stream_can_serve(p, in->dtype)) {
+    scratch_lock.lock();         // until the kernels that use the list are launched
     rc = redo_scratch(p.n_rows, st, &p.redo_list, &p.redo_count);
     if (rc) return rc;
     e = cudaMemsetAsync(p.redo_count, 0, (8 + 2 * SAKI_PHASE_COUNTERS) * sizeof(unsigned int), st);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
     g_last_redo_count = p.redo_count;
+    g_last_redo_generation = g_redo_generation.load();
     e = launch_meta_stream(p, st, &launches, &served);
     if (e != cudaSuccess) return cuda_fail(e, "streaming backward kernel launch");
     if (served) { used = 4; p.from_list = 1; }
@@ -613,11 +636,12 @@ SAKI_API int saki_redo_count(void* cuda_stream, uint64_t* n_rows) {
   g_err[0] = 0;
   if (!n_rows) return fail(SAKI_ERR_INVALID_ARG, "NULL output pointer");
   *n_rows = 0;
-  if (!g_last_redo_count) return SAKI_OK;
+  unsigned int* const counters = last_counters();
+  if (!counters) return SAKI_OK;
   cudaError_t e = cudaStreamSynchronize((cudaStream_t)cuda_stream);
   if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
   unsigned int h = 0;
-  e = cudaMemcpy(&h, g_last_redo_count, sizeof(h), cudaMemcpyDeviceToHost);
+  e = cudaMemcpy(&h, counters, sizeof(h), cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy");
   *n_rows = h;
   return SAKI_OK;
@@ -627,11 +651,12 @@ SAKI_API int saki_solve_evaluations(void* cuda_stream, uint64_t* n_passes) {
   g_err[0] = 0;
   if (!n_passes) return fail(SAKI_ERR_INVALID_ARG, "NULL output pointer");
   *n_passes = 0;
-  if (!g_last_redo_count) return SAKI_OK;
+  unsigned int* const counters = last_counters();
+  if (!counters) return SAKI_OK;
   cudaError_t e = cudaStreamSynchronize((cudaStream_t)cuda_stream);
   if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
   unsigned int h = 0;
-  e = cudaMemcpy(&h, g_last_redo_count + 3, sizeof(h), cudaMemcpyDeviceToHost);
+  e = cudaMemcpy(&h, counters + 3, sizeof(h), cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy");
   *n_passes = h;
   return SAKI_OK;
@@ -645,10 +670,11 @@ SAKI_API int saki_phase_cycles(void* cuda_stream, uint64_t* cycles) {
   g_err[0] = 0;
   if (!cycles) return fail(SAKI_ERR_INVALID_ARG, "NULL output pointer");
   memset(cycles, 0, SAKI_PHASE_COUNTERS * sizeof(uint64_t));
-  if (!g_last_redo_count) return SAKI_OK;
+  unsigned int* const counters = last_counters();
+  if (!counters) return SAKI_OK;
   cudaError_t e = cudaStreamSynchronize((cudaStream_t)cuda_stream);
   if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
-  e = cudaMemcpy(cycles, g_last_redo_count + 8, SAKI_PHASE_COUNTERS * sizeof(uint64_t), cudaMemcpyDeviceToHost);
+  e = cudaMemcpy(cycles, counters + 8, SAKI_PHASE_COUNTERS * sizeof(uint64_t), cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy");
   return SAKI_OK;
 }
@@ -659,11 +685,12 @@ SAKI_API int saki_spec_positions_routed(void* cuda_stream, uint64_t* n_positions
   g_err[0] = 0;
   if (!n_positions) return fail(SAKI_ERR_INVALID_ARG, "NULL output pointer");
   *n_positions = 0;
-  if (!g_last_redo_count) return SAKI_OK;
+  unsigned int* const counters = last_counters();
+  if (!counters) return SAKI_OK;
   cudaError_t e = cudaStreamSynchronize((cudaStream_t)cuda_stream);
   if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
   unsigned int h = 0;
-  e = cudaMemcpy(&h, g_last_redo_count + 2, sizeof(h), cudaMemcpyDeviceToHost);
+  e = cudaMemcpy(&h, counters + 2, sizeof(h), cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy");
   *n_positions = h;
   return SAKI_OK;

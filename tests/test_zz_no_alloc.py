@@ -50,6 +50,38 @@ def test_noalloc_entry_matches_regular_entry_twice_in_a_row():
         P.set_kernel(prev)
 
 
+def test_noalloc_entry_allocates_nothing_on_a_stream_the_library_has_never_seen():
+    """What the entry point is for: on a stream that no regular call has used (the regular entry would now
+    allocate that stream's row list) the call leaves the device's free memory exactly as it was, and the
+    rows that need the float64 kernel still get there through the fixed array."""
+    prev = P.set_kernel(0)
+    try:
+        w = synth.Workload("noalloc3", 512, 32000, "bf16", 0.05, 1.0, True, 313, 21)
+        d = synth.generate(w, DEV)
+        force_second_tier(d, [5, 100, 511])
+        ref_out, ref_g = P.route_fwd_bwd(d["s"], d["t"], d["proposal"], w.eps, seed=w.seed)
+        torch.cuda.synchronize()
+        out = P.alloc_outputs(w.N, DEV)
+        g = torch.empty_like(d["s"])
+        fresh = torch.cuda.Stream()
+        # once on the current stream: the address of the fixed array is looked up on a device's first call
+        P.route_fwd_bwd_noalloc(d["s"], d["t"], d["proposal"], w.eps, out, g, seed=w.seed)
+        torch.cuda.synchronize()
+        g.fill_(float("nan"))
+        free_before, _ = torch.cuda.mem_get_info()
+        P.route_fwd_bwd_noalloc(d["s"], d["t"], d["proposal"], w.eps, out, g, seed=w.seed, stream=fresh)
+        fresh.synchronize()
+        torch.cuda.synchronize()
+        free_after, _ = torch.cuda.mem_get_info()
+        assert free_after == free_before, (free_before, free_after)
+        assert P.last_kernel() == 3 and P.redo_count(fresh) == 3
+        for k in ref_out:
+            assert torch.equal(out[k], ref_out[k]), k
+        assert torch.equal(g, ref_g)
+    finally:
+        P.set_kernel(prev)
+
+
 def test_noalloc_entry_rejects_batches_beyond_its_fixed_scratch():
     s = torch.zeros((1, 2048), dtype=torch.bfloat16, device=DEV)
     big = s.expand((1 << 20) + 1, 2048)          # a view: no memory behind the extra rows, and none is read
