@@ -39,9 +39,16 @@
  *     (row lo, row hi, stage, block); stage 0 proposal Gumbel noise (word
  *     v%4 of block v/4), 1 acceptance uniform, 2 residual draw, 3 bonus draw,
  *     4 placement-control key (word 0 of block 0).  A word w gives the uniform ((w>>9)+0.5) 2^-23.
- *     `row` is the GLOBAL row id row_offset + i, so results do not depend on
- *     how a batch is chunked or sharded.
- *   - Results are deterministic: same inputs, same GPU model, same outputs.
+ *     `row` is the GLOBAL row id row_offset + i, so the random numbers a position
+ *     sees do not depend on how a batch is chunked or sharded.
+ *   - Results are deterministic: same call (inputs, sizes), same GPU model, same bits.  Chunking or
+ *     sharding a batch leaves every output bit-identical as long as each piece is served by the same
+ *     kernel as the whole; the library picks the kernel from the call's size (calls of at most 32 rows
+ *     with V >= 65536 run one row per thread-block cluster, larger ones one row per SM), so a tail piece
+ *     of 32 long rows or fewer agrees with the same rows inside a large call to the tolerances of the
+ *     arithmetic (float outputs to ~1e-6, flags and ids wherever the decision is not within 1e-6 of
+ *     its threshold), not to the bit.  saki_set_kernel pins the choice where bit-identity across pieces
+ *     matters.
  */
 #ifndef SAKI_H_
 #define SAKI_H_

@@ -9,7 +9,8 @@ Tolerances (written here so that the tests state them):
   lambda, TV          |delta| <= 1e-5
   other fp32 scalars  |delta| <= 1e-5 (kl, accept_prob) or 1e-5 (1+|ref|) (log-probs)
   loss                |delta| <= 1e-4 |ref| + 1e-6 (1 + |k1| + |log p(x)|), k1 = log p(x) - log T(x): the loss is
-                      k1 log p(x), and a log-sum-exp taken from float32 sums resolves each factor to ~1e-7
+                      k1 log p(x), and a log-sum-exp taken from float32 sums resolves each factor to ~1e-7;
+                      rows that need the absolute term are counted, and must have |loss| < 0.25
   gradient, fp32      |delta| <= 1e-6 + 2e-6 |ref|
   gradient, bf16      |delta| <= 2e-3 where |g_ref| < 1; elsewhere within one
                       bf16 ulp of the oracle's rounded value; and relative
@@ -52,17 +53,28 @@ def grad_check(g_gpu: np.ndarray, g_ref: np.ndarray, dtype: str, tok=None):
     big_ok = d[~small] <= bf16_ulp(g_ref[~small]) * 1.0000001
     assert np.all(big_ok), "bf16 gradient entry with |g|>=1 off by more than one ulp"
     nz = np.abs(g_ref) >= 1e-30
+    n_tok_abs_only = 0
     if tok is not None:
-        nz[np.arange(len(tok)), np.asarray(tok)] = False
+        ti, tj = np.arange(len(tok)), np.asarray(tok)
+        at_tok = nz[ti, tj]
+        n_tok_abs_only = int(np.count_nonzero(d[ti, tj][at_tok] > 2.0 ** -7 * 1.0000001 * np.abs(g_ref[ti, tj][at_tok])))
+        nz[ti, tj] = False
     rel = d[nz] / np.abs(g_ref[nz])
     assert np.all(rel <= 2.0 ** -7 * 1.0000001), f"bf16 gradient relative error {rel.max():.3e}"
     return dict(max_abs=float(d[small].max()) if small.any() else 0.0,
-                n_ulp=int(np.count_nonzero(g_gpu != g_ref)))
+                n_ulp=int(np.count_nonzero(g_gpu != g_ref)),
+                n_tok_abs_only=n_tok_abs_only)   # supervised-token entries held by the absolute bound alone
 
 
-def compare_rows(gpu: dict, ref: dict, rows=None, check_loss=True):
+LOSS_FLOOR_MAX = 0.25   # a row that meets the loss bound only through its absolute floor has a loss this small
+
+
+def compare_rows(gpu: dict, ref: dict, rows=None, check_loss=True, report=None):
     """gpu: dict of torch tensors (all rows); ref: oracle dict over `rows`.
-    Returns the number of margin-exempt rows."""
+    Returns the number of margin-exempt rows.  `report` (a dict) receives the counts a reader of the test
+    output wants: rows compared, margin-exempt rows by decision, rows whose loss error exceeds the pure
+    relative bound (they pass by the absolute floor, and only if their loss is below LOSS_FLOOR_MAX), and
+    the largest errors."""
     n_total = len(gpu["token"])
     rows = np.arange(n_total) if rows is None else np.asarray(list(rows))
     g = {k: v.detach().cpu().numpy()[rows] for k, v in gpu.items() if isinstance(v, torch.Tensor)}
@@ -82,10 +94,21 @@ def compare_rows(gpu: dict, ref: dict, rows=None, check_loss=True):
     for name in ("logp_x", "logq_x", "logT_x", "logp_y", "logq_y", "logT_y"):
         d = np.abs(g[name].astype(np.float64) - ref[name])[same]
         assert np.all(d <= 1e-5 * (1 + np.abs(ref[name][same]))), f"{name}: max error {d.max():.3e}"
+    n_loss_floor = 0
     if check_loss:
         d = np.abs(g["loss"].astype(np.float64) - ref["loss"])[same]
         floor = 1e-6 * (1.0 + np.abs(ref["logp_x"] - ref["logT_x"]) + np.abs(ref["logp_x"]))[same]   # the ~1e-7 resolution of a
         assert np.all(d <= 1e-4 * np.abs(ref["loss"][same]) + floor), f"loss: max error {d.max():.3e}"   # float32 lse
+        by_floor = d > 1e-4 * np.abs(ref["loss"][same])
+        n_loss_floor = int(by_floor.sum())
+        assert np.all(np.abs(ref["loss"][same][by_floor]) < LOSS_FLOOR_MAX), "a large loss met its bound only by the floor"
+    if report is not None:
+        report.update(rows=int(len(rows)), margin_exempt=int(exempt.sum()),
+                      margin_exempt_accept=int(np.sum(ref["margin_accept"] < MARGIN)),
+                      margin_exempt_draw=int(np.sum(ref["margin_draw"] < MARGIN)),
+                      loss_by_floor_only=n_loss_floor,
+                      max_abs_dlambda=float(np.abs(g["lambda"].astype(np.float64) - ref["lam"]).max()),
+                      max_abs_dtv=float(np.abs(g["tv"].astype(np.float64) - ref["tv"]).max()))
     return int(exempt.sum())
 
 

@@ -1,11 +1,14 @@
 """Parity at the benchmark's sizes, in the launch configuration bench.py times (automatic kernel
 selection, one call over the whole batch), on sampled rows the oracle computes one by one.
 
-cfg1 runs in test_gpu_parity.py (all 64 rows).  cfg2, cfg3 and cfg5 run at full size here.  The
-throughput sweep (cfg4) keeps its full vocabulary and all 9 regime x radius cells but routes the
-first 2368 positions of each regime (16 rows per SM) instead of 65536: the per-row work and the launch shape
-per SM are the same, only the row loop is shorter; one cell (the mixed one) also runs at the full
-65536 positions in one call when the device has room for it."""
+cfg1 runs in test_gpu_parity.py (all 64 rows).  cfg2, cfg3 and cfg5 run at full size here: 1024 rows
+of each of the first two against the oracle, every sequence of cfg5.  The throughput sweep (cfg4) keeps its
+full vocabulary and all 9 regime x radius cells but routes the first 2368 positions of each regime (16 rows per
+SM) instead of 65536, 263 of them against the oracle: the per-row work and the launch shape per SM are the
+same, only the row loop is shorter; one cell (the mixed one) also runs at the full 65536 positions in one call
+when the device has room for it, the rows r % 32 == 0 against the oracle.  The oracle runs in a pool of
+processes (oracle_pool.py); each test prints its counts: margin-exempt rows, rows whose loss met its bound only
+through the absolute floor, supervised-token gradient entries held by the absolute bound alone."""
 import numpy as np
 import pytest
 import torch
@@ -13,38 +16,39 @@ import torch
 import oracle as O
 import paper_2609_36601_b200 as P
 from paper_2609_36601_b200 import synth
+from oracle_pool import route_rows, spec_verify_seqs
 from parity import compare_rows, grad_check, to_np64
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-def _sampled(w, d, rows, eps=None):
+def _sampled(w, d, rows, eps=None, label=None):
+    """One call over the whole batch, then the float64 oracle (a pool of processes over the host's cores) on the
+    rows `rows`: every per-position output and the gradient row.  Prints the counts a reader wants to see."""
     e = w.eps if eps is None else eps
     out, g = P.route_fwd_bwd(d["s"], d["t"], d["proposal"], e, w.temperature, w.seed, grad_scale=1.0 / w.N)
     torch.cuda.synchronize()
     assert P.check() == 0
-    idx = torch.as_tensor(rows, device=DEV)
-    s64, t64 = to_np64(d["s"][idx]), to_np64(d["t"][idx])
-    x = d["proposal"][idx].cpu().numpy()
-    ref = {k: [] for k in ()}
-    res = [O.route_row(s64[i], t64[i], int(x[i]), e, w.temperature, w.seed, int(rows[i]), 1, 1.0 / w.N, True, w.dtype)
-           for i in range(len(rows))]
-    ref = {k: np.array([r[k] for r in res]) for k in res[0] if k != "grad"}
-    ref["grad"] = np.stack([r["grad"] for r in res])
-    n_exempt = compare_rows(out, ref, rows)
-    gg = to_np64(g[idx])
-    same = out["corrected"].cpu().numpy()[rows] == ref["corrected"]
-    grad_check(gg[same], ref["grad"][same], w.dtype, np.where(ref["corrected"] == 1, ref["teacher_top1"], ref["token"])[same])
+    ref = route_rows(d, rows, e, w.temperature, w.seed, 1.0 / w.N, w.dtype, g=g, corrected_gpu=out["corrected"])
+    report = {}
+    n_exempt = compare_rows(out, ref, rows, report=report)
+    bad = [(int(r), m) for r, m in zip(rows, ref["grad_error"]) if m]
+    assert not bad, f"gradient rows off: {bad[:3]}"
+    gs = [st for st in ref["grad_stats"] if st]
+    report.update(grad_rows_checked=len(gs), grad_entries_not_the_oracles_rounding=sum(st["n_ulp"] for st in gs),
+                  supervised_entries_by_absolute_bound_only=sum(st["n_tok_abs_only"] for st in gs),
+                  second_tier_rows=P.redo_count())
+    print(f"\n[parity] {label or w.name} eps={e:g}: {report}")
     return out, ref, n_exempt
 
 
 def test_cfg2_full():
     w = synth.WORKLOADS["cfg2"]
     d = synth.generate(w, DEV)
-    rows = list(range(0, w.N, 64))
+    rows = list(range(0, w.N, 4))                                 # 1024 rows
     out, ref, n_exempt = _sampled(w, d, rows)
-    assert P.last_kernel() == 3 and n_exempt <= 1
+    assert P.last_kernel() == 3 and n_exempt <= 3 + 0.25 * int(ref['corrected'].sum())
     tv = out["tv"].cpu().numpy()
     assert np.all(tv <= np.sqrt(w.eps / 2) + 1e-5)              # Pinsker cap on the whole batch
     assert abs(out["corrected"].float().mean().item() - tv.mean()) < 4 * np.sqrt(0.12 * 0.88 / w.N)
@@ -53,9 +57,9 @@ def test_cfg2_full():
 def test_cfg3_full():
     w = synth.WORKLOADS["cfg3"]
     d = synth.generate(w, DEV)
-    rows = list(range(5, w.N, 341))                               # 48 rows
+    rows = list(range(5, w.N, 16))                                # 1024 rows
     out, ref, n_exempt = _sampled(w, d, rows)
-    assert P.last_kernel() == 3 and n_exempt <= 1
+    assert P.last_kernel() == 3 and n_exempt <= 3 + 0.25 * int(ref['corrected'].sum())   # a draw's target lies within 1e-6 of a cell edge in ~5 % of the corrected rows: most cells of the residual are narrower than that
     tv = out["tv"].cpu().numpy()
     assert 0.15 < np.median(tv) < 0.2237                          # the workload's "median TV roughly 0.2"
     assert np.all(tv <= np.sqrt(w.eps / 2) + 1e-5)
@@ -75,8 +79,9 @@ def test_cfg4_cells(regime):
         w = synth.shrink(synth.WORKLOADS[f"cfg4_{regime}_e{eps:g}"], n)
         if d is None:
             d = synth.generate(w, DEV)                            # one input set per regime
-        rows = list(range(3, n, 148))                             # 16 rows
-        out, ref, _ = _sampled(w, d, rows)
+        rows = list(range(3, n, 9))                               # 263 rows
+        out, ref, n_exempt = _sampled(w, d, rows)
+        assert n_exempt <= 3 + 0.25 * int(ref['corrected'].sum())   # exempt rows are draws: see test_cfg3_full
         saturated[eps] = float(((out["row_status"] & 1) != 0).float().mean().item())
     if regime == "s05":
         assert saturated[1.0] > 0.99 and 0.0 < saturated[0.1] < 0.99   # an (almost) saturated and a mixed cell
@@ -90,9 +95,9 @@ def test_cfg4_one_cell_at_65536_positions():
     if torch.cuda.mem_get_info(0)[0] < need:
         pytest.skip("needs %.0f GB of free device memory" % (need / 1e9))
     d = synth.generate(w, DEV)
-    rows = list(range(11, w.N, 2731))                             # 24 rows over the whole batch
+    rows = list(range(0, w.N, 32))                                # the r % 32 == 0 subset: 2048 rows
     out, ref, n_exempt = _sampled(w, d, rows)
-    assert P.last_kernel() == 3 and n_exempt <= 1
+    assert P.last_kernel() == 3 and n_exempt <= 3 + 0.25 * int(ref['corrected'].sum())
     st = out["row_status"]
     assert int((st & ~1).max().item()) == 0                       # no status bit but "saturated" on any of the rows
     tv = out["tv"].cpu().numpy()
@@ -112,24 +117,24 @@ def test_cfg5_full():
     res = P.spec_verify(s3, t3, draft, w.eps, seed=w.seed)
     torch.cuda.synchronize()
     assert P.check() == 0 and P.last_kernel() == 3
-    seqs = list(range(0, B, 22))                                  # 24 sequences
-    idx = torch.as_tensor(seqs, device=DEV)
-    ref = O.spec_verify(to_np64(s3[idx]), to_np64(t3[idx]), draft[idx].cpu().numpy(), w.eps, seed=w.seed)
-    # the oracle keys random streams by global sequence: recompute per sequence with its own offset
+    seqs = list(range(B))                                         # every sequence
+    refs = spec_verify_seqs(s3, t3, draft, seqs, w.eps, w.temperature, w.seed)
     n_acc = res["n_accept"].cpu().numpy()
     nxt = res["next_token"].cpu().numpy()
     isc = res["next_is_correction"].cpu().numpy()
-    for j, b in enumerate(seqs):
-        r = O.spec_verify(to_np64(s3[b:b + 1]), to_np64(t3[b:b + 1]), draft[b:b + 1].cpu().numpy(), w.eps,
-                          seed=w.seed, seq_offset=b)
+    per_all = {k: v.cpu().numpy().reshape(B, K + 1) for k, v in res["per_pos"].items()}
+    n_exempt = 0
+    for b, r in zip(seqs, refs):
         if r["margin"][0] < 1e-6:
+            n_exempt += 1
             continue
         assert n_acc[b] == r["n_accept"][0] and nxt[b] == r["next_token"][0] and isc[b] == r["next_is_correction"][0]
-        per = {k: v.cpu().numpy().reshape(B, K + 1)[b] for k, v in res["per_pos"].items()}
         for p in range(K + 1):
             rr = r["per_pos"][0][p]
-            assert per["row_status"][p] == rr["status"] and per["token"][p] == rr["token"]
-            assert abs(per["lambda"][p] - rr["lam"]) <= 1e-5 and abs(per["tv"][p] - rr["tv"]) <= 1e-5
+            assert per_all["row_status"][b][p] == rr["status"] and per_all["token"][b][p] == rr["token"]
+            assert abs(per_all["lambda"][b][p] - rr["lam"]) <= 1e-5 and abs(per_all["tv"][b][p] - rr["tv"]) <= 1e-5
+    print(f"\n[parity] cfg5: {B} sequences checked, {n_exempt} margin-exempt")
+    assert n_exempt <= 0.1 * B
     # law of the accepted-prefix length over the whole batch: mean acceptance ~ 1 - TV
     assert 0 < n_acc.mean() < K
     assert set(np.unique(n_acc)) <= set(range(K + 1))

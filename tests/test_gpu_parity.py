@@ -171,6 +171,49 @@ def test_determinism_and_chunk_invariance(kernel):
     assert torch.equal(ga, gb) and torch.equal(ga[17:], gc)
 
 
+def test_rows_alone_and_inside_a_larger_call_when_the_kernel_changes_with_the_size():
+    """Automatic dispatch serves a call of at most 32 long rows with the cluster kernel and a larger one with
+    the row-per-SM kernel.  The two agree with the oracle, and therefore with each other, to the tolerances,
+    not to the bit: flags and ids wherever the oracle's decision is outside the margin, floats to 2e-5."""
+    w = synth.Workload("piece", 40, 151936, "bf16", 0.1, 1.5, True, 83, 15)
+    d = synth.generate(w, DEV)
+    lo, hi = 14, 26                                   # 12 rows
+    prev = P.set_kernel(0)
+    try:
+        big, g_big = P.route_fwd_bwd(d["s"], d["t"], d["proposal"], w.eps, seed=w.seed)
+        k_big = P.last_kernel()
+        piece, g_piece = P.route_fwd_bwd(d["s"][lo:hi], d["t"][lo:hi], d["proposal"][lo:hi], w.eps, seed=w.seed,
+                                         row_offset=lo)
+        k_piece = P.last_kernel()
+        # pinned to one kernel, the piece is bit-identical to the rows inside the large call
+        P.set_kernel(3)
+        pinned, g_pinned = P.route_fwd_bwd(d["s"][lo:hi], d["t"][lo:hi], d["proposal"][lo:hi], w.eps, seed=w.seed,
+                                           row_offset=lo)
+        torch.cuda.synchronize()
+    finally:
+        P.set_kernel(prev)
+    assert (k_big, k_piece) == (3, 2)
+    for k in big:
+        assert torch.equal(big[k][lo:hi], pinned[k]), k
+    assert torch.equal(g_big[lo:hi], g_pinned)
+    rows = list(range(lo, hi))
+    ref = _route_oracle(d, w, rows)
+    n1 = compare_rows(big, ref, rows)
+    ref_piece = dict(ref)
+    n2 = compare_rows(piece, ref_piece)
+    ok = np.minimum(ref["margin_accept"], ref["margin_draw"]) >= 1e-6
+    okt = torch.as_tensor(ok, device=DEV)
+    for k in ("corrected", "token", "teacher_top1", "row_status"):
+        assert torch.equal(big[k][lo:hi][okt], piece[k][okt]), k
+    for k in ("lambda", "tv", "kl", "accept_prob"):
+        assert float((big[k][lo:hi] - piece[k]).abs().max()) <= 2e-5, k
+    same = okt & (big["corrected"][lo:hi] == piece["corrected"])
+    dg = (g_big[lo:hi][same].float() - g_piece[same].float()).abs()
+    assert float(dg.max()) <= 4e-3
+    print(f"\n[parity] piece vs whole, V=151936: margin-exempt {n1}/{n2} of 12; gradient entries that differ "
+          f"{int((dg > 0).sum())} of {dg.numel()}, max {float(dg.max()):.2e}")
+
+
 def test_spec_verify_small(kernel):
     B, K, V = 48, 4, 3000
     w = synth.Workload("t", B * (K + 1), V, "bf16", 0.2, 1.5, True, 82, 14, K=K)
