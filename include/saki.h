@@ -227,6 +227,54 @@ typedef struct {
 /* selected: [N] uint8 (required); m: [B] int32 or NULL.  Asynchronous on the stream. */
 SAKI_API int saki_select_tm(const saki_select_in* in, uint8_t* selected, int32_t* m, void* cuda_stream);
 
+/* Vocabulary-sharded rows (the paper fixes only the [B,K,V] -> [BK,V] shape of the engine's logits,
+ * Appendix K "Engine-Resident q Backend"; with a tensor-parallel lm-head each GPU holds a slice of every
+ * row).  Rank r of `world` holds columns [v0, v0 + V_local) of both logit tensors; the slices of the ranks,
+ * taken in rank order, tile [0, V) without gaps.  A row is routed without gathering it, in stages; in each
+ * stage every rank reduces its slice to SAKI_VSHARD_PARTIALS doubles per row (saki_vshard_partial), the
+ * ranks exchange them (the caller's all-gather into [world][N][SAKI_VSHARD_PARTIALS], rank-major) and
+ * every rank folds the gathered partials, in rank order, into the same per-row state of
+ * SAKI_VSHARD_STATE doubles (saki_vshard_combine).  Stages, run in this order:
+ *   0  maxima, teacher argmax, sums of exponentials and moments of the logit difference (Section 3.1)
+ *   1  one evaluation of KL(q_beta || p) at every unsettled row's current beta (Eqs. "bridge",
+ *      "trust_region"); repeat stage 1 until the combine reports no row still solving
+ *   2  shares of TV(p, q) and KL(q || p); the combine decides acceptance (Eq. "accept"), the routed loss
+ *      (Eqs. "k1_loss_token", "teacher_mode_loss") and which rank owns the residual draw (Eq. "residual")
+ *   3  the gradient slice (Eq. "general_objective": dlogits_slice [N, V_local], same dtype, may be NULL) and,
+ *      on the owning rank, the drawn token; the combine writes the per-position outputs
+ * Everything is float64; results equal the unsharded call's to rounding (float outputs ~1e-12 before the
+ * cast to float32; flags and ids wherever the decision is not within rounding of its threshold) and do not
+ * depend on the number of ranks beyond that.  Arguments: `proposal` holds GLOBAL token ids; `state` and
+ * `partial` are caller-owned buffers ([N][SAKI_VSHARD_STATE], [N][SAKI_VSHARD_PARTIALS] doubles); `state`
+ * may be NULL at stage 0 of saki_vshard_partial.  saki_vshard_partial and saki_vshard_combine take DEVICE
+ * pointers and run asynchronously on the stream; `n_solving` (device, may be NULL) receives the number of
+ * rows that need another stage-1 wave (meaningful after stages 0 and 1).  saki_vshard_combine_host is the
+ * same combine for HOST buffers (every pointer, `proposal` and `mask` of `in` and the arrays of `out`
+ * included, is a host pointer; the logits pointers of `in` are not read): for callers that exchange
+ * through host memory.  Errors: SAKI_ERR_INVALID_ARG for NULL required pointers, a stage outside 0..3,
+ * sizes or strides that do not fit; SAKI_ERR_CUDA for a failed launch. */
+#define SAKI_VSHARD_PARTIALS 12
+#define SAKI_VSHARD_STATE 32
+typedef struct {
+  const void* student_logits;  /* DEVICE [N, V_local]: this rank's columns, unit column stride, row stride ld_s elements */
+  const void* teacher_logits;  /* DEVICE [N, V_local], row stride ld_t */
+  int64_t ld_s, ld_t, N;
+  int32_t V;                   /* the whole vocabulary */
+  int32_t V_local, v0;         /* this rank's columns are [v0, v0 + V_local) */
+  int32_t dtype;               /* SAKI_F32 or SAKI_BF16 */
+  const int32_t* proposal;     /* [N] global ids of the student's sampled tokens */
+  const uint8_t* mask;         /* [N] or NULL */
+  float eps, temperature;
+  uint64_t seed, row_offset;
+  int32_t rank, world;
+} saki_vshard_in;
+SAKI_API int saki_vshard_partial(const saki_vshard_in* in, int stage, const double* state, double* partial,
+                                 void* dlogits_slice, int64_t ld_g, float grad_scale, void* cuda_stream);
+SAKI_API int saki_vshard_combine(const saki_vshard_in* in, int stage, const double* gathered, double* state,
+                                 const saki_out* out, uint32_t* n_solving, void* cuda_stream);
+SAKI_API int saki_vshard_combine_host(const saki_vshard_in* in, int stage, const double* gathered, double* state,
+                                      const saki_out* out, int32_t* n_solving);
+
 /* Block verification (Section 3.5, Appendix I) of B drafted blocks of K tokens. */
 typedef struct {
   const void* student_logits; /* [B,K+1,V]: position j of sequence b at element offset

@@ -21,6 +21,7 @@ ROW_SATURATED, ROW_EPS_ZERO, ROW_MASKED, ROW_NONFINITE, ROW_BAD_ID, ROW_TIMEOUT,
 _FLOAT_FIELDS = ("lambda", "kl", "tv", "accept_prob", "logp_x", "logq_x", "logT_x", "logp_y", "logq_y", "logT_y", "loss")
 EXPORTS = ("saki_route_fwd", "saki_route_fwd_bwd", "saki_route_fwd_bwd_noalloc", "saki_route_host",
            "saki_route_bwd_from_meta", "saki_select_tm", "saki_spec_verify",
+           "saki_vshard_partial", "saki_vshard_combine", "saki_vshard_combine_host",
            "saki_sample_proposal", "saki_check", "saki_set_kernel", "saki_last_kernel", "saki_redo_count",
            "saki_set_spec_early_out", "saki_spec_positions_routed", "saki_solve_evaluations", "saki_set_wait_limit", "saki_set_phase_clock", "saki_phase_cycles",
            "saki_launch_count",
@@ -63,6 +64,19 @@ class SakiSelectIn(C.Structure):
     _fields_ = [("N", C.c_int64), ("B", C.c_int64), ("seq_start", C.c_void_p), ("corrected", C.c_void_p),
                 ("tv", C.c_void_p), ("mask", C.c_void_p), ("rollout_status", C.c_void_p), ("mode", C.c_int32),
                 ("seed", C.c_uint64), ("row_offset", C.c_uint64)]
+
+
+class SakiVshardIn(C.Structure):
+    _fields_ = [("student_logits", C.c_void_p), ("teacher_logits", C.c_void_p),
+                ("ld_s", C.c_int64), ("ld_t", C.c_int64), ("N", C.c_int64),
+                ("V", C.c_int32), ("V_local", C.c_int32), ("v0", C.c_int32), ("dtype", C.c_int32),
+                ("proposal", C.c_void_p), ("mask", C.c_void_p),
+                ("eps", C.c_float), ("temperature", C.c_float),
+                ("seed", C.c_uint64), ("row_offset", C.c_uint64),
+                ("rank", C.c_int32), ("world", C.c_int32)]
+
+
+VSHARD_PARTIALS, VSHARD_STATE = 12, 32
 
 
 class SakiSpecIn(C.Structure):
@@ -111,6 +125,15 @@ def load_library(path: str | None = None):
     lib.saki_spec_positions_routed.restype = C.c_int
     lib.saki_solve_evaluations.argtypes = [C.c_void_p, C.POINTER(C.c_uint64)]
     lib.saki_solve_evaluations.restype = C.c_int
+    lib.saki_vshard_partial.argtypes = [C.POINTER(SakiVshardIn), C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
+                                        C.c_float, C.c_void_p]
+    lib.saki_vshard_partial.restype = C.c_int
+    lib.saki_vshard_combine.argtypes = [C.POINTER(SakiVshardIn), C.c_int, C.c_void_p, C.c_void_p, C.POINTER(SakiOut),
+                                        C.c_void_p, C.c_void_p]
+    lib.saki_vshard_combine.restype = C.c_int
+    lib.saki_vshard_combine_host.argtypes = [C.POINTER(SakiVshardIn), C.c_int, C.c_void_p, C.c_void_p, C.POINTER(SakiOut),
+                                             C.POINTER(C.c_int32)]
+    lib.saki_vshard_combine_host.restype = C.c_int
     lib.saki_set_wait_limit.argtypes = [C.c_int64]
     lib.saki_set_wait_limit.restype = C.c_int64
     lib.saki_set_phase_clock.argtypes = [C.c_int]
@@ -297,6 +320,57 @@ def route_fwd_bwd_noalloc(s, t, proposal, eps, out, dlogits, temperature=1.0, se
     _raise(lib, lib.saki_route_fwd_bwd_noalloc(C.byref(si), C.byref(so), dlogits.data_ptr(), ld_g, grad_scale,
                                                _stream_ptr(stream)))
     return out, dlogits
+
+
+def vshard_in(s_loc, t_loc, v0, V, proposal, eps, temperature=1.0, seed=0, row_offset=0, mask=None, rank=0, world=1,
+              dtype=None, n_rows=None) -> SakiVshardIn:
+    """The argument record of the vocabulary-sharded calls: this rank's columns [v0, v0 + V_local) of both logit
+    tensors.  `s_loc` / `t_loc` may be None for the host-side combine (which reads no logits); then `dtype`
+    ("bf16" / "f32") and `n_rows` say what the slices hold."""
+    si = SakiVshardIn()
+    if s_loc is not None:
+        si.student_logits, si.teacher_logits = s_loc.data_ptr(), t_loc.data_ptr()
+        si.ld_s = s_loc.stride(0) if s_loc.shape[0] > 1 else max(1, s_loc.shape[1])
+        si.ld_t = t_loc.stride(0) if t_loc.shape[0] > 1 else max(1, t_loc.shape[1])
+        si.N, si.V_local, si.dtype = s_loc.shape[0], s_loc.shape[1], _dtype_code(s_loc)
+    else:
+        si.N, si.V_local, si.dtype = n_rows, 0, (SAKI_BF16 if dtype == "bf16" else SAKI_F32)
+    si.V, si.v0 = V, v0
+    si.proposal = proposal.data_ptr()
+    si.mask = mask.data_ptr() if mask is not None else None
+    si.eps, si.temperature, si.seed, si.row_offset = eps, temperature, seed, row_offset
+    si.rank, si.world = rank, world
+    return si
+
+
+def vshard_partial(si: SakiVshardIn, stage: int, state, partial, dlogits=None, grad_scale=1.0, stream=None):
+    """saki_vshard_partial: this rank's partial vectors of one stage (device tensors, float64)."""
+    lib = load_library()
+    ld_g = 0
+    if dlogits is not None:
+        ld_g = dlogits.stride(0) if dlogits.shape[0] > 1 else max(1, dlogits.shape[1])
+    _raise(lib, lib.saki_vshard_partial(C.byref(si), stage, state.data_ptr() if state is not None else None,
+                                        partial.data_ptr(), dlogits.data_ptr() if dlogits is not None else None, ld_g,
+                                        grad_scale, _stream_ptr(stream)))
+
+
+def vshard_combine(si: SakiVshardIn, stage: int, gathered, state, out=None, n_solving=None, stream=None):
+    """saki_vshard_combine: folds the gathered partials [world, N, 12] into the per-row state (device tensors)."""
+    lib = load_library()
+    so = _out_struct(out) if out is not None else None
+    _raise(lib, lib.saki_vshard_combine(C.byref(si), stage, gathered.data_ptr(), state.data_ptr(),
+                                        C.byref(so) if so is not None else None,
+                                        n_solving.data_ptr() if n_solving is not None else None, _stream_ptr(stream)))
+
+
+def vshard_combine_host(si: SakiVshardIn, stage: int, gathered, state, out=None) -> int:
+    """saki_vshard_combine_host: the same combine on host tensors; returns the number of rows still solving."""
+    lib = load_library()
+    so = _out_struct(out) if out is not None else None
+    n = C.c_int32(0)
+    _raise(lib, lib.saki_vshard_combine_host(C.byref(si), stage, gathered.data_ptr(), state.data_ptr(),
+                                             C.byref(so) if so is not None else None, C.byref(n)))
+    return int(n.value)
 
 
 def route_host(s, t, proposal, eps, temperature=1.0, seed=0, row_offset=0, mask=None, grad_scale=1.0,

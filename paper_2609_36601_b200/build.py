@@ -12,9 +12,9 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsaki.so")
 SOURCES = ("saki_api.cu", "saki_general.cu", "saki_cluster.cu", "saki_rowsm.cu", "saki_rowsm_half.cu", "saki_meta.cu",
-           "saki_select.cu")
+           "saki_select.cu", "saki_vshard.cu")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-         "--use_fast_math=false", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
+         "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 
 
 def _nvcc():
@@ -38,7 +38,7 @@ def build(verbose: bool = False, force: bool = False) -> str:
         return LIB
     objs = []
     procs = []
-    flags = [f for f in FLAGS if f != "--use_fast_math=false"]
+    flags = list(FLAGS)
     for src in SOURCES:
         obj = os.path.join(CSRC, src.replace(".cu", ".o"))
         cmd = [_nvcc(), *flags, "-c", os.path.join(CSRC, src), "-o", obj]

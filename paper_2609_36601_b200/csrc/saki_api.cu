@@ -436,6 +436,81 @@ SAKI_API int saki_select_tm(const saki_select_in* in, uint8_t* selected, int32_t
   return SAKI_OK;
 }
 
+static int vshard_check(const saki_vshard_in* in, int stage) {
+  if (!in) return fail(SAKI_ERR_INVALID_ARG, "NULL argument struct");
+  if (stage < 0 || stage > 3) return fail(SAKI_ERR_INVALID_ARG, "stage must be 0..3 (got %d)", stage);
+  if (in->N < 0) return fail(SAKI_ERR_INVALID_ARG, "negative row count");
+  if (in->V < 2) return fail(SAKI_ERR_INVALID_ARG, "V must be >= 2 (got %d)", in->V);
+  if (in->world < 1 || in->rank < 0 || in->rank >= in->world) return fail(SAKI_ERR_INVALID_ARG, "rank %d outside [0, %d)", in->rank, in->world);
+  if (in->V_local < 0 || in->v0 < 0 || (int64_t)in->v0 + in->V_local > in->V)
+    return fail(SAKI_ERR_INVALID_ARG, "slice [%d, %d) outside [0, %d)", in->v0, in->v0 + in->V_local, in->V);
+  if (in->dtype != SAKI_F32 && in->dtype != SAKI_BF16) return fail(SAKI_ERR_INVALID_ARG, "unknown dtype %d", in->dtype);
+  if (!(in->eps >= 0.f)) return fail(SAKI_ERR_INVALID_ARG, "eps must be >= 0 and not NaN");
+  if (!(in->temperature > 0.f) || std::isinf(in->temperature)) return fail(SAKI_ERR_INVALID_ARG, "temperature must be finite and > 0");
+  if (in->N > 0 && !in->proposal) return fail(SAKI_ERR_INVALID_ARG, "NULL proposal pointer");
+  return SAKI_OK;
+}
+
+SAKI_API int saki_vshard_partial(const saki_vshard_in* in, int stage, const double* state, double* partial,
+                                 void* dlogits_slice, int64_t ld_g, float grad_scale, void* cuda_stream) {
+  g_err[0] = 0;
+  int rc = vshard_check(in, stage);
+  if (rc) return rc;
+  if (in->N == 0) return SAKI_OK;
+  if (in->V_local > 0 && (!in->student_logits || !in->teacher_logits)) return fail(SAKI_ERR_INVALID_ARG, "NULL logits pointer");
+  if (in->ld_s < in->V_local || in->ld_t < in->V_local) return fail(SAKI_ERR_INVALID_ARG, "row stride smaller than the slice");
+  if (!partial || (stage > 0 && !state)) return fail(SAKI_ERR_INVALID_ARG, "NULL partial or state pointer");
+  if (dlogits_slice && (ld_g < in->V_local || !std::isfinite(grad_scale))) return fail(SAKI_ERR_INVALID_ARG, "bad gradient stride or scale");
+  unsigned long long* flagged = nullptr;
+  rc = device_ready(&flagged);
+  if (rc) return rc;
+  cudaError_t e = launch_vshard_partial(*in, stage, state, partial, stage == 3 ? dlogits_slice : nullptr, ld_g, grad_scale,
+                                        (cudaStream_t)cuda_stream);
+  if (e != cudaSuccess) return cuda_fail(e, "vocabulary-sharded partial kernel launch");
+  g_launches += 1;
+  return SAKI_OK;
+}
+
+SAKI_API int saki_vshard_combine(const saki_vshard_in* in, int stage, const double* gathered, double* state,
+                                 const saki_out* out, uint32_t* n_solving, void* cuda_stream) {
+  g_err[0] = 0;
+  int rc = vshard_check(in, stage);
+  if (rc) return rc;
+  if (in->N == 0) return SAKI_OK;
+  if (!gathered || !state) return fail(SAKI_ERR_INVALID_ARG, "NULL gathered or state pointer");
+  if (stage == 3 && (!out || !out->corrected || !out->token)) return fail(SAKI_ERR_INVALID_ARG, "out.corrected and out.token are required at stage 3");
+  unsigned long long* flagged = nullptr;
+  rc = device_ready(&flagged);
+  if (rc) return rc;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (n_solving) {
+    cudaError_t e0 = cudaMemsetAsync(n_solving, 0, sizeof(uint32_t), st);
+    if (e0 != cudaSuccess) return cuda_fail(e0, "cudaMemsetAsync");
+  }
+  saki_out none;
+  memset(&none, 0, sizeof(none));
+  cudaError_t e = launch_vshard_combine(*in, stage, gathered, state, out ? *out : none, n_solving, st);
+  if (e != cudaSuccess) return cuda_fail(e, "vocabulary-sharded combine kernel launch");
+  g_launches += 1;
+  return SAKI_OK;
+}
+
+SAKI_API int saki_vshard_combine_host(const saki_vshard_in* in, int stage, const double* gathered, double* state,
+                                      const saki_out* out, int32_t* n_solving) {
+  g_err[0] = 0;
+  int rc = vshard_check(in, stage);
+  if (rc) return rc;
+  if (n_solving) *n_solving = 0;
+  if (in->N == 0) return SAKI_OK;
+  if (!gathered || !state) return fail(SAKI_ERR_INVALID_ARG, "NULL gathered or state pointer");
+  if (stage == 3 && (!out || !out->corrected || !out->token)) return fail(SAKI_ERR_INVALID_ARG, "out.corrected and out.token are required at stage 3");
+  saki_out none;
+  memset(&none, 0, sizeof(none));
+  const int solving = vshard_combine_host(*in, stage, gathered, state, out ? *out : none);
+  if (n_solving) *n_solving = solving;
+  return SAKI_OK;
+}
+
 SAKI_API int saki_spec_verify(const saki_spec_in* in, const saki_spec_out* out, void* cuda_stream) {
   g_err[0] = 0;
   if (!in || !out) return fail(SAKI_ERR_INVALID_ARG, "NULL argument struct");

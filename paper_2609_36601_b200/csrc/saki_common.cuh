@@ -131,7 +131,7 @@ struct RowResult {
   uint32_t status;
 };
 
-__device__ inline void write_row(const saki_out& o, int64_t i, const RowResult& r, bool write_loss) {
+__host__ __device__ inline void write_row(const saki_out& o, int64_t i, const RowResult& r, bool write_loss) {
   o.corrected[i] = (uint8_t)r.corrected;
   o.token[i] = r.token;
   if (o.teacher_top1) o.teacher_top1[i] = r.vstar;
@@ -149,7 +149,7 @@ __device__ inline void write_row(const saki_out& o, int64_t i, const RowResult& 
   if (o.row_status) o.row_status[i] = r.status;
 }
 
-__device__ inline RowResult zero_row(uint32_t status) {
+__host__ __device__ inline RowResult zero_row(uint32_t status) {
   RowResult r;
   r.corrected = 0; r.token = -1; r.vstar = -1;
   r.lambda = r.kl = r.tv = r.accept = r.logp_x = r.logq_x = r.logT_x = r.logp_y = r.logq_y = r.logT_y = r.loss = 0.f;
@@ -169,5 +169,10 @@ cudaError_t launch_meta_general(const MetaParams& p, int dtype, cudaStream_t st,
 cudaError_t launch_meta_stream(const MetaParams& p, cudaStream_t st, int* n_launches, bool* served);
 bool meta_stream_can_serve(const MetaParams& p, int dtype);
 cudaError_t launch_select(const SelectParams& p, cudaStream_t st, int* n_launches);
+cudaError_t launch_vshard_partial(const saki_vshard_in& in, int stage, const double* state, double* partial, void* dlogits,
+                                  int64_t ld_g, float grad_scale, cudaStream_t st);
+cudaError_t launch_vshard_combine(const saki_vshard_in& in, int stage, const double* gathered, double* state, const saki_out& out,
+                                  unsigned int* n_solving, cudaStream_t st);
+int vshard_combine_host(const saki_vshard_in& in, int stage, const double* gathered, double* state, const saki_out& out);
 
 }  // namespace saki

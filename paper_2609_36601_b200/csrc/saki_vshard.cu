@@ -1,0 +1,438 @@
+// Vocabulary-sharded routing: every rank holds a contiguous slice [v0, v0 + V_local) of each logit row
+// (as a tensor-parallel lm-head produces them) and the row is routed without ever gathering it.  The work
+// is cut into stages; in each stage a rank reduces its slice to a few numbers per row (a "partial", a
+// kernel here), the ranks exchange the partials (the caller's all-gather: ~100 bytes per row and stage),
+// and every rank combines them, in rank order, into the same per-row state (a kernel here, and the same
+// function compiled for the host).  What is computed is the definition (Eqs. "bridge", "trust_region",
+// "accept", "residual", "k1_loss_token", "teacher_mode_loss", "general_objective"), in float64, with the
+// solver of the float64 row kernel (Newton on KL(q_beta||p) = eps inside a bisection bracket):
+//   stage A  maxima, teacher argmax, the two sums of exponentials and the moments of the logit
+//            difference under p and T (each under the slice's own shift; the combine rescales)
+//   stage B  one evaluation of q_beta per wave: sum e, sum e delta, sum e delta^2; repeated until every
+//            row's lambda has settled
+//   stage C  the slice's share of TV = sum [q - p]_+ and of KL(q||p), the student's logit at the teacher's
+//            argmax; the combine decides acceptance and finds the rank that owns the inverse-CDF target
+//   stage D  the gradient slice, and on the owning rank the residual draw; the last combine writes the outputs
+// One thread block per row; float64 throughout.  This path is built for correctness and for the shape of
+// the exchange, not yet for speed.
+#include "saki_common.cuh"
+#include <math_constants.h>
+#include <cmath>
+
+namespace saki {
+
+// per-row state, in doubles (the same on every rank after each combine)
+enum { VS_MODE = 0,      // 0 solving, 1 settled, 2 flagged
+       VS_STATUS, VS_MS, VS_MT, VS_VSTAR, VS_LSE_S, VS_LSE_T, VS_SX, VS_TX, VS_SV,
+       VS_BETA, VS_LO, VS_HI, VS_ITER, VS_LAM, VS_LOGZ, VS_KL, VS_TV, VS_ACC, VS_CORR,
+       VS_OWNER, VS_BEFORE, VS_TARGET, VS_TAKE_LAST, VS_TOK, VS_COEF, VS_LOSS, VS_Y, VS_SY, VS_TY,
+       VS_COUNT };
+static_assert(VS_COUNT <= SAKI_VSHARD_STATE, "state record too small");
+enum { VS_SOLVING = 0, VS_SETTLED = 1, VS_FLAGGED = 2 };
+
+struct VsConsts {
+  int64_t N;
+  int32_t V, world;
+  double eps, tau;
+  uint64_t seed, row_offset;
+  const int32_t* proposal;
+  const uint8_t* mask;
+};
+
+// ---------------------------------------------------------------- the combine steps (host and device)
+// `part`: [world][N][SAKI_VSHARD_PARTIALS] gathered partials; row i of rank r at part[(r * N + i) * P].
+__host__ __device__ inline void vs_combine_a(const VsConsts& c, int64_t i, const double* part, double* st) {
+  const int P = SAKI_VSHARD_PARTIALS;
+  for (int k = 0; k < SAKI_VSHARD_STATE; ++k) st[k] = 0.0;
+  double ms = -INFINITY, mt = -INFINITY, am = 2147483647.0;
+  bool finite = true;
+  for (int r = 0; r < c.world; ++r) {
+    const double* p = part + ((int64_t)r * c.N + i) * P;
+    if (p[3] == 0.0) finite = false;
+    if (p[0] > ms) ms = p[0];
+    if (p[1] > mt || (p[1] == mt && p[2] < am)) { mt = p[1]; am = p[2]; }   // lowest index among ties
+  }
+  const int x = c.proposal[i];
+  uint32_t status = 0;
+  if (!finite || !(ms > -INFINITY) || !(mt > -INFINITY)) status = SAKI_ROW_NONFINITE;
+  else if (x < 0 || x >= c.V) status = SAKI_ROW_BAD_ID;
+  st[VS_MS] = ms; st[VS_MT] = mt; st[VS_VSTAR] = am < 2147483647.0 ? am : 0.0;
+  if (status) { st[VS_STATUS] = (double)status; st[VS_MODE] = VS_FLAGGED; return; }
+  double Ss = 0.0, St = 0.0, Td = 0.0, Sd = 0.0, Sd2 = 0.0, sx = 0.0, tx = 0.0;
+  for (int r = 0; r < c.world; ++r) {      // rank order: the summation order is part of the protocol
+    const double* p = part + ((int64_t)r * c.N + i) * P;
+    const double fs = exp((p[0] - ms) / c.tau), ft = exp((p[1] - mt) / c.tau);
+    if (p[4] > 0.0) { Ss += fs * p[4]; Sd += fs * p[7]; Sd2 += fs * p[8]; }
+    if (p[5] > 0.0) { St += ft * p[5]; Td += ft * p[6]; }
+    sx += p[9]; tx += p[10];
+  }
+  const double lse_s = ms / c.tau + log(Ss), lse_t = mt / c.tau + log(St);
+  st[VS_LSE_S] = lse_s; st[VS_LSE_T] = lse_t; st[VS_SX] = sx; st[VS_TX] = tx;
+  if (!(c.eps > 0.0)) { st[VS_STATUS] = (double)SAKI_ROW_EPS_ZERO; st[VS_MODE] = VS_SETTLED; return; }   // lambda = 0, log Z = 0
+  const double cc = lse_t - lse_s;                       // d = delta - cc with delta = (t - s) / tau
+  const double kl1 = Td / St - cc;                       // KL(T || p)
+  if (kl1 <= c.eps) {                                    // teacher endpoint: q = T, log Z(1) = 0
+    st[VS_LAM] = 1.0; st[VS_STATUS] = (double)SAKI_ROW_SATURATED; st[VS_MODE] = VS_SETTLED;
+    return;
+  }
+  const double m1 = Sd / Ss, var = Sd2 / Ss - m1 * m1;   // the variance of delta is the variance of d
+  double beta = sqrt(2.0 * c.eps / fmax(var, 1e-300));
+  if (!(beta > 0.0 && beta < 1.0)) beta = 0.5;
+  st[VS_BETA] = beta; st[VS_LO] = 0.0; st[VS_HI] = 1.0; st[VS_MODE] = VS_SOLVING;
+}
+
+// one Newton step on KL(q_beta || p) = eps inside the bisection bracket; returns 1 if the row is still solving
+__host__ __device__ inline int vs_combine_b(const VsConsts& c, int64_t i, const double* part, double* st) {
+  if ((int)st[VS_MODE] != VS_SOLVING) return 0;
+  const int P = SAKI_VSHARD_PARTIALS;
+  double a0 = 0.0, a1 = 0.0, a2 = 0.0;
+  for (int r = 0; r < c.world; ++r) {
+    const double* p = part + ((int64_t)r * c.N + i) * P;
+    a0 += p[0]; a1 += p[1]; a2 += p[2];
+  }
+  const double beta = st[VS_BETA], cc = st[VS_LSE_T] - st[VS_LSE_S];
+  const double kb = ((1.0 - beta) * st[VS_MS] + beta * st[VS_MT]) / c.tau;    // the shift the partials were taken under
+  const double md = a1 / a0, E = md - cc, var = a2 / a0 - md * md;
+  const double logZ = log(a0) + kb - (1.0 - beta) * st[VS_LSE_S] - beta * st[VS_LSE_T];
+  const double kl = beta * E - logZ;
+  double lo = st[VS_LO], hi = st[VS_HI];
+  if (kl <= c.eps) lo = beta; else hi = beta;
+  const int it = (int)st[VS_ITER] + 1;
+  double lam = -1.0;
+  const double step = (c.eps - kl) / (beta * var);
+  if (hi - lo < 1e-13 || it >= 100) lam = beta;
+  else if (fabs(step) < 1e-12) lam = fmin(fmax(beta + step, lo), hi);   // a wave is a pass and an exchange: stop at 1e-12
+  else {
+    double nb = beta + step;
+    if (!(nb > lo && nb < hi)) nb = 0.5 * (lo + hi);
+    st[VS_BETA] = nb; st[VS_LO] = lo; st[VS_HI] = hi; st[VS_ITER] = (double)it;
+    return 1;
+  }
+  st[VS_LAM] = lam;
+  st[VS_LOGZ] = logZ + (lam - beta) * E;                 // |lam - beta| < 1e-12: first order is exact to rounding
+  st[VS_MODE] = VS_SETTLED;
+  return 0;
+}
+
+// TV, KL, the coupling decision, the routed loss and the owner of the residual draw
+__host__ __device__ inline void vs_combine_c(const VsConsts& c, int64_t i, const double* part, double* st) {
+  if ((int)st[VS_MODE] == VS_FLAGGED) return;
+  const int P = SAKI_VSHARD_PARTIALS;
+  double tv = 0.0, kl = 0.0, sv = 0.0;
+  for (int r = 0; r < c.world; ++r) {
+    const double* p = part + ((int64_t)r * c.N + i) * P;
+    tv += p[0]; kl += p[1]; sv += p[2];
+  }
+  const double lam = st[VS_LAM], logZ = st[VS_LOGZ];
+  const int x = c.proposal[i];
+  const uint64_t rid = c.row_offset + (uint64_t)i;
+  const double lp_x = st[VS_SX] / c.tau - st[VS_LSE_S], lT_x = st[VS_TX] / c.tau - st[VS_LSE_T];
+  double acc = 1.0;
+  int corrected = 0;
+  if (lam > 0.0) {
+    acc = exp(fmin(0.0, lam * (lT_x - lp_x) - logZ));
+    corrected = (scalar_uniform(c.seed, rid, STAGE_ACCEPT) < acc) ? 0 : 1;
+  } else { tv = 0.0; kl = 0.0; }
+  st[VS_SV] = sv; st[VS_TV] = tv; st[VS_KL] = kl; st[VS_ACC] = acc; st[VS_CORR] = (double)corrected;
+  st[VS_OWNER] = -1.0; st[VS_Y] = (double)x; st[VS_SY] = st[VS_SX]; st[VS_TY] = st[VS_TX];
+  if (corrected) {        // inverse CDF in index order: slices are contiguous, so rank order is index order
+    const double target = scalar_uniform(c.seed, rid, STAGE_RESIDUAL) * tv;
+    int owner = -1;
+    double before = 0.0;
+    for (int r = 0; r < c.world; ++r) {
+      const double w = part[((int64_t)r * c.N + i) * P];
+      if (before + w > target) { owner = r; break; }
+      before += w;
+    }
+    double take_last = 0.0;
+    if (owner < 0) {      // rounding left no crossing: the last index with positive weight
+      take_last = 1.0; before = 0.0;
+      for (int r = c.world - 1; r >= 0; --r) if (part[((int64_t)r * c.N + i) * P] > 0.0) { owner = r; break; }
+      if (owner < 0) owner = c.world - 1;
+    }
+    st[VS_OWNER] = (double)owner; st[VS_BEFORE] = before; st[VS_TARGET] = target; st[VS_TAKE_LAST] = take_last;
+  }
+  const bool masked = c.mask != nullptr && c.mask[i] == 0;
+  uint32_t status = (uint32_t)st[VS_STATUS];
+  double loss = 0.0, coef = 0.0;
+  int tok = -1;
+  if (masked) status |= SAKI_ROW_MASKED;
+  else if (!corrected) { loss = (lp_x - lT_x) * lp_x; coef = -(lp_x - lT_x); tok = x; }
+  else { loss = -(sv / c.tau - st[VS_LSE_S]); coef = 1.0; tok = (int)st[VS_VSTAR]; }
+  st[VS_STATUS] = (double)status; st[VS_LOSS] = loss; st[VS_COEF] = coef; st[VS_TOK] = (double)tok;
+}
+
+// the drawn token and the per-position outputs
+__host__ __device__ inline void vs_combine_d(const VsConsts& c, int64_t i, const double* part, double* st, const saki_out& o) {
+  if ((int)st[VS_MODE] == VS_FLAGGED) { write_row(o, i, zero_row((uint32_t)st[VS_STATUS]), true); return; }
+  const int P = SAKI_VSHARD_PARTIALS;
+  if (st[VS_CORR] != 0.0) {
+    double y = -1.0, sy = 0.0, ty = 0.0;
+    for (int r = 0; r < c.world; ++r) {
+      const double* p = part + ((int64_t)r * c.N + i) * P;
+      if (p[0] >= 0.0) { y = p[0]; sy = p[1]; ty = p[2]; }
+    }
+    st[VS_Y] = y; st[VS_SY] = sy; st[VS_TY] = ty;
+  }
+  const double lam = st[VS_LAM], logZ = st[VS_LOGZ];
+  RowResult r;
+  r.corrected = (int)st[VS_CORR]; r.token = (int)st[VS_Y]; r.vstar = (int)st[VS_VSTAR];
+  r.lambda = (float)lam; r.kl = (float)st[VS_KL]; r.tv = (float)st[VS_TV]; r.accept = (float)st[VS_ACC];
+  const double lp_x = st[VS_SX] / c.tau - st[VS_LSE_S], lT_x = st[VS_TX] / c.tau - st[VS_LSE_T];
+  const double lp_y = st[VS_SY] / c.tau - st[VS_LSE_S], lT_y = st[VS_TY] / c.tau - st[VS_LSE_T];
+  r.logp_x = (float)lp_x; r.logT_x = (float)lT_x; r.logq_x = (float)(lp_x + lam * (lT_x - lp_x) - logZ);
+  r.logp_y = (float)lp_y; r.logT_y = (float)lT_y; r.logq_y = (float)(lp_y + lam * (lT_y - lp_y) - logZ);
+  r.loss = (float)st[VS_LOSS]; r.status = (uint32_t)st[VS_STATUS];
+  write_row(o, i, r, true);
+}
+
+// ---------------------------------------------------------------- partial kernels: one block per row
+constexpr int VT = 512, VW = VT / 32;
+
+template <int NV>
+__device__ __forceinline__ void vs_block_sum(double (&v)[NV], double* sh) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int k = 0; k < NV; ++k) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v[k] += __shfl_xor_sync(0xffffffffu, v[k], o);
+  }
+  if (lane == 0) {
+#pragma unroll
+    for (int k = 0; k < NV; ++k) sh[k * VW + warp] = v[k];
+  }
+  __syncthreads();
+#pragma unroll
+  for (int k = 0; k < NV; ++k) {
+    double a = 0.0;
+#pragma unroll
+    for (int w = 0; w < VW; ++w) a += sh[k * VW + w];
+    v[k] = a;
+  }
+  __syncthreads();
+}
+
+struct VsSlice {
+  const void *s, *t;
+  int64_t ld_s, ld_t, N;
+  int32_t V_local, v0, rank;
+  double tau;
+  const int32_t* proposal;
+};
+
+template <typename T>
+__global__ void __launch_bounds__(VT) vs_partial_kernel(const VsSlice S, const int stage, const double* state, double* partial,
+                                                        void* dlogits, const int64_t ld_g, const double grad_scale) {
+  __shared__ double red[6 * VW];
+  __shared__ float smax[2][VW];
+  __shared__ int sarg[VW];
+  __shared__ int stoken;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int Vl = S.V_local;
+  const double rtau = 1.0 / S.tau;
+  for (int64_t row = blockIdx.x; row < S.N; row += gridDim.x) {
+    const T* s = (const T*)S.s + row * S.ld_s;
+    const T* t = (const T*)S.t + row * S.ld_t;
+    double* out = partial + row * SAKI_VSHARD_PARTIALS;
+    const double* st = state ? state + row * SAKI_VSHARD_STATE : nullptr;
+    if (stage == 0) {
+      // ---- stage A: maxima and argmax, then the sums under this slice's own shifts
+      float ms = -CUDART_INF_F, mt = -CUDART_INF_F;
+      int am = 0x7fffffff, finite = 1;
+      for (int v = tid; v < Vl; v += VT) {
+        const float a = ld_as_float(s, v), c = ld_as_float(t, v);
+        finite &= (isfinite(a) && isfinite(c)) ? 1 : 0;
+        ms = fmaxf(ms, a);
+        if (c > mt) { mt = c; am = v; }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        ms = fmaxf(ms, __shfl_xor_sync(0xffffffffu, ms, o));
+        const float omt = __shfl_xor_sync(0xffffffffu, mt, o);
+        const int oam = __shfl_xor_sync(0xffffffffu, am, o);
+        if (omt > mt || (omt == mt && oam < am)) { mt = omt; am = oam; }
+      }
+      if (lane == 0) { smax[0][warp] = ms; smax[1][warp] = mt; sarg[warp] = am; }
+      finite = __syncthreads_and(finite);
+      ms = smax[0][0]; mt = smax[1][0]; am = sarg[0];
+      for (int w = 1; w < VW; ++w) {
+        ms = fmaxf(ms, smax[0][w]);
+        if (smax[1][w] > mt || (smax[1][w] == mt && sarg[w] < am)) { mt = smax[1][w]; am = sarg[w]; }
+      }
+      __syncthreads();
+      double a[5] = {0.0, 0.0, 0.0, 0.0, 0.0};
+      if (finite && Vl > 0) {
+        const double zms = (double)ms * rtau, zmt = (double)mt * rtau;
+        for (int v = tid; v < Vl; v += VT) {
+          const double zs = (double)ld_as_float(s, v) * rtau, zt = (double)ld_as_float(t, v) * rtau;
+          const double es = exp(zs - zms), et = exp(zt - zmt), dl = zt - zs;
+          a[0] += es; a[1] += et; a[2] += et * dl; a[3] += es * dl; a[4] += es * dl * dl;
+        }
+      }
+      vs_block_sum<5>(a, red);
+      if (tid == 0) {
+        const int x = S.proposal[row] - S.v0;
+        const bool own = x >= 0 && x < Vl;
+        out[0] = (double)ms; out[1] = (double)mt; out[2] = am == 0x7fffffff ? 2147483647.0 : (double)(S.v0 + am);
+        out[3] = finite ? 1.0 : 0.0;
+        out[4] = a[0]; out[5] = a[1]; out[6] = a[2]; out[7] = a[3]; out[8] = a[4];
+        out[9] = own ? (double)ld_as_float(s, x) : 0.0; out[10] = own ? (double)ld_as_float(t, x) : 0.0;
+        out[11] = own ? 1.0 : 0.0;
+      }
+    } else if (stage == 1) {
+      // ---- stage B: one evaluation at the row's current beta, under the row's global shift
+      double a[3] = {0.0, 0.0, 0.0};
+      if ((int)st[VS_MODE] == VS_SOLVING) {
+        const double beta = st[VS_BETA];
+        const double kb = ((1.0 - beta) * st[VS_MS] + beta * st[VS_MT]) * rtau;
+        for (int v = tid; v < Vl; v += VT) {
+          const double zs = (double)ld_as_float(s, v) * rtau, zt = (double)ld_as_float(t, v) * rtau;
+          const double dl = zt - zs, e = exp(zs + beta * dl - kb);
+          a[0] += e; a[1] += e * dl; a[2] += e * dl * dl;
+        }
+      }
+      vs_block_sum<3>(a, red);
+      if (tid == 0) {
+        for (int k = 0; k < SAKI_VSHARD_PARTIALS; ++k) out[k] = 0.0;
+        out[0] = a[0]; out[1] = a[1]; out[2] = a[2];
+      }
+    } else if (stage == 2) {
+      // ---- stage C: the slice's share of TV and KL(q||p); the student's logit at the teacher's argmax
+      double a[2] = {0.0, 0.0};
+      const bool live = (int)st[VS_MODE] == VS_SETTLED;
+      const double lam = st[VS_LAM];
+      if (live && lam > 0.0) {
+        const double lse_s = st[VS_LSE_S], lse_t = st[VS_LSE_T], logZ = st[VS_LOGZ];
+        // per-warp segments in index order, summed in warp order: close to the index-order sum of the definition
+        const int seg = (Vl + VW - 1) / VW, v_lo = warp * seg, v_hi = min(Vl, v_lo + seg);
+        for (int v = v_lo + lane; v < v_hi; v += 32) {
+          const double lp = (double)ld_as_float(s, v) * rtau - lse_s, lT = (double)ld_as_float(t, v) * rtau - lse_t;
+          const double lq = lp + lam * (lT - lp) - logZ, q = exp(lq);
+          a[0] += fmax(q - exp(lp), 0.0);
+          a[1] += q * (lq - lp);
+        }
+      }
+      vs_block_sum<2>(a, red);
+      if (tid == 0) {
+        for (int k = 0; k < SAKI_VSHARD_PARTIALS; ++k) out[k] = 0.0;
+        const int vs = (int)st[VS_VSTAR] - S.v0;
+        out[0] = a[0]; out[1] = a[1];
+        out[2] = (live && vs >= 0 && vs < Vl) ? (double)ld_as_float(s, vs) : 0.0;
+      }
+    } else {
+      // ---- stage D: the gradient slice; on the owning rank the residual draw
+      const int mode = (int)st[VS_MODE];
+      T* g = dlogits ? (T*)dlogits + row * ld_g : nullptr;
+      if (g) {
+        const double sc = mode == VS_FLAGGED ? 0.0 : grad_scale * st[VS_COEF] * rtau;
+        const double lse_s = st[VS_LSE_S];
+        const int tok = mode == VS_FLAGGED ? -1 : (int)st[VS_TOK] - S.v0;
+        for (int v = tid; v < Vl; v += VT) {
+          double gv = 0.0;
+          if (sc != 0.0) gv = sc * (exp((double)ld_as_float(s, v) * rtau - lse_s) - (v == tok ? 1.0 : 0.0));
+          if constexpr (sizeof(T) == 2) g[v] = __double2bfloat16(gv);
+          else g[v] = (float)gv;
+        }
+      }
+      if (tid == 0) stoken = -1;
+      __syncthreads();
+      const bool mine = mode == VS_SETTLED && st[VS_CORR] != 0.0 && (int)st[VS_OWNER] == S.rank;
+      if (mine && warp == 0) {
+        const double lam = st[VS_LAM], lse_s = st[VS_LSE_S], lse_t = st[VS_LSE_T], logZ = st[VS_LOGZ];
+        const double target = st[VS_TARGET];
+        const bool take_last = st[VS_TAKE_LAST] != 0.0;
+        double running = st[VS_BEFORE];
+        int last_pos = -1, found = -1;
+        for (int v0 = 0; v0 < Vl && found < 0; v0 += 32) {
+          const int v = v0 + lane;
+          double r = 0.0;
+          if (v < Vl) {
+            const double lp = (double)ld_as_float(s, v) * rtau - lse_s, lT = (double)ld_as_float(t, v) * rtau - lse_t;
+            r = fmax(exp(lp + lam * (lT - lp) - logZ) - exp(lp), 0.0);
+          }
+          double inc = r;
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const double up = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += up;
+          }
+          const unsigned pos = __ballot_sync(0xffffffffu, r > 0.0);
+          const unsigned hit = take_last ? 0u : __ballot_sync(0xffffffffu, (running + inc > target) && v < Vl);
+          if (pos) last_pos = v0 + 31 - __clz(pos);
+          if (hit) found = v0 + __ffs(hit) - 1;
+          running += __shfl_sync(0xffffffffu, inc, 31);
+        }
+        if (found < 0) found = last_pos >= 0 ? last_pos : max(Vl - 1, 0);
+        if (lane == 0) stoken = found;
+      }
+      __syncthreads();
+      if (tid == 0) {
+        for (int k = 0; k < SAKI_VSHARD_PARTIALS; ++k) out[k] = 0.0;
+        out[0] = -1.0;
+        if (mine && stoken >= 0 && stoken < Vl) {
+          out[0] = (double)(S.v0 + stoken);
+          out[1] = (double)ld_as_float(s, stoken); out[2] = (double)ld_as_float(t, stoken);
+        }
+      }
+      __syncthreads();
+    }
+  }
+}
+
+__global__ void vs_combine_kernel(const VsConsts C, const int stage, const double* part, double* state, const saki_out o,
+                                  unsigned int* n_solving) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= C.N) return;
+  double* st = state + i * SAKI_VSHARD_STATE;
+  if (stage == 0) { vs_combine_a(C, i, part, st); if ((int)st[VS_MODE] == VS_SOLVING && n_solving) atomicAdd(n_solving, 1u); }
+  else if (stage == 1) { if (vs_combine_b(C, i, part, st) && n_solving) atomicAdd(n_solving, 1u); }
+  else if (stage == 2) vs_combine_c(C, i, part, st);
+  else vs_combine_d(C, i, part, st, o);
+}
+
+cudaError_t launch_vshard_partial(const saki_vshard_in& in, int stage, const double* state, double* partial, void* dlogits,
+                                  int64_t ld_g, float grad_scale, cudaStream_t st) {
+  VsSlice S;
+  S.s = in.student_logits; S.t = in.teacher_logits; S.ld_s = in.ld_s; S.ld_t = in.ld_t; S.N = in.N;
+  S.V_local = in.V_local; S.v0 = in.v0; S.rank = in.rank; S.tau = (double)in.temperature; S.proposal = in.proposal;
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int grid = (int)(in.N < 3LL * sms ? in.N : 3LL * sms);
+  if (in.dtype == SAKI_BF16)
+    vs_partial_kernel<__nv_bfloat16><<<dim3(grid, 1, 1), VT, 0, st>>>(S, stage, state, partial, dlogits, ld_g, (double)grad_scale);
+  else
+    vs_partial_kernel<float><<<dim3(grid, 1, 1), VT, 0, st>>>(S, stage, state, partial, dlogits, ld_g, (double)grad_scale);
+  return cudaGetLastError();
+}
+
+static VsConsts consts_of(const saki_vshard_in& in) {
+  VsConsts c;
+  c.N = in.N; c.V = in.V; c.world = in.world; c.eps = (double)in.eps; c.tau = (double)in.temperature;
+  c.seed = in.seed; c.row_offset = in.row_offset; c.proposal = in.proposal; c.mask = in.mask;
+  return c;
+}
+
+cudaError_t launch_vshard_combine(const saki_vshard_in& in, int stage, const double* gathered, double* state, const saki_out& out,
+                                  unsigned int* n_solving, cudaStream_t st) {
+  const VsConsts c = consts_of(in);
+  const int th = 128;
+  vs_combine_kernel<<<(unsigned)((in.N + th - 1) / th), th, 0, st>>>(c, stage, gathered, state, out, n_solving);
+  return cudaGetLastError();
+}
+
+// the same combine on HOST buffers (a caller without a GPU at hand, and the multi-process tests of the exchange)
+int vshard_combine_host(const saki_vshard_in& in, int stage, const double* gathered, double* state, const saki_out& out) {
+  const VsConsts c = consts_of(in);
+  int solving = 0;
+  for (int64_t i = 0; i < in.N; ++i) {
+    double* st = state + i * SAKI_VSHARD_STATE;
+    if (stage == 0) { vs_combine_a(c, i, gathered, st); solving += (int)st[VS_MODE] == VS_SOLVING; }
+    else if (stage == 1) solving += vs_combine_b(c, i, gathered, st);
+    else if (stage == 2) vs_combine_c(c, i, gathered, st);
+    else vs_combine_d(c, i, gathered, st, out);
+  }
+  return solving;
+}
+
+}  // namespace saki

@@ -1,0 +1,87 @@
+"""Vocabulary-sharded routing on the GPU: the rows' columns cut into 2, 8 and uneven slices, every slice
+reduced by its own kernel calls (one rank after the other on the one device: the same calls, in the same
+order, that one rank per GPU makes around its all-gather), against the float64 oracle on the whole rows and
+against the unsharded call."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+import paper_2609_36601_b200 as P
+from paper_2609_36601_b200 import synth
+from paper_2609_36601_b200.vshard import route_vocab_sharded_local, split_columns
+from parity import compare_rows, grad_check, oracle_inputs, to_np64
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _slices(d, cuts):
+    return [(d["s"][:, a:a + n], d["t"][:, a:a + n], a) for a, n in cuts]
+
+
+def _special_rows(d, w):
+    mask = torch.ones(w.N, dtype=torch.uint8, device=DEV)
+    mask[3] = 0
+    d["proposal"][5] = w.V + 1                                    # bad id
+    d["s"][6, w.V // 2 + 11] = float("nan")                        # non-finite, in the second half of the row
+    d["t"][8] = (d["s"][8].float() + 0.01).to(d["t"].dtype)        # teacher = student up to a constant: lambda = 1
+    return mask
+
+
+@pytest.mark.parametrize("V,world", [(151936, 2), (151936, 8), (32000, 3), (1000, 7)])
+def test_sliced_rows_match_the_oracle_and_the_unsharded_call(V, world):
+    w = synth.Workload("vs", 40, V, "bf16", 0.1, 1.5, True, 900 + world, 40 + world)
+    d = synth.generate(w, DEV)
+    mask = _special_rows(d, w)
+    cuts = split_columns(V, world)
+    if world == 7:                                               # uneven, with an empty slice in the middle
+        cuts = [(0, 100), (100, 0), (100, 250), (350, 1), (351, 349), (700, 299), (999, 1)]
+    out, gs, waves = route_vocab_sharded_local(_slices(d, cuts), V, d["proposal"], w.eps, w.temperature, w.seed, mask=mask,
+                                               grad_scale=0.5)
+    torch.cuda.synchronize()
+    g = torch.cat(gs, dim=1)
+    assert 3 <= waves <= 12
+    s64, t64 = oracle_inputs(d)
+    ref = O.route(s64, t64, d["proposal"].cpu().numpy(), w.eps, w.temperature, w.seed, 0, mask=mask.cpu().numpy(),
+                  grad_scale=0.5, want_grad=True, grad_dtype=w.dtype)
+    n_exempt = compare_rows(out, ref)
+    assert n_exempt <= 2
+    same = out["corrected"].cpu().numpy() == ref["corrected"]
+    live = same & (ref["status"] & (8 | 16) == 0)
+    tok = np.where(ref["corrected"] == 1, ref["teacher_top1"], ref["token"])
+    grad_check(to_np64(g)[live], ref["grad"][live], w.dtype, tok[live])
+    assert torch.all(g[5] == 0) and torch.all(g[6] == 0) and torch.all(g[3] == 0)      # flagged and masked rows
+    assert np.max(np.abs(out["lambda"].cpu().numpy() - ref["lam"])) <= 1e-6          # float64 all the way
+    st = ref["status"]
+    assert st[3] & 4 and st[5] == 16 and st[6] == 8 and st[8] & 1
+    # the unsharded float64 kernel on the same rows: same flags and ids, floats to float32 rounding
+    prev = P.set_kernel(1)
+    try:
+        whole, g_whole = P.route_fwd_bwd(d["s"], d["t"], d["proposal"], w.eps, w.temperature, w.seed, mask=mask, grad_scale=0.5)
+        torch.cuda.synchronize()
+    finally:
+        P.set_kernel(prev)
+    ok = torch.as_tensor(np.minimum(ref["margin_accept"], ref["margin_draw"]) >= 1e-6, device=DEV)
+    for k in ("corrected", "token", "teacher_top1", "row_status"):
+        assert torch.equal(out[k][ok], whole[k][ok]), k
+    for k in ("lambda", "tv", "kl", "accept_prob", "loss", "logp_x", "logq_y"):
+        assert float((out[k] - whole[k]).abs().max()) <= 1e-6 * (1 + float(whole[k].abs().max())), k
+    print(f"\n[parity] vocabulary-sharded V={V} world={world}: {waves} evaluation waves, margin-exempt {n_exempt}, "
+          f"corrected {int(ref['corrected'].sum())} of {w.N}")
+
+
+@pytest.mark.parametrize("eps", [0.0, 5.0])
+def test_endpoints_need_no_evaluation_wave(eps):
+    w = synth.Workload("vs", 16, 8192, "bf16", eps, 1.0, True, 77, 9)
+    d = synth.generate(w, DEV)
+    out, gs, waves = route_vocab_sharded_local(_slices(d, split_columns(w.V, 4)), w.V, d["proposal"], eps, seed=w.seed)
+    torch.cuda.synchronize()
+    s64, t64 = oracle_inputs(d)
+    ref = O.route(s64, t64, d["proposal"].cpu().numpy(), eps, 1.0, w.seed, want_grad=True, grad_dtype=w.dtype)
+    compare_rows(out, ref)
+    if eps == 0.0:
+        assert waves == 0 and int(out["corrected"].sum()) == 0
+    else:
+        assert np.all(ref["lam"] == 1.0) and waves == 0
+    grad_check(to_np64(torch.cat(gs, dim=1)), ref["grad"], w.dtype, np.where(ref["corrected"] == 1, ref["teacher_top1"], ref["token"]))
