@@ -18,6 +18,7 @@ def test_expired_wait_flags_rows_and_leaves_the_library_usable(V, N):
     w = synth.Workload("limit", N, V, "bf16", 0.1, 1.5, True, 4100 + V % 97, 9)
     d = synth.generate(w, DEV)
     prev_k = P.set_kernel(3)
+    P.check()                                       # clears what earlier tests may have left
     try:
         ref, g_ref = P.route_fwd_bwd(d["s"], d["t"], d["proposal"], w.eps, seed=w.seed)
         torch.cuda.synchronize()
