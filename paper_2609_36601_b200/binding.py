@@ -436,11 +436,13 @@ def check(stream=None) -> int:
 
 
 def set_kernel(which: int) -> int:
+    """saki_set_kernel: 0 automatic, 1 general (float64), 2 cluster, 3 row-per-SM; returns the previous choice."""
     return load_library().saki_set_kernel(which)
 
 
 def last_kernel() -> int:
-    """1 = general kernel, 2 = cluster kernel (the calling thread's last routing call)."""
+    """The kernel that served the calling thread's last routing call: 1 general (float64), 2 cluster, 3 row-per-SM,
+    4 the streaming kernel of route_bwd_from_meta."""
     return load_library().saki_last_kernel()
 
 

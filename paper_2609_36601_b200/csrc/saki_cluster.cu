@@ -1,4 +1,4 @@
-// Register-resident cluster kernel for bf16 rows (the hot path).
+// Register-resident cluster kernel for bf16 rows: the latency path (calls of a few long rows).
 //
 // One vocabulary row per thread-block cluster of CS CTAs x 256 threads, two
 // CTAs resident per SM.  Each CTA owns a contiguous slice of the row; each
@@ -14,9 +14,10 @@
 //            pass runs), moments of the teacher-student logit difference under
 //            p (initial guess of lambda), KL(T||p) (saturation test), teacher
 //            argmax index
-//   solve    1 exponential/element per evaluation of KL(q_beta||p) and its
-//            slope; Newton on sqrt(KL) inside a bisection bracket, typically
-//            two evaluations (Eqs. "bridge", "trust_region")
+//   solve    1 exponential/element per evaluation of KL(q_beta||p) and the first
+//            four cumulants of the logit difference under q_beta; lambda = root of
+//            the fourth-order Taylor model inside a bisection bracket, one
+//            evaluation for most rows (Eqs. "bridge", "trust_region")
 //   final    2 exponentials/element: TV = sum [q-p]_+ with per-thread ordered
 //            partial sums for the inverse-CDF residual draw (Eqs. "accept",
 //            "residual"), and the gradient row written straight from

@@ -1,8 +1,8 @@
 // General row kernel: one thread block per position, any V, dtype and strides.
 // All arithmetic is float64 and every pass re-reads the row from global
 // memory (L2 after the first pass).  It is the library's fallback for layouts
-// the register-resident cluster kernel does not serve, and the slow, careful
-// path.  Steps follow the method's definition:
+// the bf16 streaming kernels do not serve (fp32 logits, odd strides, ragged V), their second tier
+// (rows they hand over through the row list), and the slow, careful path.  Steps follow the method's definition:
 //   log-softmax x2 -> lambda (Eqs. "bridge", "trust_region") -> TV and the
 //   maximal coupling (Eqs. "accept", "residual") -> routed loss (Eqs.
 //   "k1_loss_token", "teacher_mode_loss") -> gradient (Eq. "general_objective").
@@ -162,11 +162,13 @@ __global__ void __launch_bounds__(GT) general_kernel(const RowParams P) {
           const double kl = beta * E - log(a[0]);
           if (kl <= eps) lo = beta; else hi = beta;
           if (hi - lo < 1e-15) break;
-          double nb = beta + (eps - kl) / (beta * var);
+          const double step = (eps - kl) / (beta * var);
+          // at the root to rounding: stop here (a step that small can fall outside the bracket, and the
+          // bisection that would follow costs some thirty more passes for nothing)
+          if (fabs(step) < 1e-13) { beta = fmin(fmax(beta + step, lo), hi); break; }
+          double nb = beta + step;
           if (!(nb > lo && nb < hi)) nb = 0.5 * (lo + hi);
-          const bool done = fabs(nb - beta) < 1e-15;
           beta = nb;
-          if (done) break;
         }
         lam = beta;
       }
