@@ -275,6 +275,29 @@ SAKI_API int saki_vshard_combine(const saki_vshard_in* in, int stage, const doub
 SAKI_API int saki_vshard_combine_host(const saki_vshard_in* in, int stage, const double* gathered, double* state,
                                       const saki_out* out, int32_t* n_solving);
 
+/* The step in front of the path (Section 3.5, Appendix K: drafting and verification leave full-vocabulary
+ * logits): logits = hidden x weight^T in bf16 on the tensor cores, fp32 accumulation, with the row
+ * statistics of the first pass of routing (Section 3.1: p = softmax(logits / tau)) taken in the GEMM's
+ * epilogue from the ROUNDED bf16 values that are stored: row_max[i] = max_v logits[i, v] and
+ * lse[i] = log sum_v exp(logits[i, v] / temperature).  All pointers are DEVICE pointers owned by the caller:
+ *   hidden  [N, d] bf16, unit stride along d, row stride ld_h elements
+ *   weight  [V, d] bf16 (one row per vocabulary entry), row stride ld_w
+ *   logits  [N, V] bf16 out, row stride ld_l; row_max, lse: [N] float out (either may be NULL)
+ *   scratch saki_lmhead_scratch_bytes(N, V) bytes, 256-byte aligned (per-tile partial statistics)
+ * Requirements: 16-byte aligned hidden / weight / logits, ld_h, ld_w, ld_l and V multiples of 8, d >= 8.
+ * Asynchronous on the stream.  Errors: SAKI_ERR_INVALID_ARG (NULL pointers, sizes, strides, scratch too
+ * small), SAKI_ERR_UNSUPPORTED (alignment), SAKI_ERR_CUDA.  Every wait inside the kernel is bounded; should
+ * one run out (a fault of the machine, not of the data) the kernel still returns and row_max and lse are NaN. */
+typedef struct {
+  const void* hidden; int64_t ld_h;
+  const void* weight; int64_t ld_w;
+  int64_t N; int32_t d; int32_t V;
+  float temperature;
+} saki_lmhead_in;
+SAKI_API int64_t saki_lmhead_scratch_bytes(int64_t N, int32_t V);
+SAKI_API int saki_lmhead_lse(const saki_lmhead_in* in, void* logits, int64_t ld_l, float* row_max, float* lse,
+                             void* scratch, int64_t scratch_bytes, void* cuda_stream);
+
 /* Block verification (Section 3.5, Appendix I) of B drafted blocks of K tokens. */
 typedef struct {
   const void* student_logits; /* [B,K+1,V]: position j of sequence b at element offset

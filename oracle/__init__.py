@@ -14,4 +14,5 @@ from .saki_oracle import (  # noqa: F401
     route_row, route, sample_proposal_row, sample_proposal, spec_verify,
     bwd_from_meta_row, bwd_from_meta,
     STAGE_SELECT, SELECT_RANDOM, SELECT_TV_WEIGHTED, select_tm,
+    lmhead_lse,
 )

@@ -29,6 +29,10 @@ T = teacher distribution, both full-vocabulary softmaxes of the logit rows):
      gradient for freshly computed student
      logits, from the rollout's metadata only  Section 3.5; Eqs. "k1_loss_token",
                                                "teacher_mode_loss"
+  9. the step in front of the path: logits =
+     hidden x W^T as the models' lm-heads
+     leave them (stored in bf16), with the row
+     maximum and log-sum-exp of step 1         Section 3.5, Appendix K; Section 3.1
 
 Readings where the paper is silent are stated next to the code that takes them.
 The random numbers are a counter-based Philox4x32-10 stream keyed by
@@ -43,7 +47,9 @@ enumeration and by Monte Carlo over seeds; losses and gradient against
 torch.autograd in float64 and central differences; block verification by the
 product law of the acceptance probabilities; the metadata-driven backward
 against torch's cross-entropy (a library routine), central differences, the
-zero row sum of a softmax gradient and route() itself on unchanged logits.  The
+zero row sum of a softmax gradient and route() itself on unchanged logits; the
+lm-head step against scipy's logsumexp, torch's float64 matmul, one-hot hidden
+states (the logits are then a column of W) and equal weight rows (log V).  The
 paper prints no worked numeric example for any of these quantities.
 """
 from __future__ import annotations
@@ -599,3 +605,24 @@ def spec_verify(s, t, draft, eps, temperature=1.0, seed=0, seq_offset=0):
     return dict(n_accept=n_accept, next_token=next_token,
                 next_is_correction=next_is_corr, margin=margins,
                 per_pos=per_pos)
+
+
+# --------------------------------------------------------------------------
+# The step in front of the path: the lm-head that leaves the logits
+# --------------------------------------------------------------------------
+def lmhead_lse(hidden, weight, temperature: float = 1.0):
+    """`hidden`: [N, d], `weight`: [V, d] (one row per vocabulary entry), the
+    stored (bf16) values widened exactly to float64.  Section 3.5 / Appendix K:
+    the student and the teacher each leave full-vocabulary logits
+    logits[i, v] = sum_k hidden[i, k] weight[v, k]; they are stored in bf16
+    (round to nearest even), and Section 3.1's softmax is taken of the STORED
+    values: row_max[i] = max_v logits[i, v], lse[i] = log sum_v
+    exp(logits[i, v] / temperature).  Returns (logits as float64 holding bf16
+    values, row_max, lse)."""
+    h = np.asarray(hidden, dtype=np.float64)
+    w = np.asarray(weight, dtype=np.float64)
+    logits = round_to_bf16(h @ w.T)
+    z = logits / temperature
+    m = z.max(axis=1)
+    lse = m + np.log(np.exp(z - m[:, None]).sum(axis=1))
+    return logits, logits.max(axis=1), lse

@@ -22,6 +22,7 @@ _FLOAT_FIELDS = ("lambda", "kl", "tv", "accept_prob", "logp_x", "logq_x", "logT_
 EXPORTS = ("saki_route_fwd", "saki_route_fwd_bwd", "saki_route_fwd_bwd_noalloc", "saki_route_host",
            "saki_route_bwd_from_meta", "saki_select_tm", "saki_spec_verify",
            "saki_vshard_partial", "saki_vshard_combine", "saki_vshard_combine_host",
+           "saki_lmhead_scratch_bytes", "saki_lmhead_lse",
            "saki_sample_proposal", "saki_check", "saki_set_kernel", "saki_last_kernel", "saki_redo_count",
            "saki_set_spec_early_out", "saki_spec_positions_routed", "saki_solve_evaluations", "saki_set_wait_limit", "saki_set_phase_clock", "saki_phase_cycles",
            "saki_launch_count",
@@ -79,6 +80,11 @@ class SakiVshardIn(C.Structure):
 VSHARD_PARTIALS, VSHARD_STATE = 12, 32
 
 
+class SakiLmheadIn(C.Structure):
+    _fields_ = [("hidden", C.c_void_p), ("ld_h", C.c_int64), ("weight", C.c_void_p), ("ld_w", C.c_int64),
+                ("N", C.c_int64), ("d", C.c_int32), ("V", C.c_int32), ("temperature", C.c_float)]
+
+
 class SakiSpecIn(C.Structure):
     _fields_ = [("student_logits", C.c_void_p), ("teacher_logits", C.c_void_p),
                 ("ss_seq", C.c_int64), ("ss_pos", C.c_int64), ("ts_seq", C.c_int64), ("ts_pos", C.c_int64),
@@ -134,6 +140,11 @@ def load_library(path: str | None = None):
     lib.saki_vshard_combine_host.argtypes = [C.POINTER(SakiVshardIn), C.c_int, C.c_void_p, C.c_void_p, C.POINTER(SakiOut),
                                              C.POINTER(C.c_int32)]
     lib.saki_vshard_combine_host.restype = C.c_int
+    lib.saki_lmhead_scratch_bytes.argtypes = [C.c_int64, C.c_int32]
+    lib.saki_lmhead_scratch_bytes.restype = C.c_int64
+    lib.saki_lmhead_lse.argtypes = [C.POINTER(SakiLmheadIn), C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
+                                    C.c_int64, C.c_void_p]
+    lib.saki_lmhead_lse.restype = C.c_int
     lib.saki_set_wait_limit.argtypes = [C.c_int64]
     lib.saki_set_wait_limit.restype = C.c_int64
     lib.saki_set_phase_clock.argtypes = [C.c_int]
@@ -371,6 +382,34 @@ def vshard_combine_host(si: SakiVshardIn, stage: int, gathered, state, out=None)
     _raise(lib, lib.saki_vshard_combine_host(C.byref(si), stage, gathered.data_ptr(), state.data_ptr(),
                                              C.byref(so) if so is not None else None, C.byref(n)))
     return int(n.value)
+
+
+def lmhead_lse(hidden, weight, temperature=1.0, logits=None, scratch=None, stream=None):
+    """saki_lmhead_lse: logits = hidden @ weight.T (bf16 in, fp32 accumulation, bf16 out) with each row's maximum and
+    log-sum-exp (of the stored bf16 values / temperature) from the GEMM's epilogue.  hidden [N, d], weight [V, d] on
+    the GPU.  Returns (logits, row_max, lse)."""
+    lib = load_library()
+    if hidden.dtype != torch.bfloat16 or weight.dtype != torch.bfloat16 or hidden.shape[1] != weight.shape[1]:
+        raise ValueError("hidden [N, d] and weight [V, d] must be bf16 with the same d")
+    if hidden.stride(1) != 1 or weight.stride(1) != 1:
+        raise ValueError("hidden and weight need unit stride along d")
+    N, d = hidden.shape
+    V = weight.shape[0]
+    dev = hidden.device
+    logits = logits if logits is not None else torch.empty((N, V), dtype=torch.bfloat16, device=dev)
+    need = int(lib.saki_lmhead_scratch_bytes(N, V))
+    if scratch is None or scratch.numel() * scratch.element_size() < need:
+        scratch = torch.empty(need, dtype=torch.uint8, device=dev)
+    row_max = torch.empty(N, dtype=torch.float32, device=dev)
+    lse = torch.empty(N, dtype=torch.float32, device=dev)
+    li = SakiLmheadIn()
+    li.hidden, li.ld_h = hidden.data_ptr(), (hidden.stride(0) if N > 1 else d)
+    li.weight, li.ld_w = weight.data_ptr(), (weight.stride(0) if V > 1 else d)
+    li.N, li.d, li.V, li.temperature = N, d, V, temperature
+    ld_l = logits.stride(0) if N > 1 else V
+    _raise(lib, lib.saki_lmhead_lse(C.byref(li), logits.data_ptr(), ld_l, row_max.data_ptr(), lse.data_ptr(),
+                                    scratch.data_ptr(), scratch.numel() * scratch.element_size(), _stream_ptr(stream)))
+    return logits, row_max, lse
 
 
 def route_host(s, t, proposal, eps, temperature=1.0, seed=0, row_offset=0, mask=None, grad_scale=1.0,

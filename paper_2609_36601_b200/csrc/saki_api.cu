@@ -511,6 +511,35 @@ SAKI_API int saki_vshard_combine_host(const saki_vshard_in* in, int stage, const
   return SAKI_OK;
 }
 
+SAKI_API int64_t saki_lmhead_scratch_bytes(int64_t N, int32_t V) {
+  if (N < 0 || V < 1) return 0;
+  return lmhead_scratch_bytes(N, V);
+}
+
+SAKI_API int saki_lmhead_lse(const saki_lmhead_in* in, void* logits, int64_t ld_l, float* row_max, float* lse,
+                             void* scratch, int64_t scratch_bytes, void* cuda_stream) {
+  g_err[0] = 0;
+  if (!in) return fail(SAKI_ERR_INVALID_ARG, "NULL argument struct");
+  if (in->N < 0) return fail(SAKI_ERR_INVALID_ARG, "negative row count");
+  if (in->V < 8 || in->d < 8) return fail(SAKI_ERR_INVALID_ARG, "V and d must be >= 8 (got %d, %d)", in->V, in->d);
+  if (!(in->temperature > 0.f) || std::isinf(in->temperature)) return fail(SAKI_ERR_INVALID_ARG, "temperature must be finite and > 0");
+  if (in->ld_h < in->d || in->ld_w < in->d || ld_l < in->V) return fail(SAKI_ERR_INVALID_ARG, "row stride smaller than the row");
+  if (in->N == 0) return SAKI_OK;
+  if (!in->hidden || !in->weight || !logits || !scratch) return fail(SAKI_ERR_INVALID_ARG, "NULL hidden, weight, logits or scratch pointer");
+  if (scratch_bytes < lmhead_scratch_bytes(in->N, in->V)) return fail(SAKI_ERR_INVALID_ARG, "scratch too small: %lld bytes needed", (long long)lmhead_scratch_bytes(in->N, in->V));
+  auto al = [](const void* q, uintptr_t a) { return ((uintptr_t)q & (a - 1)) == 0; };
+  if (!al(in->hidden, 16) || !al(in->weight, 16) || !al(logits, 16) || !al(scratch, 256) || in->ld_h % 8 || in->ld_w % 8 || ld_l % 8 || in->V % 8)
+    return fail(SAKI_ERR_UNSUPPORTED, "pointers must be 16-byte aligned (scratch 256), strides and V multiples of 8");
+  unsigned long long* flagged = nullptr;
+  int rc = device_ready(&flagged);
+  if (rc) return rc;
+  const char* why = nullptr;
+  cudaError_t e = launch_lmhead(*in, logits, ld_l, row_max, lse, scratch, (cudaStream_t)cuda_stream, &why);
+  if (e != cudaSuccess) return why ? fail(SAKI_ERR_CUDA, "%s", why) : cuda_fail(e, "lm-head kernel launch");
+  g_launches += 2;
+  return SAKI_OK;
+}
+
 SAKI_API int saki_spec_verify(const saki_spec_in* in, const saki_spec_out* out, void* cuda_stream) {
   g_err[0] = 0;
   if (!in || !out) return fail(SAKI_ERR_INVALID_ARG, "NULL argument struct");

@@ -173,6 +173,9 @@ cudaError_t launch_vshard_partial(const saki_vshard_in& in, int stage, const dou
                                   int64_t ld_g, float grad_scale, cudaStream_t st);
 cudaError_t launch_vshard_combine(const saki_vshard_in& in, int stage, const double* gathered, double* state, const saki_out& out,
                                   unsigned int* n_solving, cudaStream_t st);
+int64_t lmhead_scratch_bytes(int64_t N, int32_t V);
+cudaError_t launch_lmhead(const saki_lmhead_in& in, void* logits, int64_t ld_l, float* row_max, float* lse, void* scratch,
+                          cudaStream_t st, const char** why);
 int vshard_combine_host(const saki_vshard_in& in, int stage, const double* gathered, double* state, const saki_out& out);
 
 }  // namespace saki

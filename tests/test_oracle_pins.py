@@ -537,3 +537,40 @@ def test_select_tm_uniform_fill_when_too_few_positive():
         hits += sel
     zeros = [0, 2, 3, 5]                            # two of the four zero-TV positions, uniformly
     assert np.all(np.abs(hits[zeros] / 3000 - 0.5) < 0.03)
+
+
+# ---- the lm-head step (logits as stored, row maximum, log-sum-exp)
+def _bf16_values(shape, seed, scale=1.0):
+    g = torch.Generator().manual_seed(seed)
+    return (scale * torch.randn(shape, generator=g)).to(torch.bfloat16).to(torch.float64).numpy()
+
+
+def test_lmhead_against_library_routines():
+    h, w = _bf16_values((7, 48), 1), _bf16_values((300, 48), 2, 0.3)
+    for tau in (1.0, 0.7):
+        logits, row_max, lse = O.lmhead_lse(h, w, tau)
+        full = (torch.as_tensor(h) @ torch.as_tensor(w).T)                   # torch's float64 matmul
+        stored = full.to(torch.bfloat16).to(torch.float64).numpy()           # torch's rounding to bf16
+        assert np.array_equal(logits, stored)
+        assert np.array_equal(row_max, stored.max(axis=1))
+        assert np.allclose(lse, scipy.special.logsumexp(stored / tau, axis=1), rtol=0, atol=1e-12)
+
+
+def test_lmhead_closed_forms():
+    # a one-hot hidden state picks a column of W: the logits are that column, exactly
+    w = _bf16_values((64, 16), 3)
+    h = np.zeros((2, 16))
+    h[0, 5] = 1.0
+    h[1, 11] = -2.0
+    logits, row_max, lse = O.lmhead_lse(h, w, 1.0)
+    assert np.array_equal(logits[0], w[:, 5]) and np.array_equal(logits[1], -2.0 * w[:, 11])
+    assert row_max[0] == w[:, 5].max()
+    # equal weight rows: constant logits, lse = logit / tau + log V
+    w2 = np.tile(_bf16_values((1, 16), 4), (40, 1))
+    h2 = _bf16_values((3, 16), 5)
+    logits2, _, lse2 = O.lmhead_lse(h2, w2, 2.0)
+    assert np.all(logits2 == logits2[:, :1])
+    assert np.allclose(lse2, logits2[:, 0] / 2.0 + math.log(40), rtol=0, atol=1e-12)
+    # and the result is what route_row's own log-softmax starts from
+    lp = O.log_softmax(logits[0] / 1.0)
+    assert abs(-lp.max() - (lse[0] - row_max[0])) < 1e-12
