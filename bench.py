@@ -20,6 +20,9 @@ positions: one saki_route_fwd_bwd call.  Prints ONE JSON line.
             timed the same way beside the headline: saki_route_bwd_from_meta on
             the same logits, saki_spec_verify on its own workload with and
             without early out, and the latency of saki_route_fwd on 8 rows
+  lm_head, vocab_sharded  (rank 0, unless --no-sweep) the lm-head GEMM with the row statistics
+            in its epilogue, against the measured dense bf16 GEMM rate; vocabulary-sharded
+            routing with the ranks run one after the other on this GPU
   sweep     (rank 0, unless --no-sweep) the throughput sweep at its full size
             (65536 positions, three disagreement regimes x three radii) and the
             V = 32000 workload: positions/s, fraction of the copy bandwidth,
@@ -66,6 +69,18 @@ def _peaks():
             return float(json.load(f)["hbm_gbs"]), "measured"
     except Exception:
         return FALLBACK_HBM_GBS, "fallback"
+
+
+FALLBACK_BF16_TFLOPS = 1590.0
+
+
+def _tensor_peak():
+    """Dense bf16 GEMM throughput of this machine's B200s (a cuBLAS GEMM run back to back for seconds), TFLOP/s."""
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["bf16_tflops_sustained"]), "measured (sustained)"
+    except Exception:
+        return FALLBACK_BF16_TFLOPS, "fallback (burst)"
 
 
 class ClockSampler:
@@ -218,6 +233,64 @@ def _config(w, world):
 def _describe(w):
     return (f"{w.name}: N={w.N} positions, V={w.V}, {w.dtype} logits, eps={w.eps}, temperature={w.temperature}, "
             f"teacher noise sigma={w.sigma}, fused fwd+bwd with {w.dtype} dlogits")
+
+
+def _lm_head(P, dev, stream, steps):
+    """saki_lmhead_lse on the teacher's lm-head shape (Qwen3-4B: d_model 2560, V 151936) for cfg3's 16384
+    positions: the bf16 GEMM that leaves the logits, row maximum and log-sum-exp from its epilogue."""
+    import torch
+    N, d, V = 16384, 2560, 151936
+    g = torch.Generator(device=dev).manual_seed(2024)
+    h = torch.randn((N, d), generator=g, device=dev).to(torch.bfloat16)
+    w = (torch.randn((V, d), generator=g, device=dev) * (2.0 / d ** 0.5)).to(torch.bfloat16)
+    logits = torch.empty((N, V), dtype=torch.bfloat16, device=dev)
+    scratch = torch.empty(int(P.load_library().saki_lmhead_scratch_bytes(N, V)), dtype=torch.uint8, device=dev)
+    for _ in range(3):
+        P.lmhead_lse(h, w, 1.0, logits=logits, scratch=scratch, stream=stream)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        _, _, lse = P.lmhead_lse(h, w, 1.0, logits=logits, scratch=scratch, stream=stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    flops = 2.0 * N * d * V
+    peak, kind = _tensor_peak()
+    tf = flops / (ms * 1e-3) / 1e12
+    ok = bool(torch.isfinite(lse).all().item())
+    return {"call": "saki_lmhead_lse", "workload": f"hidden [{N}, {d}] x weight [{V}, {d}]^T, bf16, fp32 accumulation, bf16 logits "
+            "+ row max + log-sum-exp", "ms_per_call": ms, "value": N / (ms * 1e-3), "unit": UNIT, "flops_per_call": flops,
+            "kernel": "saki::lmhead_kernel", "results_finite": ok,
+            "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
+                         "peak_kind": f"of {kind} dense bf16 GEMM, MEASURED_PEAKS.json" if kind.startswith("measured") else "of fallback",
+                         "traffic": None}}
+
+
+def _vocab_sharded(P, synth, dev, stream):
+    """Vocabulary-sharded routing of 1024 rows of the headline workload's shape cut into 8 column slices, the ranks
+    run one after the other on this GPU (the calls one rank per GPU would make around its all-gathers): time of
+    all ranks' kernels, evaluation waves, bytes a rank sends per row."""
+    import torch
+    from paper_2609_36601_b200.vshard import route_vocab_sharded_local, split_columns
+    w = synth.shrink(synth.WORKLOADS["cfg3"], 1024)
+    d = synth.generate(w, dev)
+    world = 8
+    slices = [(d["s"][:, a:a + n], d["t"][:, a:a + n], a) for a, n in split_columns(w.V, world)]
+    for _ in range(2):
+        out, gs, waves = route_vocab_sharded_local(slices, w.V, d["proposal"], w.eps, w.temperature, w.seed, grad_scale=1.0 / w.N,
+                                                   stream=stream)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    out, gs, waves = route_vocab_sharded_local(slices, w.V, d["proposal"], w.eps, w.temperature, w.seed, grad_scale=1.0 / w.N,
+                                               stream=stream)
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    stages = 3 + waves
+    return {"call": "saki_vshard_partial / saki_vshard_combine", "rows": w.N, "V": w.V, "ranks_emulated_on_one_gpu": world,
+            "ms_all_ranks": dt * 1e3, "value": w.N / dt, "unit": UNIT, "evaluation_waves": waves, "stages": stages,
+            "bytes_sent_per_row_and_rank": stages * 12 * 8, "arithmetic": "f64",
+            "note": "float64 slice kernels, one block per row: built for the exchange protocol, not yet for speed"}
 
 
 def _sweep(P, synth, dev, stream, peak, args):
@@ -515,13 +588,18 @@ def run_ours(args):
             if allc:
                 cpu["all_cores"] = allc
 
-    # ---- the throughput sweep at its full size and the V = 32000 workload: beside the headline
-    sweep = None
+    # ---- the throughput sweep at its full size and the V = 32000 workload, the step in front of the path (the
+    # lm-head GEMM with the first row statistics in its epilogue) and vocabulary-sharded rows: beside the headline
+    sweep = lm_head = vocab_sharded = None
     if not args.no_sweep and not args.rows and rank == 0:
         del s, t, g, x, d
         out = None
         torch.cuda.empty_cache()
         sweep = _sweep(P, synth, dev, stream, peak, args)
+        torch.cuda.empty_cache()
+        vocab_sharded = _vocab_sharded(P, synth, dev, stream)
+        torch.cuda.empty_cache()
+        lm_head = _lm_head(P, dev, stream, 5)      # last: a dense GEMM at the power limit would colour what follows it
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -531,6 +609,10 @@ def run_ours(args):
             "stats": stats, "achieved_gbs": achieved}
     if phases is not None:
         line["phase_cycles_per_row"] = phases
+    if lm_head is not None:
+        line["lm_head"] = lm_head
+    if vocab_sharded is not None:
+        line["vocab_sharded"] = vocab_sharded
     if sweep is not None:
         line["sweep"] = sweep
     if nxt is not None:
