@@ -235,11 +235,11 @@ def _describe(w):
             f"teacher noise sigma={w.sigma}, fused fwd+bwd with {w.dtype} dlogits")
 
 
-def _lm_head(P, dev, stream, steps):
+def _lm_head(P, dev, stream, steps, rows=0):
     """saki_lmhead_lse on the teacher's lm-head shape (Qwen3-4B: d_model 2560, V 151936) for cfg3's 16384
     positions: the bf16 GEMM that leaves the logits, row maximum and log-sum-exp from its epilogue."""
     import torch
-    N, d, V = 16384, 2560, 151936
+    N, d, V = (rows or 16384), 2560, 151936
     g = torch.Generator(device=dev).manual_seed(2024)
     h = torch.randn((N, d), generator=g, device=dev).to(torch.bfloat16)
     w = (torch.randn((V, d), generator=g, device=dev) * (2.0 / d ** 0.5)).to(torch.bfloat16)
@@ -656,13 +656,20 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-next", action="store_true", help="skip the metadata-driven backward measurement")
     ap.add_argument("--no-sweep", action="store_true", help="skip the throughput sweep and the V = 32000 workload")
+    ap.add_argument("--section", default="all", choices=["all", "lm_head"],
+                    help="lm_head: time only the lm-head GEMM (on --rows positions if given) and print its object (profiling)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-rows", type=int, default=384)
     ap.add_argument("--ref-rows", type=int, default=32)
     args = ap.parse_args()
     if args.gpus > 1 and "RANK" not in os.environ:
         sys.exit(_spawn_ranks(args.gpus))
-    if args.impl == "reference":
+    if args.section == "lm_head":
+        import torch
+        import paper_2609_36601_b200 as P
+        torch.cuda.set_device(0)
+        print(json.dumps(_lm_head(P, "cuda:0", torch.cuda.current_stream(), args.steps, args.rows)))
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
