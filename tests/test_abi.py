@@ -80,3 +80,30 @@ def test_argument_validation_returns_codes_before_any_device_work():
     sp, spo = binding.SakiSpecIn(), binding.SakiSpecOut()
     sp.B, sp.K, sp.V, sp.dtype, sp.eps, sp.temperature = 2, 17, 128, 1, 0.1, 1.0           # K outside [1,16]
     assert lib.saki_spec_verify(C.byref(sp), C.byref(spo), null) == 1
+
+
+def test_new_entry_points_validate_on_the_host():
+    """saki_vshard_* and saki_lmhead_lse reject bad arguments, and accept empty batches, before any device work."""
+    lib = binding.load_library()
+    C = ctypes
+    null = C.c_void_p(None)
+    vi = binding.SakiVshardIn()
+    vi.N, vi.V, vi.V_local, vi.v0, vi.dtype, vi.eps, vi.temperature, vi.rank, vi.world = 0, 1000, 500, 0, 1, 0.1, 1.0, 0, 2
+    assert lib.saki_vshard_partial(C.byref(vi), 0, null, null, null, 0, 1.0, null) == 0           # empty batch
+    assert lib.saki_vshard_partial(C.byref(vi), 4, null, null, null, 0, 1.0, null) == 1 and "stage" in P.last_error()
+    vi.v0 = 600                                                                                    # slice past the vocabulary
+    assert lib.saki_vshard_partial(C.byref(vi), 0, null, null, null, 0, 1.0, null) == 1
+    vi.v0, vi.rank = 0, 2                                                                          # rank outside the world
+    assert lib.saki_vshard_combine(C.byref(vi), 0, null, null, None, null, null) == 1
+    vi.rank, vi.N = 1, 4                                                                           # NULL proposal
+    n = C.c_int32(0)
+    assert lib.saki_vshard_combine_host(C.byref(vi), 0, null, null, None, C.byref(n)) == 1
+    li = binding.SakiLmheadIn()
+    li.N, li.d, li.V, li.ld_h, li.ld_w, li.temperature = 0, 64, 256, 64, 64, 1.0
+    assert lib.saki_lmhead_lse(C.byref(li), null, 256, null, null, null, 0, null) == 0             # empty batch
+    li.N = 8
+    assert lib.saki_lmhead_lse(C.byref(li), null, 256, null, null, null, 0, null) == 1             # NULL pointers
+    li.d = 4
+    assert lib.saki_lmhead_lse(C.byref(li), null, 256, null, null, null, 0, null) == 1
+    assert lib.saki_lmhead_scratch_bytes(128, 512) == 128 * 2 * 3 * 4 + 256
+    assert lib.saki_set_wait_limit(0) == 0 and lib.saki_set_phase_clock(0) == 0
