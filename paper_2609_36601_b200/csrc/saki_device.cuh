@@ -220,6 +220,27 @@ __device__ __forceinline__ void lse_of_sum(double S, double k, double& rS, doubl
   rS = rcp_fast(S);
   G = LN2 * (log2_fast(S) - k);
 }
+// The initial guess of lambda far from the student's end.  There the series in the cumulants of d under p is
+// short of terms, but the other end is known: KL at beta = 1 is KL(T||p).  A fifth-order term is chosen so that
+// the model meets it there, and the model's root is taken inside the bracket (0, 1) by safeguarded Newton (the
+// model is negative at 0 and positive at 1, the row being short of the teacher endpoint).  On the sweep's rows
+// at eps = 1 the median error of the guess goes from 5 % to 1.3 %; guesses below 0.45 (eps = 0.1 on most rows)
+// are left to the series.  Out of line: rare on the headline workload, and the caller's code stays short.
+static __device__ __noinline__ float anchored_guess(float b, float vd, float k3, float k4, float kl1, float ef) {
+  const float a2 = 0.5f * vd, a3 = (1.f / 3.f) * k3, a4 = 0.125f * k4, a5 = kl1 - (a2 + a3 + a4);
+  float lo = 0.f, hi = 1.f, x = fminf(b, 1.f);
+#pragma unroll 1
+  for (int it = 0; it < 8; ++it) {
+    const float pv = x * x * (a2 + x * (a3 + x * (a4 + x * a5))) - ef;
+    const float dv = x * (2.f * a2 + x * (3.f * a3 + x * (4.f * a4 + x * (5.f * a5))));
+    if (pv > 0.f) hi = x; else lo = x;
+    float nx = dv > 0.f ? x - __fdividef(pv, dv) : -1.f;
+    if (!(nx > lo && nx < hi)) nx = 0.5f * (lo + hi);
+    x = nx;
+  }
+  return x;
+}
+
 static __device__ __noinline__ void scalar_after_lse_tail(double* bc, const double* v, Consts K, float k0f, float k1f, int x,
                                                    bool bonus, bool masked, bool row_timeout, float e_max,
                                                    bool overflow_redo, double rSs, double rSt, double G0, double G1,
@@ -278,25 +299,7 @@ static __device__ __noinline__ void scalar_after_lse_tail(double* bc, const doub
     const float den = vd + (2.f / 3.f) * bb * k3 + 0.25f * bb * bb * k4;
     if (den > 0.25f * vd) b = sqrtf(__fdividef(e2, den));
   }
-  // Far from the student's end the series is short of terms, but the other end is known: KL at beta = 1 is
-  // KL(T||p).  A fifth-order term is chosen so that the model meets it there, and the model's root is taken
-  // inside the bracket (0, 1) by safeguarded Newton (the model is negative at 0 and positive at 1, the row
-  // being short of the teacher endpoint).  On the sweep's rows at eps = 1 the median error of the guess
-  // goes from 5 % to 1.3 %; guesses below 0.45 (eps = 0.1 on most rows) are left to the series.
-  if (b > 0.45f) {
-    const float a2 = 0.5f * vd, a3 = (1.f / 3.f) * k3, a4 = 0.125f * k4, a5 = (float)kl1 - (a2 + a3 + a4), ef = (float)eps;
-    float lo = 0.f, hi = 1.f, x = fminf(b, 1.f);
-#pragma unroll 1
-    for (int it = 0; it < 8; ++it) {
-      const float pv = x * x * (a2 + x * (a3 + x * (a4 + x * a5))) - ef;
-      const float dv = x * (2.f * a2 + x * (3.f * a3 + x * (4.f * a4 + x * (5.f * a5))));
-      if (pv > 0.f) hi = x; else lo = x;
-      float nx = dv > 0.f ? x - __fdividef(pv, dv) : -1.f;
-      if (!(nx > lo && nx < hi)) nx = 0.5f * (lo + hi);
-      x = nx;
-    }
-    b = x;
-  }
+  if (b > 0.45f) b = anchored_guess(b, vd, k3, k4, (float)kl1, (float)eps);
   if (!(b > 1e-7f)) b = 1e-7f;
   if (b > 0.98f) b = 0.98f;
   const float cb = (float)(K.c64 * (double)b);
@@ -440,7 +443,12 @@ static __device__ __noinline__ void scalar_after_solve4(double* bc, const double
   const double kl_err = 3e-7 * (eps < 5e-3 ? 1.0 : bc[BC_PMAX]);
   if (done && ((!by_quadrature && kl_err > kl_tol) || iter >= 40)) { bc[BC_MODE] = MODE_REDO; return; }
   if (done) {
-    const float cl = (float)(K.c64 * nb);
+    float cl = (float)(K.c64 * nb);
+    {   // rounded so that (c - cl) + cl = c exactly in float32: pass "final" of the row-per-SM kernel forms the
+        // exponent of q as (c - cl) s + cl t
+      const float cf = (float)K.c64, ccl = cf - cl;
+      cl = cf - ccl;
+    }
     const double lam = (double)cl * K.rc64;
     const double dl = lam - beta;
     // the model's predictions at lambda

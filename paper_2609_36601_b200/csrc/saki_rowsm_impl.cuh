@@ -477,9 +477,8 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const float2 sf = unpack_bf16x2(sw[i]), tf = unpack_bf16x2(tw[i]);
-      const float2 d = ffma2(sf, splat(-1.f), tf);
       const float2 ep = ex2f2(ffma2(sf, splat(c32), splat(k0p)));
-      const float2 eq = ex2f2(ffma2(d, splat(clp), ffma2(sf, splat(c32), splat(kqp))));
+      const float2 eq = ex2f2(ffma2(tf, splat(clp), ffma2(sf, splat(c32 - clp), splat(kqp))));   // as in pass "final"
       w[2 * i] = pbonus ? eq.x : fmaxf(fmaf(ep.x, -rhop, eq.x), 0.f);
       w[2 * i + 1] = pbonus ? eq.y : fmaxf(fmaf(ep.y, -rhop, eq.y), 0.f);
     }
@@ -780,8 +779,9 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
     {
       const bool want_g = (g_out != nullptr);
       float2 R = splat(0.f);
-      const float2 cc = splat(c32), cll = splat(cl), kqq = splat(kq), kk0 = splat(k0), neg1 = splat(-1.f);
+      const float2 cc = splat(c32), cll = splat(cl), kqq = splat(kq), kk0 = splat(k0);
       const float2 nrho = splat(-rho), kgg = splat(kg);
+      const float2 ccl = splat(c32 - cl);               // exact: the scalar step rounds cl so that (c - cl) + cl = c in float32
       float* step_w = (float*)(smem + ROFF_STEP) + warp * MAX_STEPS;   // draw weight of each of this warp's steps
       for_each_chunk(sg, lane, res_s, res_t, g_s, g_t, n_s, n_t, pol_last, rg, [&](const uint4& s4, const uint4& t4, int c, bool valid) {
         const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
@@ -790,9 +790,9 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const float2 sf = unpack_bf16x2(sw[i]), tf = unpack_bf16x2(tw[i]);
-          const float2 d = ffma2(sf, neg1, tf);
           const float2 ep = ex2f2(ffma2(sf, cc, kk0));
-          const float2 eq = ex2f2(ffma2(d, cll, ffma2(sf, cc, kqq)));
+          const float2 eq = ex2f2(ffma2(tf, cll, ffma2(sf, ccl, kqq)));     // c s + cl (t - s) as (c - cl) s + cl t: no difference to form
+
           sqc = fadd2(sqc, eq);
           float2 r = ffma2(ep, nrho, eq);                // (q_i - p_i) / iq
           r.x = fmaxf(r.x, 0.f); r.y = fmaxf(r.y, 0.f);
