@@ -43,6 +43,7 @@ struct RowParams {
   unsigned int* redo_count;            // scratch: their number (zeroed before the launch, with the three words
                                        // after it: [1], [2] see seq_next; [3] evaluation passes of the row-per-SM kernel)
   int32_t from_list;                   // general kernel only: route the rows of redo_list
+  int32_t list_min, list_max;          // ... and only if their number lies in [list_min, list_max] (0, 0: any number)
   long long wait_limit;                // row-per-SM kernel: SM cycles a block waits for a row's bulk copy (<= 0: ~2 s)
   unsigned long long* phase_cycles;    // row-per-SM kernel: [SAKI_PHASE_COUNTERS] cycle sums per phase (zeroed before
                                        // the launch); NULL: not wanted
