@@ -148,41 +148,49 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint32_t w) {
 constexpr uint32_t FILLER = 0xFF7FFF7Fu;          // two bf16 of the most negative finite value: exp -> 0, difference 0
 constexpr uint32_t T_OFF = RW * RES_CHUNKS * 16;  // a teacher slot lies this far behind its student slot
 
-// The streamed part of a warp's segment passes through a ring of NST steps in shared memory.  Every
-// lane owns one 16-byte slot per stage and array and fills it itself (cp.async, or the filler where
-// the row has no chunk for it), so no lane ever reads what another lane wrote: a thread's own
-// wait_group is all the synchronisation there is.  Invariant between passes: the first NST streamed
-// steps of the coming pass are in flight or landed, one committed group per step.
+// The streamed part of a warp's segment passes through a ring in shared memory, two steps (a "double
+// step": 64 chunks, two per lane) at a time: NSD double steps fill the NST steps of the ring.  Every lane
+// owns two 16-byte slots per double stage and array and fills them itself (cp.async, or the filler where
+// the row has no chunk for it), so no lane ever reads what another lane wrote: a thread's own wait_group is
+// all the synchronisation there is, and the bookkeeping of a ring step (wait, commit, offsets, wrap) is
+// paid once per two chunks.  A streamed part is a whole number of double steps (the resident part gives up
+// a step where it would not be).  Invariant between passes: the first NSD double steps of the coming
+// pass are in flight or landed, one committed group per double step.
+constexpr int NSD = NST / 2;
+static_assert(NST == 2 * NSD && NSD >= 2, "the ring holds whole double steps");
 struct Ring {
-  uint32_t base;   // shared-memory address of this lane's student slot of stage 0 (a stage is 512 bytes on)
-  uint32_t slot;   // slot of the next step to consume
+  uint32_t base;   // shared-memory address of this lane's first student slot of double stage 0 (a double stage is 1024 bytes on)
+  uint32_t slot;   // slot of the next double step to consume
 };
 
-// request the first NST streamed steps of a row (g_s == nullptr: no row) once everything in flight has landed
+// request the first NSD double steps of a row (g_s == nullptr: no row) once everything in flight has landed
 __device__ __forceinline__ void ring_prime(Ring& rg, const Seg& sg, int lane, const __nv_bfloat16* g_s,
                                            const __nv_bfloat16* g_t, uint64_t pol) {
   cp_async_wait<0>();
   if (sg.res == sg.steps) return;          // nothing is streamed
   uint32_t slot = rg.slot;
 #pragma unroll
-  for (int j = 0; j < NST; ++j) {
-    const int c = sg.c0 + (sg.res + j) * 32 + lane;
-    if (g_s != nullptr && c < sg.c1) {
-      cp_async16(slot, g_s + (size_t)c * 8, pol);
-      cp_async16(slot + T_OFF, g_t + (size_t)c * 8, pol);
-    } else {
-      sts128(slot, FILLER);
-      sts128(slot + T_OFF, FILLER);
+  for (int j = 0; j < NSD; ++j) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int c = sg.c0 + (sg.res + 2 * j + h) * 32 + lane;
+      if (g_s != nullptr && c < sg.c1) {
+        cp_async16(slot + h * 512, g_s + (size_t)c * 8, pol);
+        cp_async16(slot + h * 512 + T_OFF, g_t + (size_t)c * 8, pol);
+      } else {
+        sts128(slot + h * 512, FILLER);
+        sts128(slot + h * 512 + T_OFF, FILLER);
+      }
     }
     cp_async_commit();
-    slot += 512;
-    if (slot == rg.base + NST * 512) slot = rg.base;
+    slot += 1024;
+    if (slot == rg.base + NSD * 1024) slot = rg.base;
   }
 }
 
 // Visits this thread's chunks in step order: body(a, b, chunk, valid) with the packed student /
 // teacher words of the chunk (the filler where valid is false).  Resident steps are read from shared
-// memory; streamed steps come out of the ring, and each one consumed requests the step NST further
+// memory; streamed steps come out of the ring, and each double step consumed requests the one NSD further
 // on: of this pass, or, past its end, of the next pass, whose rows are wrap_s / wrap_t (the same row
 // again, the next row after the last pass, nullptr if nothing follows).
 // after_resident() runs once the resident steps are done.
@@ -197,52 +205,60 @@ __device__ __forceinline__ void for_each_chunk(const Seg& sg, int lane, const ui
 #pragma unroll 1
   for (int k = 0; k < sg.res; ++k, c += 32) body(res_s[k * 32 + lane], res_t[k * 32 + lane], c, c < sg.c1);
   after_resident();
-  const int T = sg.steps - sg.res;                  // streamed steps: 0 or more than NST
-  if (T <= 0) return;
+  const int TD = (sg.steps - sg.res) >> 1;          // streamed double steps: 0 or more than NSD
+  if (TD <= 0) return;
   const uint32_t first_off = (uint32_t)c * 16u;
-  uint32_t off = first_off + 512u * NST;            // byte offset, in either row, of the chunk requested next
+  uint32_t off = first_off + 1024u * NSD;           // byte offset, in either row, of the first chunk of the double step requested next
   uint32_t lim = (uint32_t)sg.c1 * 16u;
   const char* bs = reinterpret_cast<const char*>(g_s);   // (warp-uniform) rows the requests read
   const char* bt = reinterpret_cast<const char*>(g_t);
   uint32_t slot = rg.slot;
-  const uint32_t slot_end = rg.base + NST * 512;
+  const uint32_t slot_end = rg.base + NSD * 1024;
   int i = 0;
-  // all but the last NST + 1 steps: the chunk consumed and the chunk requested exist for every lane, and
-  // the requests stay inside this pass, so this copy of the loop carries none of the checks below (the
-  // body is instantiated twice; 1.7 % faster on V = 151936 in spite of the larger code)
+  // all but the last NSD + 1 double steps: the chunks consumed and the chunks requested exist for every lane,
+  // and the requests stay inside this pass, so this copy of the loop carries none of the checks below
 #pragma unroll 1
-  for (; i < T - NST - 1; ++i, c += 32) {
-    cp_async_wait<NST - 1>();
-    const uint4 a = lds128(slot), b = lds128(slot + T_OFF);
+  for (; i < TD - NSD - 1; ++i, c += 64) {
+    cp_async_wait<NSD - 1>();
+    const uint4 a0 = lds128(slot), b0 = lds128(slot + T_OFF);
+    const uint4 a1 = lds128(slot + 512), b1 = lds128(slot + 512 + T_OFF);
     cp_async16(slot, bs + off, pol);
     cp_async16(slot + T_OFF, bt + off, pol);
+    cp_async16(slot + 512, bs + off + 512, pol);
+    cp_async16(slot + 512 + T_OFF, bt + off + 512, pol);
     cp_async_commit();
-    off += 512;
-    slot += 512;
+    off += 1024;
+    slot += 1024;
     if (slot == slot_end) slot = rg.base;
-    body(a, b, c, true);
+    body(a0, b0, c, true);
+    body(a1, b1, c + 32, true);
   }
 #pragma unroll 1
-  for (; i < T; ++i, c += 32) {
-    if (i == T - NST) {   // from here on the requests belong to the pass that follows
+  for (; i < TD; ++i, c += 64) {
+    if (i == TD - NSD) {   // from here on the requests belong to the pass that follows
       off = first_off;
       if (wrap_s != nullptr) { bs = reinterpret_cast<const char*>(wrap_s); bt = reinterpret_cast<const char*>(wrap_t); }
       else lim = 0;
     }
-    cp_async_wait<NST - 1>();
-    const uint4 a = lds128(slot), b = lds128(slot + T_OFF);
-    if (off < lim) {
-      cp_async16(slot, bs + off, pol);
-      cp_async16(slot + T_OFF, bt + off, pol);
-    } else {
-      sts128(slot, FILLER);
-      sts128(slot + T_OFF, FILLER);
+    cp_async_wait<NSD - 1>();
+    const uint4 a0 = lds128(slot), b0 = lds128(slot + T_OFF);
+    const uint4 a1 = lds128(slot + 512), b1 = lds128(slot + 512 + T_OFF);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      if (off + h * 512 < lim) {
+        cp_async16(slot + h * 512, bs + off + h * 512, pol);
+        cp_async16(slot + h * 512 + T_OFF, bt + off + h * 512, pol);
+      } else {
+        sts128(slot + h * 512, FILLER);
+        sts128(slot + h * 512 + T_OFF, FILLER);
+      }
     }
     cp_async_commit();
-    off += 512;
-    slot += 512;
+    off += 1024;
+    slot += 1024;
     if (slot == slot_end) slot = rg.base;
-    body(a, b, c, c < sg.c1);
+    body(a0, b0, c, c < sg.c1);
+    body(a1, b1, c + 32, c + 32 < sg.c1);
   }
   rg.slot = slot;
 }
@@ -290,7 +306,9 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
   };
   Seg sg;
   seg_of(warp, sg);
-  sg.res = sg.steps <= KS_MAX ? sg.steps : KS_RES;   // a segment that does not fit leaves NST steps to the ring
+  // a segment that does not fit leaves NST steps to the ring, and one more where the streamed part would not be
+  // a whole number of double steps
+  sg.res = sg.steps <= KS_MAX ? sg.steps : KS_RES - ((sg.steps - KS_RES) & 1);
   const int res_chunks = min(sg.c1 - sg.c0, sg.res * 32);          // resident chunks of this warp
   const uint32_t res_bytes = (uint32_t)res_chunks * 16u;
   Ring rg;
