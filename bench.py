@@ -272,6 +272,7 @@ def _vocab_sharded(P, synth, dev, stream):
     run one after the other on this GPU (the calls one rank per GPU would make around its all-gathers): time of
     all ranks' kernels, evaluation waves, bytes a rank sends per row."""
     import torch
+    from paper_2609_36601_b200 import binding as B
     from paper_2609_36601_b200.vshard import route_vocab_sharded_local, split_columns
     w = synth.shrink(synth.WORKLOADS["cfg3"], 1024)
     d = synth.generate(w, dev)
@@ -288,9 +289,11 @@ def _vocab_sharded(P, synth, dev, stream):
     dt = time.perf_counter() - t0
     stages = 3 + waves
     return {"call": "saki_vshard_partial / saki_vshard_combine", "rows": w.N, "V": w.V, "ranks_emulated_on_one_gpu": world,
-            "ms_all_ranks": dt * 1e3, "value": w.N / dt, "unit": UNIT, "evaluation_waves": waves, "stages": stages,
-            "bytes_sent_per_row_and_rank": stages * 12 * 8, "arithmetic": "f64",
-            "note": "float64 slice kernels, one block per row: built for the exchange protocol, not yet for speed"}
+            "ms_all_ranks": dt * 1e3, "ms_per_rank": dt * 1e3 / world, "value": w.N / dt, "unit": UNIT,
+            "evaluation_waves": waves, "stages": stages,
+            "bytes_sent_per_row_and_rank": stages * B.VSHARD_PARTIALS * 8, "arithmetic": "f64",
+            "note": "float64 slice kernels, one block per row; value = rows / time of all 8 ranks' kernels run one after "
+                    "the other on this GPU (a rank's own share is ms_per_rank, the exchanges not included)"}
 
 
 def _sweep(P, synth, dev, stream, peak, args):

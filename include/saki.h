@@ -236,8 +236,9 @@ SAKI_API int saki_select_tm(const saki_select_in* in, uint8_t* selected, int32_t
  * every rank folds the gathered partials, in rank order, into the same per-row state of
  * SAKI_VSHARD_STATE doubles (saki_vshard_combine).  Stages, run in this order:
  *   0  maxima, teacher argmax, sums of exponentials and moments of the logit difference (Section 3.1)
- *   1  one evaluation of KL(q_beta || p) at every unsettled row's current beta (Eqs. "bridge",
- *      "trust_region"); repeat stage 1 until the combine reports no row still solving
+ *   1  one evaluation of KL(q_beta || p) and of the cumulants of the logit difference at every unsettled
+ *      row's current beta (Eqs. "bridge", "trust_region"); repeat stage 1 until the combine reports no row
+ *      still solving (each wave moves to the root of a fourth-order model: two waves as a rule)
  *   2  shares of TV(p, q) and KL(q || p); the combine decides acceptance (Eq. "accept"), the routed loss
  *      (Eqs. "k1_loss_token", "teacher_mode_loss") and which rank owns the residual draw (Eq. "residual")
  *   3  the gradient slice (Eq. "general_objective": dlogits_slice [N, V_local], same dtype, may be NULL) and,
@@ -253,7 +254,7 @@ SAKI_API int saki_select_tm(const saki_select_in* in, uint8_t* selected, int32_t
  * included, is a host pointer; the logits pointers of `in` are not read): for callers that exchange
  * through host memory.  Errors: SAKI_ERR_INVALID_ARG for NULL required pointers, a stage outside 0..3,
  * sizes or strides that do not fit; SAKI_ERR_CUDA for a failed launch. */
-#define SAKI_VSHARD_PARTIALS 12
+#define SAKI_VSHARD_PARTIALS 16
 #define SAKI_VSHARD_STATE 32
 typedef struct {
   const void* student_logits;  /* DEVICE [N, V_local]: this rank's columns, unit column stride, row stride ld_s elements */

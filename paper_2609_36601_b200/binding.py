@@ -77,7 +77,7 @@ class SakiVshardIn(C.Structure):
                 ("rank", C.c_int32), ("world", C.c_int32)]
 
 
-VSHARD_PARTIALS, VSHARD_STATE = 12, 32
+VSHARD_PARTIALS, VSHARD_STATE = 16, 32
 
 
 class SakiLmheadIn(C.Structure):
@@ -366,7 +366,7 @@ def vshard_partial(si: SakiVshardIn, stage: int, state, partial, dlogits=None, g
 
 
 def vshard_combine(si: SakiVshardIn, stage: int, gathered, state, out=None, n_solving=None, stream=None):
-    """saki_vshard_combine: folds the gathered partials [world, N, 12] into the per-row state (device tensors)."""
+    """saki_vshard_combine: folds the gathered partials [world, N, 16] into the per-row state (device tensors)."""
     lib = load_library()
     so = _out_struct(out) if out is not None else None
     _raise(lib, lib.saki_vshard_combine(C.byref(si), stage, gathered.data_ptr(), state.data_ptr(),

@@ -4,17 +4,19 @@
 // kernel here), the ranks exchange the partials (the caller's all-gather: ~100 bytes per row and stage),
 // and every rank combines them, in rank order, into the same per-row state (a kernel here, and the same
 // function compiled for the host).  What is computed is the definition (Eqs. "bridge", "trust_region",
-// "accept", "residual", "k1_loss_token", "teacher_mode_loss", "general_objective"), in float64, with the
-// solver of the float64 row kernel (Newton on KL(q_beta||p) = eps inside a bisection bracket):
+// "accept", "residual", "k1_loss_token", "teacher_mode_loss", "general_objective"), in float64.  An evaluation
+// of q_beta costs every rank a pass over its slice and the ranks an exchange, so the solver makes each one
+// count: it carries the first four cumulants of the logit difference, the first guess is the root of the
+// fourth-order series of KL(q_beta||p) at beta = 0, and each wave moves to the root of the fourth-order model
+// at its beta (inside a bisection bracket); a step shorter than VS_SETTLE_STEP is taken without another look.
 //   stage A  maxima, teacher argmax, the two sums of exponentials and the moments of the logit
-//            difference under p and T (each under the slice's own shift; the combine rescales)
-//   stage B  one evaluation of q_beta per wave: sum e, sum e delta, sum e delta^2; repeated until every
-//            row's lambda has settled
+//            difference under p (four) and T (one), each under the slice's own shift; the combine rescales
+//   stage B  one evaluation of q_beta per wave: sum e delta^k, k = 0..4; repeated until every
+//            row's lambda has settled (two waves as a rule)
 //   stage C  the slice's share of TV = sum [q - p]_+ and of KL(q||p), the student's logit at the teacher's
 //            argmax; the combine decides acceptance and finds the rank that owns the inverse-CDF target
 //   stage D  the gradient slice, and on the owning rank the residual draw; the last combine writes the outputs
-// One thread block per row; float64 throughout.  This path is built for correctness and for the shape of
-// the exchange, not yet for speed.
+// One thread block per row; float64 throughout.
 #include "saki_common.cuh"
 #include <math_constants.h>
 #include <cmath>
@@ -39,6 +41,19 @@ struct VsConsts {
   const uint8_t* mask;
 };
 
+// the second to fourth cumulants of delta from the sums  a_k = sum w delta^k, k = 0..4
+__host__ __device__ inline void vs_cumulants(double a0, double a1, double a2, double a3, double a4, double& k2, double& k3,
+                                             double& k4) {
+  const double m1 = a1 / a0, r2 = a2 / a0, r3 = a3 / a0, r4 = a4 / a0;
+  const double mu2 = r2 - m1 * m1;
+  const double mu3 = r3 - 3.0 * m1 * r2 + 2.0 * m1 * m1 * m1;
+  const double mu4 = r4 - 4.0 * m1 * r3 + 6.0 * m1 * m1 * r2 - 3.0 * m1 * m1 * m1 * m1;
+  k2 = mu2; k3 = mu3; k4 = mu4 - 3.0 * mu2 * mu2;
+}
+// a wave's step shorter than this is taken without another evaluation: the model's error in lambda is of
+// the order of (k5 / k2) step^4 / 24
+constexpr double VS_SETTLE_STEP = 3e-3;
+
 // ---------------------------------------------------------------- the combine steps (host and device)
 // `part`: [world][N][SAKI_VSHARD_PARTIALS] gathered partials; row i of rank r at part[(r * N + i) * P].
 __host__ __device__ inline void vs_combine_a(const VsConsts& c, int64_t i, const double* part, double* st) {
@@ -58,11 +73,11 @@ __host__ __device__ inline void vs_combine_a(const VsConsts& c, int64_t i, const
   else if (x < 0 || x >= c.V) status = SAKI_ROW_BAD_ID;
   st[VS_MS] = ms; st[VS_MT] = mt; st[VS_VSTAR] = am < 2147483647.0 ? am : 0.0;
   if (status) { st[VS_STATUS] = (double)status; st[VS_MODE] = VS_FLAGGED; return; }
-  double Ss = 0.0, St = 0.0, Td = 0.0, Sd = 0.0, Sd2 = 0.0, sx = 0.0, tx = 0.0;
+  double Ss = 0.0, St = 0.0, Td = 0.0, Sd = 0.0, Sd2 = 0.0, Sd3 = 0.0, Sd4 = 0.0, sx = 0.0, tx = 0.0;
   for (int r = 0; r < c.world; ++r) {      // rank order: the summation order is part of the protocol
     const double* p = part + ((int64_t)r * c.N + i) * P;
     const double fs = exp((p[0] - ms) / c.tau), ft = exp((p[1] - mt) / c.tau);
-    if (p[4] > 0.0) { Ss += fs * p[4]; Sd += fs * p[7]; Sd2 += fs * p[8]; }
+    if (p[4] > 0.0) { Ss += fs * p[4]; Sd += fs * p[7]; Sd2 += fs * p[8]; Sd3 += fs * p[12]; Sd4 += fs * p[13]; }
     if (p[5] > 0.0) { St += ft * p[5]; Td += ft * p[6]; }
     sx += p[9]; tx += p[10];
   }
@@ -75,41 +90,78 @@ __host__ __device__ inline void vs_combine_a(const VsConsts& c, int64_t i, const
     st[VS_LAM] = 1.0; st[VS_STATUS] = (double)SAKI_ROW_SATURATED; st[VS_MODE] = VS_SETTLED;
     return;
   }
-  const double m1 = Sd / Ss, var = Sd2 / Ss - m1 * m1;   // the variance of delta is the variance of d
-  double beta = sqrt(2.0 * c.eps / fmax(var, 1e-300));
+  // First guess: d KL(q_beta||p) / d beta = beta Var_{q_beta}(d) and the variance under q_beta is
+  // k2 + k3 beta + k4 beta^2 / 2 + ... in the cumulants of d under p (those of delta: d differs by a constant),
+  // so KL = k2 beta^2 / 2 + k3 beta^3 / 3 + k4 beta^4 / 8 + ...; the root of that polynomial at eps, by Newton
+  // from the root of its first term.
+  double k2, k3, k4;
+  vs_cumulants(Ss, Sd, Sd2, Sd3, Sd4, k2, k3, k4);
+  double beta = sqrt(2.0 * c.eps / fmax(k2, 1e-300));
   if (!(beta > 0.0 && beta < 1.0)) beta = 0.5;
+  {
+    double b = beta;
+    bool ok = true;
+    for (int it = 0; it < 12 && ok; ++it) {
+      const double f = b * b * (0.5 * k2 + b * (k3 / 3.0 + b * 0.125 * k4)) - c.eps;
+      const double fp = b * (k2 + b * (k3 + b * 0.5 * k4));
+      if (!(fp > 0.0)) { ok = false; break; }
+      const double nb = b - f / fp;
+      if (!(nb > 0.0 && nb < 1.0)) { ok = false; break; }
+      const bool done = fabs(nb - b) < 1e-9;
+      b = nb;
+      if (done) break;
+    }
+    if (ok) beta = b;
+  }
   st[VS_BETA] = beta; st[VS_LO] = 0.0; st[VS_HI] = 1.0; st[VS_MODE] = VS_SOLVING;
 }
 
-// one Newton step on KL(q_beta || p) = eps inside the bisection bracket; returns 1 if the row is still solving
+// One wave of the solver: from the sums at beta, KL(q_beta||p), the cumulants of d under q_beta and with them
+// the model  KL(beta + h) = KL(beta) + int_0^h (beta + u) (k2 + k3 u + k4 u^2 / 2) du;  h = its root at eps (Newton
+// from the first-order step), kept inside the bisection bracket.  Returns 1 if the row needs another wave.
 __host__ __device__ inline int vs_combine_b(const VsConsts& c, int64_t i, const double* part, double* st) {
   if ((int)st[VS_MODE] != VS_SOLVING) return 0;
   const int P = SAKI_VSHARD_PARTIALS;
-  double a0 = 0.0, a1 = 0.0, a2 = 0.0;
+  double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0, a4 = 0.0;
   for (int r = 0; r < c.world; ++r) {
     const double* p = part + ((int64_t)r * c.N + i) * P;
-    a0 += p[0]; a1 += p[1]; a2 += p[2];
+    a0 += p[0]; a1 += p[1]; a2 += p[2]; a3 += p[3]; a4 += p[4];
   }
   const double beta = st[VS_BETA], cc = st[VS_LSE_T] - st[VS_LSE_S];
   const double kb = ((1.0 - beta) * st[VS_MS] + beta * st[VS_MT]) / c.tau;    // the shift the partials were taken under
-  const double md = a1 / a0, E = md - cc, var = a2 / a0 - md * md;
+  double k2, k3, k4;
+  vs_cumulants(a0, a1, a2, a3, a4, k2, k3, k4);
+  const double E = a1 / a0 - cc;
   const double logZ = log(a0) + kb - (1.0 - beta) * st[VS_LSE_S] - beta * st[VS_LSE_T];
   const double kl = beta * E - logZ;
   double lo = st[VS_LO], hi = st[VS_HI];
   if (kl <= c.eps) lo = beta; else hi = beta;
   const int it = (int)st[VS_ITER] + 1;
-  double lam = -1.0;
-  const double step = (c.eps - kl) / (beta * var);
-  if (hi - lo < 1e-13 || it >= 100) lam = beta;
-  else if (fabs(step) < 1e-12) lam = fmin(fmax(beta + step, lo), hi);   // a wave is a pass and an exchange: stop at 1e-12
-  else {
-    double nb = beta + step;
-    if (!(nb > lo && nb < hi)) nb = 0.5 * (lo + hi);
-    st[VS_BETA] = nb; st[VS_LO] = lo; st[VS_HI] = hi; st[VS_ITER] = (double)it;
+  double h = (c.eps - kl) / (beta * k2);
+  {
+    double u = h;
+    bool ok = isfinite(u);
+    for (int n = 0; n < 12 && ok; ++n) {
+      const double g = kl - c.eps + beta * u * (k2 + u * (0.5 * k3 + u * k4 / 6.0)) + u * u * (0.5 * k2 + u * (k3 / 3.0 + u * 0.125 * k4));
+      const double gp = (beta + u) * (k2 + u * (k3 + u * 0.5 * k4));
+      if (!(gp > 0.0)) { ok = false; break; }
+      const double nu = u - g / gp;
+      if (!isfinite(nu)) { ok = false; break; }
+      const bool done = fabs(nu - u) < 1e-15;
+      u = nu;
+      if (done) break;
+    }
+    if (ok && fabs(u) <= 2.0 * fabs(h) + 1e-300) h = u;     // the model's root, unless it ran away from the first-order step
+  }
+  const bool inside = isfinite(h) && beta + h > lo && beta + h < hi;
+  if (hi - lo < 1e-13 || it >= 100) h = 0.0;
+  else if (!(inside && fabs(h) < VS_SETTLE_STEP)) {
+    st[VS_BETA] = inside ? beta + h : 0.5 * (lo + hi);
+    st[VS_LO] = lo; st[VS_HI] = hi; st[VS_ITER] = (double)it;
     return 1;
   }
-  st[VS_LAM] = lam;
-  st[VS_LOGZ] = logZ + (lam - beta) * E;                 // |lam - beta| < 1e-12: first order is exact to rounding
+  st[VS_LAM] = beta + h;
+  st[VS_LOGZ] = logZ + h * (E + h * (0.5 * k2 + h * (k3 / 6.0 + h * k4 / 24.0)));   // log Z along beta: the cumulant series of d under q_beta
   st[VS_MODE] = VS_SETTLED;
   return 0;
 }
@@ -223,7 +275,7 @@ struct VsSlice {
 template <typename T>
 __global__ void __launch_bounds__(VT) vs_partial_kernel(const VsSlice S, const int stage, const double* state, double* partial,
                                                         void* dlogits, const int64_t ld_g, const double grad_scale) {
-  __shared__ double red[6 * VW];
+  __shared__ double red[7 * VW];
   __shared__ float smax[2][VW];
   __shared__ int sarg[VW];
   __shared__ int stoken;
@@ -260,16 +312,16 @@ __global__ void __launch_bounds__(VT) vs_partial_kernel(const VsSlice S, const i
         if (smax[1][w] > mt || (smax[1][w] == mt && sarg[w] < am)) { mt = smax[1][w]; am = sarg[w]; }
       }
       __syncthreads();
-      double a[5] = {0.0, 0.0, 0.0, 0.0, 0.0};
+      double a[7] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
       if (finite && Vl > 0) {
         const double zms = (double)ms * rtau, zmt = (double)mt * rtau;
         for (int v = tid; v < Vl; v += VT) {
           const double zs = (double)ld_as_float(s, v) * rtau, zt = (double)ld_as_float(t, v) * rtau;
-          const double es = exp(zs - zms), et = exp(zt - zmt), dl = zt - zs;
-          a[0] += es; a[1] += et; a[2] += et * dl; a[3] += es * dl; a[4] += es * dl * dl;
+          const double es = exp(zs - zms), et = exp(zt - zmt), dl = zt - zs, ed = es * dl, ed2 = ed * dl;
+          a[0] += es; a[1] += et; a[2] += et * dl; a[3] += ed; a[4] += ed2; a[5] += ed2 * dl; a[6] += ed2 * dl * dl;
         }
       }
-      vs_block_sum<5>(a, red);
+      vs_block_sum<7>(a, red);
       if (tid == 0) {
         const int x = S.proposal[row] - S.v0;
         const bool own = x >= 0 && x < Vl;
@@ -278,23 +330,24 @@ __global__ void __launch_bounds__(VT) vs_partial_kernel(const VsSlice S, const i
         out[4] = a[0]; out[5] = a[1]; out[6] = a[2]; out[7] = a[3]; out[8] = a[4];
         out[9] = own ? (double)ld_as_float(s, x) : 0.0; out[10] = own ? (double)ld_as_float(t, x) : 0.0;
         out[11] = own ? 1.0 : 0.0;
+        out[12] = a[5]; out[13] = a[6]; out[14] = 0.0; out[15] = 0.0;
       }
     } else if (stage == 1) {
       // ---- stage B: one evaluation at the row's current beta, under the row's global shift
-      double a[3] = {0.0, 0.0, 0.0};
+      double a[5] = {0.0, 0.0, 0.0, 0.0, 0.0};
       if ((int)st[VS_MODE] == VS_SOLVING) {
         const double beta = st[VS_BETA];
         const double kb = ((1.0 - beta) * st[VS_MS] + beta * st[VS_MT]) * rtau;
         for (int v = tid; v < Vl; v += VT) {
           const double zs = (double)ld_as_float(s, v) * rtau, zt = (double)ld_as_float(t, v) * rtau;
-          const double dl = zt - zs, e = exp(zs + beta * dl - kb);
-          a[0] += e; a[1] += e * dl; a[2] += e * dl * dl;
+          const double dl = zt - zs, e = exp(zs + beta * dl - kb), ed = e * dl, ed2 = ed * dl;
+          a[0] += e; a[1] += ed; a[2] += ed2; a[3] += ed2 * dl; a[4] += ed2 * dl * dl;
         }
       }
-      vs_block_sum<3>(a, red);
+      vs_block_sum<5>(a, red);
       if (tid == 0) {
         for (int k = 0; k < SAKI_VSHARD_PARTIALS; ++k) out[k] = 0.0;
-        out[0] = a[0]; out[1] = a[1]; out[2] = a[2];
+        out[0] = a[0]; out[1] = a[1]; out[2] = a[2]; out[3] = a[3]; out[4] = a[4];
       }
     } else if (stage == 2) {
       // ---- stage C: the slice's share of TV and KL(q||p); the student's logit at the teacher's argmax

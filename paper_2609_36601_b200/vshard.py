@@ -1,7 +1,7 @@
 """Vocabulary-sharded routing: the exchange around the library's stage calls.
 
 Every rank holds a contiguous column slice of the logit rows (as a tensor-parallel lm-head leaves them).  A
-row is routed in four stages; per stage a rank reduces its slice to 12 float64 numbers per row
+row is routed in four stages; per stage a rank reduces its slice to 16 float64 numbers per row
 (`vshard_partial`, a kernel), the ranks all-gather those (96 bytes per row, rank and stage; NCCL over NVLink on
 GPUs, no logits ever cross), and every rank folds the gathered partials in rank order into the same per-row
 state (`vshard_combine`, a kernel).  Stage 1 (one evaluation of the trust-region constraint) repeats until no

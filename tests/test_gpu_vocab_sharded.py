@@ -41,7 +41,7 @@ def test_sliced_rows_match_the_oracle_and_the_unsharded_call(V, world):
                                                grad_scale=0.5)
     torch.cuda.synchronize()
     g = torch.cat(gs, dim=1)
-    assert 3 <= waves <= 12
+    assert 1 <= waves <= 4
     s64, t64 = oracle_inputs(d)
     ref = O.route(s64, t64, d["proposal"].cpu().numpy(), w.eps, w.temperature, w.seed, 0, mask=mask.cpu().numpy(),
                   grad_scale=0.5, want_grad=True, grad_dtype=w.dtype)

@@ -136,7 +136,7 @@ def test_two_gloo_ranks_route_column_slices_and_agree_with_the_oracle():
     (_, out0, g0, waves0), (_, out1, g1, waves1) = got
     for k in out0:                                    # every rank ends with the same outputs, bit for bit
         assert np.array_equal(out0[k], out1[k]), k
-    assert waves0 == waves1 and 3 <= waves0 <= 12     # the float64 Newton iteration settles in a few waves
+    assert waves0 == waves1 and 1 <= waves0 <= 4      # a wave moves to the root of a fourth-order model: two as a rule
     w, s, t, x, mask = _workload()
     ref = _check_against_oracle(w, s, t, x, mask, out0, np.concatenate([g0, g1], axis=1))
     st = ref["status"]

@@ -1,17 +1,17 @@
 """A numpy stand-in for the GPU's vocabulary-slice kernels (saki_vshard_partial), for the multi-process tests
-of the exchange that run without a GPU: given a slice of the logit rows and the per-row state, the 12 numbers
+of the exchange that run without a GPU: given a slice of the logit rows and the per-row state, the 16 numbers
 per row of each stage, as the header defines them.  The combine is NOT modelled here: the tests call the
 library's own host combine (saki_vshard_combine_host)."""
 import numpy as np
 
-P, S = 12, 32
+P, S = 16, 32
 (MODE, STATUS, MS, MT, VSTAR, LSE_S, LSE_T, SX, TX, SV, BETA, LO, HI, ITER, LAM, LOGZ, KL, TV, ACC, CORR,
  OWNER, BEFORE, TARGET, TAKE_LAST, TOK, COEF, LOSS, Y, SY, TY) = range(30)
 SOLVING, SETTLED, FLAGGED = 0, 1, 2
 
 
 def partial(stage, s, t, v0, tau, proposal, state, rank, grad_scale=1.0, want_grad=False):
-    """s, t: [N, V_local] float64 copies of the stored slice values.  Returns ([N, 12] partials, gradient
+    """s, t: [N, V_local] float64 copies of the stored slice values.  Returns ([N, 16] partials, gradient
     slice or None)."""
     N, Vl = s.shape
     out = np.zeros((N, P))
@@ -30,16 +30,18 @@ def partial(stage, s, t, v0, tau, proposal, state, rank, grad_scale=1.0, want_gr
             if fin and Vl:
                 es, et = np.exp(zs - ms / tau), np.exp(zt - mt / tau)
                 sums = [es.sum(), et.sum(), (et * dl).sum(), (es * dl).sum(), (es * dl * dl).sum()]
+                high = [(es * dl ** 3).sum(), (es * dl ** 4).sum()]
             else:
-                sums = [0.0] * 5
+                sums, high = [0.0] * 5, [0.0] * 2
             out[i, :12] = [ms, mt, am, 1.0 if fin else 0.0, *sums, s[i, x] if own else 0.0, t[i, x] if own else 0.0,
                            1.0 if own else 0.0]
+            out[i, 12:14] = high
         elif stage == 1:
             if int(st[MODE]) == SOLVING:
                 b = st[BETA]
                 kb = ((1 - b) * st[MS] + b * st[MT]) / tau
                 e = np.exp(zs + b * dl - kb)
-                out[i, :3] = [e.sum(), (e * dl).sum(), (e * dl * dl).sum()]
+                out[i, :5] = [(e * dl ** k).sum() for k in range(5)]
         elif stage == 2:
             live = int(st[MODE]) == SETTLED
             if live and st[LAM] > 0:
