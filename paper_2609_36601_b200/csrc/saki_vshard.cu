@@ -383,40 +383,68 @@ __global__ void __launch_bounds__(VT) vs_partial_kernel(const VsSlice S, const i
         for (int v = tid; v < Vl; v += VT) {
           double gv = 0.0;
           if (sc != 0.0) gv = sc * (exp((double)ld_as_float(s, v) * rtau - lse_s) - (v == tok ? 1.0 : 0.0));
-          if constexpr (sizeof(T) == 2) g[v] = __double2bfloat16(gv);
-          else g[v] = (float)gv;
+          if constexpr (sizeof(T) == 2) {
+            // float64 -> bf16, round to nearest even: through a float rounded to odd (truncate, and keep in the
+            // last bit whether anything was cut off), which the second rounding cannot mistake for a tie
+            float f = __double2float_rz(gv);
+            if ((double)f != gv) f = __uint_as_float(__float_as_uint(f) | 1u);
+            g[v] = __float2bfloat16_rn(f);
+          } else g[v] = (float)gv;
         }
       }
       if (tid == 0) stoken = -1;
       __syncthreads();
       const bool mine = mode == VS_SETTLED && st[VS_CORR] != 0.0 && (int)st[VS_OWNER] == S.rank;
-      if (mine && warp == 0) {
+      if (mine) {
+        // The inverse-CDF target lies in this slice.  Every warp adds up the residual weights of its contiguous
+        // segment; the warp whose segment holds the target (segments in index order) walks it 32 elements at a time.
         const double lam = st[VS_LAM], lse_s = st[VS_LSE_S], lse_t = st[VS_LSE_T], logZ = st[VS_LOGZ];
         const double target = st[VS_TARGET];
         const bool take_last = st[VS_TAKE_LAST] != 0.0;
-        double running = st[VS_BEFORE];
-        int last_pos = -1, found = -1;
-        for (int v0 = 0; v0 < Vl && found < 0; v0 += 32) {
-          const int v = v0 + lane;
-          double r = 0.0;
-          if (v < Vl) {
-            const double lp = (double)ld_as_float(s, v) * rtau - lse_s, lT = (double)ld_as_float(t, v) * rtau - lse_t;
-            r = fmax(exp(lp + lam * (lT - lp) - logZ) - exp(lp), 0.0);
-          }
-          double inc = r;
+        const int seg = (Vl + VW - 1) / VW, v_lo = min(Vl, warp * seg), v_hi = min(Vl, v_lo + seg);
+        auto weight = [&](int v) {
+          const double lp = (double)ld_as_float(s, v) * rtau - lse_s, lT = (double)ld_as_float(t, v) * rtau - lse_t;
+          return fmax(exp(lp + lam * (lT - lp) - logZ) - exp(lp), 0.0);
+        };
+        double wsum = 0.0;
+        for (int v = v_lo + lane; v < v_hi; v += 32) wsum += weight(v);
 #pragma unroll
-          for (int o = 1; o < 32; o <<= 1) {
-            const double up = __shfl_up_sync(0xffffffffu, inc, o);
-            if (lane >= o) inc += up;
-          }
-          const unsigned pos = __ballot_sync(0xffffffffu, r > 0.0);
-          const unsigned hit = take_last ? 0u : __ballot_sync(0xffffffffu, (running + inc > target) && v < Vl);
-          if (pos) last_pos = v0 + 31 - __clz(pos);
-          if (hit) found = v0 + __ffs(hit) - 1;
-          running += __shfl_sync(0xffffffffu, inc, 31);
+        for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
+        if (lane == 0) red[warp] = wsum;
+        __syncthreads();
+        // the first warp whose running total passes the target; none (rounding, or the rule "last positive
+        // element"): the last warp with weight
+        double before = st[VS_BEFORE];
+        int own_w = -1, last_w = -1;
+        for (int w = 0; w < VW; ++w) {
+          if (red[w] > 0.0) last_w = w;
+          if (own_w < 0 && !take_last && before + red[w] > target) own_w = w;
+          if (own_w < 0) before += red[w];
         }
-        if (found < 0) found = last_pos >= 0 ? last_pos : max(Vl - 1, 0);
-        if (lane == 0) stoken = found;
+        const bool walk_last = own_w < 0;
+        if (walk_last) own_w = last_w;
+        if (warp == own_w) {
+          double running = before;
+          int last_pos = -1, found = -1;
+          for (int v0 = v_lo; v0 < v_hi && found < 0; v0 += 32) {
+            const int v = v0 + lane;
+            const double r = v < v_hi ? weight(v) : 0.0;
+            double inc = r;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+              const double up = __shfl_up_sync(0xffffffffu, inc, o);
+              if (lane >= o) inc += up;
+            }
+            const unsigned pos = __ballot_sync(0xffffffffu, r > 0.0);
+            const unsigned hit = walk_last ? 0u : __ballot_sync(0xffffffffu, (running + inc > target) && v < v_hi);
+            if (pos) last_pos = v0 + 31 - __clz(pos);
+            if (hit) found = v0 + __ffs(hit) - 1;
+            running += __shfl_sync(0xffffffffu, inc, 31);
+          }
+          if (found < 0) found = last_pos >= 0 ? last_pos : max(v_hi - 1, 0);   // rounding: the last element with weight in the segment
+          if (lane == 0) stoken = found;
+        }
+        if (own_w < 0 && tid == 0) stoken = max(Vl - 1, 0);   // no weight anywhere in the slice
       }
       __syncthreads();
       if (tid == 0) {

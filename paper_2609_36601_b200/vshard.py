@@ -2,10 +2,10 @@
 
 Every rank holds a contiguous column slice of the logit rows (as a tensor-parallel lm-head leaves them).  A
 row is routed in four stages; per stage a rank reduces its slice to 16 float64 numbers per row
-(`vshard_partial`, a kernel), the ranks all-gather those (96 bytes per row, rank and stage; NCCL over NVLink on
+(`vshard_partial`, a kernel), the ranks all-gather those (128 bytes per row, rank and stage; NCCL over NVLink on
 GPUs, no logits ever cross), and every rank folds the gathered partials in rank order into the same per-row
 state (`vshard_combine`, a kernel).  Stage 1 (one evaluation of the trust-region constraint) repeats until no
-row is still solving: 5 to 8 waves for the float64 Newton iteration.  This module holds no arithmetic: it
+row is still solving: two waves as a rule (each moves to the root of a fourth-order model of the constraint).  This module holds no arithmetic: it
 sequences the stages, moves the partials, and reads one counter per wave.
 
 `route_vocab_sharded` is the one-rank-per-process form over `torch.distributed`; `route_vocab_sharded_local`
