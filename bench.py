@@ -55,10 +55,11 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one rowsm_kernel launch divided by the positions it
 # routed, from an ncu capture on 2220 rows of the same workload (the kernel's ncu summary gives the
 # command); traffic grows in proportion to the rows, so a full launch is this figure times N
-TRAFFIC_BYTES_PER_POSITION = 945005
+TRAFFIC_BYTES_PER_POSITION = 958203
 # rows up to this length are served by the instances of the two streaming kernels that run two CTAs per SM
 # (namespace half_sm, meta_stream_kernel<16>); the names below are the ones a profiler shows
 TWO_CTA_MAX_V = 98304
+FOUR_CTA_MAX_V = 49152      # and the row kernel's instance with four (namespace quarter_sm) up to this length
 # the same for one meta_stream_kernel launch
 META_TRAFFIC_BYTES_PER_POSITION = 581046
 
@@ -539,7 +540,7 @@ def run_ours(args):
                 "peak_kind": f"of {peak_kind} (device-to-device copy, MEASURED_PEAKS.json)"
                 if peak_kind == "measured" else "of fallback",
                 "traffic": (TRAFFIC_BYTES_PER_POSITION * w.N) if TRAFFIC_BYTES_PER_POSITION else None,
-                "algorithmic_bytes_per_launch": bpp * w.N, "kernel": {3: "saki::%s::rowsm_kernel<false>" % ("half_sm" if w.V <= TWO_CTA_MAX_V else "full_sm"),
+                "algorithmic_bytes_per_launch": bpp * w.N, "kernel": {3: "saki::%s::rowsm_kernel<false>" % ("quarter_sm" if w.V <= FOUR_CTA_MAX_V else "half_sm" if w.V <= TWO_CTA_MAX_V else "full_sm"),
                            2: "saki::cluster_kernel"}.get(kernel_used, "saki::general_kernel"),
                 "kernel_ms": kern_ms,
                 "frac_of_nominal_8TBs": achieved / 8000.0}

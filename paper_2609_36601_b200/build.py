@@ -11,7 +11,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsaki.so")
-SOURCES = ("saki_api.cu", "saki_general.cu", "saki_cluster.cu", "saki_rowsm.cu", "saki_rowsm_half.cu", "saki_meta.cu",
+SOURCES = ("saki_api.cu", "saki_general.cu", "saki_cluster.cu", "saki_rowsm.cu", "saki_rowsm_half.cu", "saki_rowsm_quarter.cu", "saki_meta.cu",
            "saki_select.cu", "saki_vshard.cu", "saki_lmhead.cu")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]

@@ -165,6 +165,7 @@ bool cluster_can_serve(const RowParams& p, int dtype);
 cudaError_t launch_rowsm(const RowParams& p, cudaStream_t st, int* n_launches, bool* served);
 namespace full_sm { cudaError_t launch(const RowParams& p, cudaStream_t st, int* n_launches, bool* served); int max_v(); }
 namespace half_sm { cudaError_t launch(const RowParams& p, cudaStream_t st, int* n_launches, bool* served); int max_v(); }
+namespace quarter_sm { cudaError_t launch(const RowParams& p, cudaStream_t st, int* n_launches, bool* served); int max_v(); }
 bool rowsm_can_serve(const RowParams& p, int dtype);
 cudaError_t launch_meta_general(const MetaParams& p, int dtype, cudaStream_t st, int* n_launches);
 cudaError_t launch_meta_stream(const MetaParams& p, cudaStream_t st, int* n_launches, bool* served);

@@ -1,4 +1,4 @@
-// Row-per-SM kernel, the variant with one CTA of 512 threads per SM, and the choice between the two
+// Row-per-SM kernel, the variant with one CTA of 512 threads per SM, and the choice between the three
 // variants (the implementation is saki_rowsm_impl.cuh).
 #include "saki_rowsm_impl.cuh"
 
@@ -11,6 +11,10 @@ namespace saki {
 // one / two CTAs per SM): V = 8192 15.9 / 25.3, 32000 9.9 / 12.7, 65536 6.5 / 7.5, 81920 5.6 / 6.3,
 // 100000 4.85 / 5.06, 131072 3.95 / 3.76.
 constexpr int HALF_MAX_V = 98304;
+// Shorter rows still go to the variant with four CTAs of 128 threads per SM: more of the SM's rows are in a
+// pass at any time.  Measured (M rows/s, two / four CTAs per SM): V = 4096 29.7 / 44.4, 8192 26.0 / 35.0,
+// 16384 19.6 / 21.7, 32000 13.1 / 14.3, 49152 9.8 / 10.0, 65536 7.8 / 7.5.
+constexpr int QUARTER_MAX_V = 49152;
 
 bool rowsm_can_serve(const RowParams& p, int dtype) {
   if (dtype != SAKI_BF16) return false;
@@ -24,6 +28,7 @@ bool rowsm_can_serve(const RowParams& p, int dtype) {
 }
 
 cudaError_t launch_rowsm(const RowParams& p, cudaStream_t st, int* n_launches, bool* served) {
+  if (p.V <= QUARTER_MAX_V && p.V <= quarter_sm::max_v()) return quarter_sm::launch(p, st, n_launches, served);
   if (p.V <= HALF_MAX_V && p.V <= half_sm::max_v()) return half_sm::launch(p, st, n_launches, served);
   return full_sm::launch(p, st, n_launches, served);
 }

@@ -3,6 +3,7 @@
 //   saki_rowsm_half.cu  two persistent CTAs of 256 threads per SM (namespace half_sm, SAKI_ROWSM_HALF):
 //                       for short rows, whose passes are short against the serial phases between them,
 //                       so that one CTA's scalar phases run under the other CTA's passes
+//   saki_rowsm_quarter.cu  four of 128 threads (namespace quarter_sm, SAKI_ROWSM_QUARTER): shorter rows still
 //
 // A persistent CTA routes whole rows, one after the
 // other.  A row pair (student + teacher, e.g. 608 KB at V = 151936) does not
@@ -32,7 +33,11 @@
 #include "saki_device.cuh"
 #include <mutex>
 
-#ifdef SAKI_ROWSM_HALF
+#if defined(SAKI_ROWSM_QUARTER)
+#define SAKI_ROWSM_NS quarter_sm
+#define SAKI_ROWSM_THREADS 128
+#define SAKI_ROWSM_CTAS 4
+#elif defined(SAKI_ROWSM_HALF)
 #define SAKI_ROWSM_NS half_sm
 #define SAKI_ROWSM_THREADS 256
 #define SAKI_ROWSM_CTAS 2
@@ -52,7 +57,7 @@ constexpr int KS_MAX = 208 / (RW * CTAS_PER_SM);   // steps per warp that fit in
 constexpr int MAX_STEPS = 64;            // steps per warp the draw bookkeeping can hold (V <= 64*32*8*RW)
 constexpr int RES_CHUNKS = KS_MAX * 32; // resident chunks per warp and row
 constexpr int RNV = 9;                  // doubles per partial vector
-static_assert(RW >= 14 || RW == 8, "warps 0-7 gather; the side work has warps of its own, or is shared out among those eight");
+static_assert(RW >= 14 || RW == 8 || RW == 4, "the eight gather roles go round the first eight warps; the side work has warps of its own, or is shared out");
 // Who does what beside the passes.  With 14 warps or more the row scalars that do not depend on the
 // passes (uniforms, the logits at the proposal) are fetched by warps 8-10 while warps 0-7 gather; with
 // eight warps, by warps 1-3 before the block barrier that ends pass "lse".  After the gather, while
@@ -60,7 +65,7 @@ static_assert(RW >= 14 || RW == 8, "warps 0-7 gather; the side work has warps of
 // block verification, lane 0 of SV_WARP fetches the student's logit at the teacher's argmax.
 constexpr bool SIDE_WARPS = RW >= 14;
 constexpr int UACC_WARP = SIDE_WARPS ? 8 : 1, UDRAW_WARP = SIDE_WARPS ? 9 : 2, SX_WARP = SIDE_WARPS ? 10 : 3;
-constexpr int RES_WARP = SIDE_WARPS ? 11 : 5, SV_WARP = SIDE_WARPS ? 13 : 6;
+constexpr int RES_WARP = SIDE_WARPS ? 11 : (RW == 8 ? 5 : 2), SV_WARP = SIDE_WARPS ? 13 : (RW == 8 ? 6 : 3);
 static_assert(KS_MAX - 4 >= 1, "every warp keeps at least its first step resident");
 
 constexpr int ROFF_S = 0;                                        // [RW][RES_CHUNKS] uint4
@@ -72,7 +77,7 @@ constexpr int ROFF_WMAX = ROFF_BC + 2 * BC_DOUBLES * 8;          // [3][RW]: tea
 constexpr int ROFF_STEP = ROFF_WMAX + 4 * RW * 4;                // [RW][MAX_STEPS] floats: draw weight of each step
 constexpr int ROFF_FIN = ROFF_STEP + RW * MAX_STEPS * 4;          // [2][2][RW] doubles: what pass "final" leaves per warp, by row parity
 constexpr int ROFF_MBAR = ROFF_FIN + 2 * 2 * RW * 8;
-constexpr int FIN_WARP = SIDE_WARPS ? 12 : 4;   // the warp that finishes the previous row
+constexpr int FIN_WARP = SIDE_WARPS ? 12 : (RW == 8 ? 4 : 1);   // the warp that finishes the previous row
 constexpr int ROFF_SEQ = ROFF_MBAR + 16;   // [4] ints: block verification, the CTA's reservation state
 constexpr int ROFF_PH = ROFF_SEQ + 16;     // [PH_WORDS] 64-bit words: the phase clock of thread 0
 constexpr int RSMEM_BYTES = ROFF_PH + PH_WORDS * 8;
@@ -350,9 +355,10 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
       for (int k = 0; k < RNV; ++k) if (k < n) red[k * RW + warp] = v[k];
     }
     __syncthreads();
-    if (warp < n) {
-      const double a = warp_sum_d(lane < RW ? red[warp * RW + lane] : 0.0);
-      if (lane == 0) gat[warp] = a;
+#pragma unroll 1
+    for (int k = warp; k < n; k += RW) {
+      const double a = warp_sum_d(lane < RW ? red[k * RW + lane] : 0.0);
+      if (lane == 0) gat[k] = a;
     }
     __syncthreads();
   };
@@ -653,20 +659,22 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
       if (!SIDE_WARPS && lane == 0) side_work();
       const int any_dead = __syncthreads_or(dead ? 1 : 0);
       RTS(PH_LSE_REDUCE);
-      if (warp < 8) {   // block level: warps 0-6 add up one sum each on the row's shifts, warp 7 finds the argmax
+      if (warp < 8) {   // block level, eight roles dealt round the first eight warps: 0-6 add up one sum each on the row's shifts, 7 finds the argmax
+#pragma unroll 1
+       for (int role = warp; role < 8; role += RW) {
         const int wl = lane < RW ? lane : 0;       // lanes beyond the warp count carry zero weight
         const float* wm = (const float*)(smem + ROFF_WMAX);
-        if (warp < 7) {
+        if (role < 7) {
           // From here on the row's shifts are those of its true maxima (the largest term of each sum has
           // its exponent argument in (-1, 0], where float32 resolves it best); a warp's shift came from an
           // element of the row, so it is never below the row's, and the factor is an exact power of two <= 1.
-          const bool teacher = (warp == 1 || warp == 5);
+          const bool teacher = (role == 1 || role == 5);
           const float mx = warp_max_f(lane < RW ? wm[teacher ? wl : 2 * RW + wl] : -CUDART_INF_F);
           const double kr = (double)-ceilf(c32 * fmaxf(mx, -1e30f));
           const double kw = lane < RW ? red[(teacher ? 8 : 7) * RW + wl] : 1e30;
           const double f = kw < 1e29 ? (double)pow2f_exact((float)(kr - kw)) : 0.0;
-          const double a = warp_sum_d(f * red[warp * RW + wl]);
-          if (lane == 0) { gat[warp < 6 ? warp : 9] = a; if (warp < 2) gat[7 + warp] = kr; }   // gat[9]: the fourth moment
+          const double a = warp_sum_d(f * red[role * RW + wl]);
+          if (lane == 0) { gat[role < 6 ? role : 9] = a; if (role < 2) gat[7 + role] = kr; }   // gat[9]: the fourth moment
         } else {
           float gmt = lane < RW ? wm[wl] : -CUDART_INF_F;
           int garg = ((const int*)wm)[RW + wl];
@@ -691,6 +699,7 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
             gat[6] = (double)best;
           }
         }
+       }
       } else if (SIDE_WARPS && lane == 0) {
         side_work();                             // meanwhile, on warps that would only wait
       }

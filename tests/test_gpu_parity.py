@@ -339,8 +339,9 @@ def test_small_radii_on_the_row_per_sm_kernel(eps):
         assert P.last_kernel() == 3
         assert P.redo_count() <= 20
         lam = out["lambda"].cpu().numpy()[list(rows)].astype(np.float64)
-        # below 5e-3 every row is settled by the quadrature or by the float64 kernel
-        assert np.max(np.abs(lam - ref["lam"])) <= (5e-7 if eps < 5e-3 else 1e-5)
+        # below 5e-3 every row is settled by the quadrature or by the float64 kernel: held to a tenth of the
+        # tolerance on lambda (1e-5)
+        assert np.max(np.abs(lam - ref["lam"])) <= (1e-6 if eps < 5e-3 else 1e-5)
     finally:
         P.set_kernel(prev)
 
