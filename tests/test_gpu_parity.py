@@ -102,6 +102,21 @@ def test_rowsm_streamed_shapes(V):
         P.set_kernel(prev)
 
 
+@pytest.mark.parametrize("V", [13320, 14344, 26808, 49152])
+def test_rowsm_streamed_shapes_four_blocks_per_sm(V):
+    """The same for the instance with four blocks of four warps per SM (rows up to 49152 elements): one warp
+    of four with a streamed part, the shortest streamed part with a ragged last step, an odd number of streamed
+    steps, the longest row it serves; more rows than blocks, so the ring runs over into the next row."""
+    prev = P.set_kernel(3)
+    try:
+        w = synth.Workload("t", 700, V, "bf16", 0.1, 1.5, True, 137, 43)
+        d = synth.generate(w, DEV)
+        _check_fwd_bwd(d, w, rows=range(0, 700, 41), row_offset=3)
+        assert P.last_kernel() == 3
+    finally:
+        P.set_kernel(prev)
+
+
 def test_strided_rows_and_mask(kernel):
     w = synth.Workload("t", 12, 3000, "bf16", 0.05, 1.0, True, 78, 10)
     d = synth.generate(w, DEV)
