@@ -60,6 +60,8 @@ TRAFFIC_BYTES_PER_POSITION = 958203
 # (namespace half_sm, meta_stream_kernel<16>); the names below are the ones a profiler shows
 TWO_CTA_MAX_V = 98304
 FOUR_CTA_MAX_V = 49152      # and the row kernel's instance with four (namespace quarter_sm) up to this length
+# warp-instructions the row kernel's one-CTA instance issues per 32 vocabulary elements, from the same capture
+ISSUED_PER_32_ELEMENTS = 37.75
 # the same for one meta_stream_kernel launch
 META_TRAFFIC_BYTES_PER_POSITION = 581046
 
@@ -268,14 +270,15 @@ def _lm_head(P, dev, stream, steps, rows=0):
                          "traffic": None}}
 
 
-def _vocab_sharded(P, synth, dev, stream):
-    """Vocabulary-sharded routing of 1024 rows of the headline workload's shape cut into 8 column slices, the ranks
+def _vocab_sharded(P, synth, dev, stream, peak):
+    """Vocabulary-sharded routing of 4096 rows of the headline workload's shape cut into 8 column slices, the ranks
     run one after the other on this GPU (the calls one rank per GPU would make around its all-gathers): time of
-    all ranks' kernels, evaluation waves, bytes a rank sends per row."""
+    all ranks' kernels, evaluation waves, bytes a rank sends per row, and the slice kernels' HBM traffic (every
+    stage reads the slice again: the rows of a call do not fit in L2) against the copy bandwidth."""
     import torch
     from paper_2609_36601_b200 import binding as B
     from paper_2609_36601_b200.vshard import route_vocab_sharded_local, split_columns
-    w = synth.shrink(synth.WORKLOADS["cfg3"], 1024)
+    w = synth.shrink(synth.WORKLOADS["cfg3"], 4096)
     d = synth.generate(w, dev)
     world = 8
     slices = [(d["s"][:, a:a + n], d["t"][:, a:a + n], a) for a, n in split_columns(w.V, world)]
@@ -289,12 +292,19 @@ def _vocab_sharded(P, synth, dev, stream):
     torch.cuda.synchronize()
     dt = time.perf_counter() - t0
     stages = 3 + waves
+    # algorithmic bytes of the staged protocol: the two slices read by stage 0 (its second sweep counted as an L2
+    # hit), by the first evaluation wave and by stage 2, the student's slice read and the gradient slice written by
+    # stage 3 (later waves touch only the rows still solving: not counted)
+    alg = w.N * w.V * 2 * (2 + 2 + 2 + 1 + 1)
+    gbs = alg / dt / 1e9
     return {"call": "saki_vshard_partial / saki_vshard_combine", "rows": w.N, "V": w.V, "ranks_emulated_on_one_gpu": world,
             "ms_all_ranks": dt * 1e3, "ms_per_rank": dt * 1e3 / world, "value": w.N / dt, "unit": UNIT,
             "evaluation_waves": waves, "stages": stages,
-            "bytes_sent_per_row_and_rank": stages * B.VSHARD_PARTIALS * 8, "arithmetic": "f64",
-            "note": "float64 slice kernels, one block per row; value = rows / time of all 8 ranks' kernels run one after "
-                    "the other on this GPU (a rank's own share is ms_per_rank, the exchanges not included)"}
+            "bytes_sent_per_row_and_rank": stages * B.VSHARD_PARTIALS * 8, "arithmetic": "f32 per element, f64 sums and scalars",
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                         "algorithmic_bytes": alg},
+            "note": "value = rows / wall time of all 8 ranks' kernels run one after the other on this GPU, host-side "
+                    "sequencing included (a rank's own share is ms_per_rank, the exchanges not included)"}
 
 
 def _sweep(P, synth, dev, stream, peak, args):
@@ -557,6 +567,15 @@ def run_ours(args):
         roofline["special_function_pipe"] = {"achieved": xu_ach, "peak": xu_peak, "unit": "G ex2/s",
                                              "frac": xu_ach / xu_peak, "evaluation_passes_per_row": evals,
                                              "ex2_per_element": 4.0 + evals}
+        # and its other near-binding bound: issue slots (4 warp-instructions per clock per SM); the instruction
+        # count per 32 elements is the profiler's (smsp__inst_executed.sum of the capture the kernel's ncu
+        # summary describes, divided by the elements of that launch), not counted live
+        if w.V > TWO_CTA_MAX_V:
+            iss_peak = 4.0 * sm_count * mhz * 1e6 / 1e9
+            iss_ach = ISSUED_PER_32_ELEMENTS * w.V * w.N / 32.0 / (kern_ms * 1e-3) / 1e9
+            roofline["issue_slots"] = {"achieved": iss_ach, "peak": iss_peak, "unit": "G warp-instructions/s",
+                                       "frac": iss_ach / iss_peak, "issued_per_32_elements": ISSUED_PER_32_ELEMENTS,
+                                       "source": "ncu capture on 2220 rows of this workload"}
 
     stats = {"correction_rate": float(out["corrected"].float().mean().item()),
              "median_tv": float(out["tv"].median().item()), "mean_lambda": float(out["lambda"].mean().item()),
@@ -601,7 +620,7 @@ def run_ours(args):
         torch.cuda.empty_cache()
         sweep = _sweep(P, synth, dev, stream, peak, args)
         torch.cuda.empty_cache()
-        vocab_sharded = _vocab_sharded(P, synth, dev, stream)
+        vocab_sharded = _vocab_sharded(P, synth, dev, stream, peak)
         torch.cuda.empty_cache()
         lm_head = _lm_head(P, dev, stream, 5)      # last: a dense GEMM at the power limit would colour what follows it
 

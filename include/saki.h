@@ -243,9 +243,13 @@ SAKI_API int saki_select_tm(const saki_select_in* in, uint8_t* selected, int32_t
  *      (Eqs. "k1_loss_token", "teacher_mode_loss") and which rank owns the residual draw (Eq. "residual")
  *   3  the gradient slice (Eq. "general_objective": dlogits_slice [N, V_local], same dtype, may be NULL) and,
  *      on the owning rank, the drawn token; the combine writes the per-position outputs
- * Everything is float64; results equal the unsharded call's to rounding (float outputs ~1e-12 before the
- * cast to float32; flags and ids wherever the decision is not within rounding of its threshold) and do not
- * depend on the number of ranks beyond that.  Arguments: `proposal` holds GLOBAL token ids; `state` and
+ * Arithmetic: bf16 slices that start on 16-byte boundaries (V_local, v0 and the strides multiples of 8) with
+ * eps >= 0.02 are reduced with the per-element arithmetic of the unsharded bf16 kernels (float32 elements,
+ * float64 sums and scalars; a row that float32 cannot resolve goes on in float64, decided in the combine);
+ * everything else, and every call under saki_set_kernel(1), is float64 throughout.  Results equal the
+ * unsharded call's within the tolerances of that arithmetic (float64: ~1e-12 before the cast to float32;
+ * flags and ids wherever the decision is not within rounding of its threshold) and do not depend on the
+ * number of ranks beyond that.  saki_set_kernel must be the same on every rank of a call.  Arguments: `proposal` holds GLOBAL token ids; `state` and
  * `partial` are caller-owned buffers ([N][SAKI_VSHARD_STATE], [N][SAKI_VSHARD_PARTIALS] doubles); `state`
  * may be NULL at stage 0 of saki_vshard_partial.  saki_vshard_partial and saki_vshard_combine take DEVICE
  * pointers and run asynchronously on the stream; `n_solving` (device, may be NULL) receives the number of

@@ -465,7 +465,7 @@ SAKI_API int saki_vshard_partial(const saki_vshard_in* in, int stage, const doub
   rc = device_ready(&flagged);
   if (rc) return rc;
   cudaError_t e = launch_vshard_partial(*in, stage, state, partial, stage == 3 ? dlogits_slice : nullptr, ld_g, grad_scale,
-                                        (cudaStream_t)cuda_stream);
+                                        g_kernel.load() != 1, (cudaStream_t)cuda_stream);
   if (e != cudaSuccess) return cuda_fail(e, "vocabulary-sharded partial kernel launch");
   g_launches += 1;
   return SAKI_OK;
@@ -489,7 +489,7 @@ SAKI_API int saki_vshard_combine(const saki_vshard_in* in, int stage, const doub
   }
   saki_out none;
   memset(&none, 0, sizeof(none));
-  cudaError_t e = launch_vshard_combine(*in, stage, gathered, state, out ? *out : none, n_solving, st);
+  cudaError_t e = launch_vshard_combine(*in, stage, gathered, state, out ? *out : none, n_solving, g_kernel.load() != 1, st);
   if (e != cudaSuccess) return cuda_fail(e, "vocabulary-sharded combine kernel launch");
   g_launches += 1;
   return SAKI_OK;
@@ -506,7 +506,7 @@ SAKI_API int saki_vshard_combine_host(const saki_vshard_in* in, int stage, const
   if (stage == 3 && (!out || !out->corrected || !out->token)) return fail(SAKI_ERR_INVALID_ARG, "out.corrected and out.token are required at stage 3");
   saki_out none;
   memset(&none, 0, sizeof(none));
-  const int solving = vshard_combine_host(*in, stage, gathered, state, out ? *out : none);
+  const int solving = vshard_combine_host(*in, stage, gathered, state, out ? *out : none, g_kernel.load() != 1);
   if (n_solving) *n_solving = solving;
   return SAKI_OK;
 }

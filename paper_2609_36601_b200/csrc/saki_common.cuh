@@ -172,12 +172,13 @@ cudaError_t launch_meta_stream(const MetaParams& p, cudaStream_t st, int* n_laun
 bool meta_stream_can_serve(const MetaParams& p, int dtype);
 cudaError_t launch_select(const SelectParams& p, cudaStream_t st, int* n_launches);
 cudaError_t launch_vshard_partial(const saki_vshard_in& in, int stage, const double* state, double* partial, void* dlogits,
-                                  int64_t ld_g, float grad_scale, cudaStream_t st);
+                                  int64_t ld_g, float grad_scale, bool allow_fast, cudaStream_t st);
 cudaError_t launch_vshard_combine(const saki_vshard_in& in, int stage, const double* gathered, double* state, const saki_out& out,
-                                  unsigned int* n_solving, cudaStream_t st);
+                                  unsigned int* n_solving, bool allow_fast, cudaStream_t st);
 int64_t lmhead_scratch_bytes(int64_t N, int32_t V);
 cudaError_t launch_lmhead(const saki_lmhead_in& in, void* logits, int64_t ld_l, float* row_max, float* lse, void* scratch,
                           cudaStream_t st, const char** why);
-int vshard_combine_host(const saki_vshard_in& in, int stage, const double* gathered, double* state, const saki_out& out);
+int vshard_combine_host(const saki_vshard_in& in, int stage, const double* gathered, double* state, const saki_out& out,
+                        bool allow_fast);
 
 }  // namespace saki

@@ -4,7 +4,8 @@
 // kernel here), the ranks exchange the partials (the caller's all-gather: ~100 bytes per row and stage),
 // and every rank combines them, in rank order, into the same per-row state (a kernel here, and the same
 // function compiled for the host).  What is computed is the definition (Eqs. "bridge", "trust_region",
-// "accept", "residual", "k1_loss_token", "teacher_mode_loss", "general_objective"), in float64.  An evaluation
+// "accept", "residual", "k1_loss_token", "teacher_mode_loss", "general_objective"); sums, scalars and every
+// combine in float64.  An evaluation
 // of q_beta costs every rank a pass over its slice and the ranks an exchange, so the solver makes each one
 // count: it carries the first four cumulants of the logit difference, the first guess is the root of the
 // fourth-order series of KL(q_beta||p) at beta = 0, and each wave moves to the root of the fourth-order model
@@ -16,8 +17,9 @@
 //   stage C  the slice's share of TV = sum [q - p]_+ and of KL(q||p), the student's logit at the teacher's
 //            argmax; the combine decides acceptance and finds the rank that owns the inverse-CDF target
 //   stage D  the gradient slice, and on the owning rank the residual draw; the last combine writes the outputs
-// One thread block per row; float64 throughout.
-#include "saki_common.cuh"
+// Two families of slice kernels: float64 throughout (one block of 16 warps per row; any dtype, any alignment),
+// and, further down, float32 per element for aligned bf16 slices.
+#include "saki_device.cuh"
 #include <math_constants.h>
 #include <cmath>
 
@@ -28,6 +30,7 @@ enum { VS_MODE = 0,      // 0 solving, 1 settled, 2 flagged
        VS_STATUS, VS_MS, VS_MT, VS_VSTAR, VS_LSE_S, VS_LSE_T, VS_SX, VS_TX, VS_SV,
        VS_BETA, VS_LO, VS_HI, VS_ITER, VS_LAM, VS_LOGZ, VS_KL, VS_TV, VS_ACC, VS_CORR,
        VS_OWNER, VS_BEFORE, VS_TARGET, VS_TAKE_LAST, VS_TOK, VS_COEF, VS_LOSS, VS_Y, VS_SY, VS_TY,
+       VS_F64,        // 1: the row is ill-conditioned for the float32 slice kernels, the float64 ones take it
        VS_COUNT };
 static_assert(VS_COUNT <= SAKI_VSHARD_STATE, "state record too small");
 enum { VS_SOLVING = 0, VS_SETTLED = 1, VS_FLAGGED = 2 };
@@ -39,6 +42,7 @@ struct VsConsts {
   uint64_t seed, row_offset;
   const int32_t* proposal;
   const uint8_t* mask;
+  int fast;          // the float32 slice kernels may be at work (a property of the call, the same on every rank)
 };
 
 // the second to fourth cumulants of delta from the sums  a_k = sum w delta^k, k = 0..4
@@ -160,6 +164,18 @@ __host__ __device__ inline int vs_combine_b(const VsConsts& c, int64_t i, const 
     st[VS_LO] = lo; st[VS_HI] = hi; st[VS_ITER] = (double)it;
     return 1;
   }
+  if (c.fast && st[VS_F64] == 0.0) {
+    // The float32 slice kernels resolve KL to a few 1e-7 x (largest probability of either row).  Where that
+    // would move lambda by more than a tenth of its tolerance (a very flat KL: nearly one-hot rows, whose TV
+    // and acceptance probability move many times faster than lambda) the row goes on in float64.
+    const double pmax = fmin(1.0, exp(fmax(st[VS_MS] / c.tau - st[VS_LSE_S], st[VS_MT] / c.tau - st[VS_LSE_T])));
+    if (3e-7 * pmax > 1e-6 * beta * k2) {
+      st[VS_F64] = 1.0;
+      st[VS_BETA] = inside ? beta + h : beta;
+      st[VS_LO] = 0.0; st[VS_HI] = 1.0; st[VS_ITER] = (double)it;     // the bracket came from float32 sums: start it over
+      return 1;
+    }
+  }
   st[VS_LAM] = beta + h;
   st[VS_LOGZ] = logZ + h * (E + h * (0.5 * k2 + h * (k3 / 6.0 + h * k4 / 24.0)));   // log Z along beta: the cumulant series of d under q_beta
   st[VS_MODE] = VS_SETTLED;
@@ -272,9 +288,65 @@ struct VsSlice {
   const int32_t* proposal;
 };
 
+// The residual draw on the rank that owns the inverse-CDF target (all threads of the block call; NW warps).
+// Every warp adds up the residual weights of its contiguous segment; the warp whose segment holds the target
+// (segments in index order) walks it 32 elements at a time.  float64, whichever kernel family calls.
+template <typename T, int NW>
+__device__ __forceinline__ void vs_draw(const T* s, const T* t, int Vl, double rtau, const double* st, double* red, int* stoken) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const double lam = st[VS_LAM], lse_s = st[VS_LSE_S], lse_t = st[VS_LSE_T], logZ = st[VS_LOGZ];
+  const double target = st[VS_TARGET];
+  const bool take_last = st[VS_TAKE_LAST] != 0.0;
+  const int seg = (Vl + NW - 1) / NW, v_lo = min(Vl, warp * seg), v_hi = min(Vl, v_lo + seg);
+  auto weight = [&](int v) {
+    const double lp = (double)ld_as_float(s, v) * rtau - lse_s, lT = (double)ld_as_float(t, v) * rtau - lse_t;
+    return fmax(exp(lp + lam * (lT - lp) - logZ) - exp(lp), 0.0);
+  };
+  double wsum = 0.0;
+  for (int v = v_lo + lane; v < v_hi; v += 32) wsum += weight(v);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
+  if (lane == 0) red[warp] = wsum;
+  __syncthreads();
+  // the first warp whose running total passes the target; none (rounding, or the rule "last positive
+  // element"): the last warp with weight
+  double before = st[VS_BEFORE];
+  int own_w = -1, last_w = -1;
+  for (int w = 0; w < NW; ++w) {
+    if (red[w] > 0.0) last_w = w;
+    if (own_w < 0 && !take_last && before + red[w] > target) own_w = w;
+    if (own_w < 0) before += red[w];
+  }
+  const bool walk_last = own_w < 0;
+  if (walk_last) own_w = last_w;
+  if (warp == own_w) {
+    double running = before;
+    int last_pos = -1, found = -1;
+    for (int v0 = v_lo; v0 < v_hi && found < 0; v0 += 32) {
+      const int v = v0 + lane;
+      const double r = v < v_hi ? weight(v) : 0.0;
+      double inc = r;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const double up = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += up;
+      }
+      const unsigned pos = __ballot_sync(0xffffffffu, r > 0.0);
+      const unsigned hit = walk_last ? 0u : __ballot_sync(0xffffffffu, (running + inc > target) && v < v_hi);
+      if (pos) last_pos = v0 + 31 - __clz(pos);
+      if (hit) found = v0 + __ffs(hit) - 1;
+      running += __shfl_sync(0xffffffffu, inc, 31);
+    }
+    if (found < 0) found = last_pos >= 0 ? last_pos : max(v_hi - 1, 0);   // rounding: the last element with weight in the segment
+    if (lane == 0) *stoken = found;
+  }
+  if (own_w < 0 && tid == 0) *stoken = max(Vl - 1, 0);   // no weight anywhere in the slice
+}
+
 template <typename T>
 __global__ void __launch_bounds__(VT) vs_partial_kernel(const VsSlice S, const int stage, const double* state, double* partial,
-                                                        void* dlogits, const int64_t ld_g, const double grad_scale) {
+                                                        void* dlogits, const int64_t ld_g, const double grad_scale,
+                                                        const bool only_flagged) {
   __shared__ double red[7 * VW];
   __shared__ float smax[2][VW];
   __shared__ int sarg[VW];
@@ -287,6 +359,7 @@ __global__ void __launch_bounds__(VT) vs_partial_kernel(const VsSlice S, const i
     const T* t = (const T*)S.t + row * S.ld_t;
     double* out = partial + row * SAKI_VSHARD_PARTIALS;
     const double* st = state ? state + row * SAKI_VSHARD_STATE : nullptr;
+    if (only_flagged && !(st != nullptr && st[VS_F64] != 0.0)) continue;   // the float32 kernel has this row
     if (stage == 0) {
       // ---- stage A: maxima and argmax, then the sums under this slice's own shifts
       float ms = -CUDART_INF_F, mt = -CUDART_INF_F;
@@ -395,57 +468,7 @@ __global__ void __launch_bounds__(VT) vs_partial_kernel(const VsSlice S, const i
       if (tid == 0) stoken = -1;
       __syncthreads();
       const bool mine = mode == VS_SETTLED && st[VS_CORR] != 0.0 && (int)st[VS_OWNER] == S.rank;
-      if (mine) {
-        // The inverse-CDF target lies in this slice.  Every warp adds up the residual weights of its contiguous
-        // segment; the warp whose segment holds the target (segments in index order) walks it 32 elements at a time.
-        const double lam = st[VS_LAM], lse_s = st[VS_LSE_S], lse_t = st[VS_LSE_T], logZ = st[VS_LOGZ];
-        const double target = st[VS_TARGET];
-        const bool take_last = st[VS_TAKE_LAST] != 0.0;
-        const int seg = (Vl + VW - 1) / VW, v_lo = min(Vl, warp * seg), v_hi = min(Vl, v_lo + seg);
-        auto weight = [&](int v) {
-          const double lp = (double)ld_as_float(s, v) * rtau - lse_s, lT = (double)ld_as_float(t, v) * rtau - lse_t;
-          return fmax(exp(lp + lam * (lT - lp) - logZ) - exp(lp), 0.0);
-        };
-        double wsum = 0.0;
-        for (int v = v_lo + lane; v < v_hi; v += 32) wsum += weight(v);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
-        if (lane == 0) red[warp] = wsum;
-        __syncthreads();
-        // the first warp whose running total passes the target; none (rounding, or the rule "last positive
-        // element"): the last warp with weight
-        double before = st[VS_BEFORE];
-        int own_w = -1, last_w = -1;
-        for (int w = 0; w < VW; ++w) {
-          if (red[w] > 0.0) last_w = w;
-          if (own_w < 0 && !take_last && before + red[w] > target) own_w = w;
-          if (own_w < 0) before += red[w];
-        }
-        const bool walk_last = own_w < 0;
-        if (walk_last) own_w = last_w;
-        if (warp == own_w) {
-          double running = before;
-          int last_pos = -1, found = -1;
-          for (int v0 = v_lo; v0 < v_hi && found < 0; v0 += 32) {
-            const int v = v0 + lane;
-            const double r = v < v_hi ? weight(v) : 0.0;
-            double inc = r;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-              const double up = __shfl_up_sync(0xffffffffu, inc, o);
-              if (lane >= o) inc += up;
-            }
-            const unsigned pos = __ballot_sync(0xffffffffu, r > 0.0);
-            const unsigned hit = walk_last ? 0u : __ballot_sync(0xffffffffu, (running + inc > target) && v < v_hi);
-            if (pos) last_pos = v0 + 31 - __clz(pos);
-            if (hit) found = v0 + __ffs(hit) - 1;
-            running += __shfl_sync(0xffffffffu, inc, 31);
-          }
-          if (found < 0) found = last_pos >= 0 ? last_pos : max(v_hi - 1, 0);   // rounding: the last element with weight in the segment
-          if (lane == 0) stoken = found;
-        }
-        if (own_w < 0 && tid == 0) stoken = max(Vl - 1, 0);   // no weight anywhere in the slice
-      }
+      if (mine) vs_draw<T, VW>(s, t, Vl, rtau, st, red, &stoken);
       __syncthreads();
       if (tid == 0) {
         for (int k = 0; k < SAKI_VSHARD_PARTIALS; ++k) out[k] = 0.0;
@@ -453,6 +476,410 @@ __global__ void __launch_bounds__(VT) vs_partial_kernel(const VsSlice S, const i
         if (mine && stoken >= 0 && stoken < Vl) {
           out[0] = (double)(S.v0 + stoken);
           out[1] = (double)ld_as_float(s, stoken); out[2] = (double)ld_as_float(t, stoken);
+        }
+      }
+      __syncthreads();
+    }
+  }
+}
+
+// ---------------------------------------------------------------- the float32 slice kernels
+// The same partials for bf16 slices that start on a 16-byte boundary, with the per-element arithmetic of the
+// row-per-SM kernel: packed f32x2 FMAs, ex2.approx under whole-number exponent shifts (the factor between such
+// a shift and the one the partial is defined under is applied once per row, in float64), float32 sums per thread,
+// float64 across threads.  One block of four warps per row slice, several blocks per SM.  A row whose state says
+// VS_F64 is left to the float64 kernel, which is launched behind this one for those rows only.
+constexpr int FT = 128, FW = FT / 32;
+constexpr uint32_t VF_FILLER = 0xFF7FFF7Fu;       // two bf16 of the most negative finite value
+constexpr double VF_LOG2E = 1.4426950408889634;
+
+template <int NV>
+__device__ __forceinline__ void vf_block_sum(double (&v)[NV], double* sh) {   // the totals are valid in thread 0
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int k = 0; k < NV; ++k) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v[k] += __shfl_xor_sync(0xffffffffu, v[k], o);
+  }
+  if (lane == 0) {
+#pragma unroll
+    for (int k = 0; k < NV; ++k) sh[k * FW + warp] = v[k];
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+#pragma unroll
+    for (int k = 0; k < NV; ++k) {
+      double a = 0.0;
+#pragma unroll
+      for (int w = 0; w < FW; ++w) a += sh[k * FW + w];
+      v[k] = a;
+    }
+  }
+  __syncthreads();
+}
+__device__ __forceinline__ uint4 vf_ld(const __nv_bfloat16* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ double vf_tot(const float2 a) { return (double)a.x + (double)a.y; }
+// sums of e (d - D)^k, k = 0..4, to sums of e d^k (in place): the kernels take the moments about a constant near the
+// mean of the logit difference, where float32 products keep their digits; the partials are defined about zero
+__device__ __forceinline__ void vf_uncentre(double D, double a0, double& a1, double& a2, double& a3, double& a4) {
+  const double D2 = D * D, D3 = D2 * D, D4 = D2 * D2;
+  a4 = a4 + 4.0 * D * a3 + 6.0 * D2 * a2 + 4.0 * D3 * a1 + D4 * a0;
+  a3 = a3 + 3.0 * D * a2 + 3.0 * D2 * a1 + D3 * a0;
+  a2 = a2 + 2.0 * D * a1 + D2 * a0;
+  a1 = a1 + D * a0;
+}
+
+// The residual draw of the float32 kernels on the owning rank (all threads of the block call): weights
+// [q - p]_+ per element in float32 (in units of fq, like stage C), sums in float64.  Every warp adds up its
+// contiguous range of chunks; the warp that holds the target walks its range 32 chunks at a time, the lane whose
+// chunk holds it walks the chunk's 8 elements.
+__device__ __forceinline__ void vf_draw(const __nv_bfloat16* s, const __nv_bfloat16* t, int n_chunks, float c32, double c64,
+                                        double tau, const double* st, double* red, int* stoken) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const double lam = st[VS_LAM], target = st[VS_TARGET];
+  const bool take_last = st[VS_TAKE_LAST] != 0.0;
+  float cl = (float)(c64 * lam);
+  const float ccl = c32 - cl;
+  cl = c32 - ccl;
+  const float msf = (float)st[VS_MS], mtf = (float)st[VS_MT];
+  // (the log-sum-exps relative to the maxima: what the sums of 2^(c s'), 2^(c t') came to)
+  const double ls = st[VS_LSE_S] - st[VS_MS] / tau, lt = st[VS_LSE_T] - st[VS_MT] / tau;
+  const double kp2 = ls * VF_LOG2E, kq2 = ((1.0 - lam) * ls + lam * lt + st[VS_LOGZ]) * VF_LOG2E;
+  const float kpi = floorf((float)kp2 - 1e-3f), kqi = floorf((float)kq2 - 1e-3f);
+  const double fp = exp2((double)kpi - kp2), fq = exp2((double)kqi - kq2);
+  const float2 cc = splat(c32), cll = splat(cl), ccll = splat(ccl), kpp = splat(-kpi), kqq = splat(-kqi);
+  const float2 nms = splat(-msf), nmt = splat(-mtf);
+  const float2 nrho = splat(-(float)(fp / fq));
+  auto weights = [&](int c, float (&w)[8]) {
+    const uint4 s4 = vf_ld(s + (size_t)c * 8), t4 = vf_ld(t + (size_t)c * 8);
+    const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 sf = fadd2(unpack_bf16x2(sw[i]), nms), tf = fadd2(unpack_bf16x2(tw[i]), nmt);
+      const float2 ep = ex2f2(ffma2(sf, cc, kpp));
+      const float2 eq = ex2f2(ffma2(tf, cll, ffma2(sf, ccll, kqq)));
+      const float2 r = ffma2(ep, nrho, eq);
+      w[2 * i] = fmaxf(r.x, 0.f); w[2 * i + 1] = fmaxf(r.y, 0.f);
+    }
+  };
+  auto total = [&](const float (&w)[8]) { return fq * (double)(((w[0] + w[1]) + (w[2] + w[3])) + ((w[4] + w[5]) + (w[6] + w[7]))); };
+  const int seg = (n_chunks + FW - 1) / FW, c_lo = min(n_chunks, warp * seg), c_hi = min(n_chunks, c_lo + seg);
+  double wsum = 0.0;
+  for (int c = c_lo + lane; c < c_hi; c += 32) {
+    float w[8];
+    weights(c, w);
+    wsum += total(w);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
+  if (lane == 0) red[warp] = wsum;
+  __syncthreads();
+  double before = st[VS_BEFORE];
+  int own_w = -1, last_w = -1;
+  for (int w = 0; w < FW; ++w) {
+    if (red[w] > 0.0) last_w = w;
+    if (own_w < 0 && !take_last && before + red[w] > target) own_w = w;
+    if (own_w < 0) before += red[w];
+  }
+  const bool walk_last = own_w < 0;
+  if (walk_last) own_w = last_w;
+  if (warp == own_w) {
+    double running = before;
+    int found = -1, last_c = -1;
+    for (int c0 = c_lo; c0 < c_hi && found < 0; c0 += 32) {
+      const int c = c0 + lane;
+      float w[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      if (c < c_hi) weights(c, w);
+      const double mine = total(w);
+      double inc = mine;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const double up = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += up;
+      }
+      const unsigned pos = __ballot_sync(0xffffffffu, mine > 0.0);
+      const unsigned hit = walk_last ? 0u : __ballot_sync(0xffffffffu, running + inc > target);
+      if (pos) last_c = c0 + 31 - __clz(pos);
+      if (hit) {
+        const int src = __ffs(hit) - 1;
+        int f = -1;
+        if (lane == src) {
+          double run = running + inc - mine;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            run += fq * (double)w[i];
+            if (f < 0 && run > target) f = c * 8 + i;
+          }
+          if (f < 0) {                                // rounding inside the chunk: its last element with weight
+#pragma unroll
+            for (int i = 0; i < 8; ++i) if (w[i] > 0.f) f = c * 8 + i;
+          }
+        }
+        found = __shfl_sync(0xffffffffu, f, src);
+      }
+      running += __shfl_sync(0xffffffffu, inc, 31);
+    }
+    if (found < 0 && last_c >= 0) {                   // no crossing: the last element with weight in the range
+      float w[8];
+      weights(last_c, w);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) if (w[i] > 0.f) found = last_c * 8 + i;
+    }
+    if (found < 0) found = max(c_hi * 8 - 1, 0);
+    if (lane == 0) *stoken = found;
+  }
+  if (own_w < 0 && tid == 0) *stoken = max(n_chunks * 8 - 1, 0);   // no weight anywhere in the slice
+}
+
+template <int STAGE>
+__global__ void __launch_bounds__(FT) vs_fast_kernel(const VsSlice S, const double* state, double* partial, void* dlogits,
+                                                     const int64_t ld_g, const double grad_scale) {
+  __shared__ double red[7 * FW];
+  __shared__ float smax[2][FW];
+  __shared__ int sarg[FW];
+  __shared__ int stoken;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int Vl = S.V_local, n_chunks = Vl >> 3;
+  const double rtau = 1.0 / S.tau;
+  const float c32 = (float)(VF_LOG2E / S.tau);
+  const double c64 = (double)c32;                  // the multiplier the elements really see
+  const float2 cc = splat(c32), neg1 = splat(-1.f);
+  // Every element enters as its distance below the row's maxima, s' = s - max s and t' = t - max t (exact in
+  // float32 for bf16 logits): exponents are then sums of small terms, and the logit difference d' = t' - s'
+  // is taken about the difference of the maxima, so float32 products keep their digits whatever offsets the two
+  // models' logits carry.  Partials that are defined about zero are converted in float64, once per row.
+  for (int64_t row = blockIdx.x; row < S.N; row += gridDim.x) {
+    const __nv_bfloat16* s = (const __nv_bfloat16*)S.s + row * S.ld_s;
+    const __nv_bfloat16* t = (const __nv_bfloat16*)S.t + row * S.ld_t;
+    double* out = partial + row * SAKI_VSHARD_PARTIALS;
+    const double* st = state ? state + row * SAKI_VSHARD_STATE : nullptr;
+    if (STAGE > 0 && st[VS_F64] != 0.0) continue;
+    if (STAGE == 0) {
+      // ---- stage A, first sweep: the slice's maxima, and the first chunk that holds the teacher's
+      uint32_t run_s = VF_FILLER;
+      float mt_run = -CUDART_INF_F;
+      int arg_c = 0x7fffffff;
+      for (int c = tid; c < n_chunks; c += FT) {
+        const uint4 s4 = vf_ld(s + (size_t)c * 8), t4 = vf_ld(t + (size_t)c * 8);
+        run_s = max_bf16x2(run_s, max_bf16x2(max_bf16x2(s4.x, s4.y), max_bf16x2(s4.z, s4.w)));
+        const float2 cmt = unpack_bf16x2(max_bf16x2(max_bf16x2(t4.x, t4.y), max_bf16x2(t4.z, t4.w)));
+        const float cm = fmaxf(cmt.x, cmt.y);
+        if (cm > mt_run) { mt_run = cm; arg_c = c; }
+      }
+      const float2 rs2 = unpack_bf16x2(run_s);
+      float ms = fmaxf(rs2.x, rs2.y), mt = mt_run;
+      int ac = arg_c;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        ms = fmaxf(ms, __shfl_xor_sync(0xffffffffu, ms, o));
+        const float omt = __shfl_xor_sync(0xffffffffu, mt, o);
+        const int oac = __shfl_xor_sync(0xffffffffu, ac, o);
+        if (omt > mt || (omt == mt && oac < ac)) { mt = omt; ac = oac; }
+      }
+      if (lane == 0) { smax[0][warp] = ms; smax[1][warp] = mt; sarg[warp] = ac; }
+      __syncthreads();
+      ms = smax[0][0]; mt = smax[1][0]; ac = sarg[0];
+#pragma unroll
+      for (int w = 1; w < FW; ++w) {
+        ms = fmaxf(ms, smax[0][w]);
+        if (smax[1][w] > mt || (smax[1][w] == mt && sarg[w] < ac)) { mt = smax[1][w]; ac = sarg[w]; }
+      }
+      __syncthreads();
+      if (n_chunks == 0) { ms = -CUDART_INF_F; mt = -CUDART_INF_F; }
+      // ---- second sweep: the sums under the slice's own shifts (the partial's definition: no factor to apply)
+      float2 Ss = splat(0.f), St = splat(0.f), Td = splat(0.f), M1 = splat(0.f), M2 = splat(0.f), M3 = splat(0.f), M4 = splat(0.f);
+      const float msc = fminf(fmaxf(ms, -1e30f), 1e30f), mtc = fminf(fmaxf(mt, -1e30f), 1e30f);
+      const float2 nms = splat(-msc), nmt = splat(-mtc);
+#pragma unroll 2
+      for (int c = tid; c < n_chunks; c += FT) {
+        const uint4 s4 = vf_ld(s + (size_t)c * 8), t4 = vf_ld(t + (size_t)c * 8);
+        const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 sf = fadd2(unpack_bf16x2(sw[i]), nms), tf = fadd2(unpack_bf16x2(tw[i]), nmt);
+          const float2 d = ffma2(sf, neg1, tf);
+          const float2 es = ex2f2(fmul2(sf, cc));
+          const float2 et = ex2f2(fmul2(tf, cc));
+          Ss = fadd2(Ss, es);
+          St = fadd2(St, et);
+          Td = ffma2(et, d, Td);
+          const float2 d2 = fmul2(d, d);
+          M1 = ffma2(es, d, M1);
+          const float2 u = fmul2(es, d2);
+          M2 = fadd2(M2, u);
+          M3 = ffma2(u, d, M3);
+          M4 = ffma2(u, d2, M4);
+        }
+      }
+      double a[7] = {vf_tot(Ss), vf_tot(St), vf_tot(Td), vf_tot(M1), vf_tot(M2), vf_tot(M3), vf_tot(M4)};
+      vf_block_sum<7>(a, red);
+      if (tid == 0) {
+        int am = 0x7fffffff;                       // lowest index of the teacher's maximum inside its first chunk
+        if (n_chunks > 0 && ac != 0x7fffffff) {
+          for (int i = 7; i >= 0; --i) if (__bfloat162float(t[(size_t)ac * 8 + i]) == mt) am = ac * 8 + i;
+        }
+        bool finite = true;
+#pragma unroll
+        for (int k = 0; k < 7; ++k) finite = finite && isfinite(a[k]);
+        finite = finite && (n_chunks == 0 || (ms > -1e30f && mt > -1e30f && ms < 1e30f && mt < 1e30f));
+        const int x = S.proposal[row] - S.v0;
+        const bool own = x >= 0 && x < Vl;
+        for (int k = 0; k < SAKI_VSHARD_PARTIALS; ++k) out[k] = 0.0;
+        out[0] = (double)ms; out[1] = (double)mt; out[2] = am == 0x7fffffff ? 2147483647.0 : (double)(S.v0 + am);
+        out[3] = finite ? 1.0 : 0.0;
+        if (finite && n_chunks > 0) {
+          const double r2 = rtau * rtau, D = (double)mtc - (double)msc;
+          a[2] += D * a[1];
+          vf_uncentre(D, a[0], a[3], a[4], a[5], a[6]);
+          out[4] = a[0]; out[5] = a[1]; out[6] = a[2] * rtau;
+          out[7] = a[3] * rtau; out[8] = a[4] * r2; out[12] = a[5] * r2 * rtau; out[13] = a[6] * r2 * r2;
+        }
+        out[9] = own ? (double)__bfloat162float(s[x]) : 0.0; out[10] = own ? (double)__bfloat162float(t[x]) : 0.0;
+        out[11] = own ? 1.0 : 0.0;
+      }
+    } else if (STAGE == 1) {
+      // ---- stage B: one evaluation at the row's current beta, under the row's shift (its maxima: no factor)
+      if ((int)st[VS_MODE] != VS_SOLVING) {        // (block-uniform)
+        if (tid < SAKI_VSHARD_PARTIALS) out[tid] = 0.0;
+        continue;
+      }
+      const double beta = st[VS_BETA];
+      float cb = (float)(c64 * beta);
+      const float ccb = c32 - cb;                  // the exponent is formed as (c - cb) s' + cb t'
+      cb = c32 - ccb;                              // (so that the pair adds up to c exactly)
+      const float msf = (float)st[VS_MS], mtf = (float)st[VS_MT];
+      const float2 cbb = splat(cb), ccbb = splat(ccb), nms = splat(-msf), nmt = splat(-mtf);
+      float2 S0 = splat(0.f), S1 = splat(0.f), S2 = splat(0.f), S3 = splat(0.f), S4 = splat(0.f);
+#pragma unroll 2
+      for (int c = tid; c < n_chunks; c += FT) {
+        const uint4 s4 = vf_ld(s + (size_t)c * 8), t4 = vf_ld(t + (size_t)c * 8);
+        const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 sf = fadd2(unpack_bf16x2(sw[i]), nms), tf = fadd2(unpack_bf16x2(tw[i]), nmt);
+          const float2 d = ffma2(sf, neg1, tf);
+          const float2 e = ex2f2(ffma2(tf, cbb, fmul2(sf, ccbb)));
+          const float2 d2 = fmul2(d, d);
+          S0 = fadd2(S0, e);
+          S1 = ffma2(e, d, S1);
+          const float2 u = fmul2(e, d2);
+          S2 = fadd2(S2, u);
+          S3 = ffma2(u, d, S3);
+          S4 = ffma2(u, d2, S4);
+        }
+      }
+      double a[5] = {vf_tot(S0), vf_tot(S1), vf_tot(S2), vf_tot(S3), vf_tot(S4)};
+      vf_block_sum<5>(a, red);
+      if (tid == 0) {
+        const double r2 = rtau * rtau;
+        vf_uncentre((double)mtf - (double)msf, a[0], a[1], a[2], a[3], a[4]);
+        for (int k = 0; k < SAKI_VSHARD_PARTIALS; ++k) out[k] = 0.0;
+        out[0] = a[0]; out[1] = a[1] * rtau; out[2] = a[2] * r2; out[3] = a[3] * r2 * rtau; out[4] = a[4] * r2 * r2;
+      }
+    } else if (STAGE == 2) {
+      // ---- stage C: the slice's share of TV and KL(q||p); the student's logit at the teacher's argmax
+      const bool live = (int)st[VS_MODE] == VS_SETTLED;
+      const double lam = st[VS_LAM];
+      double a[3] = {0.0, 0.0, 0.0};
+      double fq = 0.0, D = 0.0;
+      if (live && lam > 0.0) {
+        const double lse_s = st[VS_LSE_S], lse_t = st[VS_LSE_T], logZ = st[VS_LOGZ];
+        float cl = (float)(c64 * lam);
+        const float ccl = c32 - cl;
+        cl = c32 - ccl;
+        const float msf = (float)st[VS_MS], mtf = (float)st[VS_MT];
+        D = (double)mtf - (double)msf;
+        // p = 2^(c s' - kp2), q = 2^((c - cl) s' + cl t' - kq2); whole-number shifts kpi <= kp2, kqi <= kq2 (both
+        // arguments stay below 1), the factors between them applied in float64
+        // (with the log-sum-exps relative to the maxima: what the sums of 2^(c s'), 2^(c t') came to)
+        const double ls = lse_s - st[VS_MS] * rtau, lt = lse_t - st[VS_MT] * rtau;
+        const double kp2 = ls * VF_LOG2E, kq2 = ((1.0 - lam) * ls + lam * lt + logZ) * VF_LOG2E;
+        const float kpi = floorf((float)kp2 - 1e-3f), kqi = floorf((float)kq2 - 1e-3f);
+        const double fp = exp2((double)kpi - kp2);
+        fq = exp2((double)kqi - kq2);
+        const float2 cll = splat(cl), ccll = splat(ccl), kpp = splat(-kpi), kqq = splat(-kqi), nrho = splat(-(float)(fp / fq));
+        const float2 nms = splat(-msf), nmt = splat(-mtf);
+        float2 R = splat(0.f), Sq = splat(0.f), Sqd = splat(0.f);
+#pragma unroll 2
+        for (int c = tid; c < n_chunks; c += FT) {
+          const uint4 s4 = vf_ld(s + (size_t)c * 8), t4 = vf_ld(t + (size_t)c * 8);
+          const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float2 sf = fadd2(unpack_bf16x2(sw[i]), nms), tf = fadd2(unpack_bf16x2(tw[i]), nmt);
+            const float2 d = ffma2(sf, neg1, tf);
+            const float2 ep = ex2f2(ffma2(sf, cc, kpp));
+            const float2 eq = ex2f2(ffma2(tf, cll, ffma2(sf, ccll, kqq)));
+            float2 r = ffma2(ep, nrho, eq);          // (q_i - p_i) / fq
+            r.x = fmaxf(r.x, 0.f); r.y = fmaxf(r.y, 0.f);
+            R = fadd2(R, r);
+            Sq = fadd2(Sq, eq);
+            Sqd = ffma2(eq, d, Sqd);
+          }
+        }
+        a[0] = vf_tot(R); a[1] = vf_tot(Sq); a[2] = vf_tot(Sqd);
+      }
+      vf_block_sum<3>(a, red);
+      if (tid == 0) {
+        for (int k = 0; k < SAKI_VSHARD_PARTIALS; ++k) out[k] = 0.0;
+        if (live && lam > 0.0) {
+          const double cc0 = st[VS_LSE_T] - st[VS_LSE_S];      // log q - log p = lam ((t - s)/tau - cc0) - log Z
+          out[0] = fq * a[0];
+          out[1] = fq * (lam * rtau * (a[2] + D * a[1]) - (lam * cc0 + st[VS_LOGZ]) * a[1]);
+        }
+        const int vs = (int)st[VS_VSTAR] - S.v0;
+        out[2] = (live && vs >= 0 && vs < Vl) ? (double)__bfloat162float(s[vs]) : 0.0;
+      }
+    } else {
+      // ---- stage D: the gradient slice; on the owning rank the residual draw
+      const int mode = (int)st[VS_MODE];
+      __nv_bfloat16* g = dlogits ? (__nv_bfloat16*)dlogits + row * ld_g : nullptr;
+      if (g) {
+        const double sc = mode == VS_FLAGGED ? 0.0 : grad_scale * st[VS_COEF] * rtau;
+        if (sc == 0.0) {
+          for (int c = tid; c < n_chunks; c += FT) *reinterpret_cast<uint4*>(g + (size_t)c * 8) = make_uint4(0, 0, 0, 0);
+        } else {
+          const float msf = (float)st[VS_MS];
+          const double kp2 = (st[VS_LSE_S] - st[VS_MS] * rtau) * VF_LOG2E;
+          const float kpi = floorf((float)kp2 - 1e-3f);
+          const float kgf = (float)(sc * exp2((double)kpi - kp2)), scf = (float)sc;     // gradient entry = e_p * kgf (- sc at the token)
+          const float2 kpp = splat(-kpi), kgg = splat(kgf), nms = splat(-msf);
+          const int tok = (int)st[VS_TOK] - S.v0;
+          const int tok_c = (tok >= 0 && tok < Vl) ? (tok >> 3) : -1;
+          for (int c = tid; c < n_chunks; c += FT) {
+            const uint4 s4 = vf_ld(s + (size_t)c * 8);
+            const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w};
+            float gv[8];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float2 ep = ex2f2(ffma2(fadd2(unpack_bf16x2(sw[i]), nms), cc, kpp));
+              const float2 v = fmul2(ep, kgg);
+              gv[2 * i] = v.x; gv[2 * i + 1] = v.y;
+            }
+            if (c == tok_c) {
+#pragma unroll
+              for (int i = 0; i < 8; ++i) if (i == (tok & 7)) gv[i] -= scf;
+            }
+            *reinterpret_cast<uint4*>(g + (size_t)c * 8) =
+                make_uint4(pack_bf16x2(gv[0], gv[1]), pack_bf16x2(gv[2], gv[3]), pack_bf16x2(gv[4], gv[5]), pack_bf16x2(gv[6], gv[7]));
+          }
+        }
+      }
+      if (tid == 0) stoken = -1;
+      __syncthreads();
+      const bool mine = mode == VS_SETTLED && st[VS_CORR] != 0.0 && (int)st[VS_OWNER] == S.rank;
+      if (mine) vf_draw(s, t, n_chunks, c32, c64, S.tau, st, red, &stoken);
+      __syncthreads();
+      if (tid == 0) {
+        for (int k = 0; k < SAKI_VSHARD_PARTIALS; ++k) out[k] = 0.0;
+        out[0] = -1.0;
+        if (mine && stoken >= 0 && stoken < Vl) {
+          out[0] = (double)(S.v0 + stoken);
+          out[1] = (double)__bfloat162float(s[stoken]); out[2] = (double)__bfloat162float(t[stoken]);
         }
       }
       __syncthreads();
@@ -471,40 +898,61 @@ __global__ void vs_combine_kernel(const VsConsts C, const int stage, const doubl
   else vs_combine_d(C, i, part, st, o);
 }
 
+// the call may use the float32 slice kernels: a property of the call's arguments alone, so that every rank's
+// combine takes the same decisions (a rank whose own slice is not aligned for them simply computes in float64)
+static bool vshard_fast_call(const saki_vshard_in& in, bool allow_fast) {
+  return allow_fast && in.dtype == SAKI_BF16 && in.eps >= 0.02f;   // below, KL needs the float64 sums (or a quadrature)
+}
+
 cudaError_t launch_vshard_partial(const saki_vshard_in& in, int stage, const double* state, double* partial, void* dlogits,
-                                  int64_t ld_g, float grad_scale, cudaStream_t st) {
+                                  int64_t ld_g, float grad_scale, bool allow_fast, cudaStream_t st) {
   VsSlice S;
   S.s = in.student_logits; S.t = in.teacher_logits; S.ld_s = in.ld_s; S.ld_t = in.ld_t; S.N = in.N;
   S.V_local = in.V_local; S.v0 = in.v0; S.rank = in.rank; S.tau = (double)in.temperature; S.proposal = in.proposal;
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  auto al16 = [](const void* q) { return ((uintptr_t)q & 15) == 0; };
+  const bool fast = vshard_fast_call(in, allow_fast) && in.V_local % 8 == 0 && in.ld_s % 8 == 0 && in.ld_t % 8 == 0 &&
+                    al16(in.student_logits) && al16(in.teacher_logits) && (!dlogits || (al16(dlogits) && ld_g % 8 == 0));
+  if (fast) {
+    const int fgrid = (int)(in.N < 8LL * sms ? in.N : 8LL * sms);
+    const double gs = (double)grad_scale;
+    if (stage == 0) vs_fast_kernel<0><<<fgrid, FT, 0, st>>>(S, state, partial, dlogits, ld_g, gs);
+    else if (stage == 1) vs_fast_kernel<1><<<fgrid, FT, 0, st>>>(S, state, partial, dlogits, ld_g, gs);
+    else if (stage == 2) vs_fast_kernel<2><<<fgrid, FT, 0, st>>>(S, state, partial, dlogits, ld_g, gs);
+    else vs_fast_kernel<3><<<fgrid, FT, 0, st>>>(S, state, partial, dlogits, ld_g, gs);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess || stage == 0) return e;          // no row is marked for float64 before the first combine
+  }
   const int grid = (int)(in.N < 3LL * sms ? in.N : 3LL * sms);
   if (in.dtype == SAKI_BF16)
-    vs_partial_kernel<__nv_bfloat16><<<dim3(grid, 1, 1), VT, 0, st>>>(S, stage, state, partial, dlogits, ld_g, (double)grad_scale);
+    vs_partial_kernel<__nv_bfloat16><<<dim3(grid, 1, 1), VT, 0, st>>>(S, stage, state, partial, dlogits, ld_g, (double)grad_scale, fast);
   else
-    vs_partial_kernel<float><<<dim3(grid, 1, 1), VT, 0, st>>>(S, stage, state, partial, dlogits, ld_g, (double)grad_scale);
+    vs_partial_kernel<float><<<dim3(grid, 1, 1), VT, 0, st>>>(S, stage, state, partial, dlogits, ld_g, (double)grad_scale, false);
   return cudaGetLastError();
 }
 
-static VsConsts consts_of(const saki_vshard_in& in) {
+static VsConsts consts_of(const saki_vshard_in& in, bool allow_fast) {
   VsConsts c;
   c.N = in.N; c.V = in.V; c.world = in.world; c.eps = (double)in.eps; c.tau = (double)in.temperature;
   c.seed = in.seed; c.row_offset = in.row_offset; c.proposal = in.proposal; c.mask = in.mask;
+  c.fast = vshard_fast_call(in, allow_fast) ? 1 : 0;
   return c;
 }
 
 cudaError_t launch_vshard_combine(const saki_vshard_in& in, int stage, const double* gathered, double* state, const saki_out& out,
-                                  unsigned int* n_solving, cudaStream_t st) {
-  const VsConsts c = consts_of(in);
+                                  unsigned int* n_solving, bool allow_fast, cudaStream_t st) {
+  const VsConsts c = consts_of(in, allow_fast);
   const int th = 128;
   vs_combine_kernel<<<(unsigned)((in.N + th - 1) / th), th, 0, st>>>(c, stage, gathered, state, out, n_solving);
   return cudaGetLastError();
 }
 
 // the same combine on HOST buffers (a caller without a GPU at hand, and the multi-process tests of the exchange)
-int vshard_combine_host(const saki_vshard_in& in, int stage, const double* gathered, double* state, const saki_out& out) {
-  const VsConsts c = consts_of(in);
+int vshard_combine_host(const saki_vshard_in& in, int stage, const double* gathered, double* state, const saki_out& out,
+                        bool allow_fast) {
+  const VsConsts c = consts_of(in, allow_fast);
   int solving = 0;
   for (int64_t i = 0; i < in.N; ++i) {
     double* st = state + i * SAKI_VSHARD_STATE;

@@ -63,9 +63,10 @@ def route_vocab_sharded(s_loc, t_loc, v0: int, V: int, proposal, eps, temperatur
 
 
 def route_vocab_sharded_local(slices, V: int, proposal, eps, temperature=1.0, seed=0, row_offset=0, mask=None,
-                              grad_scale=1.0, backward=True, stream=None):
+                              grad_scale=1.0, backward=True, stream=None, state_out=None):
     """All ranks in one process: `slices` = [(s_loc, t_loc, v0)] in rank order on one device.  Returns (out,
-    [dlogits_slice per rank], waves): the calls every rank would make, one rank after the other."""
+    [dlogits_slice per rank], waves): the calls every rank would make, one rank after the other.  `state_out`: a
+    list that receives the per-row state tensor (for tests)."""
     world = len(slices)
     dev, N = slices[0][0].device, slices[0][0].shape[0]
     sis = [B.vshard_in(s, t, v0, V, proposal, eps, temperature, seed, row_offset, mask, r, world)
@@ -89,4 +90,6 @@ def route_vocab_sharded_local(slices, V: int, proposal, eps, temperature=1.0, se
         waves += 1
     wave(2)
     wave(3)
+    if state_out is not None:
+        state_out.append(state)
     return out, gs, waves
