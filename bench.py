@@ -270,7 +270,7 @@ def _lm_head(P, dev, stream, steps, rows=0):
                          "traffic": None}}
 
 
-def _vocab_sharded(P, synth, dev, stream, peak):
+def _vocab_sharded(P, synth, dev, stream, peak, rows=0):
     """Vocabulary-sharded routing of 4096 rows of the headline workload's shape cut into 8 column slices, the ranks
     run one after the other on this GPU (the calls one rank per GPU would make around its all-gathers): time of
     all ranks' kernels, evaluation waves, bytes a rank sends per row, and the slice kernels' HBM traffic (every
@@ -278,7 +278,7 @@ def _vocab_sharded(P, synth, dev, stream, peak):
     import torch
     from paper_2609_36601_b200 import binding as B
     from paper_2609_36601_b200.vshard import route_vocab_sharded_local, split_columns
-    w = synth.shrink(synth.WORKLOADS["cfg3"], 4096)
+    w = synth.shrink(synth.WORKLOADS["cfg3"], rows or 4096)
     d = synth.generate(w, dev)
     world = 8
     slices = [(d["s"][:, a:a + n], d["t"][:, a:a + n], a) for a, n in split_columns(w.V, world)]
@@ -679,14 +679,22 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-next", action="store_true", help="skip the metadata-driven backward measurement")
     ap.add_argument("--no-sweep", action="store_true", help="skip the throughput sweep and the V = 32000 workload")
-    ap.add_argument("--section", default="all", choices=["all", "lm_head"],
-                    help="lm_head: time only the lm-head GEMM (on --rows positions if given) and print its object (profiling)")
+    ap.add_argument("--section", default="all", choices=["all", "lm_head", "vocab_sharded"],
+                    help="lm_head / vocab_sharded: time only that section (on --rows positions if given) and print its object (profiling)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-rows", type=int, default=384)
     ap.add_argument("--ref-rows", type=int, default=32)
     args = ap.parse_args()
     if args.gpus > 1 and "RANK" not in os.environ:
         sys.exit(_spawn_ranks(args.gpus))
+    if args.section == "vocab_sharded":
+        import torch
+        import paper_2609_36601_b200 as P
+        from paper_2609_36601_b200 import synth
+        torch.cuda.set_device(0)
+        peak, _ = _peaks()
+        print(json.dumps(_vocab_sharded(P, synth, "cuda:0", torch.cuda.current_stream(), peak, args.rows)))
+        return
     if args.section == "lm_head":
         import torch
         import paper_2609_36601_b200 as P
