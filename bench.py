@@ -556,17 +556,18 @@ def run_ours(args):
                 "frac_of_nominal_8TBs": achieved / 8000.0}
     if kernel_used == 3:
         # What the kernel is actually bound by: exponentials on the special-function pipe.  Per vocabulary
-        # element 2 in pass lse (student, teacher), 2 in pass final (p, q) and 1 per evaluation pass, the
+        # element 2 in pass lse (student, teacher), 2 in pass final (p, q; a quarter of the p's are computed on
+        # the FMA pipe instead: 1.75 on this pipe) and 1 per evaluation pass, the
         # evaluation passes counted by the kernel itself; peak = 16 ex2 per clock per SM (the throughput of
         # base-2 exponentials on this architecture) x SMs x the SM clock sampled during the timed region.
         evals = evals_last_step / max(1, w.N)
         sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
         mhz = (clocks or {}).get("sm_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0
         xu_peak = 16.0 * sm_count * mhz * 1e6 / 1e9
-        xu_ach = (4.0 + evals) * w.V * w.N / (kern_ms * 1e-3) / 1e9
+        xu_ach = (3.75 + evals) * w.V * w.N / (kern_ms * 1e-3) / 1e9
         roofline["special_function_pipe"] = {"achieved": xu_ach, "peak": xu_peak, "unit": "G ex2/s",
                                              "frac": xu_ach / xu_peak, "evaluation_passes_per_row": evals,
-                                             "ex2_per_element": 4.0 + evals}
+                                             "ex2_per_element": 3.75 + evals, "exponentials_per_element": 4.0 + evals}
         # and its other near-binding bound: issue slots (4 warp-instructions per clock per SM); the instruction
         # count per 32 elements is the profiler's (smsp__inst_executed.sum of the capture the kernel's ncu
         # summary describes, divided by the elements of that launch), not counted live

@@ -55,6 +55,29 @@ __device__ __forceinline__ float2 fadd2(float2 a, float2 b) { return __fadd2_rn(
 __device__ __forceinline__ float2 fmul2(float2 a, float2 b) { return __fmul2_rn(a, b); }
 __device__ __forceinline__ float2 ex2f2(float2 a) { return make_float2(ex2f(a.x), ex2f(a.y)); }
 __device__ __forceinline__ float2 splat(float a) { return make_float2(a, a); }
+// 2^x for a pair on the FMA pipe, for x <= 0 (clamped at -126: the result is then 2^-126, which the callers' sums
+// ignore): x = n + f with n = round(x) by the magic-number addition, a degree-5 polynomial for 2^f on
+// [-1/2, 1/2] (near-minimax, relative error 1.0e-7; 1.8e-7 as evaluated in float32: what ex2.approx gives),
+// the exponent inserted by an integer add.  Twelve issue slots for two exponentials: worth it only where the
+// special-function pipe is the tighter bound, and only for a share of the exponentials.
+constexpr float EX2_C1 = 0.6931470632553101f, EX2_C2 = 0.24022242426872253f, EX2_C3 = 0.05550636723637581f,
+                EX2_C4 = 0.009671509265899658f, EX2_C5 = 0.0013292919611558318f;
+__device__ __forceinline__ float2 ex2_fma2(float2 x) {
+  x.x = fmaxf(x.x, -126.f); x.y = fmaxf(x.y, -126.f);
+  const float2 t = __fadd2_rn(x, make_float2(12582912.f, 12582912.f));              // 1.5 * 2^23: the low bits of t hold n
+  const float2 nf = __fadd2_rn(t, make_float2(-12582912.f, -12582912.f));
+  const float2 f = __ffma2_rn(nf, make_float2(-1.f, -1.f), x);
+  float2 p = make_float2(EX2_C5, EX2_C5);
+  p = __ffma2_rn(p, f, make_float2(EX2_C4, EX2_C4));
+  p = __ffma2_rn(p, f, make_float2(EX2_C3, EX2_C3));
+  p = __ffma2_rn(p, f, make_float2(EX2_C2, EX2_C2));
+  p = __ffma2_rn(p, f, make_float2(EX2_C1, EX2_C1));
+  p = __ffma2_rn(p, f, make_float2(1.f, 1.f));
+  float2 r;
+  r.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23));
+  r.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23));
+  return r;
+}
 
 // ---- short float64 routines for the scalar phases (one thread, latency-bound) ----
 // log2(1 + (i+0.5)/16) and 2^(i/16), i = 0..15

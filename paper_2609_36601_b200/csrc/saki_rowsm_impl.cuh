@@ -501,8 +501,8 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const float2 sf = unpack_bf16x2(sw[i]), tf = unpack_bf16x2(tw[i]);
-      const float2 ep = ex2f2(ffma2(sf, splat(c32), splat(k0p)));
-      const float2 eq = ex2f2(ffma2(tf, splat(clp), ffma2(sf, splat(c32 - clp), splat(kqp))));   // as in pass "final"
+      const float2 ep = i == 0 ? ex2_fma2(ffma2(sf, splat(c32), splat(k0p))) : ex2f2(ffma2(sf, splat(c32), splat(k0p)));   // as in pass "final"
+      const float2 eq = ex2f2(ffma2(tf, splat(clp), ffma2(sf, splat(c32 - clp), splat(kqp))));
       w[2 * i] = pbonus ? eq.x : fmaxf(fmaf(ep.x, -rhop, eq.x), 0.f);
       w[2 * i + 1] = pbonus ? eq.y : fmaxf(fmaf(ep.y, -rhop, eq.y), 0.f);
     }
@@ -817,7 +817,9 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const float2 sf = unpack_bf16x2(sw[i]), tf = unpack_bf16x2(tw[i]);
-          const float2 ep = ex2f2(ffma2(sf, cc, kk0));
+          // (one of the chunk's eight exponential pairs goes to the FMA pipe: this pass is bound by the
+          // special-function pipe, and one pair is what the issue slots have room for)
+          const float2 ep = i == 0 ? ex2_fma2(ffma2(sf, cc, kk0)) : ex2f2(ffma2(sf, cc, kk0));
           const float2 eq = ex2f2(ffma2(tf, cll, ffma2(sf, ccl, kqq)));     // c s + cl (t - s) as (c - cl) s + cl t: no difference to form
 
           sqc = fadd2(sqc, eq);
