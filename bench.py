@@ -55,13 +55,13 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one rowsm_kernel launch divided by the positions it
 # routed, from an ncu capture on 2220 rows of the same workload (the kernel's ncu summary gives the
 # command); traffic grows in proportion to the rows, so a full launch is this figure times N
-TRAFFIC_BYTES_PER_POSITION = 958203
+TRAFFIC_BYTES_PER_POSITION = 958376
 # rows up to this length are served by the instances of the two streaming kernels that run two CTAs per SM
 # (namespace half_sm, meta_stream_kernel<16>); the names below are the ones a profiler shows
 TWO_CTA_MAX_V = 98304
 FOUR_CTA_MAX_V = 49152      # and the row kernel's instance with four (namespace quarter_sm) up to this length
 # warp-instructions the row kernel's one-CTA instance issues per 32 vocabulary elements, from the same capture
-ISSUED_PER_32_ELEMENTS = 37.75
+ISSUED_PER_32_ELEMENTS = 39.09
 # the same for one meta_stream_kernel launch
 META_TRAFFIC_BYTES_PER_POSITION = 581046
 
