@@ -133,3 +133,23 @@ def test_hard_rows_in_slices(eps):
         assert state[0][8, 30] != 0        # the flat row is handed over
     print(f"\n[parity] hard rows in 4 slices, eps={eps}: {waves} waves, {n64} of {N} rows handed to the float64 slice "
           f"kernels, margin-exempt {n_exempt}, max |dlambda| {np.max(np.abs(out['lambda'].cpu().numpy() - ref['lam'])):.2e}")
+
+
+@pytest.mark.parametrize("dtype,temperature,eps", [("bf16", 0.7, 0.1), ("bf16", 1.6, 0.03), ("f32", 0.9, 0.1)])
+def test_temperature_and_dtype_in_slices(dtype, temperature, eps):
+    """Temperatures other than 1 (they scale both logit rows, the moments of the logit difference and the gradient)
+    on the float32 slice kernels, and fp32 logits, which the float64 kernels take."""
+    V = 8192 if dtype == "bf16" else 1024
+    w = synth.Workload("vs", 48, V, dtype, eps, 1.5, dtype == "bf16", 1200, 61, temperature=temperature)
+    d = synth.generate(w, DEV)
+    out, gs, waves = route_vocab_sharded_local(_slices(d, split_columns(V, 4)), V, d["proposal"], eps, temperature, w.seed,
+                                               grad_scale=0.25)
+    torch.cuda.synchronize()
+    s64, t64 = oracle_inputs(d)
+    ref = O.route(s64, t64, d["proposal"].cpu().numpy(), eps, temperature, w.seed, grad_scale=0.25, want_grad=True,
+                  grad_dtype=dtype)
+    n_exempt = compare_rows(out, ref)
+    assert n_exempt <= 2
+    same = out["corrected"].cpu().numpy() == ref["corrected"]
+    grad_check(to_np64(torch.cat(gs, dim=1))[same], ref["grad"][same], dtype,
+               np.where(ref["corrected"] == 1, ref["teacher_top1"], ref["token"])[same])
