@@ -157,7 +157,7 @@ static int dispatch_rows(RowParams p, int dtype, cudaStream_t st, int32_t* scrat
   const bool eps_ok = !(p.eps > 0.f) || p.eps >= 5e-3f;
   const bool rowsm_ok = (which == 0 || which == 3) && rowsm_can_serve(p, dtype);
   const bool fast = (which != 1) && (rowsm_ok || (eps_ok && cluster_can_serve(p, dtype)));
-  p.redo_list = nullptr; p.redo_count = nullptr; p.from_list = 0;
+  p.redo_list = nullptr; p.redo_count = nullptr; p.redo_guess = nullptr; p.from_list = 0;
   p.wait_limit = g_wait_limit.load();
   g_last_redo_count = nullptr;          // the counters below describe this call only
   std::unique_lock<std::mutex> scratch_lock(g_redo_mu, std::defer_lock);
@@ -167,6 +167,9 @@ static int dispatch_rows(RowParams p, int dtype, cudaStream_t st, int32_t* scrat
       scratch_lock.lock();       // until the kernels that use the list are launched
       const int rc = redo_scratch(p.n_rows, st, &p.redo_list, &p.redo_count);
       if (rc) return rc;
+      // the words behind the counters (one per row; block verification keeps its sequences' stops there) take
+      // what the float32 kernel made of lambda for the rows it hands over
+      if (!p.spec) p.redo_guess = (float*)(p.redo_count + 64);
     }
     // the counter, the three statistics words after it, and the phase clock's sums
     e = cudaMemsetAsync(p.redo_count, 0, (8 + 2 * SAKI_PHASE_COUNTERS) * sizeof(unsigned int), st);

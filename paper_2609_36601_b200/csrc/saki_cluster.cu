@@ -347,7 +347,11 @@ __global__ void __launch_bounds__(CT, 2) cluster_kernel(const RowParams P, const
     if ((int)bc[BC_MODE] == MODE_FLAGGED || (int)bc[BC_MODE] == MODE_REDO) {
       const bool redo = (int)bc[BC_MODE] == MODE_REDO;   // ill-conditioned for float32: the float64 kernel routes it
       if (rank == 0 && tid == 0) {
-        if (redo) P.redo_list[atomicAdd(P.redo_count, 1u)] = (int32_t)row;
+        if (redo) {
+          const unsigned int slot = atomicAdd(P.redo_count, 1u);
+          P.redo_list[slot] = (int32_t)row;
+          if (P.redo_guess) P.redo_guess[slot] = (float)bc[BC_BETA];     // where the float64 kernel starts its iteration
+        }
         else {
           write_row(P.out, row, zero_row((uint32_t)bc[BC_STATUS]), !P.spec);
           atomicAdd(P.flagged, 1ull);

@@ -42,6 +42,7 @@ struct RowParams {
   int32_t* redo_list;                  // scratch: rows the float32 kernels hand to the float64 kernel
   unsigned int* redo_count;            // scratch: their number (zeroed before the launch, with the three words
                                        // after it: [1], [2] see seq_next; [3] evaluation passes of the row-per-SM kernel)
+  float* redo_guess;                   // scratch or NULL: what the float32 kernel made of lambda for each row of redo_list (< 0: nothing)
   int32_t from_list;                   // general kernel only: route the rows of redo_list
   int32_t list_min, list_max;          // ... and only if their number lies in [list_min, list_max] (0, 0: any number)
   long long wait_limit;                // row-per-SM kernel: SM cycles a block waits for a row's bulk copy (<= 0: ~2 s)

@@ -7,6 +7,13 @@
 
 namespace saki {
 
+// Tolerances of the float32 solve (scalar_after_solve4), set against the float64 kernel on random rows (shapes,
+// radii from 1e-3 to 3, temperatures 0.7 to 1.3): the direct value of KL from float32 sums is trusted where its
+// error bound moves lambda by less than 3e-6 (its worst case is about twice the bound: 1e-5 let one call in fifty
+// have a row more than 1e-5 off); the one-panel quadrature only up to beta = 0.25 (beyond, the slope of KL of a
+// nearly one-hot row grows so fast over [0, beta] that the two rules agree to 1e-6 and are both 1e-4 off).
+constexpr double KL_TOL_REL = 3e-6;
+constexpr double QUAD_MAX_BETA = 0.25;
 constexpr int BC_DOUBLES = 56;             // doubles of one broadcast area
 constexpr double LN2 = 0.693147180559945309417232121458;
 constexpr double INV_LN2 = 1.44269504088896340735992468100;
@@ -273,7 +280,7 @@ static __device__ __noinline__ void scalar_after_lse_tail(double* bc, const doub
   const double chk = ((v[0] + v[1]) + (v[2] + v[3])) + (v[4] + v[5]);
   if (row_timeout) status = SAKI_ROW_TIMEOUT;
   else if (!(fabs(chk) < CUDART_INF) || !(SsT > 0.0) || !(StT > 0.0)) {
-    if (overflow_redo) { bc[BC_MODE] = MODE_REDO; return; }
+    if (overflow_redo) { bc[BC_BETA] = -1.0; bc[BC_MODE] = MODE_REDO; return; }      // (no estimate of lambda to hand over)
     status = SAKI_ROW_NONFINITE;
   }
   else if (!bonus && (x < 0 || x >= K.V)) status = SAKI_ROW_BAD_ID;
@@ -358,7 +365,7 @@ static __device__ __noinline__ void scalar_after_solve4(double* bc, const double
   const double G0 = bc[BC_G0], kb = bc[BC_KB];
   double lo = bc[BC_LO], hi = bc[BC_HI];
   const int iter = (int)bc[BC_ITER] + 1;
-  if (!(fabs((v[0] + v[1]) + (v[2] + v[3]) + v[4]) < CUDART_INF)) { bc[BC_MODE] = MODE_REDO; return; }   // float32 sums overflowed
+  if (!(fabs((v[0] + v[1]) + (v[2] + v[3]) + v[4]) < CUDART_INF)) { bc[BC_BETA] = -1.0; bc[BC_MODE] = MODE_REDO; return; }   // float32 sums overflowed
   // this evaluation: log-partition and cumulants of d under q at bc[BC_BETA]
   double beta = bc[BC_BETA], G, G1, G2, G3, G4;
   bool well_conditioned;
@@ -413,8 +420,8 @@ static __device__ __noinline__ void scalar_after_solve4(double* bc, const double
       const double h2 = beta * beta;
       const double i6 = 0.5 * beta * f1 + h2 * 0.1 * (f0p - f1p) + h2 * beta * (1.0 / 120.0) * (f0pp + f1pp);
       const double i7 = rule7(beta, G2, G3, G4);
-      if (i7 > 0.0 && fabs(i7 - i6) <= 2e-6 * i7) { kl = i7; by_quadrature = true; }
-      else if (i7 > 0.0 && 3e-7 * (eps < 5e-3 ? 1.0 : bc[BC_PMAX]) > (eps < 5e-3 ? 2e-6 : 1e-5) * beta * G2 && iter < 38) {
+      if (i7 > 0.0 && fabs(i7 - i6) <= 2e-6 * i7 && beta <= QUAD_MAX_BETA) { kl = i7; by_quadrature = true; }
+      else if (i7 > 0.0 && 3e-7 * (eps < 5e-3 ? 1.0 : bc[BC_PMAX]) > (eps < 5e-3 ? 2e-6 : KL_TOL_REL) * beta * G2 && iter < 38) {
         // neither form will do (see the second-tier test below): evaluate at beta/2 first
         bc[BC_QSTATE] = 1.0;
         bc[BC_E_BETA] = beta; bc[BC_E_G] = G; bc[BC_E_G1] = G1; bc[BC_E_G2] = G2; bc[BC_E_G3] = G3; bc[BC_E_G4] = G4;
@@ -462,9 +469,13 @@ static __device__ __noinline__ void scalar_after_solve4(double* bc, const double
   // Below 5e-3 the direct value, where the quadrature was not taken, is held to a fifth of the tolerance
   // and to the worst case of its error: 3e-7 absolute (a flat row, where ex2.approx errs the same way on
   // every element).
-  const double kl_tol = (eps < 5e-3 ? 2e-6 : 1e-5) * slope;
+  const double kl_tol = (eps < 5e-3 ? 2e-6 : KL_TOL_REL) * slope;
   const double kl_err = 3e-7 * (eps < 5e-3 ? 1.0 : bc[BC_PMAX]);
-  if (done && ((!by_quadrature && kl_err > kl_tol) || iter >= 40)) { bc[BC_MODE] = MODE_REDO; return; }
+  if (done && ((!by_quadrature && kl_err > kl_tol) || iter >= 40)) {
+    bc[BC_BETA] = iter >= 40 ? -1.0 : nb;     // what float32 made of lambda: the float64 kernel starts there
+    bc[BC_MODE] = MODE_REDO;
+    return;
+  }
   if (done) {
     float cl = (float)(K.c64 * nb);
     {   // rounded so that (c - cl) + cl = c exactly in float32: pass "final" of the row-per-SM kernel forms the

@@ -201,6 +201,10 @@ __global__ void __launch_bounds__(GT) general_kernel(const RowParams P) {
         double lo = 0.0, hi = 1.0;
         double beta = sqrt(2.0 * eps / fmax(varp, 1e-300));
         if (!(beta > 0.0 && beta < 1.0)) beta = 0.5;
+        if (P.from_list && P.redo_guess) {       // the float32 kernel's value of lambda, good to ~1e-5: two steps from here
+          const double g0 = (double)P.redo_guess[item];
+          if (g0 > 0.0 && g0 < 1.0) beta = g0;
+        }
         for (int it = 0; it < 100; ++it) {
           double a[3] = {0.0, 0.0, 0.0};
           for (int v = e0; v < V; v += ET) {

@@ -603,14 +603,17 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
         const float2 cmt = unpack_bf16x2(max_bf16x2(max_bf16x2(tw[0], tw[1]), max_bf16x2(tw[2], tw[3])));
         const float cm_t = fmaxf(cmt.x, cmt.y);
         if (valid && cm_t > mt_run) { mt_run = cm_t; arg_c = c; }
+        // the two sums of exponentials are formed per chunk first and then added to the running sums: a thread's
+        // running sum takes one addition per chunk, so a dominant element swamps four times fewer small ones
+        float2 cs = splat(0.f), ct = splat(0.f);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const float2 sf = unpack_bf16x2(sw[i]), tf = unpack_bf16x2(tw[i]);
           const float2 d = ffma2(sf, neg1, tf);
           const float2 es = ex2f2(ffma2(sf, cc, kk0));
           const float2 et = ex2f2(ffma2(tf, cc, kk1));
-          Ss = fadd2(Ss, es);
-          St = fadd2(St, et);
+          cs = i == 0 ? es : fadd2(cs, es);
+          ct = i == 0 ? et : fadd2(ct, et);
           const float2 d2 = fmul2(d, d);
           M1 = ffma2(es, d, M1);
           const float2 u = fmul2(es, d2);
@@ -619,6 +622,8 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
           M4 = ffma2(u, d2, M4);
           N1 = ffma2(et, d, N1);
         }
+        Ss = fadd2(Ss, cs);
+        St = fadd2(St, ct);
       }, [] {});
       RTS(PH_LSE);
       // warp: teacher maximum with the lowest chunk that holds it (a chunk belongs to one thread, so
@@ -737,19 +742,22 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
       const float2 cc = splat(c32), cbb = splat(cb), kbb = splat(kb), neg1 = splat(-1.f);
       for_each_chunk(sg, lane, res_s, res_t, g_s, g_t, g_s, g_t, pol_last, rg, [&](const uint4& s4, const uint4& t4, int, bool) {
         const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
+        float2 c0 = splat(0.f), c1 = splat(0.f);       // the chunk's share of S0 and S1 (see pass "lse")
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const float2 sf = unpack_bf16x2(sw[i]), tf = unpack_bf16x2(tw[i]);
           const float2 d = ffma2(sf, neg1, tf);
           const float2 e = ex2f2(ffma2(d, cbb, ffma2(sf, cc, kbb)));
           const float2 d2 = fmul2(d, d);
-          S0 = fadd2(S0, e);
-          S1 = ffma2(e, d, S1);
+          c0 = i == 0 ? e : fadd2(c0, e);
+          c1 = i == 0 ? fmul2(e, d) : ffma2(e, d, c1);
           const float2 u = fmul2(e, d2);
           S2 = fadd2(S2, u);
           S3 = ffma2(u, d, S3);
           S4 = ffma2(u, d2, S4);
         }
+        S0 = fadd2(S0, c0);
+        S1 = fadd2(S1, c1);
       }, [] {});
       RTS(PH_SOLVE);
       auto tot = [](const float2 a) { return (double)a.x + (double)a.y; };
@@ -774,7 +782,11 @@ __global__ void __launch_bounds__(RT, CTAS_PER_SM) rowsm_kernel(const RowParams 
     if ((int)bc[BC_MODE] == MODE_FLAGGED || (int)bc[BC_MODE] == MODE_REDO) {
       const bool redo = (int)bc[BC_MODE] == MODE_REDO;   // ill-conditioned for float32: the float64 kernel routes it
       if (tid == 0) {
-        if (redo) P.redo_list[atomicAdd(P.redo_count, 1u)] = (int32_t)row;
+        if (redo) {
+          const unsigned int slot = atomicAdd(P.redo_count, 1u);
+          P.redo_list[slot] = (int32_t)row;
+          if (P.redo_guess) P.redo_guess[slot] = (float)bc[BC_BETA];     // where the float64 kernel starts its iteration
+        }
         else {
           write_row(P.out, row, zero_row((uint32_t)bc[BC_STATUS]), !spec);
           atomicAdd(P.flagged, 1ull);

@@ -698,14 +698,15 @@ __global__ void __launch_bounds__(FT) vs_fast_kernel(const VsSlice S, const doub
       for (int c = tid; c < n_chunks; c += FT) {
         const uint4 s4 = vf_ld(s + (size_t)c * 8), t4 = vf_ld(t + (size_t)c * 8);
         const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
+        float2 cs = splat(0.f), ct = splat(0.f);     // per chunk first: a running sum takes one addition per chunk
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const float2 sf = fadd2(unpack_bf16x2(sw[i]), nms), tf = fadd2(unpack_bf16x2(tw[i]), nmt);
           const float2 d = ffma2(sf, neg1, tf);
           const float2 es = ex2f2(fmul2(sf, cc));
           const float2 et = ex2f2(fmul2(tf, cc));
-          Ss = fadd2(Ss, es);
-          St = fadd2(St, et);
+          cs = i == 0 ? es : fadd2(cs, es);
+          ct = i == 0 ? et : fadd2(ct, et);
           Td = ffma2(et, d, Td);
           const float2 d2 = fmul2(d, d);
           M1 = ffma2(es, d, M1);
@@ -714,6 +715,8 @@ __global__ void __launch_bounds__(FT) vs_fast_kernel(const VsSlice S, const doub
           M3 = ffma2(u, d, M3);
           M4 = ffma2(u, d2, M4);
         }
+        Ss = fadd2(Ss, cs);
+        St = fadd2(St, ct);
       }
       double a[7] = {vf_tot(Ss), vf_tot(St), vf_tot(Td), vf_tot(M1), vf_tot(M2), vf_tot(M3), vf_tot(M4)};
       vf_block_sum<7>(a, red);
@@ -758,19 +761,22 @@ __global__ void __launch_bounds__(FT) vs_fast_kernel(const VsSlice S, const doub
       for (int c = tid; c < n_chunks; c += FT) {
         const uint4 s4 = vf_ld(s + (size_t)c * 8), t4 = vf_ld(t + (size_t)c * 8);
         const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w}, tw[4] = {t4.x, t4.y, t4.z, t4.w};
+float2 c0 = splat(0.f), c1 = splat(0.f);      // the chunk's share of S0 and S1
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const float2 sf = fadd2(unpack_bf16x2(sw[i]), nms), tf = fadd2(unpack_bf16x2(tw[i]), nmt);
           const float2 d = ffma2(sf, neg1, tf);
           const float2 e = ex2f2(ffma2(tf, cbb, fmul2(sf, ccbb)));
           const float2 d2 = fmul2(d, d);
-          S0 = fadd2(S0, e);
-          S1 = ffma2(e, d, S1);
+          c0 = i == 0 ? e : fadd2(c0, e);
+          c1 = i == 0 ? fmul2(e, d) : ffma2(e, d, c1);
           const float2 u = fmul2(e, d2);
           S2 = fadd2(S2, u);
           S3 = ffma2(u, d, S3);
           S4 = ffma2(u, d2, S4);
         }
+        S0 = fadd2(S0, c0);
+        S1 = fadd2(S1, c1);
       }
       double a[5] = {vf_tot(S0), vf_tot(S1), vf_tot(S2), vf_tot(S3), vf_tot(S4)};
       vf_block_sum<5>(a, red);
