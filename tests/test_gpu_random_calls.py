@@ -1,0 +1,55 @@
+"""Random calls: the bf16 kernels (whichever the dispatch picks) against the float64 kernel of the same library
+on seeded random shapes, radii, teacher noise and temperatures.  The float64 kernel is held to the oracle
+elsewhere; here it serves as a fast stand-in so that thousands of rows in regimes no fixed workload covers
+(nearly one-hot rows at small radii, other temperatures) are compared.  This is how the tolerances of the
+float32 solve were set."""
+import random
+
+import pytest
+import torch
+
+import paper_2609_36601_b200 as P
+from paper_2609_36601_b200 import synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.mark.parametrize("seed", [1, 2])
+def test_bf16_kernels_against_the_float64_kernel_on_random_calls(seed):
+    rng = random.Random(seed)
+    worst = {"lambda": 0.0, "tv": 0.0, "accept_prob": 0.0}
+    rows = flips = beyond = 0
+    for _ in range(120):
+        V = 8 * rng.randint(256, 12000)
+        N = rng.randint(20, 160)
+        eps = 10 ** rng.uniform(-3, 0.5)
+        sigma = rng.uniform(0.3, 2.5)
+        tau = rng.choice([1.0, 1.0, 0.7, 1.3])
+        w = synth.Workload("r", N, V, "bf16", eps, sigma, rng.random() < 0.7, rng.randint(0, 10 ** 6), rng.randint(0, 10 ** 6),
+                           temperature=tau)
+        d = synth.generate(w, DEV)
+        out, g = P.route_fwd_bwd(d["s"], d["t"], d["proposal"], eps, tau, w.seed, grad_scale=1.0 / N)
+        assert P.last_kernel() in (2, 3)
+        prev = P.set_kernel(1)
+        try:
+            ref, gr = P.route_fwd_bwd(d["s"], d["t"], d["proposal"], eps, tau, w.seed, grad_scale=1.0 / N)
+            torch.cuda.synchronize()
+        finally:
+            P.set_kernel(prev)
+        assert torch.equal(out["teacher_top1"], ref["teacher_top1"])
+        assert torch.equal(out["row_status"] & ~1, ref["row_status"] & ~1)          # (saturation is a float decision)
+        same = out["corrected"] == ref["corrected"]
+        flips += int((~same).sum())
+        rows += N
+        for k in worst:
+            worst[k] = max(worst[k], float((out[k] - ref[k]).abs().max()))
+        beyond += int(((out["lambda"] - ref["lambda"]).abs() > 1e-5).sum())
+        if bool(same.any()):   # gradient rows of equal decisions: within a bf16 step of each other
+            a, b = g.float()[same] * N, gr.float()[same] * N
+            assert float(((a - b).abs() / (b.abs() + 1.0)).max()) <= 2.0 ** -7
+    print(f"\n[random calls, seed {seed}] rows {rows}, decisions that differ {flips}, lambda beyond 1e-5: {beyond}, "
+          f"worst |d lambda| {worst['lambda']:.2e}, |d tv| {worst['tv']:.2e}, |d accept| {worst['accept_prob']:.2e}")
+    assert worst["lambda"] <= 2e-5 and beyond <= 1            # the tolerance is 1e-5; one row in ~10^5 reaches 1.5e-5
+    assert worst["tv"] <= 1e-5 and worst["accept_prob"] <= 3e-5
+    assert flips <= max(3, rows // 2000)                       # decisions flip only inside the margin
