@@ -53,3 +53,32 @@ def test_bf16_kernels_against_the_float64_kernel_on_random_calls(seed):
     assert worst["lambda"] <= 2e-5 and beyond <= 1            # the tolerance is 1e-5; one row in ~10^5 reaches 1.5e-5
     assert worst["tv"] <= 1e-5 and worst["accept_prob"] <= 3e-5
     assert flips <= max(3, rows // 2000)                       # decisions flip only inside the margin
+
+
+def test_float64_kernel_against_the_oracle_on_random_calls():
+    """The stand-in itself: the float64 kernel against the oracle on random small calls of the same regimes."""
+    import numpy as np
+    import oracle as O
+    from parity import compare_rows, oracle_inputs
+    rng = random.Random(7)
+    worst = 0.0
+    prev = P.set_kernel(1)
+    try:
+        for _ in range(40):
+            V = rng.choice([rng.randint(2, 40), 8 * rng.randint(16, 900)])
+            N = rng.randint(1, 12)
+            dtype = "bf16" if V >= 128 and rng.random() < 0.7 else "f32"
+            eps = 10 ** rng.uniform(-3, 0.5)
+            tau = rng.choice([1.0, 0.7, 1.3])
+            w = synth.Workload("r", N, V, dtype, eps, rng.uniform(0.3, 2.5), V >= 128 and rng.random() < 0.7, rng.randint(0, 10 ** 6),
+                               rng.randint(0, 10 ** 6), temperature=tau)
+            d = synth.generate(w, DEV)
+            out = P.route_fwd(d["s"], d["t"], d["proposal"], eps, tau, w.seed, row_offset=3)
+            torch.cuda.synchronize()
+            s64, t64 = oracle_inputs(d)
+            ref = O.route(s64, t64, d["proposal"].cpu().numpy(), eps, tau, w.seed, 3)
+            compare_rows(out, ref)
+            worst = max(worst, float(np.max(np.abs(out["lambda"].cpu().numpy() - ref["lam"]))))
+    finally:
+        P.set_kernel(prev)
+    assert worst <= 1e-6, worst
